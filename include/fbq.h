@@ -1,0 +1,149 @@
+/*
+ * fbq.h -- C ABI of the B200 (sm_100a) FBQuant inference linear.
+ *
+ * The layer (paper: Algorithm 1 step 6, Z' = Q(W - BA) X^T + B A X^T with the
+ * low-rank sub-branch Sigma = B.A of Section 4.2; Section 4.3 "Kernel Fusion"
+ * describes the inference kernel this library replaces), for row-major tokens:
+ *
+ *     y[m][n] = sum_k x[m][k] * s[n][k/group] * ( q[n][k] - z[n][k/group] )
+ *             + sum_j ( sum_k x[m][k] * A[j][k] ) * B[n][j]
+ *
+ *   x  M x K   activations           A  rank x K  down-projection
+ *   q  N x K   3- or 4-bit codes     B  N x rank  up-projection
+ *   s,z N x (K/group) fp16 scale and (integer-valued) zero point of each group of
+ *       `group` consecutive input channels of one output row (Section 5.1: 128)
+ *   y  M x N   written once, rounded to nearest even from fp32 accumulators
+ *
+ * General rules for every entry point
+ *   - All matrices are dense row-major.  Unless a comment says HOST, pointers
+ *     are DEVICE pointers owned by the caller; the library never frees or keeps
+ *     them after the work queued on `stream` has run.  They must be 16-byte
+ *     aligned.  y must not overlap any input.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls are asynchronous: the return value reports host-side validation and
+ *     launch errors only.  Calls on one stream run in order; calls on different
+ *     streams may run concurrently (each stream gets its own scratch space).
+ *   - Return value: FBQ_OK or a negative fbq_status.
+ *   - The library runs CUDA kernels only.  There is no CPU fallback: without a
+ *     usable device every compute entry point returns FBQ_ERR_CUDA.
+ *
+ * Packed code formats (the paper does not define storage; these are fixed here)
+ *   INT4  row n = K/8 consecutive uint32; code k in word k/8, bits 4*(k%8)..+3.
+ *   INT3  row n = 3*K/32 consecutive uint32; each run of 32 codes c[0..31] is
+ *         three words; word i (0..2): bits 3f..3f+2 = c[10i+f] and bits
+ *         16+3f..16+3f+2 = c[10i+5+f] for f = 0..4; bit 15 = bit i of c[30];
+ *         bit 31 = bit i of c[31].
+ */
+#ifndef FBQ_H
+#define FBQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FBQ_OK = 0,
+    FBQ_ERR_BADARG = -1,      /* NULL pointer, non-positive size, bits not 3/4, ...      */
+    FBQ_ERR_UNSUPPORTED = -2, /* shape outside every kernel's domain                     */
+    FBQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned                        */
+    FBQ_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, launch error)    */
+    FBQ_ERR_TIMEOUT = -5      /* device side: a bounded wait on a bulk copy expired      */
+} fbq_status;
+
+typedef enum {
+    FBQ_KERNEL_NONE = -1,
+    FBQ_KERNEL_GENERIC = 0,   /* any supported shape, CUDA cores, two launches if rank>0 */
+    FBQ_KERNEL_DECODE = 1,    /* M <= 16: fused split-K streaming kernel, one launch      */
+    FBQ_KERNEL_PREFILL = 2    /* M > 16: tcgen05 / TMEM tensor-core kernel                */
+} fbq_kernel;
+
+/* Number of uint32 words of a packed N x K code matrix: N*K/8 (4 bits) or
+ * 3*N*K/32 (3 bits).  Returns 0 for unsupported arguments (bits not 3/4, K not
+ * a multiple of 8 resp. 32). */
+size_t fbq_packed_words(int N, int K, int bits);
+
+/* Pack one code per byte (codes: N x K uint8, values 0..2^bits-1; higher bits
+ * are ignored) into the formats above.  Offline step of the weight-only
+ * quantised storage (Section 1: weights kept in INT3/4). */
+int fbq_pack_int4(const uint8_t *codes, uint32_t *qweight, int N, int K, void *stream);
+int fbq_pack_int3(const uint8_t *codes, uint32_t *qweight, int N, int K, void *stream);
+
+/* Inverse of the packers (test and tooling aid). */
+int fbq_unpack(const uint32_t *qweight, uint8_t *codes, int N, int K, int bits, void *stream);
+
+/* Dense fp32 weights W[n][k] = s*(q - z) of the group-wise linear quantiser
+ * (Algorithm 1 "linear quantizer").  The product is exact in fp32.  scales and
+ * zeros hold fp16 bit patterns.  Test and tooling aid; the linear entry points
+ * never materialise W. */
+int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t *zeros,
+                float *W, int N, int K, int group, int bits, void *stream);
+
+/* The fused layer, fp16 activations: x, A, B, y are fp16; scales, zeros fp16.
+ *   rank == 0: A and B are ignored (may be NULL); y is the main path alone.
+ *   M == 0: nothing is done.
+ * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128
+ * and rank a multiple of 8 not above 256 -> decode kernel for M <= 16, prefill
+ * kernel for M > 16; everything else that is well formed -> generic kernel.
+ * Well formed means bits in {3,4}, group a multiple of 8 (4 bits) or 32
+ * (3 bits) dividing K, rank >= 0.  The decode and prefill kernels assume
+ * integer-valued zero points in [0, 127]; the generic kernel accepts any
+ * fp16 value.  Accumulation is fp32; t = x.A^T stays fp32 in the decode and
+ * generic kernels and is rounded once to the activation type in the prefill
+ * kernel.  Summation order is fixed for a given shape (results are
+ * reproducible run to run) except for t in the decode kernel, which is
+ * accumulated with floating-point atomics. */
+int fbq_linear(const void *x, const uint32_t *qweight, const void *scales, const void *zeros,
+               const void *A, const void *B, void *y, int M, int N, int K, int group, int bits,
+               int rank, void *stream);
+
+/* Same layer with bf16 x, A, B and y (scales and zeros stay fp16). */
+int fbq_linear_bf16(const void *x, const uint32_t *qweight, const void *scales,
+                    const void *zeros, const void *A, const void *B, void *y, int M, int N,
+                    int K, int group, int bits, int rank, void *stream);
+
+/* End-to-end convenience: x_host (M x K) and y_host (M x N) are HOST buffers
+ * (pinned memory makes the copies asynchronous); the weights stay on the
+ * device.  Copies x to a per-stream staging buffer, runs the layer, copies y
+ * back, all queued on `stream`; the caller synchronises the stream before
+ * reading y_host.  act_is_bf16 selects fbq_linear_bf16. */
+int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *scales,
+                      const void *zeros, const void *A, const void *B, void *y_host, int M,
+                      int N, int K, int group, int bits, int rank, int act_is_bf16,
+                      void *stream);
+
+/* Which kernel fbq_linear / fbq_linear_bf16 would run for this shape, or
+ * FBQ_KERNEL_NONE when the shape is rejected.  Pure host logic. */
+int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int act_is_bf16);
+
+/* Tuning and test switches (host side, process wide).  Known names:
+ *   "force_kernel"  -1 = automatic, else an fbq_kernel value (shapes outside the
+ *                   forced kernel's domain still fall back to the generic one)
+ *   "decode_sk"     0 = automatic, else the number of K slices of the decode kernel
+ *   "decode_chunk"  0 = automatic, else quantisation groups per smem stage
+ *   "decode_depth"  0 = automatic, else stages in flight per warp
+ *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
+ *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
+ * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name. */
+int fbq_set_option(const char *name, int value);
+int fbq_get_option(const char *name, int *value);
+
+/* Number of kernels the library has launched since load (all streams). */
+long long fbq_launch_count(void);
+
+/* Synchronises `stream` and returns the device-side status word of its scratch
+ * space: FBQ_OK, or FBQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up
+ * (the affected outputs are then undefined).  Reading clears the word. */
+int fbq_poll_status(void *stream);
+
+/* Frees every per-stream scratch buffer (synchronises the device first). */
+int fbq_release_workspaces(void);
+
+const char *fbq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FBQ_H */

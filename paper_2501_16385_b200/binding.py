@@ -1,0 +1,169 @@
+"""ctypes binding of libfbq.so.  Argument marshalling only.
+
+Tensors are torch CUDA tensors (PyTorch supplies device memory and streams);
+their data pointers and the current stream's handle are passed straight to the
+C ABI declared in include/fbq.h.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import build as _build
+
+KERNEL_NONE, KERNEL_GENERIC, KERNEL_DECODE, KERNEL_PREFILL = -1, 0, 1, 2
+STATUS = {0: "FBQ_OK", -1: "FBQ_ERR_BADARG", -2: "FBQ_ERR_UNSUPPORTED", -3: "FBQ_ERR_ALIGN",
+          -4: "FBQ_ERR_CUDA", -5: "FBQ_ERR_TIMEOUT"}
+
+_lib = None
+
+
+class FbqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, STATUS.get(code, "?"), code))
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libfbq.so (building it with nvcc when absent).  Raises if the
+    library cannot be had: there is no other implementation to run."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            path = _build.build()
+        L = ctypes.CDLL(path)
+        vp, i32 = ctypes.c_void_p, ctypes.c_int
+        L.fbq_packed_words.restype = ctypes.c_size_t
+        L.fbq_packed_words.argtypes = [i32, i32, i32]
+        for name in ("fbq_pack_int4", "fbq_pack_int3"):
+            getattr(L, name).argtypes = [vp, vp, i32, i32, vp]
+        L.fbq_unpack.argtypes = [vp, vp, i32, i32, i32, vp]
+        L.fbq_dequant.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        for name in ("fbq_linear", "fbq_linear_bf16"):
+            getattr(L, name).argtypes = [vp] * 7 + [i32] * 6 + [vp]
+        L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
+        L.fbq_select_kernel.argtypes = [i32] * 7
+        L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
+        L.fbq_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32)]
+        L.fbq_launch_count.restype = ctypes.c_longlong
+        L.fbq_poll_status.argtypes = [vp]
+        L.fbq_status_string.restype = ctypes.c_char_p
+        L.fbq_status_string.argtypes = [i32]
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise FbqError(code, where)
+
+
+def _stream(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def packed_words(N: int, K: int, bits: int) -> int:
+    return int(lib().fbq_packed_words(N, K, bits))
+
+
+def pack(codes, bits: int, stream=None):
+    """fbq_pack_int4 / fbq_pack_int3: codes uint8 [N, K] (cuda) -> qweight int32 words (cuda)."""
+    import torch
+    assert codes.is_cuda and codes.dtype == torch.uint8 and codes.is_contiguous()
+    N, K = codes.shape
+    nw = packed_words(N, K, bits)
+    if nw == 0:
+        raise FbqError(-1, "fbq_packed_words")
+    q = torch.empty(nw, dtype=torch.int32, device=codes.device)
+    fn = lib().fbq_pack_int4 if bits == 4 else lib().fbq_pack_int3
+    _check(fn(_ptr(codes), _ptr(q), N, K, _stream(stream)), "fbq_pack_int%d" % bits)
+    return q
+
+
+def unpack(qweight, N: int, K: int, bits: int, stream=None):
+    import torch
+    codes = torch.empty((N, K), dtype=torch.uint8, device=qweight.device)
+    _check(lib().fbq_unpack(_ptr(qweight), _ptr(codes), N, K, bits, _stream(stream)), "fbq_unpack")
+    return codes
+
+
+def dequant(qweight, scales, zeros, N: int, K: int, group: int, bits: int, stream=None):
+    import torch
+    W = torch.empty((N, K), dtype=torch.float32, device=qweight.device)
+    _check(lib().fbq_dequant(_ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(W), N, K, group, bits,
+                             _stream(stream)), "fbq_dequant")
+    return W
+
+
+def linear(x, qweight, scales, zeros, A, B, N: int, group: int, bits: int, y=None, stream=None):
+    """fbq_linear (fp16 x) or fbq_linear_bf16 (bf16 x).  x: [M, K]; A: [rank, K] or None;
+    B: [N, rank] or None.  Returns y [M, N] in the dtype of x."""
+    import torch
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 2
+    M, K = x.shape
+    rank = 0 if A is None else A.shape[0]
+    if y is None:
+        y = torch.empty((M, N), dtype=x.dtype, device=x.device)
+    if x.dtype == torch.float16:
+        fn, name = lib().fbq_linear, "fbq_linear"
+    elif x.dtype == torch.bfloat16:
+        fn, name = lib().fbq_linear_bf16, "fbq_linear_bf16"
+    else:
+        raise TypeError("x must be float16 or bfloat16")
+    _check(fn(_ptr(x), _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(A), _ptr(B), _ptr(y),
+              M, N, K, group, bits, rank, _stream(stream)), name)
+    return y
+
+
+def linear_hostio(x_host, qweight, scales, zeros, A, B, y_host, N: int, group: int, bits: int,
+                  stream=None):
+    """fbq_linear_hostio: x_host / y_host are (pinned) CPU tensors, weights stay on the device."""
+    import torch
+    M, K = x_host.shape
+    rank = 0 if A is None else A.shape[0]
+    bf16 = 1 if x_host.dtype == torch.bfloat16 else 0
+    _check(lib().fbq_linear_hostio(_ptr(x_host), _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(A),
+                                   _ptr(B), _ptr(y_host), M, N, K, group, bits, rank, bf16,
+                                   _stream(stream)), "fbq_linear_hostio")
+    return y_host
+
+
+def select_kernel(M, N, K, group, bits, rank, bf16=False) -> int:
+    return int(lib().fbq_select_kernel(M, N, K, group, bits, rank, 1 if bf16 else 0))
+
+
+def set_option(name: str, value: int) -> None:
+    _check(lib().fbq_set_option(name.encode(), int(value)), "fbq_set_option(%s)" % name)
+
+
+def get_option(name: str) -> int:
+    v = ctypes.c_int(0)
+    _check(lib().fbq_get_option(name.encode(), ctypes.byref(v)), "fbq_get_option(%s)" % name)
+    return v.value
+
+
+def launch_count() -> int:
+    return int(lib().fbq_launch_count())
+
+
+def poll_status(stream=None) -> int:
+    return int(lib().fbq_poll_status(_stream(stream)))
+
+
+def release_workspaces() -> None:
+    _check(lib().fbq_release_workspaces(), "fbq_release_workspaces")
+
+
+def status_string(code: int) -> str:
+    return lib().fbq_status_string(code).decode()

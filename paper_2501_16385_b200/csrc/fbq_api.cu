@@ -1,0 +1,331 @@
+// extern "C" boundary of libfbq: argument validation, kernel selection,
+// per-stream scratch space, launch bookkeeping.  Declarations and the contract
+// of every entry point are in include/fbq.h.
+#include <atomic>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
+
+#include "fbq_common.cuh"
+
+namespace fbq {
+void decode_set_test_switch(int t_late);
+
+namespace {
+
+std::mutex g_mu;
+std::map<std::pair<int, cudaStream_t>, Workspace> g_ws;
+std::atomic<long long> g_launches{0};
+
+struct Options {
+    int force_kernel = -1;
+    DecodeTuning decode;
+    int decode_t_late = 0;
+} g_opt;
+
+bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+bool well_formed(int M, int N, int K, int group, int bits, int rank)
+{
+    if (M < 0 || N < 1 || K < 1 || group < 1 || rank < 0) return false;
+    if (bits != 3 && bits != 4) return false;
+    const int unit = (bits == 4) ? 8 : 32;
+    if (group % unit != 0 || K % group != 0) return false;
+    return true;
+}
+
+int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
+{
+    if (!well_formed(M, N, K, group, bits, rank)) return FBQ_KERNEL_NONE;
+    LinearArgs a{};
+    a.M = M; a.N = N; a.K = K; a.group = group; a.bits = bits; a.rank = rank; a.bf16 = bf16;
+    const bool fast_group = (group == kGroupFast) && rank % 8 == 0 && rank <= kMaxRank;
+    const bool decode_ok = fast_group && M >= 1 && M <= kDecodeMaxM;
+    const bool prefill_ok = fast_group && M >= 1 && prefill_supported(a);
+    if (g_opt.force_kernel == FBQ_KERNEL_GENERIC) return FBQ_KERNEL_GENERIC;
+    if (g_opt.force_kernel == FBQ_KERNEL_DECODE && decode_ok) return FBQ_KERNEL_DECODE;
+    if (g_opt.force_kernel == FBQ_KERNEL_PREFILL && prefill_ok) return FBQ_KERNEL_PREFILL;
+    if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
+    if (decode_ok) return FBQ_KERNEL_DECODE;
+    if (prefill_ok && M > kDecodeMaxM) return FBQ_KERNEL_PREFILL;
+    return FBQ_KERNEL_GENERIC;
+}
+
+// Grows a device buffer; zero-fills it on `s` (the invariants of the decode
+// kernel's scratch space start from zero).  The old buffer is released only
+// after the stream has drained.
+template <typename P>
+cudaError_t grow(P *&ptr, size_t &have, size_t need, size_t elem, cudaStream_t s)
+{
+    if (need <= have) return cudaSuccess;
+    cudaError_t e;
+    if (ptr) {
+        if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return e;
+        if ((e = cudaFree(ptr)) != cudaSuccess) return e;
+        ptr = nullptr;
+        have = 0;
+    }
+    void *q = nullptr;
+    if ((e = cudaMalloc(&q, need * elem)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(q, 0, need * elem, s)) != cudaSuccess) {
+        cudaFree(q);
+        return e;
+    }
+    ptr = static_cast<P *>(q);
+    have = need;
+    return cudaSuccess;
+}
+
+Workspace *workspace_for(cudaStream_t s)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lk(g_mu);
+    return &g_ws[std::make_pair(dev, s)];
+}
+
+int run_linear(const LinearArgs &a, cudaStream_t s)
+{
+    if (!well_formed(a.M, a.N, a.K, a.group, a.bits, a.rank)) return FBQ_ERR_BADARG;
+    if (a.M == 0) return FBQ_OK;
+    if (!a.x || !a.qw || !a.scales || !a.zeros || !a.y) return FBQ_ERR_BADARG;
+    if (a.rank > 0 && (!a.A || !a.B)) return FBQ_ERR_BADARG;
+    if (misaligned16(a.x) || misaligned16(a.qw) || misaligned16(a.y) || (a.rank > 0 && (misaligned16(a.A) || misaligned16(a.B))))
+        return FBQ_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(a.scales) & 1u) || (reinterpret_cast<uintptr_t>(a.zeros) & 1u)) return FBQ_ERR_ALIGN;
+
+    Workspace *ws = workspace_for(s);
+    if (!ws) return FBQ_ERR_CUDA;
+    int kernel = select_kernel(a.M, a.N, a.K, a.group, a.bits, a.rank, a.bf16);
+    if (kernel == FBQ_KERNEL_NONE) return FBQ_ERR_UNSUPPORTED;
+    int launches = 0;
+    cudaError_t e = cudaSuccess;
+
+    if (kernel == FBQ_KERNEL_DECODE) {
+        size_t pf = 0;
+        int nc = 0;
+        decode_workspace_need(a, g_opt.decode, &pf, &nc);
+        size_t have_c = (size_t)ws->n_counters;
+        if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->t, ws->t_floats, (size_t)kDecodeMaxM * kMaxRank, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        ws->n_counters = (int)have_c;
+        e = launch_decode(a, *ws, g_opt.decode, s, &launches);
+        if (e == cudaErrorInvalidConfiguration) {
+            (void)cudaGetLastError();
+            kernel = FBQ_KERNEL_GENERIC;          // plan does not fit shared memory
+        } else if (e != cudaSuccess) {
+            return FBQ_ERR_CUDA;
+        }
+    }
+    if (kernel == FBQ_KERNEL_PREFILL) {
+        e = launch_prefill(a, *ws, s, &launches);
+        if (e == cudaErrorInvalidConfiguration) {
+            (void)cudaGetLastError();
+            kernel = FBQ_KERNEL_GENERIC;
+        } else if (e != cudaSuccess) {
+            return FBQ_ERR_CUDA;
+        }
+    }
+    if (kernel == FBQ_KERNEL_GENERIC) {
+        if (a.rank > 0 &&
+            (e = grow(ws->t_gen, ws->t_gen_floats, (size_t)a.M * a.rank, sizeof(float), s)) != cudaSuccess)
+            return FBQ_ERR_CUDA;
+        if ((e = launch_generic(a, *ws, s, &launches)) != cudaSuccess) return FBQ_ERR_CUDA;
+    }
+    g_launches += launches;
+    return FBQ_OK;
+}
+
+int *option_slot(const char *name)
+{
+    if (!name) return nullptr;
+    if (!strcmp(name, "force_kernel")) return &g_opt.force_kernel;
+    if (!strcmp(name, "decode_sk")) return &g_opt.decode.sk;
+    if (!strcmp(name, "decode_chunk")) return &g_opt.decode.chunk;
+    if (!strcmp(name, "decode_depth")) return &g_opt.decode.depth;
+    if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
+    if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
+    if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
+    return nullptr;
+}
+
+}  // namespace
+}  // namespace fbq
+
+using namespace fbq;
+
+extern "C" {
+
+size_t fbq_packed_words(int N, int K, int bits)
+{
+    if (N < 1 || K < 1) return 0;
+    if (bits == 4 && K % 8 == 0) return (size_t)N * K / 8;
+    if (bits == 3 && K % 32 == 0) return (size_t)N * K / 32 * 3;
+    return 0;
+}
+
+static int pack_common(const uint8_t *codes, uint32_t *qweight, int N, int K, int bits, void *stream)
+{
+    if (!codes || !qweight || fbq_packed_words(N, K, bits) == 0) return FBQ_ERR_BADARG;
+    if (misaligned16(codes) || misaligned16(qweight)) return FBQ_ERR_ALIGN;
+    if (launch_pack(codes, qweight, N, K, bits, static_cast<cudaStream_t>(stream)) != cudaSuccess) return FBQ_ERR_CUDA;
+    ++g_launches;
+    return FBQ_OK;
+}
+
+int fbq_pack_int4(const uint8_t *codes, uint32_t *qweight, int N, int K, void *stream)
+{
+    return pack_common(codes, qweight, N, K, 4, stream);
+}
+
+int fbq_pack_int3(const uint8_t *codes, uint32_t *qweight, int N, int K, void *stream)
+{
+    return pack_common(codes, qweight, N, K, 3, stream);
+}
+
+int fbq_unpack(const uint32_t *qweight, uint8_t *codes, int N, int K, int bits, void *stream)
+{
+    if (!codes || !qweight || fbq_packed_words(N, K, bits) == 0) return FBQ_ERR_BADARG;
+    if (misaligned16(codes) || misaligned16(qweight)) return FBQ_ERR_ALIGN;
+    if (launch_unpack(qweight, codes, N, K, bits, static_cast<cudaStream_t>(stream)) != cudaSuccess) return FBQ_ERR_CUDA;
+    ++g_launches;
+    return FBQ_OK;
+}
+
+int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t *zeros, float *W, int N, int K,
+                int group, int bits, void *stream)
+{
+    if (!qweight || !scales || !zeros || !W) return FBQ_ERR_BADARG;
+    if (!well_formed(1, N, K, group, bits, 0)) return FBQ_ERR_BADARG;
+    if (misaligned16(qweight) || misaligned16(W)) return FBQ_ERR_ALIGN;
+    if (launch_dequant(qweight, reinterpret_cast<const __half *>(scales), reinterpret_cast<const __half *>(zeros), W, N,
+                       K, group, bits, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FBQ_ERR_CUDA;
+    ++g_launches;
+    return FBQ_OK;
+}
+
+static int linear_common(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
+                         const void *B, void *y, int M, int N, int K, int group, int bits, int rank, bool bf16,
+                         void *stream)
+{
+    LinearArgs a{};
+    a.x = x; a.qw = qweight;
+    a.scales = static_cast<const __half *>(scales);
+    a.zeros = static_cast<const __half *>(zeros);
+    a.A = rank > 0 ? A : nullptr;
+    a.B = rank > 0 ? B : nullptr;
+    a.y = y;
+    a.M = M; a.N = N; a.K = K; a.group = group; a.bits = bits; a.rank = rank; a.bf16 = bf16;
+    decode_set_test_switch(g_opt.decode_t_late);
+    return run_linear(a, static_cast<cudaStream_t>(stream));
+}
+
+int fbq_linear(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
+               const void *B, void *y, int M, int N, int K, int group, int bits, int rank, void *stream)
+{
+    return linear_common(x, qweight, scales, zeros, A, B, y, M, N, K, group, bits, rank, false, stream);
+}
+
+int fbq_linear_bf16(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
+                    const void *B, void *y, int M, int N, int K, int group, int bits, int rank, void *stream)
+{
+    return linear_common(x, qweight, scales, zeros, A, B, y, M, N, K, group, bits, rank, true, stream);
+}
+
+int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *scales, const void *zeros,
+                      const void *A, const void *B, void *y_host, int M, int N, int K, int group, int bits, int rank,
+                      int act_is_bf16, void *stream)
+{
+    if (!well_formed(M, N, K, group, bits, rank)) return FBQ_ERR_BADARG;
+    if (M == 0) return FBQ_OK;
+    if (!x_host || !y_host) return FBQ_ERR_BADARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace *ws = workspace_for(s);
+    if (!ws) return FBQ_ERR_CUDA;
+    const size_t xb = (size_t)M * K * 2, yb = (size_t)M * N * 2;
+    char *sx = static_cast<char *>(ws->stage_x), *sy = static_cast<char *>(ws->stage_y);
+    if (grow(sx, ws->stage_x_bytes, xb, 1, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    if (grow(sy, ws->stage_y_bytes, yb, 1, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    ws->stage_x = sx;
+    ws->stage_y = sy;
+    if (cudaMemcpyAsync(sx, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    const int rc = linear_common(sx, qweight, scales, zeros, A, B, sy, M, N, K, group, bits, rank, act_is_bf16 != 0, stream);
+    if (rc != FBQ_OK) return rc;
+    if (cudaMemcpyAsync(y_host, sy, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    return FBQ_OK;
+}
+
+int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int act_is_bf16)
+{
+    return select_kernel(M, N, K, group, bits, rank, act_is_bf16 != 0);
+}
+
+int fbq_set_option(const char *name, int value)
+{
+    int *slot = option_slot(name);
+    if (!slot) return FBQ_ERR_BADARG;
+    *slot = value;
+    return FBQ_OK;
+}
+
+int fbq_get_option(const char *name, int *value)
+{
+    int *slot = option_slot(name);
+    if (!slot || !value) return FBQ_ERR_BADARG;
+    *value = *slot;
+    return FBQ_OK;
+}
+
+long long fbq_launch_count(void) { return g_launches.load(); }
+
+int fbq_poll_status(void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FBQ_ERR_CUDA;
+    Workspace *ws = workspace_for(s);
+    if (!ws) return FBQ_ERR_CUDA;
+    if (!ws->counters) return FBQ_OK;
+    int st = 0;
+    if (cudaMemcpy(&st, ws->counters + kCtrStatus, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FBQ_ERR_CUDA;
+    if (st != 0) {
+        // a kernel gave up half way: its bookkeeping is unfinished, start from a clean slate
+        cudaMemset(ws->counters, 0, sizeof(int) * (size_t)ws->n_counters);
+        if (ws->t) cudaMemset(ws->t, 0, sizeof(float) * ws->t_floats);
+    }
+    return st;
+}
+
+int fbq_release_workspaces(void)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess) return FBQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (auto &kv : g_ws) {
+        Workspace &w = kv.second;
+        cudaFree(w.partial);
+        cudaFree(w.t);
+        cudaFree(w.t_gen);
+        cudaFree(w.counters);
+        cudaFree(w.stage_x);
+        cudaFree(w.stage_y);
+    }
+    g_ws.clear();
+    return FBQ_OK;
+}
+
+const char *fbq_status_string(int status)
+{
+    switch (status) {
+    case FBQ_OK: return "ok";
+    case FBQ_ERR_BADARG: return "bad argument";
+    case FBQ_ERR_UNSUPPORTED: return "unsupported shape";
+    case FBQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case FBQ_ERR_CUDA: return "CUDA runtime error";
+    case FBQ_ERR_TIMEOUT: return "device-side wait expired";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Shared declarations of the CUDA sources of libfbq (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/fbq.h"
+
+namespace fbq {
+
+constexpr int kGroupFast = 128;   // group size of the decode / prefill kernels (Section 5.1)
+constexpr int kMaxRank = 256;
+constexpr int kDecodeMaxM = 16;
+
+// Activation-type helpers ---------------------------------------------------
+template <typename T> struct ActTraits;
+template <> struct ActTraits<__half> {
+    using T2 = __half2;
+    static __device__ __forceinline__ float to_float(__half v) { return __half2float(v); }
+    static __device__ __forceinline__ __half from_float(float v) { return __float2half_rn(v); }
+};
+template <> struct ActTraits<__nv_bfloat16> {
+    using T2 = __nv_bfloat162;
+    static __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+    static __device__ __forceinline__ __nv_bfloat16 from_float(float v) { return __float2bfloat16_rn(v); }
+};
+
+// Per-stream scratch space (device memory owned by the library).
+struct Workspace {
+    float *partial = nullptr;     // split-K partial sums  [SK][M][N]
+    size_t partial_floats = 0;
+    float *t = nullptr;           // down-projection t = x.A^T, [M][rank] fp32 (kept zero between calls)
+    float *t_gen = nullptr;       // t of the generic path (no invariant), grows on demand
+    size_t t_floats = 0, t_gen_floats = 0;
+    int *counters = nullptr;      // [0]=t arrivals [1]=retired tiles [2]=status [3]=t ready [4]=parked; [8..] per tile
+    int n_counters = 0;
+    void *stage_x = nullptr;      // staging for the host-buffer entry point
+    void *stage_y = nullptr;
+    size_t stage_x_bytes = 0, stage_y_bytes = 0;
+};
+constexpr int kCtrT = 0, kCtrDone = 1, kCtrStatus = 2;   // the decode kernel defines the rest
+
+struct LinearArgs {
+    const void *x;
+    const uint32_t *qw;
+    const __half *scales;
+    const __half *zeros;
+    const void *A;
+    const void *B;
+    void *y;
+    int M, N, K, group, bits, rank;
+    bool bf16;
+};
+
+// Launchers implemented in the kernel files.  Each returns a cudaError_t from
+// the launch and adds the number of kernels it launched to *launches.
+cudaError_t launch_pack(const uint8_t *codes, uint32_t *qw, int N, int K, int bits, cudaStream_t s);
+cudaError_t launch_unpack(const uint32_t *qw, uint8_t *codes, int N, int K, int bits, cudaStream_t s);
+cudaError_t launch_dequant(const uint32_t *qw, const __half *sc, const __half *ze, float *W, int N,
+                           int K, int group, int bits, cudaStream_t s);
+cudaError_t launch_generic(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
+
+struct DecodeTuning {
+    int sk = 0, chunk = 0, depth = 0, max_ctas = 0, pdl = 1;
+};
+// Returns cudaErrorInvalidConfiguration when no plan fits (caller falls back).
+cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning &tune,
+                          cudaStream_t s, int *launches);
+// Scratch the decode kernel needs for a shape (floats of partial sums, ints of counters).
+void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t *partial_floats,
+                           int *counters);
+
+bool prefill_supported(const LinearArgs &a);
+cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
+
+}  // namespace fbq
