@@ -126,6 +126,10 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "decode_depth"  0 = automatic, else stages in flight per warp
  *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
+ *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
+ *                   every tile through the parked-tile branch of the combine protocol
+ *   "decode_trace"  tuning aid: 1 = the decode kernel records phase timestamps
+ *                   (globaltimer, ns) per CTA and warp, read with fbq_debug_read_trace
  * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name. */
 int fbq_set_option(const char *name, int value);
 int fbq_get_option(const char *name, int *value);
@@ -137,6 +141,11 @@ long long fbq_launch_count(void);
  * space: FBQ_OK, or FBQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up
  * (the affected outputs are then undefined).  Reading clears the word. */
 int fbq_poll_status(void *stream);
+
+/* Tuning aid: copies the phase timestamps of the last decode launch on `stream`
+ * (recorded while "decode_trace" is 1) to host_buf: uint64 [cta][10 warps][16 marks],
+ * zero where a mark was not reached.  Synchronises the stream. */
+int fbq_debug_read_trace(void *stream, void *host_buf, size_t bytes);
 
 /* Frees every per-stream scratch buffer (synchronises the device first). */
 int fbq_release_workspaces(void);

@@ -22,7 +22,9 @@ struct Options {
     int force_kernel = -1;
     DecodeTuning decode;
     int decode_t_late = 0;
+    int decode_trace = 0;
 } g_opt;
+constexpr size_t kTraceBytes = 2 * 512 * 10 * 16 * 8;   // two launches (alternating) x 512 CTAs x 10 warps x 16 marks
 
 bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -111,6 +113,16 @@ int run_linear(const LinearArgs &a, cudaStream_t s)
         if ((e = grow(ws->t, ws->t_floats, (size_t)kDecodeMaxM * kMaxRank, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         ws->n_counters = (int)have_c;
+        if (g_opt.decode_trace && !ws->trace) {
+            if (cudaMalloc(&ws->trace, kTraceBytes) != cudaSuccess) return FBQ_ERR_CUDA;
+        }
+        if (ws->trace) {
+            if (!g_opt.decode_trace) {
+                cudaStreamSynchronize(s);
+                cudaFree(ws->trace);
+                ws->trace = nullptr;
+            }
+        }
         e = launch_decode(a, *ws, g_opt.decode, s, &launches);
         if (e == cudaErrorInvalidConfiguration) {
             (void)cudaGetLastError();
@@ -148,6 +160,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
+    if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
 
@@ -298,6 +311,15 @@ int fbq_poll_status(void *stream)
     return st;
 }
 
+int fbq_debug_read_trace(void *stream, void *host_buf, size_t bytes)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FBQ_ERR_CUDA;
+    Workspace *ws = workspace_for(s);
+    if (!ws || !ws->trace || !host_buf || bytes > kTraceBytes) return FBQ_ERR_BADARG;
+    return cudaMemcpy(host_buf, ws->trace, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? FBQ_OK : FBQ_ERR_CUDA;
+}
+
 int fbq_release_workspaces(void)
 {
     if (cudaDeviceSynchronize() != cudaSuccess) return FBQ_ERR_CUDA;
@@ -308,6 +330,7 @@ int fbq_release_workspaces(void)
         cudaFree(w.t);
         cudaFree(w.t_gen);
         cudaFree(w.counters);
+        cudaFree(w.trace);
         cudaFree(w.stage_x);
         cudaFree(w.stage_y);
     }

@@ -36,6 +36,7 @@ struct Workspace {
     size_t t_floats = 0, t_gen_floats = 0;
     int *counters = nullptr;      // [0]=t arrivals [1]=retired tiles [2]=status [3]=t ready [4]=parked; [8..] per tile
     int n_counters = 0;
+    void *trace = nullptr;        // optional phase timestamps of the decode kernel (tuning aid)
     void *stage_x = nullptr;      // staging for the host-buffer entry point
     void *stage_y = nullptr;
     size_t stage_x_bytes = 0, stage_y_bytes = 0;

@@ -6,35 +6,49 @@
 // a second launch; here t is produced by the same launch, so a decode step costs
 // one launch per linear and y is written exactly once.
 //
-// Work split.  The grid is R x SK CTAs: CTA (rr, s) owns the 16-row output tiles
-// of row range rr and the quantisation groups of K slice s.  Inside a CTA each
-// warp owns whole (tile, slice) tasks.  A task's packed codes are fetched with
-// bulk asynchronous copies (one per weight row, mbarrier completion) into a
-// small per-warp ring in shared memory, so that every SM keeps tens of KB of
-// HBM requests in flight without tying up registers.  Codes are expanded with
-// the exponent trick ((w & mask) | 0x6400 is 1024+q in fp16), the zero point is
-// subtracted exactly, and the integers q-z are contracted with x by warp-level
-// m16n8k16 tensor-core MMAs (16 weight rows x 8 tokens, fp32 accumulation); the
-// group scale multiplies the fp32 partial sum once per group.  The k order
-// inside an MMA is a fixed permutation chosen so that a lane's packed word IS
-// its operand fragment; x is stored in shared memory in the matching order.
+// Work split (stream-K).  The grid is R x SK CTAs, about one per SM.  K is cut
+// into SK slices (SK = 1 unless x is too large for shared memory); inside a
+// slice the (16-row tile, quantisation group) units are dealt out tile-major in
+// equal contiguous ranges, so every CTA streams the same number of bytes and at
+// most its first and last tile are shared with a neighbour.  A CTA walks its
+// range tile by tile ("segments").
 //
-// Cross-CTA combination is wait-free (no spinning on other CTAs): every task
-// writes its fp32 partial tile to scratch and bumps the tile's arrival counter;
-// whoever arrives last sums the SK partials in slice order, adds t.B^T and
-// stores y.  t is accumulated with fp32 atomics by the warps that own rows of A;
-// the warp that completes t publishes a flag and finishes any tile that was
-// parked waiting for it.  The only waits in the kernel are on this CTA's own
-// bulk copies, and they are bounded.
+// Warp roles.  A producer warp streams the packed codes of the range with bulk
+// asynchronous copies (one per weight row and stage, 1-2 KB each, mbarrier
+// completion) into a ring of shared-memory stages, and also fetches this CTA's
+// rows of A and B once.  Eight compute warps share every stage: each takes an
+// eighth of its groups, expands the codes with the exponent trick ((w & mask) |
+// 0x6400 is 1024+q in fp16), subtracts the zero point exactly and contracts the
+// integers q-z with x by warp-level m16n8k16 tensor-core MMAs (16 weight rows x
+// 8 tokens, fp32 accumulation); the group scale multiplies the fp32 partial sum
+// once per group.  The k order inside an MMA is a fixed permutation chosen so
+// that a lane's packed word IS its operand fragment; x is kept in shared memory
+// in the matching order.  An epilogue warp owns everything else: it computes
+// this CTA's share of t = x.A^T, and for every segment adds the eight warps'
+// partial tiles (fixed order), then finishes the tile (adds t.B^T, rounds,
+// stores y) or, for a tile shared with other CTAs, combines through scratch:
+// whoever finds all other contributions already there finishes the tile
+// directly; otherwise it leaves its partial and an arrival count, and the last
+// arrival finishes.  Nothing in the kernel spins on another CTA: a tile that
+// is complete before t is waits in a local list and, at worst, is handed to
+// the warp that completes t.  The only waits are on this CTA's own copies and
+// warps, and they are bounded.
 #include "fbq_common.cuh"
 
 namespace fbq {
 namespace {
 
-constexpr int kNW = 8;                 // warps per CTA
-constexpr int kThreads = kNW * 32;
+constexpr int kCW = 8;                       // compute warps per CTA
+constexpr int kProdWarp = kCW + 1;         // warp kCW is the epilogue warp
+constexpr int kWarps = kCW + 2;
+constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 16;
-constexpr uint32_t kWaitLimit = 1u << 24;
+constexpr int kMaxSeg = 64;                  // segments (tiles touched) per CTA
+constexpr int kNBuf = 4;                     // segment partial buffers in flight
+constexpr int kTUnitK = 1024;                // k extent of one unit of the down-projection
+constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr int kEarlyStages = 1;              // weight stages prefetched before x has been requested
+constexpr int kTPolls = 64;                  // looks at the "t complete" flag before a finished tile is parked
 
 // counters[] layout (ints) inside the per-stream scratch
 constexpr int kCtrReady = 3, kCtrPendingN = 4, kCtrFirstTile = 8;
@@ -47,17 +61,22 @@ struct DecodeParams {
     const void *A;
     const void *B;
     void *y;
-    float *partial;     // [SK][M][N]
+    float *partial;     // [NT][maxslots][M][16]
     float *t;           // [M][rank], zero on entry, zero again on exit
     int *ctr;           // counters, see above; all zero on entry and on exit
     int M, N, K, G, rank;
-    int SK, R, NT, CH, D;
-    int t_target;       // number of warps that contribute to t
+    int SK, R, NT, CHG, NS;
+    int maxslots;
+    int t_target;       // number of CTAs that contribute to t
     int t_late;         // test switch: contribute to t after the main loop
-    int meta_pitch;     // 8-byte entries per meta row (odd)
+    int vt;             // lanes per quad whose accumulators are exchanged (tokens 2tq, 2tq+1 valid)
     int x_pitch;        // elements per token in shared memory
-    int slot_bytes;
-    int off_list, off_meta, off_x, off_ring;
+    int stage_bytes;
+    int meta_rows;      // rows of the shared-memory scale / zero tables
+    int a_cap;          // units of A held in shared memory
+    int b_cap_rows;     // rows of B held in shared memory (0: read B from global memory)
+    int off_tab, off_def, off_meta, off_x, off_px, off_segbuf, off_A, off_B, off_t, off_ring;
+    unsigned long long *trace;   // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -70,6 +89,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -86,6 +109,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: returns false when the limit is hit (never spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
+#pragma unroll 1
     for (uint32_t i = 0; i < kWaitLimit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
@@ -95,10 +119,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async()
-{
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -173,84 +193,97 @@ template <> struct Pk<__nv_bfloat16> {
 };
 
 // ------------------------------------------------------------------ unpackers
-// unpack(words, z) fills h[0..15] with the pairs (q - z) of one lane's 32 codes
-// of one weight row, as packed 16-bit floats, in "fragment order":
+// run(words, h) fills h[0..15] with one lane's 32 codes of one weight row as
+// packed 16-bit floats in "fragment order", using nothing but shifts and one
+// LOP3 per pair: a code field sitting at bit 3f (or 4e) of a 16-bit half is
+// OR-ed into the mantissa of MAGIC = 1024 (fp16) or 128 (bf16), which yields
+//        MAGIC + c*q      with c = 2^(field offset)  (kDiv below).
 //   INT4: h[4i+e]  = codes (8i+e , 8i+e+4)  of word i          (i = 0..3, e = 0..3)
 //   INT3: h[5i+f]  = codes (10i+f, 10i+5+f) of word i          (i = 0..2, f = 0..4)
 //         h[15]    = codes (30, 31)
-// z is the integer zero point of the group.  All arithmetic is exact.
+// No arithmetic is spent on removing MAGIC, c or the zero point per element:
+// x is stored in shared memory already divided by c (a power of two), so the
+// MMA yields  sum_k x_k*q_k + sum_k (MAGIC/c_k)*x_k ; the second sum and
+// sum_k x_k depend on the token and group only and are tabulated once per CTA
+// (P and X0), and the group's value is  s*(mma - P) - (s*z)*X0.
 template <int BITS, typename T> struct Unpack;
 
 template <> struct Unpack<4, __half> {
     static constexpr int kWords = 4;
-    static __device__ __forceinline__ void run(const uint32_t *w, float z, uint32_t *h)
+    static constexpr float kMagic = 1024.f;
+    static __device__ __forceinline__ int div_log2(int c) { return ((c & 7) & 1) ? 4 : 0; }   // odd nibbles sit 4 bits up
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
     {
-        const uint32_t c0 = Pk<__half>::splat(1024.f + z), c1 = Pk<__half>::splat(64.f + z);
-        const uint32_t sixteenth = 0x2C002C00u;                      // 1/16
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t a = w[i], b = w[i] >> 8;
-            h[4 * i + 0] = Pk<__half>::sub(lop3_and_or(a, 0x000F000Fu, 0x64006400u), c0);
-            h[4 * i + 1] = Pk<__half>::fma(lop3_and_or(a, 0x00F000F0u, 0x64006400u), sixteenth, c1 ^ 0x80008000u);
-            h[4 * i + 2] = Pk<__half>::sub(lop3_and_or(b, 0x000F000Fu, 0x64006400u), c0);
-            h[4 * i + 3] = Pk<__half>::fma(lop3_and_or(b, 0x00F000F0u, 0x64006400u), sixteenth, c1 ^ 0x80008000u);
+            h[4 * i + 0] = lop3_and_or(a, 0x000F000Fu, 0x64006400u);
+            h[4 * i + 1] = lop3_and_or(a, 0x00F000F0u, 0x64006400u);
+            h[4 * i + 2] = lop3_and_or(b, 0x000F000Fu, 0x64006400u);
+            h[4 * i + 3] = lop3_and_or(b, 0x00F000F0u, 0x64006400u);
         }
     }
 };
 template <> struct Unpack<4, __nv_bfloat16> {
     static constexpr int kWords = 4;
-    static __device__ __forceinline__ void run(const uint32_t *w, float z, uint32_t *h)
+    static constexpr float kMagic = 128.f;                     // 0x4300 | q  is 128 + q in bf16 (7 mantissa bits)
+    static __device__ __forceinline__ int div_log2(int) { return 0; }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
     {
-        const uint32_t c0 = Pk<__nv_bfloat16>::splat(128.f + z);     // 0x4300 | q  is 128 + q in bf16
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                h[4 * i + e] = Pk<__nv_bfloat16>::sub(lop3_and_or(w[i] >> (4 * e), 0x000F000Fu, 0x43004300u), c0);
+            for (int e = 0; e < 4; ++e) h[4 * i + e] = lop3_and_or(w[i] >> (4 * e), 0x000F000Fu, 0x43004300u);
     }
 };
 template <> struct Unpack<3, __half> {
     static constexpr int kWords = 3;
-    static __device__ __forceinline__ void run(const uint32_t *w, float z, uint32_t *h)
+    static constexpr float kMagic = 1024.f;
+    static __device__ __forceinline__ int div_log2(int c)
     {
-        const uint32_t c0 = Pk<__half>::splat(1024.f + z);
-        const uint32_t n1 = Pk<__half>::splat(-(128.f + z)), n2 = Pk<__half>::splat(-(16.f + z));
-        const uint32_t eighth = 0x30003000u, sixtyfourth = 0x24002400u;   // 1/8, 1/64
+        if (c >= 30) return 0;
+        const int f = (c % 10) % 5;                             // fields 0,3: bit 0; 1,4: bit 3; 2: bit 6 (3,4 after >> 9)
+        return (f == 2) ? 6 : ((f == 1 || f == 4) ? 3 : 0);
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
             const uint32_t a = w[i], b = w[i] >> 9;
-            h[5 * i + 0] = Pk<__half>::sub(lop3_and_or(a, 0x00070007u, 0x64006400u), c0);
-            h[5 * i + 1] = Pk<__half>::fma(lop3_and_or(a, 0x00380038u, 0x64006400u), eighth, n1);
-            h[5 * i + 2] = Pk<__half>::fma(lop3_and_or(a, 0x01C001C0u, 0x64006400u), sixtyfourth, n2);
-            h[5 * i + 3] = Pk<__half>::sub(lop3_and_or(b, 0x00070007u, 0x64006400u), c0);
-            h[5 * i + 4] = Pk<__half>::fma(lop3_and_or(b, 0x00380038u, 0x64006400u), eighth, n1);
+            h[5 * i + 0] = lop3_and_or(a, 0x00070007u, 0x64006400u);
+            h[5 * i + 1] = lop3_and_or(a, 0x00380038u, 0x64006400u);
+            h[5 * i + 2] = lop3_and_or(a, 0x01C001C0u, 0x64006400u);
+            h[5 * i + 3] = lop3_and_or(b, 0x00070007u, 0x64006400u);
+            h[5 * i + 4] = lop3_and_or(b, 0x00380038u, 0x64006400u);
         }
         uint32_t l = lop3_and_or(w[0] >> 15, 0x00010001u, 0x64006400u);
         l = lop3_and_or(w[1] >> 14, 0x00020002u, l);
-        l = lop3_and_or(w[2] >> 13, 0x00040004u, l);
-        h[15] = Pk<__half>::sub(l, c0);
+        h[15] = lop3_and_or(w[2] >> 13, 0x00040004u, l);
     }
 };
 template <> struct Unpack<3, __nv_bfloat16> {
     static constexpr int kWords = 3;
-    static __device__ __forceinline__ void run(const uint32_t *w, float z, uint32_t *h)
+    static constexpr float kMagic = 128.f;
+    static __device__ __forceinline__ int div_log2(int c)
     {
-        const uint32_t c0 = Pk<__nv_bfloat16>::splat(128.f + z);
-        const uint32_t n1 = Pk<__nv_bfloat16>::splat(-(16.f + z));
-        const uint32_t eighth = 0x3E003E00u;                          // 1/8 in bf16
+        if (c >= 30) return 0;
+        const int f = (c % 10) % 5;                             // shifts 0, 6, 12: fields 0,2,4 at bit 0; 1,3 at bit 3
+        return (f == 1 || f == 3) ? 3 : 0;
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
             const uint32_t a = w[i], b = w[i] >> 6, c = w[i] >> 12;
-            h[5 * i + 0] = Pk<__nv_bfloat16>::sub(lop3_and_or(a, 0x00070007u, 0x43004300u), c0);
-            h[5 * i + 1] = Pk<__nv_bfloat16>::fma(lop3_and_or(a, 0x00380038u, 0x43004300u), eighth, n1);
-            h[5 * i + 2] = Pk<__nv_bfloat16>::sub(lop3_and_or(b, 0x00070007u, 0x43004300u), c0);
-            h[5 * i + 3] = Pk<__nv_bfloat16>::fma(lop3_and_or(b, 0x00380038u, 0x43004300u), eighth, n1);
-            h[5 * i + 4] = Pk<__nv_bfloat16>::sub(lop3_and_or(c, 0x00070007u, 0x43004300u), c0);
+            h[5 * i + 0] = lop3_and_or(a, 0x00070007u, 0x43004300u);
+            h[5 * i + 1] = lop3_and_or(a, 0x00380038u, 0x43004300u);
+            h[5 * i + 2] = lop3_and_or(b, 0x00070007u, 0x43004300u);
+            h[5 * i + 3] = lop3_and_or(b, 0x00380038u, 0x43004300u);
+            h[5 * i + 4] = lop3_and_or(c, 0x00070007u, 0x43004300u);
         }
         uint32_t l = lop3_and_or(w[0] >> 15, 0x00010001u, 0x43004300u);
         l = lop3_and_or(w[1] >> 14, 0x00020002u, l);
-        l = lop3_and_or(w[2] >> 13, 0x00040004u, l);
-        h[15] = Pk<__nv_bfloat16>::sub(l, c0);
+        h[15] = lop3_and_or(w[2] >> 13, 0x00040004u, l);
     }
 };
 
@@ -283,82 +316,102 @@ __device__ __forceinline__ int ld_acquire(const int *p)
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void named_barrier_arrive(int id, int nthreads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ void trace_mark(const DecodeParams &p, int slot)
+{
+    if (p.trace && (threadIdx.x & 31) == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = t;
+    }
+}
 
 // --------------------------------------------------------------- tile epilogue
-// Sums the SK partial tiles in slice order (or takes `own` when the task was
-// not split), adds the up-projection t.B^T and stores y.  Lane (g,t) owns rows
-// g and g+8 of the tile and tokens 8b+2t, 8b+2t+1.
+// Main-path sums of the tile: slot i of scratch for i != myslot, `own` (this
+// warp's registers) for i == myslot (own == nullptr: every slot from scratch),
+// always added in slot order.  Then the up-projection t.B^T is added and y is
+// stored.  Lane (g,tq) owns rows g and g+8 and tokens 8b+2tq, 8b+2tq+1.
+// t is read from shared memory (s_t); B from shared memory when b_smem != 0
+// (rows of this CTA's own tiles), else from global memory.
 template <typename T, int MT>
-__device__ __forceinline__ void tile_epilogue(const DecodeParams &p, int tile, int lane, const float (*own)[4])
+__device__ __forceinline__ void tile_epilogue(const DecodeParams &p, int tile, int lane, const float (*own)[4], int myslot,
+                                              int cnt, const float *s_t, const T *b_smem)
 {
     const int g = lane >> 2, tq = lane & 3;
-    const T *B = static_cast<const T *>(p.B);
     T *y = static_cast<T *>(p.y);
+    const float *slots = p.partial + (size_t)tile * p.maxslots * p.M * kTileRows;
+    const size_t stride = (size_t)p.M * kTileRows;
 #pragma unroll
     for (int b = 0; b < MT; ++b) {
 #pragma unroll
-        for (int half_row = 0; half_row < 2; ++half_row) {
-            const int n = tile * kTileRows + g + 8 * half_row;
+        for (int hr = 0; hr < 2; ++hr) {
+            const int row = g + 8 * hr, n = tile * kTileRows + row;
 #pragma unroll
             for (int tk = 0; tk < 2; ++tk) {
                 const int m = 8 * b + 2 * tq + tk;
                 if (m >= p.M || n >= p.N) continue;
-                float v;
-                if (own) {
-                    v = own[b][2 * half_row + tk];
+                const float mine = own ? own[b][2 * hr + tk] : 0.f;
+                float v = 0.f;
+                const float *sp = slots + (size_t)m * kTileRows + row;
+                if (cnt == 1 && own) {
+                    v = mine;
                 } else {
-                    v = 0.f;
-                    for (int s = 0; s < p.SK; ++s) v += ld_cg_f32(p.partial + ((size_t)s * p.M + m) * p.N + n);
+                    for (int i0 = 0; i0 < cnt; i0 += 4) {
+                        float a[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int i = i0 + u;
+                            a[u] = (i < cnt && !(own && i == myslot)) ? ld_cg_f32(sp + i * stride) : 0.f;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int i = i0 + u;
+                            if (i < cnt) v += (own && i == myslot) ? mine : a[u];
+                        }
+                    }
                 }
                 if (p.rank > 0) {
-                    const uint4 *brow = reinterpret_cast<const uint4 *>(B + (size_t)n * p.rank);
-                    const float4 *trow = reinterpret_cast<const float4 *>(p.t + (size_t)m * p.rank);
+                    const float4 *trow = reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank);
                     float sub = 0.f;
-                    for (int c = 0; c < p.rank / 8; ++c) {
-                        const uint4 bv = __ldg(brow + c);
-                        const float4 t0 = __ldcg(trow + 2 * c), t1 = __ldcg(trow + 2 * c + 1);
-                        const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
-                        const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
-                        sub = fmaf(t0.x, b0.x, sub);
-                        sub = fmaf(t0.y, b0.y, sub);
-                        sub = fmaf(t0.z, b1.x, sub);
-                        sub = fmaf(t0.w, b1.y, sub);
-                        sub = fmaf(t1.x, b2.x, sub);
-                        sub = fmaf(t1.y, b2.y, sub);
-                        sub = fmaf(t1.z, b3.x, sub);
-                        sub = fmaf(t1.w, b3.y, sub);
+                    if (b_smem) {
+                        const uint4 *brow = reinterpret_cast<const uint4 *>(b_smem + (size_t)row * p.rank);
+#pragma unroll 2
+                        for (int c = 0; c < p.rank / 8; ++c) {
+                            const uint4 bv = brow[c];
+                            const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
+                            const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
+                            const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
+                            sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
+                            sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
+                            sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
+                            sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
+                        }
+                    } else {
+                        const uint4 *brow = reinterpret_cast<const uint4 *>(static_cast<const T *>(p.B) + (size_t)n * p.rank);
+#pragma unroll 4
+                        for (int c = 0; c < p.rank / 8; ++c) {
+                            const uint4 bv = __ldg(brow + c);
+                            const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
+                            const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
+                            const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
+                            sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
+                            sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
+                            sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
+                            sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
+                        }
                     }
                     v += sub;
                 }
                 y[(size_t)m * p.N + n] = ActTraits<T>::from_float(v);
             }
-        }
-    }
-}
-
-// Bookkeeping after a tile's y has been stored (and, once per call when there is
-// a sub-branch, after the t-completing warp has left its parked-tile loop).
-// Whoever retires last restores the scratch invariants (all counters, flags and
-// t equal to zero) for the next call on this stream; nobody else is touching the
-// scratch space any more at that point.
-__device__ __forceinline__ void retire_one(const DecodeParams &p, int lane)
-{
-    __syncwarp();
-    const int target = p.NT + (p.rank > 0 ? 1 : 0);
-    int last = 0;
-    if (lane == 0) {
-        __threadfence();
-        last = (atomicAdd(p.ctr + kCtrDone, 1) == target - 1);
-    }
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (last) {
-        __threadfence();
-        for (int i = lane; i < 2 * p.NT; i += 32) p.ctr[kCtrFirstTile + i] = 0;   // arrivals + parked list
-        for (int i = lane; i < p.M * p.rank; i += 32) p.t[i] = 0.f;
-        if (lane == 0) {
-            p.ctr[kCtrDone] = 0;
-            p.ctr[kCtrReady] = 0;
-            p.ctr[kCtrPendingN] = 0;
         }
     }
 }
@@ -378,90 +431,439 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int GB = (BITS == 4) ? 64 : 48;          // packed bytes of one group of one row
     constexpr int NWORDS = Unpack<BITS, T>::kWords;    // words per lane per group
+    // Row pitch of a stage in shared memory: the packed bytes of the row, padded so that the
+    // eight rows a warp reads at once start in different banks (64-byte offset per row pair
+    // for the 128-bit loads of INT4, 48-byte for the three 32-bit loads of INT3).
+    constexpr int RP = (BITS == 4) ? 64 : 48;
+    auto row_pitch = [](int ng) { const int b = ng * GB; return (b % 128 == 0) ? b + RP : b; };
+    constexpr int NACC = 2;                            // independent MMA accumulator chains
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, tq = lane & 3;
-    const int s = blockIdx.x % p.SK, rr = blockIdx.x / p.SK;
+    const int s = blockIdx.x % p.SK, r = blockIdx.x / p.SK;
     const int g0 = (int)((long long)s * p.G / p.SK), g1 = (int)((long long)(s + 1) * p.G / p.SK);
     const int ngs = g1 - g0;
-    const int tile0 = (int)((long long)rr * p.NT / p.R), tile1 = (int)((long long)(rr + 1) * p.NT / p.R);
-    const int ntiles = tile1 - tile0;
-    const int nchunks = (ngs + p.CH - 1) / p.CH;
-    const int my_tiles = (ntiles > warp) ? (ntiles - warp + kNW - 1) / kNW : 0;
-    const int n_items = my_tiles * nchunks;
+    // whole 16-row tiles, dealt out in contiguous ranges; a "segment" is one tile of the range
+    const int tile_first = (int)((long long)r * p.NT / p.R);
+    const int nseg = (int)((long long)(r + 1) * p.NT / p.R) - tile_first;
     const size_t row_bytes = (size_t)p.G * GB;
 
+    // units of the down-projection owned by this CTA: (row j of A, 1024-wide k chunk of the slice)
+    const int kslice = ngs * kGroupFast;
+    const int nkc = (kslice + kTUnitK - 1) / kTUnitK;
+    const long long TU = (long long)p.rank * nkc;
+    const int tu0 = (int)((long long)r * TU / p.R), tu1 = (int)((long long)(r + 1) * TU / p.R);
+    const bool has_t = (p.rank > 0) && (tu1 > tu0);
+    // few tokens: the down-projection reads x straight from global memory and need not wait
+    // for the compute warps' permuted copy
+    const bool t_from_global = (p.M <= 2);
+
+    // shared memory: barriers | table | deferred list | meta | x | segbuf | A | B | t | ring
+    trace_mark(p, 0);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
-    uint2 *s_meta = reinterpret_cast<uint2 *>(smem + p.off_meta);
+    const uint32_t st_full = smem_u32(bars), st_empty = st_full + 8u * p.NS;
+    const uint32_t seg_full = st_empty + 8u * p.NS, seg_free = seg_full + 8u * kNBuf;
+    const uint32_t a_full = seg_free + 8u * kNBuf, b_full = a_full + 8u, x_req = b_full + 8u;
+    int *s_def = reinterpret_cast<int *>(smem + p.off_def);
+    float2 *s_mf = reinterpret_cast<float2 *>(smem + p.off_meta);         // (s, s*z) [segment row][slice group]
+    float2 *s_px = reinterpret_cast<float2 *>(smem + p.off_px);           // (P, X0)  [slice group][token]
     T *s_x = reinterpret_cast<T *>(smem + p.off_x);
-    const uint32_t ring_base = smem_u32(smem + p.off_ring) + (uint32_t)(warp * p.D) * p.slot_bytes;
-    const uint8_t *ring_ptr = smem + p.off_ring + (size_t)(warp * p.D) * p.slot_bytes;
-    const uint32_t bar_base = smem_u32(bars + warp * p.D);
+    float *s_seg = reinterpret_cast<float *>(smem + p.off_segbuf);
+    T *s_A = reinterpret_cast<T *>(smem + p.off_A);
+    T *s_B = reinterpret_cast<T *>(smem + p.off_B);
+    float *s_t = reinterpret_cast<float *>(smem + p.off_t);
+    const int segbuf_floats = kCW * 8 * p.vt * 4 * MT;
 
     if (tid == 0) {
-        for (int i = 0; i < kNW * p.D; ++i) mbar_init(smem_u32(bars + i), 1);
+        for (int i = 0; i < p.NS; ++i) {
+            mbar_init(st_full + 8u * i, 1);
+            mbar_init(st_empty + 8u * i, kCW);
+        }
+        for (int i = 0; i < kNBuf; ++i) {
+            mbar_init(seg_full + 8u * i, kCW);
+            mbar_init(seg_free + 8u * i, 1);
+        }
+        mbar_init(a_full, 1);
+        mbar_init(b_full, 1);
+        mbar_init(x_req, kCW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    trace_mark(p, 1);
 
-    // ---- producer side of this warp's ring ---------------------------------
-    auto issue = [&](int it) {
-        const int tile = tile0 + warp + (it / nchunks) * kNW;
-        const int cg0 = g0 + (it % nchunks) * p.CH;
-        const int ng = min(p.CH, g1 - cg0);
-        const int slot = it % p.D;
-        const uint32_t bar = bar_base + 8u * slot;
-        const uint32_t bytes_row = (uint32_t)ng * GB;
-        if (lane == 0) mbar_expect_tx(bar, bytes_row * kTileRows);
-        __syncwarp();
-        if (lane < kTileRows) {
-            const int n = min(tile * kTileRows + lane, p.N - 1);
-            bulk_g2s(ring_base + slot * p.slot_bytes + lane * bytes_row, p.qw + (size_t)n * row_bytes + (size_t)cg0 * GB,
-                     bytes_row, bar);
+    const int b_rows = min(p.N, (tile_first + nseg) * kTileRows) - tile_first * kTileRows;   // weight rows of our tiles
+    const bool b_in_smem = (p.rank > 0) && nseg > 0 && b_rows <= p.b_cap_rows;
+
+    if (warp == kProdWarp) {
+        // =================================================== producer warp
+        // A and B of this CTA (weights: independent of earlier kernels of the stream)
+        if (has_t) {
+            const T *A = static_cast<const T *>(p.A);
+            const int na = min(tu1 - tu0, p.a_cap);
+            uint32_t total = 0;
+            for (int i = 0; i < na; ++i) {
+                const int kc = (tu0 + i) % nkc;
+                total += (uint32_t)min(kTUnitK, kslice - kc * kTUnitK) * 2u;
+            }
+            if (lane == 0) mbar_expect_tx(a_full, total);
+            __syncwarp();
+            for (int i = lane; i < na; i += 32) {
+                const int u = tu0 + i, j = u / nkc, kc = u - j * nkc;
+                const int nk = min(kTUnitK, kslice - kc * kTUnitK);
+                bulk_g2s(smem_u32(s_A + (size_t)i * kTUnitK), A + (size_t)j * p.K + g0 * kGroupFast + kc * kTUnitK,
+                         (uint32_t)nk * 2u, a_full);
+            }
         }
-    };
-    for (int it = 0; it < min(p.D, n_items); ++it) issue(it);
+        if (b_in_smem && lane == 0) {
+            const uint32_t bytes = (uint32_t)b_rows * p.rank * 2u;
+            mbar_expect_tx(b_full, bytes);
+            bulk_g2s(smem_u32(s_B), static_cast<const T *>(p.B) + (size_t)tile_first * kTileRows * p.rank, bytes, b_full);
+        }
+        // the weight stream
+        const uint32_t ring = smem_u32(smem + p.off_ring);
+        int it = 0;
+        bool dead = false;
+        for (int seg = 0; seg < nseg && !dead; ++seg) {
+            const int tile = tile_first + seg;
+            for (int pos = 0; pos < ngs; pos += p.CHG, ++it) {
+                const int ng = min(p.CHG, ngs - pos);
+                const int slot = it % p.NS;
+                // Until the compute warps have put their loads of x (which everything waits for)
+                // into the memory system, keep the prefetch shallow: x must not queue behind
+                // megabytes of weights that cannot be used before it arrives.
+                if (it == kEarlyStages && !mbar_wait(x_req, 0)) {
+                    dead = true;
+                    break;
+                }
+                if (it >= p.NS && !mbar_wait(st_empty + 8u * slot, (uint32_t)(it / p.NS - 1) & 1u)) {
+                    dead = true;
+                    break;
+                }
+                const uint32_t bytes_row = (uint32_t)ng * GB;
+                if (lane == 0) mbar_expect_tx(st_full + 8u * slot, bytes_row * kTileRows);
+                __syncwarp();
+                if (lane < kTileRows) {
+                    const int n = min(tile * kTileRows + lane, p.N - 1);
+                    bulk_g2s(ring + slot * p.stage_bytes + lane * row_pitch(ng),
+                             p.qw + (size_t)n * row_bytes + (size_t)(g0 + pos) * GB, bytes_row, st_full + 8u * slot);
+                }
+            }
+        }
+        if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+        trace_mark(p, 9);
+        return;
+    }
 
-    // Everything above touches only the weights, which no earlier kernel of the
-    // stream writes; from here on x may come from the previous kernel.
+    if (warp < kCW) {
+        // =================================================== compute warps
+        // ---- fill shared memory.  The (s, s*z) table comes from weights, so its loads go out
+        // before the wait on the previous kernel; x (divided by the field weights, permuted
+        // into fragment order) and the per-group sums P, X0 after it.  All global loads of a
+        // batch are issued before the first dependent instruction. ----
+        constexpr int MB = 8;
+        const int nthr = kCW * 32;
+        const int mpitch = ngs | 1;                  // odd pitch: the eight rows of a warp hit different banks
+        const int nmeta = nseg * kTileRows * ngs;
+        const uint16_t *sc = reinterpret_cast<const uint16_t *>(p.scales);
+        const uint16_t *ze = reinterpret_cast<const uint16_t *>(p.zeros);
+        auto meta_batch = [&](int mbase, bool load, uint16_t (&msc)[MB], uint16_t (&mze)[MB]) {
+#pragma unroll
+            for (int i = 0; i < MB; ++i) {
+                const int idx = mbase + i * nthr + tid;
+                if (idx < nmeta) {
+                    if (load) {
+                        const int row = idx / ngs, gl = idx - row * ngs;
+                        const int n = min(tile_first * kTileRows + row, p.N - 1);
+                        const size_t mi = (size_t)n * p.G + g0 + gl;
+                        msc[i] = sc[mi];
+                        mze[i] = ze[mi];
+                    } else {
+                        const float sf = __half2float(__ushort_as_half(msc[i]));
+                        const float zf = __half2float(__ushort_as_half(mze[i]));
+                        const int row = idx / ngs, gl = idx - row * ngs;
+                        s_mf[row * mpitch + gl] = make_float2(sf, sf * zf);
+                    }
+                }
+            }
+        };
+        uint16_t msc0[MB], mze0[MB];
+        meta_batch(0, true, msc0, mze0);
+
+        // From here on x may come from the previous kernel of the stream.
+        pdl_wait();
+        pdl_launch_dependents();
+        trace_mark(p, 3);
+        {
+            // One thread prepares one 32-element run of x: 64 contiguous bytes in, the run's 16
+            // fragment-order pairs (four 16-byte units) out, with compile-time positions.
+            const T *x = static_cast<const T *>(p.x);
+            const int runs_per_tok = kslice / 32, nruns = p.M * runs_per_tok;     // multiples of 4
+            const int mp = 8 * MT;                                                // token slots of the (P, X0) table
+            for (int i = tid; i < ngs * mp; i += nthr)                            // tokens beyond M contribute nothing
+                if (i % mp >= p.M) s_px[i] = make_float2(0.f, 0.f);
+            for (int base = 0; base < nruns; base += nthr) {
+                const int idx = base + tid;                                       // whole quads are valid or not
+                const bool valid = idx < nruns;
+                const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+                uint4 xv[4];
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + g0 * kGroupFast + run * 32);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+                if (base == 0) {                                  // our loads of x are on their way
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(x_req);
+                }
+                const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
+                uint32_t h[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) h[i] = 0u;
+                float psum = 0.f, xsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const int pos = frag_pos<BITS>(c);                            // folds to a constant
+                    T xe;
+                    *reinterpret_cast<uint16_t *>(&xe) = e[c];
+                    const float xf = ActTraits<T>::to_float(xe);
+                    // exact division by the field weight (a power of two; up to fp16 underflow).
+                    // P is summed from the stored value, so the MMA's bias term cancels exactly.
+                    const T xs = ActTraits<T>::from_float(ldexpf(xf, -Unpack<BITS, T>::div_log2(c)));
+                    h[pos >> 1] |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&xs)) << (16 * (pos & 1));
+                    psum = fmaf(Unpack<BITS, T>::kMagic, ActTraits<T>::to_float(xs), psum);
+                    xsum += xf;
+                }
+                if (valid) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(s_x + (size_t)m * p.x_pitch + (run >> 2) * kGroupFast);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        dst[q4 * 4 + (run & 3)] = make_uint4(h[4 * q4], h[4 * q4 + 1], h[4 * q4 + 2], h[4 * q4 + 3]);
+                }
+                // the four runs of one (token, group) sit in four consecutive lanes
+                psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+                psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+                if (valid && (run & 3) == 0) s_px[(run >> 2) * mp + m] = make_float2(psum, xsum);
+            }
+        }
+        meta_batch(0, false, msc0, mze0);
+        for (int mbase = MB * nthr; mbase < nmeta; mbase += MB * nthr) {
+            uint16_t msc[MB], mze[MB];
+            meta_batch(mbase, true, msc, mze);
+            meta_batch(mbase, false, msc, mze);
+        }
+        trace_mark(p, 4);
+        bool dead = false;
+        named_barrier_sync(1, kCW * 32);
+        if (p.rank > 0 && !(p.M <= 2 && !p.t_late))
+            named_barrier_arrive(2, (kCW + 1) * 32);                   // x is in place for the epilogue warp
+        trace_mark(p, 5);
+
+        // ---- consumer: every stage is shared; this warp takes an eighth of its groups ----
+        const uint8_t *ring_ptr = smem + p.off_ring;
+        int it = 0;
+        for (int seg = 0; seg < nseg && !dead; ++seg) {
+            float acc[MT][4];
+#pragma unroll
+            for (int b = 0; b < MT; ++b)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[b][i] = 0.f;
+            for (int pos = 0; pos < ngs; pos += p.CHG, ++it) {
+                const int ng = min(p.CHG, ngs - pos);
+                const int slot = it % p.NS;
+                if (!mbar_wait(st_full + 8u * slot, (uint32_t)(it / p.NS) & 1u)) {
+                    dead = true;
+                    break;
+                }
+                if (it == 0) trace_mark(p, 6);
+                const uint8_t *slot_ptr = ring_ptr + (size_t)slot * p.stage_bytes;
+                const uint32_t bytes_row = (uint32_t)row_pitch(ng);
+                const int gbeg = warp * ng / kCW, gend = (warp + 1) * ng / kCW;     // this warp's groups of the stage
+                const float2 *meta_a = s_mf + (size_t)(seg * kTileRows + g) * mpitch + pos;   // row g; row g+8 is 8 rows on
+                const float2 *meta_b = meta_a + 8 * mpitch;
+
+                for (int gi = gbeg; gi < gend; ++gi) {
+                    const float2 fa = meta_a[gi], fb = meta_b[gi];          // (s, s*z) of rows g and g+8
+                    uint32_t wa[NWORDS], wb[NWORDS];
+                    const uint8_t *pa = slot_ptr + (size_t)g * bytes_row + gi * GB + tq * (GB / 4);
+                    const uint8_t *pb = pa + (size_t)8 * bytes_row;
+                    if constexpr (BITS == 4) {
+                        const uint4 va = *reinterpret_cast<const uint4 *>(pa), vb = *reinterpret_cast<const uint4 *>(pb);
+                        wa[0] = va.x; wa[1] = va.y; wa[2] = va.z; wa[3] = va.w;
+                        wb[0] = vb.x; wb[1] = vb.y; wb[2] = vb.z; wb[3] = vb.w;
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < NWORDS; ++i) {
+                            wa[i] = reinterpret_cast<const uint32_t *>(pa)[i];
+                            wb[i] = reinterpret_cast<const uint32_t *>(pb)[i];
+                        }
+                    }
+                    uint32_t ha[16], hb[16];
+                    Unpack<BITS, T>::run(wa, ha);
+                    Unpack<BITS, T>::run(wb, hb);
+
+#pragma unroll
+                    for (int b = 0; b < MT; ++b) {
+                        float tmp[NACC][4];
+#pragma unroll
+                        for (int c = 0; c < NACC; ++c) tmp[c][0] = tmp[c][1] = tmp[c][2] = tmp[c][3] = 0.f;
+                        const int token = 8 * b + g;
+                        const uint4 *xg = reinterpret_cast<const uint4 *>(s_x + (size_t)token * p.x_pitch +
+                                                                          (size_t)(pos + gi) * kGroupFast);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                            if (token < p.M) xv = xg[q4 * 4 + tq];
+                            const uint32_t a0[4] = {ha[4 * q4 + 0], hb[4 * q4 + 0], ha[4 * q4 + 1], hb[4 * q4 + 1]};
+                            const uint32_t a1[4] = {ha[4 * q4 + 2], hb[4 * q4 + 2], ha[4 * q4 + 3], hb[4 * q4 + 3]};
+                            Pk<T>::mma(tmp[q4 % NACC], a0, xv.x, xv.y);
+                            Pk<T>::mma(tmp[q4 % NACC], a1, xv.z, xv.w);
+                        }
+                        // (P, X0) of tokens 8b+2tq and 8b+2tq+1 for this group
+                        const float4 px = *reinterpret_cast<const float4 *>(s_px + (size_t)(pos + gi) * (8 * MT) + 8 * b + 2 * tq);
+                        float d[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            d[i] = tmp[0][i];
+#pragma unroll
+                            for (int c = 1; c < NACC; ++c) d[i] += tmp[c][i];
+                        }
+                        // s*(mma - P) - (s*z)*X0
+                        acc[b][0] = fmaf(-fa.y, px.y, fmaf(fa.x, d[0] - px.x, acc[b][0]));
+                        acc[b][1] = fmaf(-fa.y, px.w, fmaf(fa.x, d[1] - px.z, acc[b][1]));
+                        acc[b][2] = fmaf(-fb.y, px.y, fmaf(fb.x, d[2] - px.x, acc[b][2]));
+                        acc[b][3] = fmaf(-fb.y, px.w, fmaf(fb.x, d[3] - px.z, acc[b][3]));
+                    }
+                }
+                // stage consumed by this warp
+                __syncwarp();
+                if (lane == 0) mbar_arrive(st_empty + 8u * slot);
+            }
+            if (dead) break;
+
+            // ---- deposit this warp's partial tile for the epilogue warp ---------------
+            const int buf = seg % kNBuf;
+            if (seg >= kNBuf && !mbar_wait(seg_free + 8u * buf, (uint32_t)(seg / kNBuf - 1) & 1u)) {
+                dead = true;
+                break;
+            }
+            if (tq < p.vt) {
+                float4 *dst = reinterpret_cast<float4 *>(s_seg + (size_t)buf * segbuf_floats +
+                                                         (size_t)((warp * 8 + g) * p.vt + tq) * 4 * MT);
+#pragma unroll
+                for (int b = 0; b < MT; ++b) dst[b] = make_float4(acc[b][0], acc[b][1], acc[b][2], acc[b][3]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(seg_full + 8u * buf);
+            trace_mark(p, seg == 0 ? 7 : 8);
+        }
+        trace_mark(p, 9);
+        if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+        return;
+    }
+
+    // ======================================================= epilogue warp
     pdl_wait();
     pdl_launch_dependents();
+    trace_mark(p, 2);
+    int n_retired = 0;          // tiles finished by this warp (+1 token if it completed t)
+    int n_def = 0;              // tiles this warp must finish once t is complete (s_def[])
+    bool t_local = (p.rank == 0);   // t is complete and copied to shared memory
+    bool dead = false;
 
-    // ---- which warps own rows of A (down-projection share) ------------------
-    const int j0 = (int)((long long)rr * p.rank / p.R), j1 = (int)((long long)(rr + 1) * p.rank / p.R);
-    const int nj = j1 - j0;
-    const int ntw = min(nj, kNW);                      // t-warps are the LAST ntw warps
-    const bool is_tw = warp >= kNW - ntw;
-    const int nfill_warps = (ntw < kNW && !p.t_late) ? kNW - ntw : kNW;   // warps that fill shared memory
+    // Looks at the "t complete" flag; on the first sighting copies t to shared memory.
+    auto t_poll = [&]() -> bool {
+        if (t_local) return true;
+        int ready = 0;
+        if (lane == 0) ready = ld_acquire(p.ctr + kCtrReady);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (!ready) return false;
+        for (int i = lane; i < p.M * p.rank; i += 32) s_t[i] = ld_cg_f32(p.t + i);
+        __syncwarp();
+        t_local = true;
+        return true;
+    };
+    auto own_b = [&](int tile) -> const T * {
+        return (b_in_smem && tile >= tile_first && tile < tile_first + nseg)
+                   ? s_B + (size_t)(tile - tile_first) * kTileRows * p.rank
+                   : nullptr;
+    };
+    // Finish `tile` from scratch slots (all contributions are there and visible).
+    auto finish_from_slots = [&](int tile) {
+        tile_epilogue<T, MT>(p, tile, lane, nullptr, 0, p.SK, s_t, own_b(tile));
+        ++n_retired;
+        if (p.rank == 0 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;   // nobody else will touch it again
+    };
 
     auto t_share = [&]() {
-        // t[m][j] += sum_{k in slice} x[m][k] * A[j][k] for this warp's rows j
+        // t[m][j] += sum over this CTA's units (j, k chunk) of x[m][k] * A[j][k]
+        if (!mbar_wait(a_full, 0)) {
+            dead = true;
+            return;
+        }
         const T *A = static_cast<const T *>(p.A);
-        const T *x = static_cast<const T *>(p.x);
-        const int k0 = g0 * kGroupFast, k1 = g1 * kGroupFast;
-        for (int j = j0 + (kNW - 1 - warp); j < j1; j += ntw) {
+        for (int u = tu0; u < tu1; ++u) {
+            const int j = u / nkc, kc = u - j * nkc;
+            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
+            const bool in_smem = (u - tu0) < p.a_cap;
+            const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
             float acc[MT * 8];
 #pragma unroll
             for (int m = 0; m < MT * 8; ++m) acc[m] = 0.f;
-            for (int k = k0 + lane * 8; k < k1; k += 256) {
-                const uint4 av = __ldg(reinterpret_cast<const uint4 *>(A + (size_t)j * p.K + k));
-                const float2 a0 = Pk<T>::to_float2(av.x), a1 = Pk<T>::to_float2(av.y);
-                const float2 a2 = Pk<T>::to_float2(av.z), a3 = Pk<T>::to_float2(av.w);
+            if (t_from_global && !p.t_late) {
+                const T *xg = static_cast<const T *>(p.x) + g0 * kGroupFast + kbeg;
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {
+                    if (m < p.M) {
+                        uint4 xv[4], av[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int k = lane * 8 + 256 * i;
+                            xv[i] = make_uint4(0u, 0u, 0u, 0u);
+                            av[i] = xv[i];
+                            if (k < nk) {
+                                xv[i] = __ldcg(reinterpret_cast<const uint4 *>(xg + (size_t)m * p.K + k));
+                                av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
+                                                : __ldg(reinterpret_cast<const uint4 *>(arow + k));
+                            }
+                        }
+                        float v = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
+                            const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
+                                v = fmaf(xf.x, af.x, v);
+                                v = fmaf(xf.y, af.y, v);
+                            }
+                        }
+                        acc[m] = v;
+                    }
+                }
+            } else
+            for (int k = lane * 8; k < nk; k += 256) {
+                const uint4 av = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
+                                         : __ldg(reinterpret_cast<const uint4 *>(arow + k));
+                const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+                const int kl = kbeg + k;                              // slice-local k of the first element
+                const int xoff = (kl >> 7) * kGroupFast;
+                int slot8[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) slot8[q] = xoff + x_slot<BITS>((kl & 127) + q);
 #pragma unroll
                 for (int m = 0; m < MT * 8; ++m) {
                     if (m < p.M) {
-                        const uint4 xv = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + k));
-                        const float2 x0 = Pk<T>::to_float2(xv.x), x1 = Pk<T>::to_float2(xv.y);
-                        const float2 x2 = Pk<T>::to_float2(xv.z), x3 = Pk<T>::to_float2(xv.w);
+                        const T *xr = s_x + (size_t)m * p.x_pitch;
                         float v = acc[m];
-                        v = fmaf(x0.x, a0.x, v);
-                        v = fmaf(x0.y, a0.y, v);
-                        v = fmaf(x1.x, a1.x, v);
-                        v = fmaf(x1.y, a1.y, v);
-                        v = fmaf(x2.x, a2.x, v);
-                        v = fmaf(x2.y, a2.y, v);
-                        v = fmaf(x3.x, a3.x, v);
-                        v = fmaf(x3.y, a3.y, v);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            // shared memory holds x divided by the field weight: undo it
+                            const float2 af = Pk<T>::to_float2(aw[q]);
+                            const int c0 = ((kl & 127) + 2 * q) & 31, c1 = c0 + 1;
+                            v = fmaf(ldexpf(ActTraits<T>::to_float(xr[slot8[2 * q]]), Unpack<BITS, T>::div_log2(c0)), af.x, v);
+                            v = fmaf(ldexpf(ActTraits<T>::to_float(xr[slot8[2 * q + 1]]), Unpack<BITS, T>::div_log2(c1)), af.y, v);
+                        }
                         acc[m] = v;
                     }
                 }
@@ -476,8 +878,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             }
         }
     };
-    // After this warp's share of t is in: count it; the warp that completes t
-    // publishes the flag and finishes every tile parked before the flag was up.
+    // After this CTA's share of t is in: count it; the warp that completes t publishes
+    // the flag and finishes every tile that was parked (by any CTA) before the flag was up.
     auto t_arrive = [&]() {
         __syncwarp();
         int done = 0;
@@ -496,6 +898,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             npend = ld_acquire(p.ctr + kCtrPendingN);
         }
         npend = __shfl_sync(0xffffffffu, npend, 0);
+        (void)t_poll();
         for (int i = 0; i < npend; ++i) {
             int tile = 0;
             if (lane == 0) tile = ld_acquire(p.ctr + kCtrFirstTile + p.NT + i) - 1;
@@ -503,181 +906,190 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             if (tile < 0) continue;                    // entry not visible yet: its owner will see the flag
             if (!tile_claim(p, tile, lane)) continue;
             __threadfence();
-            tile_epilogue<T, MT>(p, tile, lane, nullptr);
-            retire_one(p, lane);
+            finish_from_slots(tile);
         }
-        retire_one(p, lane);                           // the completer's own slot in the retire count
+        ++n_retired;                                   // the completer's own token in the retire count
     };
 
-    if (p.rank > 0 && is_tw && !p.t_late) t_share();
-
-    // ---- fill shared memory: permuted x slice and (scale, zero) table --------
-    if (warp < nfill_warps) {
-        const int nthr = nfill_warps * 32;
-        const T *x = static_cast<const T *>(p.x);
-        const int kslice = ngs * kGroupFast;
-        for (int idx = tid; idx < p.M * (kslice / 8); idx += nthr) {
-            const int m = idx / (kslice / 8), kk = (idx - m * (kslice / 8)) * 8;
-            const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + g0 * kGroupFast + kk));
-            const uint16_t *e = reinterpret_cast<const uint16_t *>(&v);
-            uint16_t *dst = reinterpret_cast<uint16_t *>(s_x + (size_t)m * p.x_pitch + (kk >> 7) * kGroupFast);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[x_slot<BITS>((kk & 127) + i)] = e[i];
-        }
-        const int nrows = ntiles * kTileRows;
-        for (int idx = tid; idx < nrows * ngs; idx += nthr) {
-            const int r = idx / ngs, gl = idx - r * ngs;
-            const int n = min(tile0 * kTileRows + r, p.N - 1);
-            const float sc = __half2float(p.scales[(size_t)n * p.G + g0 + gl]);
-            const float ze = __half2float(p.zeros[(size_t)n * p.G + g0 + gl]);
-            s_meta[(size_t)r * p.meta_pitch + gl] = make_uint2(__float_as_uint(sc), __float_as_uint(ze));
-        }
+    if (p.rank > 0 && !(t_from_global && !p.t_late)) named_barrier_sync(2, (kCW + 1) * 32);   // permuted x is in place
+    if (has_t && !p.t_late) {
+        t_share();
+        trace_mark(p, 3);
+        t_arrive();
     }
-    __syncthreads();
-    if (p.rank > 0 && is_tw && !p.t_late) t_arrive();
+    trace_mark(p, 4);
+    if (b_in_smem && !mbar_wait(b_full, 0)) dead = true;
 
-    // ---- consumer: stream this warp's tasks ---------------------------------
-    bool dead = false;
-    int it = 0;
-    for (int ti = 0; ti < my_tiles && !dead; ++ti) {
-        const int tile = tile0 + warp + ti * kNW;
+    // Arrival results of the first segment are looked at only after the loop, so that the
+    // round trip of its atomic does not sit in front of the other segments.
+    int old0 = 0, tile0 = -1, cnt0 = 0;
+
+    for (int seg = 0; seg < nseg && !dead; ++seg) {
+        const int buf = seg % kNBuf;
+        const int tile = tile_first + seg;
+        const int cnt = p.SK, myslot = s;       // one contribution per K slice
+        // While the compute warps still work on the segment, look whether every other
+        // contribution of a shared tile has already arrived.
+        int others_in = 0;
+        if (cnt > 1) {
+            if (lane == 0) others_in = ((ld_acquire(p.ctr + kCtrFirstTile + tile) & 0xFFFF) == cnt - 1);
+            others_in = __shfl_sync(0xffffffffu, others_in, 0);
+        }
+        if (!mbar_wait(seg_full + 8u * buf, (uint32_t)(seg / kNBuf) & 1u)) {
+            dead = true;
+            break;
+        }
+        trace_mark(p, seg == 0 ? 5 : 7);
         float acc[MT][4];
 #pragma unroll
-        for (int b = 0; b < MT; ++b)
+        for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+        if (tq < p.vt) {
+            const float4 *src = reinterpret_cast<const float4 *>(s_seg + (size_t)buf * segbuf_floats);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[b][i] = 0.f;
-
-        for (int ch = 0; ch < nchunks; ++ch, ++it) {
-            const int slot = it % p.D;
-            if (!mbar_wait(bar_base + 8u * slot, (uint32_t)(it / p.D) & 1u)) {
-                dead = true;
-                break;
-            }
-            const int cgl = ch * p.CH;                          // first group of the chunk, slice-local
-            const int ng = min(p.CH, ngs - cgl);
-            const uint8_t *slot_ptr = ring_ptr + (size_t)slot * p.slot_bytes;
-            const uint32_t bytes_row = (uint32_t)ng * GB;
-            const uint2 *meta_a = s_meta + (size_t)((tile - tile0) * kTileRows + g) * p.meta_pitch + cgl;
-            const uint2 *meta_b = meta_a + (size_t)8 * p.meta_pitch;
-
-            for (int gi = 0; gi < ng; ++gi) {
-                const uint2 ma = meta_a[gi], mb = meta_b[gi];
-                uint32_t wa[NWORDS], wb[NWORDS];
-                const uint8_t *pa = slot_ptr + (size_t)g * bytes_row + gi * GB + tq * (GB / 4);
-                const uint8_t *pb = pa + (size_t)8 * bytes_row;
-                if constexpr (BITS == 4) {
-                    const uint4 va = *reinterpret_cast<const uint4 *>(pa), vb = *reinterpret_cast<const uint4 *>(pb);
-                    wa[0] = va.x; wa[1] = va.y; wa[2] = va.z; wa[3] = va.w;
-                    wb[0] = vb.x; wb[1] = vb.y; wb[2] = vb.z; wb[3] = vb.w;
-                } else {
-#pragma unroll
-                    for (int i = 0; i < NWORDS; ++i) {
-                        wa[i] = reinterpret_cast<const uint32_t *>(pa)[i];
-                        wb[i] = reinterpret_cast<const uint32_t *>(pb)[i];
-                    }
-                }
-                uint32_t ha[16], hb[16];
-                Unpack<BITS, T>::run(wa, __uint_as_float(ma.y), ha);
-                Unpack<BITS, T>::run(wb, __uint_as_float(mb.y), hb);
-
-                float tmp[MT][4];
+            for (int w = 0; w < kCW; ++w)
 #pragma unroll
                 for (int b = 0; b < MT; ++b) {
-                    tmp[b][0] = tmp[b][1] = tmp[b][2] = tmp[b][3] = 0.f;
-                    const int token = 8 * b + g;
-                    const uint4 *xg = reinterpret_cast<const uint4 *>(s_x + (size_t)token * p.x_pitch +
-                                                                      (size_t)(cgl + gi) * kGroupFast);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 xv = make_uint4(0u, 0u, 0u, 0u);
-                        if (token < p.M) xv = xg[q4 * 4 + tq];
-                        const uint32_t a0[4] = {ha[4 * q4 + 0], hb[4 * q4 + 0], ha[4 * q4 + 1], hb[4 * q4 + 1]};
-                        const uint32_t a1[4] = {ha[4 * q4 + 2], hb[4 * q4 + 2], ha[4 * q4 + 3], hb[4 * q4 + 3]};
-                        Pk<T>::mma(tmp[b], a0, xv.x, xv.y);
-                        Pk<T>::mma(tmp[b], a1, xv.z, xv.w);
-                    }
-                    const float sa = __uint_as_float(ma.x), sb = __uint_as_float(mb.x);
-                    acc[b][0] = fmaf(sa, tmp[b][0], acc[b][0]);
-                    acc[b][1] = fmaf(sa, tmp[b][1], acc[b][1]);
-                    acc[b][2] = fmaf(sb, tmp[b][2], acc[b][2]);
-                    acc[b][3] = fmaf(sb, tmp[b][3], acc[b][3]);
+                    const float4 v = src[(size_t)((w * 8 + g) * p.vt + tq) * MT + b];
+                    acc[b][0] += v.x; acc[b][1] += v.y; acc[b][2] += v.z; acc[b][3] += v.w;
                 }
-            }
-            // slot consumed: refill it with the task D items ahead
-            __syncwarp();
-            if (it + p.D < n_items) {
-                fence_proxy_async();
-                issue(it + p.D);
-            }
         }
-        if (dead) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(seg_free + 8u * buf);
 
-        // ---- hand the finished (tile, slice) task over ------------------------
-        if (p.SK == 1 && p.rank == 0) {
-            tile_epilogue<T, MT>(p, tile, lane, acc);
+        if (cnt == 1 || others_in) {
+            // This warp finishes the tile: straight from registers if t is complete ...
+            if (t_poll()) {
+                tile_epilogue<T, MT>(p, tile, lane, acc, myslot, cnt, s_t, own_b(tile));
+                ++n_retired;
+                if (p.rank == 0 && cnt > 1 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;
+                continue;
+            }
+            // ... else its sums wait in scratch on a local list until t is.
+            float *slot = p.partial + ((size_t)tile * p.maxslots + myslot) * p.M * kTileRows;
+#pragma unroll
+            for (int b = 0; b < MT; ++b)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = g + 8 * (i >> 1), m = 8 * b + 2 * tq + (i & 1);
+                    if (m < p.M) slot[(size_t)m * kTileRows + row] = acc[b][i];
+                }
+            if (lane == 0) s_def[n_def] = tile;
+            ++n_def;
+            __syncwarp();
             continue;
         }
+        // Shared tile, others still missing: leave the partial and an arrival count.
+        float *slot = p.partial + ((size_t)tile * p.maxslots + myslot) * p.M * kTileRows;
 #pragma unroll
         for (int b = 0; b < MT; ++b)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int n = tile * kTileRows + g + 8 * (i >> 1), m = 8 * b + 2 * tq + (i & 1);
-                if (m < p.M && n < p.N) p.partial[((size_t)s * p.M + m) * p.N + n] = acc[b][i];
+                const int row = g + 8 * (i >> 1), m = 8 * b + 2 * tq + (i & 1);
+                if (m < p.M) slot[(size_t)m * kTileRows + row] = acc[b][i];
             }
         __syncwarp();
-        int last = 0;
+        int old = 0;
         if (lane == 0) {
             __threadfence();
-            last = ((atomicAdd(p.ctr + kCtrFirstTile + tile, 1) & 0xFFFF) == p.SK - 1);
+            old = atomicAdd(p.ctr + kCtrFirstTile + tile, 1) & 0xFFFF;
         }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (!last) continue;
-        if (p.rank > 0) {
-            int ready = 0;
-            if (lane == 0) {
-                __threadfence();
-                ready = ld_acquire(p.ctr + kCtrReady);
-                if (!ready) {
-                    // park the tile, then look again: either we see the flag now, or the
-                    // warp that raises it will see our entry (both sides fence in between)
-                    const int idx = atomicAdd(p.ctr + kCtrPendingN, 1);
-                    atomicExch(p.ctr + kCtrFirstTile + p.NT + idx, tile + 1);
-                    __threadfence();
-                    ready = ld_acquire(p.ctr + kCtrReady) ? 2 : 0;
-                }
-            }
-            ready = __shfl_sync(0xffffffffu, ready, 0);
-            if (ready == 0) continue;                               // parked: finished by the t-completing warp
-            if (ready == 2 && !tile_claim(p, tile, lane)) continue; // parked and already taken
+        if (seg == 0 && nseg > 1) {          // look at the result after the loop
+            old0 = old;
+            tile0 = tile;
+            cnt0 = cnt;
+            continue;
         }
-        __threadfence();
-        tile_epilogue<T, MT>(p, tile, lane, nullptr);
-        retire_one(p, lane);
+        const int last = __shfl_sync(0xffffffffu, (int)(old == cnt - 1), 0);
+        if (last) {
+            if (lane == 0) s_def[n_def] = tile;
+            ++n_def;
+            __syncwarp();
+        }
     }
+    if (tile0 >= 0) {
+        const int last = __shfl_sync(0xffffffffu, (int)(old0 == cnt0 - 1), 0);
+        if (last) {
+            if (lane == 0) s_def[n_def] = tile0;
+            ++n_def;
+            __syncwarp();
+        }
+    }
+    trace_mark(p, 8);
 
-    if (dead) {
-        // A bulk copy did not complete in time: report, give copies already in flight a
-        // last bounded chance to land (the CTA must not exit under them), and stop.
-        if (lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
-        for (int j = it; j < min(it + p.D, n_items); ++j)
-            (void)mbar_wait(bar_base + 8u * (j % p.D), (uint32_t)(j / p.D) & 1u);
-    }
-    if (p.rank > 0 && is_tw && p.t_late) {
+    if (has_t && p.t_late) {
         t_share();
         t_arrive();
     }
+    // ---- tiles this warp still owes: finish them if t is complete by now, else park them
+    // globally for the warp that completes t ----
+    if (n_def > 0) {
+        __threadfence();
+        // t is normally complete within a microsecond or two of the first tiles: look a bounded
+        // number of times before handing the tiles over (every CTA contributes to t before it
+        // waits for anything, so this cannot block the contributors)
+        bool ready = t_poll();
+        for (int spin = 0; spin < kTPolls && !ready; ++spin) ready = t_poll();
+        for (int i = 0; i < n_def; ++i) {
+            const int tile = s_def[i];
+            if (ready) {
+                finish_from_slots(tile);
+                continue;
+            }
+            int st = 0;
+            if (lane == 0) {
+                // park the tile, then look again: either we see the flag now, or the warp
+                // that raises it will see our entry (both sides fence in between)
+                const int idx = atomicAdd(p.ctr + kCtrPendingN, 1);
+                atomicExch(p.ctr + kCtrFirstTile + p.NT + idx, tile + 1);
+                __threadfence();
+                st = ld_acquire(p.ctr + kCtrReady);
+            }
+            st = __shfl_sync(0xffffffffu, st, 0);
+            if (st && tile_claim(p, tile, lane)) {
+                __threadfence();
+                (void)t_poll();
+                finish_from_slots(tile);
+            }
+        }
+    }
+    if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+
+    // ---- retire: whoever brings the count to NT + 1 (every tile finished, and the t-completing
+    // warp out of its parked-tile loop) restores the scratch invariants for the next call ----
+    if (p.rank > 0 && n_retired > 0) {
+        __syncwarp();
+        int fin = 0;
+        if (lane == 0) {
+            __threadfence();
+            fin = (atomicAdd(p.ctr + kCtrDone, n_retired) + n_retired == p.NT + 1);
+        }
+        fin = __shfl_sync(0xffffffffu, fin, 0);
+        if (fin) {
+            __threadfence();
+            for (int i = lane; i < 2 * p.NT; i += 32) p.ctr[kCtrFirstTile + i] = 0;   // arrivals + parked list
+            for (int i = lane; i < p.M * p.rank; i += 32) p.t[i] = 0.f;
+            if (lane == 0) {
+                p.ctr[kCtrDone] = 0;
+                p.ctr[kCtrReady] = 0;
+                p.ctr[kCtrPendingN] = 0;
+            }
+        }
+    }
+    trace_mark(p, 9);
 }
 
 // ------------------------------------------------------------------ host side
 struct Plan {
-    int SK, R, NT, CH, D, t_target;
-    int meta_pitch, x_pitch, slot_bytes;
-    int off_list, off_meta, off_x, off_ring;
+    int SK, R, NT, CHG, NS, t_target, maxslots, vt, a_cap, b_cap_rows, meta_rows;
+    int x_pitch, stage_bytes;
+    int off_tab, off_def, off_meta, off_x, off_px, off_segbuf, off_A, off_B, off_t, off_ring;
     size_t smem;
     bool ok;
 };
 
 int g_sm_count = 0;
+constexpr size_t kSmemBudget = 110 * 1024;   // two CTAs (this launch and the next one) fit on an SM
+constexpr size_t kSmemMax = 227 * 1024;      // everything an SM has
 
 Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
 {
@@ -690,52 +1102,84 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     }
     const int GB = (a.bits == 4) ? 64 : 48;
     const int G = a.K / kGroupFast;
+    const int mt = (a.M <= 8) ? 1 : 2;
     pl.NT = (a.N + kTileRows - 1) / kTileRows;
-    int max_ctas = 2 * g_sm_count;
+    int max_ctas = 2 * g_sm_count;            // two CTAs per SM: one streams while the other starts or ends
     if (tune.max_ctas > 0) max_ctas = min(max_ctas, tune.max_ctas);
-    // K slices: enough (tile, slice) tasks to give every warp of the grid about
-    // two, but never more slices than groups, and fewer for many tokens (each
-    // slice costs one fp32 partial tile per output tile).
-    int sk = tune.sk;
-    if (sk <= 0) {
-        const long long want_tasks = 2LL * max_ctas * kNW;
-        sk = (int)((want_tasks + pl.NT - 1) / pl.NT);
-        const int cap = (a.M <= 2) ? 16 : (a.M <= 8 ? 8 : 4);
-        sk = max(1, min(sk, cap));
+    pl.vt = (mt == 2) ? 4 : min(4, (a.M + 1) / 2);
+    // K slices: one, unless the x slice and the other tables do not fit next to the ring.
+    // First try to stay within half an SM's shared memory (so that this launch and the next
+    // one can be resident together) with few slices; otherwise take the whole SM.
+    auto layout = [&](int sk, size_t budget) {
+        pl.SK = sk;
+        const int ngs_max = (G + sk - 1) / sk;
+        pl.R = max(1, min(max_ctas / sk, pl.NT));
+        const int nseg_max = (pl.NT + pl.R - 1) / pl.R;
+        pl.maxslots = sk;
+        pl.CHG = max(1, min(tune.chunk > 0 ? tune.chunk : 16, ngs_max));
+        pl.stage_bytes = kTileRows * (pl.CHG * GB + 64);      // rows are padded by up to 64 bytes
+        pl.x_pitch = ngs_max * kGroupFast + 32;    // +64 bytes: tokens 2j, 2j+1 land in different bank halves
+        const int nkc = (ngs_max * kGroupFast + kTUnitK - 1) / kTUnitK;
+        const long long tu_max = ((long long)a.rank * nkc + pl.R - 1) / pl.R;
+        pl.a_cap = (int)min(tu_max, 8LL);
+        size_t off = (size_t)(2 * 8 + 2 * kNBuf + 3) * 8;      // room for up to 8 stages' barriers
+        off = (off + 15) & ~(size_t)15;
+        pl.off_tab = (int)off;
+        pl.off_def = (int)off;
+        off += (size_t)(kMaxSeg + 2) * sizeof(int);
+        off = (off + 15) & ~(size_t)15;
+        pl.off_meta = (int)off;
+        pl.meta_rows = nseg_max * kTileRows;
+        off += (size_t)pl.meta_rows * (ngs_max | 1) * 8;
+        off = (off + 127) & ~(size_t)127;
+        pl.off_x = (int)off;
+        off += (size_t)a.M * pl.x_pitch * 2;
+        off = (off + 127) & ~(size_t)127;
+        pl.off_px = (int)off;
+        off += (size_t)ngs_max * 8 * mt * 8;
+        off = (off + 127) & ~(size_t)127;
+        pl.off_segbuf = (int)off;
+        off += (size_t)kNBuf * kCW * 8 * pl.vt * 4 * mt * 4;
+        off = (off + 127) & ~(size_t)127;
+        pl.off_A = (int)off;
+        off += (size_t)pl.a_cap * kTUnitK * 2;
+        off = (off + 127) & ~(size_t)127;
+        pl.off_t = (int)off;
+        off += (size_t)a.M * a.rank * 4;
+        off = (off + 127) & ~(size_t)127;
+        // what is left goes to the ring first (at least 2 stages), then to B
+        pl.off_B = (int)off;
+        const size_t b_bytes = (size_t)nseg_max * kTileRows * a.rank * 2;
+        int ns_want = tune.depth > 0 ? tune.depth : 4;
+        ns_want = max(2, min(ns_want, 8));
+        pl.b_cap_rows = 0;
+        if (off + b_bytes + (size_t)ns_want * pl.stage_bytes <= budget) {
+            pl.b_cap_rows = nseg_max * kTileRows;
+            off += b_bytes;
+            off = (off + 127) & ~(size_t)127;
+        }
+        pl.off_ring = (int)off;
+        pl.NS = ns_want;
+        while (pl.NS > 2 && off + (size_t)pl.NS * pl.stage_bytes > budget) --pl.NS;
+        off += (size_t)pl.NS * pl.stage_bytes;
+        pl.smem = off;
+        return nseg_max <= kMaxSeg && pl.smem <= budget;
+    };
+    if (tune.sk > 0) {
+        pl.ok = layout(min(tune.sk, G), kSmemMax);
+    } else {
+        for (int sk = 1; sk <= min(G, 4) && !pl.ok; ++sk) pl.ok = layout(sk, kSmemBudget);
+        for (int sk = 1; sk <= G && !pl.ok; ++sk) pl.ok = layout(sk, kSmemMax);
     }
-    sk = max(1, min(sk, G));
-    pl.SK = sk;
-    pl.R = max(1, min(max_ctas / sk, pl.NT));
-    const int ngs_max = (G + sk - 1) / sk;
-    pl.CH = tune.chunk > 0 ? tune.chunk : 3;
-    pl.CH = max(1, min(pl.CH, ngs_max));
-    pl.D = tune.depth > 0 ? tune.depth : 2;
-    pl.slot_bytes = kTileRows * pl.CH * GB;
-    const int tiles_max = (pl.NT + pl.R - 1) / pl.R;
-    pl.meta_pitch = ngs_max | 1;
-    pl.x_pitch = ngs_max * kGroupFast + 32;    // +64 bytes: tokens 2j, 2j+1 land in different bank halves
-    size_t off = (size_t)kNW * pl.D * 8;
-    pl.off_list = (int)off;
-    off = (off + 15) & ~(size_t)15;
-    pl.off_meta = (int)off;
-    off += (size_t)tiles_max * kTileRows * pl.meta_pitch * 8;
-    off = (off + 127) & ~(size_t)127;
-    pl.off_x = (int)off;
-    off += (size_t)a.M * pl.x_pitch * 2;
-    off = (off + 127) & ~(size_t)127;
-    pl.off_ring = (int)off;
-    off += (size_t)kNW * pl.D * pl.slot_bytes;
-    pl.smem = off;
-    // warps that own at least one row of A
+    // CTAs that own at least one unit of the down-projection
     pl.t_target = 0;
     if (a.rank > 0) {
-        for (int rr = 0; rr < pl.R; ++rr) {
-            const int nj = (int)((long long)(rr + 1) * a.rank / pl.R) - (int)((long long)rr * a.rank / pl.R);
-            pl.t_target += min(nj, kNW);
+        for (int s = 0; s < pl.SK; ++s) {
+            const int ngs = (int)((long long)(s + 1) * G / pl.SK) - (int)((long long)s * G / pl.SK);
+            const long long TU = (long long)a.rank * ((ngs * kGroupFast + kTUnitK - 1) / kTUnitK);
+            pl.t_target += (int)min((long long)pl.R, TU);
         }
-        pl.t_target *= pl.SK;
     }
-    pl.ok = pl.smem <= 110 * 1024;
     return pl;
 }
 
@@ -745,7 +1189,7 @@ cudaError_t launch_variant(const DecodeParams &p, const Plan &pl, bool pdl, cuda
     auto kern = decode_kernel<BITS, T, MT>;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -771,7 +1215,7 @@ void decode_set_test_switch(int t_late) { g_t_late = t_late; }
 void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t *partial_floats, int *counters)
 {
     const Plan pl = make_plan(a, tune);
-    *partial_floats = (size_t)pl.SK * a.M * a.N;
+    *partial_floats = (size_t)pl.NT * pl.maxslots * a.M * kTileRows;
     *counters = kCtrFirstTile + 2 * pl.NT;
 }
 
@@ -791,11 +1235,17 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     p.t = ws.t;
     p.ctr = ws.counters;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.K / kGroupFast; p.rank = a.rank;
-    p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CH = pl.CH; p.D = pl.D;
+    p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CHG = pl.CHG; p.NS = pl.NS;
+    p.maxslots = pl.maxslots;
     p.t_target = pl.t_target;
     p.t_late = g_t_late;
-    p.meta_pitch = pl.meta_pitch; p.x_pitch = pl.x_pitch; p.slot_bytes = pl.slot_bytes;
-    p.off_list = pl.off_list; p.off_meta = pl.off_meta; p.off_x = pl.off_x; p.off_ring = pl.off_ring;
+    p.vt = pl.vt;
+    p.x_pitch = pl.x_pitch; p.stage_bytes = pl.stage_bytes;
+    p.a_cap = pl.a_cap; p.b_cap_rows = pl.b_cap_rows;
+    p.meta_rows = pl.meta_rows;
+    p.off_tab = pl.off_tab; p.off_def = pl.off_def; p.off_meta = pl.off_meta; p.off_x = pl.off_x; p.off_px = pl.off_px;
+    p.off_segbuf = pl.off_segbuf; p.off_A = pl.off_A; p.off_B = pl.off_B; p.off_t = pl.off_t; p.off_ring = pl.off_ring;
+    p.trace = reinterpret_cast<unsigned long long *>(ws.trace);
     const bool pdl = tune.pdl != 0;
     cudaError_t e;
     const int mt = (a.M <= 8) ? 1 : 2;
