@@ -114,6 +114,29 @@ int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *s
                       int N, int K, int group, int bits, int rank, int act_is_bf16,
                       void *stream);
 
+/* (The paper has no counterpart: this entry point exists for integration reasons only.)
+ * The same fused layer for callers that must not allocate device memory: a process that
+ * gave all of it to its own pool at start-up, a latency-critical loop that cannot take the
+ * device-wide synchronisation an allocation may imply, a plug-in whose host forbids driver
+ * allocations after initialisation.  fbq_linear keeps its scratch space in buffers it
+ * allocates per stream on first use; this variant runs the decode kernel with its scratch in
+ * one fixed array that is part of the library image (about 2.1 MiB, held by every GPU that
+ * loads the library until the process exits), and never calls an allocating routine.
+ *   - Domain: the decode kernel's (M <= 16, group == 128, rank a multiple of 8 up to 256),
+ *     and the scratch it needs must fit the array: N <= 65536 and roughly M * N * (number
+ *     of K slices, 1 unless x is too large for shared memory) <= 524288.  Anything else
+ *     returns FBQ_ERR_UNSUPPORTED and runs nothing; use fbq_linear for those.
+ *   - The first call on each device looks up the array's device address (a cheap query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - Every call uses the same array and begins by clearing the part that must start at
+ *     zero (a memset queued on `stream`).  Calls that can overlap on the GPU (different
+ *     streams, or several host threads) therefore race on it: run them one after another.
+ *   - Arguments, layouts, dtypes (act_is_bf16 selects bf16 x, A, B, y) and results are
+ *     those of fbq_linear / fbq_linear_bf16. */
+int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const void *scales,
+                       const void *zeros, const void *A, const void *B, void *y, int M, int N,
+                       int K, int group, int bits, int rank, int act_is_bf16, void *stream);
+
 /* Which kernel fbq_linear / fbq_linear_bf16 would run for this shape, or
  * FBQ_KERNEL_NONE when the shape is rejected.  Pure host logic. */
 int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int act_is_bf16);

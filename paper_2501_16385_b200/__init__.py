@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     library_path,
     linear,
     linear_hostio,
+    linear_noalloc,
     pack,
     packed_words,
     poll_status,

@@ -47,6 +47,7 @@ def lib() -> ctypes.CDLL:
         for name in ("fbq_linear", "fbq_linear_bf16"):
             getattr(L, name).argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
+        L.fbq_linear_noalloc.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_select_kernel.argtypes = [i32] * 7
         L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
         L.fbq_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32)]
@@ -137,6 +138,20 @@ def linear_hostio(x_host, qweight, scales, zeros, A, B, y_host, N: int, group: i
                                    _ptr(B), _ptr(y_host), M, N, K, group, bits, rank, bf16,
                                    _stream(stream)), "fbq_linear_hostio")
     return y_host
+
+
+def linear_noalloc(x, qweight, scales, zeros, A, B, N: int, group: int, bits: int, y, stream=None):
+    """fbq_linear_noalloc: like ``linear`` for decode shapes, but the library allocates nothing
+    (its scratch lives in a fixed array inside the library).  The caller passes y.  Calls must
+    not overlap on the GPU: they all share that one array."""
+    import torch
+    M, K = x.shape
+    rank = 0 if A is None else A.shape[0]
+    bf16 = 1 if x.dtype == torch.bfloat16 else 0
+    _check(lib().fbq_linear_noalloc(_ptr(x), _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(A), _ptr(B),
+                                    _ptr(y), M, N, K, group, bits, rank, bf16, _stream(stream)),
+           "fbq_linear_noalloc")
+    return y
 
 
 def select_kernel(M, N, K, group, bits, rank, bf16=False) -> int:

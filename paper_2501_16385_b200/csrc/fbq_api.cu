@@ -165,6 +165,9 @@ int *option_slot(const char *name)
 }
 
 }  // namespace
+
+void count_launches(int n) { g_launches += n; }
+
 }  // namespace fbq
 
 using namespace fbq;
