@@ -323,9 +323,10 @@ def gpu_arm(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per step measured with ncu on the seven decode launches of one
-# step (profiles/decode_int3_r64_m1.md); None until a capture has been taken.
-TRAFFIC_BYTES_PER_STEP = None
+# DRAM bytes (read + write) per step measured with ncu (--set full) on the seven decode
+# launches of one step: 4 x 7.971 MB + 2 x 20.373 MB + 20.388 MB
+# (profiles/decode_int3_r64_m1_bench.md).
+TRAFFIC_BYTES_PER_STEP = 93_018_000
 
 
 # ---------------------------------------------------------------------- reference arm
