@@ -299,15 +299,9 @@ template <int BITS> __device__ __forceinline__ int frag_pos(int c)
     const int i = c / 10, f = c - 10 * i;
     return (f < 5) ? 2 * (5 * i + f) : 2 * (5 * i + f - 5) + 1;
 }
-// Shared-memory element offset of x[k] inside its 128-element group block:
-// 16-byte units are laid out [h_index / 4][lane t][h_index % 4] so that one
-// 128-bit load per lane fetches the operands of two MMAs, conflict free.
-template <int BITS> __device__ __forceinline__ int x_slot(int k_in_group)
-{
-    const int t = k_in_group >> 5, pos = frag_pos<BITS>(k_in_group & 31);
-    const int hidx = pos >> 1;
-    return (((hidx >> 2) * 4 + t) * 4 + (hidx & 3)) * 2 + (pos & 1);
-}
+// x in shared memory: per token and 128-element group, 16-byte units are laid out
+// [h_index / 4][lane t][h_index % 4], so that one 128-bit load per lane fetches the
+// operands of two MMAs, conflict free.
 
 __device__ __forceinline__ float ld_cg_f32(const float *p) { return __ldcg(p); }
 __device__ __forceinline__ int ld_acquire(const int *p)
@@ -320,11 +314,6 @@ __device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
-__device__ __forceinline__ void named_barrier_arrive(int id, int nthreads)
-{
-    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-
 __device__ __forceinline__ void trace_mark(const DecodeParams &p, int slot)
 {
     if (p.trace && (threadIdx.x & 31) == 0) {
@@ -335,84 +324,47 @@ __device__ __forceinline__ void trace_mark(const DecodeParams &p, int slot)
 }
 
 // --------------------------------------------------------------- tile epilogue
-// Main-path sums of the tile: slot i of scratch for i != myslot, `own` (this
-// warp's registers) for i == myslot (own == nullptr: every slot from scratch),
-// always added in slot order.  Then the up-projection t.B^T is added and y is
-// stored.  Lane (g,tq) owns rows g and g+8 and tokens 8b+2tq, 8b+2tq+1.
-// t is read from shared memory (s_t); B from shared memory when b_smem != 0
-// (rows of this CTA's own tiles), else from global memory.
-template <typename T, int MT>
-__device__ __forceinline__ void tile_epilogue(const DecodeParams &p, int tile, int lane, const float (*own)[4], int myslot,
-                                              int cnt, const float *s_t, const T *b_smem)
+// Finishes one 16-row tile: main-path sums (slot i of scratch for i != myslot,
+// the staged sums of this warp for i == myslot; staged == nullptr: every slot
+// from scratch; always added in slot order), plus the up-projection t.B^T, one
+// rounding, one store.  A lane handles (row, token) pairs idx = lane, lane+32, ..
+// t comes from shared memory (s_t); B from shared memory when b_smem != nullptr
+// (rows of this CTA's own tiles), else from global memory.  Kept out of line
+// and free of unrolling on purpose: it runs once per tile, and the kernel's
+// code must stay small enough for the instruction cache.
+template <typename T>
+__device__ __forceinline__ void finish_tile(const DecodeParams &p, int tile, int lane, const float *staged, int myslot, int cnt,
+                                         const float *s_t, const T *b_smem)
 {
-    const int g = lane >> 2, tq = lane & 3;
     T *y = static_cast<T *>(p.y);
     const float *slots = p.partial + (size_t)tile * p.maxslots * p.M * kTileRows;
     const size_t stride = (size_t)p.M * kTileRows;
-#pragma unroll
-    for (int b = 0; b < MT; ++b) {
-#pragma unroll
-        for (int hr = 0; hr < 2; ++hr) {
-            const int row = g + 8 * hr, n = tile * kTileRows + row;
-#pragma unroll
-            for (int tk = 0; tk < 2; ++tk) {
-                const int m = 8 * b + 2 * tq + tk;
-                if (m >= p.M || n >= p.N) continue;
-                const float mine = own ? own[b][2 * hr + tk] : 0.f;
-                float v = 0.f;
-                const float *sp = slots + (size_t)m * kTileRows + row;
-                if (cnt == 1 && own) {
-                    v = mine;
-                } else {
-                    for (int i0 = 0; i0 < cnt; i0 += 4) {
-                        float a[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int i = i0 + u;
-                            a[u] = (i < cnt && !(own && i == myslot)) ? ld_cg_f32(sp + i * stride) : 0.f;
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int i = i0 + u;
-                            if (i < cnt) v += (own && i == myslot) ? mine : a[u];
-                        }
-                    }
-                }
-                if (p.rank > 0) {
-                    const float4 *trow = reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank);
-                    float sub = 0.f;
-                    if (b_smem) {
-                        const uint4 *brow = reinterpret_cast<const uint4 *>(b_smem + (size_t)row * p.rank);
+#pragma unroll 1
+    for (int idx = lane; idx < kTileRows * p.M; idx += 32) {
+        const int row = idx & (kTileRows - 1), m = idx >> 4, n = tile * kTileRows + row;
+        if (n >= p.N) continue;
+        float v = 0.f;
+#pragma unroll 1
+        for (int i = 0; i < cnt; ++i) v += (staged && i == myslot) ? staged[idx] : ld_cg_f32(slots + i * stride + idx);
+        if (p.rank > 0) {
+            const float4 *trow = reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank);
+            const uint4 *brow = b_smem ? reinterpret_cast<const uint4 *>(b_smem + (size_t)row * p.rank)
+                                       : reinterpret_cast<const uint4 *>(static_cast<const T *>(p.B) + (size_t)n * p.rank);
+            float sub = 0.f;
 #pragma unroll 2
-                        for (int c = 0; c < p.rank / 8; ++c) {
-                            const uint4 bv = brow[c];
-                            const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
-                            const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
-                            const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
-                            sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
-                            sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
-                            sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
-                            sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
-                        }
-                    } else {
-                        const uint4 *brow = reinterpret_cast<const uint4 *>(static_cast<const T *>(p.B) + (size_t)n * p.rank);
-#pragma unroll 4
-                        for (int c = 0; c < p.rank / 8; ++c) {
-                            const uint4 bv = __ldg(brow + c);
-                            const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
-                            const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
-                            const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
-                            sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
-                            sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
-                            sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
-                            sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
-                        }
-                    }
-                    v += sub;
-                }
-                y[(size_t)m * p.N + n] = ActTraits<T>::from_float(v);
+            for (int c = 0; c < p.rank / 8; ++c) {
+                const uint4 bv = brow[c];
+                const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
+                const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
+                const float2 b2 = Pk<T>::to_float2(bv.z), b3 = Pk<T>::to_float2(bv.w);
+                sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
+                sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
+                sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
+                sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
             }
+            v += sub;
         }
+        y[(size_t)m * p.N + n] = ActTraits<T>::from_float(v);
     }
 }
 
@@ -454,9 +406,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     const long long TU = (long long)p.rank * nkc;
     const int tu0 = (int)((long long)r * TU / p.R), tu1 = (int)((long long)(r + 1) * TU / p.R);
     const bool has_t = (p.rank > 0) && (tu1 > tu0);
-    // few tokens: the down-projection reads x straight from global memory and need not wait
-    // for the compute warps' permuted copy
-    const bool t_from_global = (p.M <= 2);
 
     // shared memory: barriers | table | deferred list | meta | x | segbuf | A | B | t | ring
     trace_mark(p, 0);
@@ -654,8 +603,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         trace_mark(p, 4);
         bool dead = false;
         named_barrier_sync(1, kCW * 32);
-        if (p.rank > 0 && !(p.M <= 2 && !p.t_late))
-            named_barrier_arrive(2, (kCW + 1) * 32);                   // x is in place for the epilogue warp
         trace_mark(p, 5);
 
         // ---- consumer: every stage is shared; this warp takes an eighth of its groups ----
@@ -769,6 +716,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     int n_def = 0;              // tiles this warp must finish once t is complete (s_def[])
     bool t_local = (p.rank == 0);   // t is complete and copied to shared memory
     bool dead = false;
+    float *s_stage = s_t + (size_t)p.M * p.rank;     // this warp's staged main sums [token][16]
 
     // Looks at the "t complete" flag; on the first sighting copies t to shared memory.
     auto t_poll = [&]() -> bool {
@@ -789,92 +737,63 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     };
     // Finish `tile` from scratch slots (all contributions are there and visible).
     auto finish_from_slots = [&](int tile) {
-        tile_epilogue<T, MT>(p, tile, lane, nullptr, 0, p.SK, s_t, own_b(tile));
+        finish_tile<T>(p, tile, lane, nullptr, 0, p.SK, s_t, own_b(tile));
         ++n_retired;
         if (p.rank == 0 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;   // nobody else will touch it again
     };
+    // Copies the staged sums of this warp to its scratch slot of `tile`.
+    auto stage_to_slot = [&](int tile) {
+        float *slot = p.partial + ((size_t)tile * p.maxslots + s) * p.M * kTileRows;
+        for (int idx = lane; idx < kTileRows * p.M; idx += 32) slot[idx] = s_stage[idx];
+        __syncwarp();
+    };
 
+    // This CTA's share of t = x.A^T:  t[m][j] += sum over its units (row j of A, k chunk).
+    // A comes from shared memory (bulk copy) for the first a_cap units, x from global memory.
     auto t_share = [&]() {
-        // t[m][j] += sum over this CTA's units (j, k chunk) of x[m][k] * A[j][k]
         if (!mbar_wait(a_full, 0)) {
             dead = true;
             return;
         }
         const T *A = static_cast<const T *>(p.A);
+        const T *x = static_cast<const T *>(p.x) + g0 * kGroupFast;
+#pragma unroll 1
         for (int u = tu0; u < tu1; ++u) {
             const int j = u / nkc, kc = u - j * nkc;
             const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
             const bool in_smem = (u - tu0) < p.a_cap;
             const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
-            float acc[MT * 8];
+            uint4 av[4];
 #pragma unroll
-            for (int m = 0; m < MT * 8; ++m) acc[m] = 0.f;
-            if (t_from_global && !p.t_late) {
-                const T *xg = static_cast<const T *>(p.x) + g0 * kGroupFast + kbeg;
-#pragma unroll
-                for (int m = 0; m < 2; ++m) {
-                    if (m < p.M) {
-                        uint4 xv[4], av[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int k = lane * 8 + 256 * i;
-                            xv[i] = make_uint4(0u, 0u, 0u, 0u);
-                            av[i] = xv[i];
-                            if (k < nk) {
-                                xv[i] = __ldcg(reinterpret_cast<const uint4 *>(xg + (size_t)m * p.K + k));
-                                av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
-                                                : __ldg(reinterpret_cast<const uint4 *>(arow + k));
-                            }
-                        }
-                        float v = 0.f;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
-                            const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
-                                v = fmaf(xf.x, af.x, v);
-                                v = fmaf(xf.y, af.y, v);
-                            }
-                        }
-                        acc[m] = v;
-                    }
-                }
-            } else
-            for (int k = lane * 8; k < nk; k += 256) {
-                const uint4 av = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
-                                         : __ldg(reinterpret_cast<const uint4 *>(arow + k));
-                const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
-                const int kl = kbeg + k;                              // slice-local k of the first element
-                const int xoff = (kl >> 7) * kGroupFast;
-                int slot8[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) slot8[q] = xoff + x_slot<BITS>((kl & 127) + q);
-#pragma unroll
-                for (int m = 0; m < MT * 8; ++m) {
-                    if (m < p.M) {
-                        const T *xr = s_x + (size_t)m * p.x_pitch;
-                        float v = acc[m];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            // shared memory holds x divided by the field weight: undo it
-                            const float2 af = Pk<T>::to_float2(aw[q]);
-                            const int c0 = ((kl & 127) + 2 * q) & 31, c1 = c0 + 1;
-                            v = fmaf(ldexpf(ActTraits<T>::to_float(xr[slot8[2 * q]]), Unpack<BITS, T>::div_log2(c0)), af.x, v);
-                            v = fmaf(ldexpf(ActTraits<T>::to_float(xr[slot8[2 * q + 1]]), Unpack<BITS, T>::div_log2(c1)), af.y, v);
-                        }
-                        acc[m] = v;
-                    }
-                }
+            for (int i = 0; i < 4; ++i) {
+                const int k = lane * 8 + 256 * i;
+                av[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (k < nk) av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
+                                            : __ldg(reinterpret_cast<const uint4 *>(arow + k));
             }
+#pragma unroll 1
+            for (int m = 0; m < p.M; ++m) {
+                uint4 xv[4];
 #pragma unroll
-            for (int m = 0; m < MT * 8; ++m) {
-                if (m < p.M) {
-                    float v = acc[m];
-                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + j, v);
+                for (int i = 0; i < 4; ++i) {
+                    const int k = lane * 8 + 256 * i;
+                    xv[i] = make_uint4(0u, 0u, 0u, 0u);
+                    if (k < nk) xv[i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + kbeg + k));
                 }
+                float v = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
+                    const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
+                        v = fmaf(xf.x, af.x, v);
+                        v = fmaf(xf.y, af.y, v);
+                    }
+                }
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + j, v);
             }
         }
     };
@@ -899,6 +818,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         }
         npend = __shfl_sync(0xffffffffu, npend, 0);
         (void)t_poll();
+#pragma unroll 1
         for (int i = 0; i < npend; ++i) {
             int tile = 0;
             if (lane == 0) tile = ld_acquire(p.ctr + kCtrFirstTile + p.NT + i) - 1;
@@ -911,7 +831,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         ++n_retired;                                   // the completer's own token in the retire count
     };
 
-    if (p.rank > 0 && !(t_from_global && !p.t_late)) named_barrier_sync(2, (kCW + 1) * 32);   // permuted x is in place
     if (has_t && !p.t_late) {
         t_share();
         trace_mark(p, 3);
@@ -920,10 +839,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     trace_mark(p, 4);
     if (b_in_smem && !mbar_wait(b_full, 0)) dead = true;
 
-    // Arrival results of the first segment are looked at only after the loop, so that the
-    // round trip of its atomic does not sit in front of the other segments.
-    int old0 = 0, tile0 = -1, cnt0 = 0;
-
+#pragma unroll 1
     for (int seg = 0; seg < nseg && !dead; ++seg) {
         const int buf = seg % kNBuf;
         const int tile = tile_first + seg;
@@ -940,10 +856,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             break;
         }
         trace_mark(p, seg == 0 ? 5 : 7);
-        float acc[MT][4];
-#pragma unroll
-        for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+        // add the eight warps' partial tiles in warp order and stage the result as [token][row]
         if (tq < p.vt) {
+            float acc[MT][4];
+#pragma unroll
+            for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
             const float4 *src = reinterpret_cast<const float4 *>(s_seg + (size_t)buf * segbuf_floats);
 #pragma unroll
             for (int w = 0; w < kCW; ++w)
@@ -952,64 +869,43 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                     const float4 v = src[(size_t)((w * 8 + g) * p.vt + tq) * MT + b];
                     acc[b][0] += v.x; acc[b][1] += v.y; acc[b][2] += v.z; acc[b][3] += v.w;
                 }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(seg_free + 8u * buf);
-
-        if (cnt == 1 || others_in) {
-            // This warp finishes the tile: straight from registers if t is complete ...
-            if (t_poll()) {
-                tile_epilogue<T, MT>(p, tile, lane, acc, myslot, cnt, s_t, own_b(tile));
-                ++n_retired;
-                if (p.rank == 0 && cnt > 1 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;
-                continue;
-            }
-            // ... else its sums wait in scratch on a local list until t is.
-            float *slot = p.partial + ((size_t)tile * p.maxslots + myslot) * p.M * kTileRows;
 #pragma unroll
             for (int b = 0; b < MT; ++b)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int row = g + 8 * (i >> 1), m = 8 * b + 2 * tq + (i & 1);
-                    if (m < p.M) slot[(size_t)m * kTileRows + row] = acc[b][i];
+                    if (m < p.M) s_stage[m * kTileRows + row] = acc[b][i];
                 }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(seg_free + 8u * buf);
+
+        if (cnt == 1 || others_in) {
+            // This warp finishes the tile: straight from the staged sums if t is complete ...
+            if (t_poll()) {
+                finish_tile<T>(p, tile, lane, s_stage, myslot, cnt, s_t, own_b(tile));
+                ++n_retired;
+                if (p.rank == 0 && cnt > 1 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;
+                __syncwarp();
+                continue;
+            }
+            // ... else its sums wait in scratch on a local list until t is.
+            stage_to_slot(tile);
             if (lane == 0) s_def[n_def] = tile;
             ++n_def;
             __syncwarp();
             continue;
         }
         // Shared tile, others still missing: leave the partial and an arrival count.
-        float *slot = p.partial + ((size_t)tile * p.maxslots + myslot) * p.M * kTileRows;
-#pragma unroll
-        for (int b = 0; b < MT; ++b)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = g + 8 * (i >> 1), m = 8 * b + 2 * tq + (i & 1);
-                if (m < p.M) slot[(size_t)m * kTileRows + row] = acc[b][i];
-            }
-        __syncwarp();
-        int old = 0;
+        stage_to_slot(tile);
+        int last = 0;
         if (lane == 0) {
             __threadfence();
-            old = atomicAdd(p.ctr + kCtrFirstTile + tile, 1) & 0xFFFF;
+            last = ((atomicAdd(p.ctr + kCtrFirstTile + tile, 1) & 0xFFFF) == cnt - 1);
         }
-        if (seg == 0 && nseg > 1) {          // look at the result after the loop
-            old0 = old;
-            tile0 = tile;
-            cnt0 = cnt;
-            continue;
-        }
-        const int last = __shfl_sync(0xffffffffu, (int)(old == cnt - 1), 0);
+        last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
             if (lane == 0) s_def[n_def] = tile;
-            ++n_def;
-            __syncwarp();
-        }
-    }
-    if (tile0 >= 0) {
-        const int last = __shfl_sync(0xffffffffu, (int)(old0 == cnt0 - 1), 0);
-        if (last) {
-            if (lane == 0) s_def[n_def] = tile0;
             ++n_def;
             __syncwarp();
         }
@@ -1020,7 +916,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         t_share();
         t_arrive();
     }
-    // ---- tiles this warp still owes: finish them if t is complete by now, else park them
+    // ---- tiles this warp still owes: finish them once t is complete, else park them
     // globally for the warp that completes t ----
     if (n_def > 0) {
         __threadfence();
@@ -1028,7 +924,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         // number of times before handing the tiles over (every CTA contributes to t before it
         // waits for anything, so this cannot block the contributors)
         bool ready = t_poll();
+#pragma unroll 1
         for (int spin = 0; spin < kTPolls && !ready; ++spin) ready = t_poll();
+#pragma unroll 1
         for (int i = 0; i < n_def; ++i) {
             const int tile = s_def[i];
             if (ready) {
@@ -1145,7 +1043,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         off += (size_t)pl.a_cap * kTUnitK * 2;
         off = (off + 127) & ~(size_t)127;
         pl.off_t = (int)off;
-        off += (size_t)a.M * a.rank * 4;
+        off += (size_t)a.M * a.rank * 4 + (size_t)kTileRows * kDecodeMaxM * 4;   // t, then the epilogue warp's staging tile
         off = (off + 127) & ~(size_t)127;
         // what is left goes to the ring first (at least 2 stages), then to B
         pl.off_B = (int)off;
