@@ -32,6 +32,11 @@ if ROOT not in sys.path:
 BITS, RANK, GROUP, M_TOKENS = 3, 64, 128, 1
 WORKLOAD = "llama2-7b decoder-layer linears, M=1, INT3 g128, rank 64 (7 linears per step)"
 GRAPH_STEPS = 100
+# The seven linears of a step are independent (each has its own x), so a step issues them
+# round-robin over N_STREAMS CUDA streams (fbq_linear keeps separate scratch per stream) with
+# the decode grid limited to DECODE_CTAS, which lets launches of different streams share the SMs.
+N_STREAMS = int(os.environ.get("FBQ_BENCH_STREAMS", "7"))
+DECODE_CTAS = int(os.environ.get("FBQ_BENCH_CTAS", "74"))
 NVSMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                 "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                 "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -138,17 +143,41 @@ def build_pool(fbq, torch, n_layers: int, seed0: int = 1000):
     return pool, host0
 
 
-def run_step(fbq, layer, with_branch: bool = True):
-    for d in layer:
+_SIDE_STREAMS = []
+
+
+def side_streams(torch):
+    while len(_SIDE_STREAMS) < N_STREAMS - 1:
+        _SIDE_STREAMS.append(torch.cuda.Stream())
+    return _SIDE_STREAMS
+
+
+def run_step(fbq, layer, with_branch: bool = True, streams=None):
+    """One step: the seven fbq_linear calls of one layer instance.  With `streams` (the
+    current stream first), call j goes to stream j % len(streams)."""
+    import torch
+    for j, d in enumerate(layer):
+        st = streams[j % len(streams)] if streams else None
         fbq.linear(d.x, d.qweight, d.scales, d.zeros, d.A if with_branch else None,
-                   d.B if with_branch else None, d.N, GROUP, BITS, y=d.y)
+                   d.B if with_branch else None, d.N, GROUP, BITS, y=d.y, stream=st)
+
+
+def run_steps_forked(fbq, torch, pool, n_steps: int, main, with_branch: bool):
+    """n_steps steps with the side streams forked from / joined to `main` once around them."""
+    sides = side_streams(torch)
+    streams = [main] + sides
+    for st in sides:
+        st.wait_stream(main)
+    for i in range(n_steps):
+        run_step(fbq, pool[i % len(pool)], with_branch, streams)
+    for st in sides:
+        main.wait_stream(st)
 
 
 def capture_graph(fbq, torch, pool, n_steps: int, stream, with_branch: bool):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g, stream=stream):
-        for i in range(n_steps):
-            run_step(fbq, pool[i % len(pool)], with_branch)
+        run_steps_forked(fbq, torch, pool, n_steps, stream, with_branch)
     return g
 
 
@@ -158,8 +187,8 @@ def time_graph_steps(fbq, torch, pool, steps: int, warmup: int, barrier, with_br
     chunk = max(1, min((GRAPH_STEPS // L) * L, steps))
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
-        for i in range(min(max(warmup, 3), 2 * L)):
-            run_step(fbq, pool[i % L], with_branch)   # plain launches: first-call set-up, scratch growth
+        # plain launches: first-call set-up and scratch growth on every stream used later
+        run_steps_forked(fbq, torch, pool, min(max(warmup, 3), 2 * L), stream, with_branch)
         stream.synchronize()
         g_main = capture_graph(fbq, torch, pool, chunk, stream, with_branch)
         rem = steps % chunk
@@ -188,8 +217,9 @@ def time_plain_steps(fbq, torch, pool, steps: int):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     e0.record()
+    main = torch.cuda.current_stream()
     for i in range(steps):
-        run_step(fbq, pool[i % L])
+        run_steps_forked(fbq, torch, pool[i % L:i % L + 1], 1, main, True)
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1)
@@ -201,11 +231,15 @@ def time_e2e(fbq, torch, pool, steps: int, warmup: int):
     xs = [[d.x.cpu().pin_memory() for d in layer] for layer in pool]
     ys = [[torch.empty((M_TOKENS, d.N), dtype=torch.float16).pin_memory() for d in layer] for layer in pool]
 
+    streams = [torch.cuda.current_stream()] + side_streams(torch)
+
     def one(i):
         layer = pool[i % L]
         for j, d in enumerate(layer):
-            fbq.linear_hostio(xs[i % L][j], d.qweight, d.scales, d.zeros, d.A, d.B, ys[i % L][j], d.N, GROUP, BITS)
-        torch.cuda.current_stream().synchronize()      # the step's result is read on the host
+            fbq.linear_hostio(xs[i % L][j], d.qweight, d.scales, d.zeros, d.A, d.B, ys[i % L][j], d.N, GROUP, BITS,
+                              stream=streams[j % len(streams)])
+        for st in streams:
+            st.synchronize()                          # the step's results are read on the host
 
     for i in range(max(3, warmup)):
         one(i)
@@ -249,6 +283,7 @@ def gpu_arm(args):
             dist.barrier()
 
     import paper_2501_16385_b200 as fbq
+    fbq.set_option("decode_ctas", DECODE_CTAS)
     peaks, peak_kind = measured_peaks()
     bytes_step = step_bytes()
     pool_layers = max(2, -(-3 * 126_000_000 // bytes_step))        # pool >= 3 x L2 (126 MB)
@@ -303,7 +338,9 @@ def gpu_arm(args):
                    "linears_per_step": n_linears, "pool_layers": pool_layers,
                    "cold": "pool of %d layer instances (%.0f MB) > 3x L2, visited round-robin" %
                            (pool_layers, pool_layers * bytes_step / 1e6),
-                   "launch": "CUDA graph replay of fbq_linear calls (programmatic dependent launch)",
+                   "launch": "CUDA graph replay of fbq_linear calls (programmatic dependent launch); the 7 "
+                             "independent linears of a step go round-robin over %d streams, decode grid <= %d CTAs"
+                             % (N_STREAMS, DECODE_CTAS),
                    "parallelism": "replicas only (no collective on the path)" if world > 1 else "1 GPU"},
         "gpu_launches": args.steps * n_linears,       # one fused decode launch per linear per step
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",

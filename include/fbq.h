@@ -151,8 +151,8 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol
- *   "decode_trace"  tuning aid: 1 = the decode kernel records phase timestamps
- *                   (globaltimer, ns) per CTA and warp, read with fbq_debug_read_trace
+ *   "decode_trace"  tuning aid: 1 = the decode kernel records, per CTA and warp, the SM cycle
+ *                   counter at its phases, read with fbq_debug_read_trace
  * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name. */
 int fbq_set_option(const char *name, int value);
 int fbq_get_option(const char *name, int *value);
@@ -165,9 +165,10 @@ long long fbq_launch_count(void);
  * (the affected outputs are then undefined).  Reading clears the word. */
 int fbq_poll_status(void *stream);
 
-/* Tuning aid: copies the phase timestamps of the last decode launch on `stream`
- * (recorded while "decode_trace" is 1) to host_buf: uint64 [cta][10 warps][16 marks],
- * zero where a mark was not reached.  Synchronises the stream. */
+/* Tuning aid: copies the phase marks of the last decode launch on `stream` (recorded while
+ * "decode_trace" is 1) to host_buf: uint64 [cta][10 warps][16 marks] of SM cycle counts, zero
+ * where a mark was not reached; mark 15 of warp 0 is the global timer (ns) at kernel entry.
+ * bytes <= 512*10*16*8.  Synchronises the stream. */
 int fbq_debug_read_trace(void *stream, void *host_buf, size_t bytes);
 
 /* Frees every per-stream scratch buffer (synchronises the device first). */

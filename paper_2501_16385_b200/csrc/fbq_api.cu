@@ -24,7 +24,7 @@ struct Options {
     int decode_t_late = 0;
     int decode_trace = 0;
 } g_opt;
-constexpr size_t kTraceBytes = 2 * 512 * 10 * 16 * 8;   // two launches (alternating) x 512 CTAs x 10 warps x 16 marks
+constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
 
 bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 

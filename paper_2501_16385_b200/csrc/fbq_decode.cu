@@ -47,7 +47,7 @@ constexpr int kMaxSeg = 64;                  // segments (tiles touched) per CTA
 constexpr int kNBuf = 4;                     // segment partial buffers in flight
 constexpr int kTUnitK = 1024;                // k extent of one unit of the down-projection
 constexpr uint32_t kWaitLimit = 1u << 22;
-constexpr int kEarlyStages = 1;              // weight stages prefetched before x has been requested
+constexpr int kEarlyStages = 1;                // weight stages prefetched before x has been requested
 constexpr int kTPolls = 64;                  // looks at the "t complete" flag before a finished tile is parked
 
 // counters[] layout (ints) inside the per-stream scratch
@@ -314,12 +314,18 @@ __device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+// Tuning aid: SM cycle counter of this warp at a phase (cheap to read, unlike %globaltimer).
+// Slot 15 of warp 0 additionally holds the global timer at kernel entry, to line CTAs up.
 __device__ __forceinline__ void trace_mark(const DecodeParams &p, int slot)
 {
     if (p.trace && (threadIdx.x & 31) == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = t;
+        unsigned long long *row = p.trace + ((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16;
+        row[slot] = (unsigned long long)clock64();
+        if (slot == 0 && threadIdx.x == 0) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+            row[15] = t;
+        }
     }
 }
 
@@ -332,27 +338,27 @@ __device__ __forceinline__ void trace_mark(const DecodeParams &p, int slot)
 // (rows of this CTA's own tiles), else from global memory.  Kept out of line
 // and free of unrolling on purpose: it runs once per tile, and the kernel's
 // code must stay small enough for the instruction cache.
+// (Arguments are passed one by one, not as the parameter struct, so that the call needs no
+// stack.)  slots = scratch of this tile, Bg = B in global memory.
 template <typename T>
-__device__ __forceinline__ void finish_tile(const DecodeParams &p, int tile, int lane, const float *staged, int myslot, int cnt,
-                                         const float *s_t, const T *b_smem)
+__device__ __noinline__ void finish_tile(T *y, const float *slots, const T *Bg, int M, int N, int rank, int tile, int lane,
+                                         const float *staged, int myslot, int cnt, const float *s_t, const T *b_smem)
 {
-    T *y = static_cast<T *>(p.y);
-    const float *slots = p.partial + (size_t)tile * p.maxslots * p.M * kTileRows;
-    const size_t stride = (size_t)p.M * kTileRows;
+    const size_t stride = (size_t)M * kTileRows;
 #pragma unroll 1
-    for (int idx = lane; idx < kTileRows * p.M; idx += 32) {
+    for (int idx = lane; idx < kTileRows * M; idx += 32) {
         const int row = idx & (kTileRows - 1), m = idx >> 4, n = tile * kTileRows + row;
-        if (n >= p.N) continue;
+        if (n >= N) continue;
         float v = 0.f;
 #pragma unroll 1
         for (int i = 0; i < cnt; ++i) v += (staged && i == myslot) ? staged[idx] : ld_cg_f32(slots + i * stride + idx);
-        if (p.rank > 0) {
-            const float4 *trow = reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank);
-            const uint4 *brow = b_smem ? reinterpret_cast<const uint4 *>(b_smem + (size_t)row * p.rank)
-                                       : reinterpret_cast<const uint4 *>(static_cast<const T *>(p.B) + (size_t)n * p.rank);
+        if (rank > 0) {
+            const float4 *trow = reinterpret_cast<const float4 *>(s_t + (size_t)m * rank);
+            const uint4 *brow = b_smem ? reinterpret_cast<const uint4 *>(b_smem + (size_t)row * rank)
+                                       : reinterpret_cast<const uint4 *>(Bg + (size_t)n * rank);
             float sub = 0.f;
 #pragma unroll 2
-            for (int c = 0; c < p.rank / 8; ++c) {
+            for (int c = 0; c < rank / 8; ++c) {
                 const uint4 bv = brow[c];
                 const float4 t0 = trow[2 * c], t1 = trow[2 * c + 1];
                 const float2 b0 = Pk<T>::to_float2(bv.x), b1 = Pk<T>::to_float2(bv.y);
@@ -364,7 +370,7 @@ __device__ __forceinline__ void finish_tile(const DecodeParams &p, int tile, int
             }
             v += sub;
         }
-        y[(size_t)m * p.N + n] = ActTraits<T>::from_float(v);
+        y[(size_t)m * N + n] = ActTraits<T>::from_float(v);
     }
 }
 
@@ -509,34 +515,23 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         // before the wait on the previous kernel; x (divided by the field weights, permuted
         // into fragment order) and the per-group sums P, X0 after it.  All global loads of a
         // batch are issued before the first dependent instruction. ----
-        constexpr int MB = 8;
         const int nthr = kCW * 32;
         const int mpitch = ngs | 1;                  // odd pitch: the eight rows of a warp hit different banks
-        const int nmeta = nseg * kTileRows * ngs;
-        const uint16_t *sc = reinterpret_cast<const uint16_t *>(p.scales);
-        const uint16_t *ze = reinterpret_cast<const uint16_t *>(p.zeros);
-        auto meta_batch = [&](int mbase, bool load, uint16_t (&msc)[MB], uint16_t (&mze)[MB]) {
-#pragma unroll
-            for (int i = 0; i < MB; ++i) {
-                const int idx = mbase + i * nthr + tid;
-                if (idx < nmeta) {
-                    if (load) {
-                        const int row = idx / ngs, gl = idx - row * ngs;
-                        const int n = min(tile_first * kTileRows + row, p.N - 1);
-                        const size_t mi = (size_t)n * p.G + g0 + gl;
-                        msc[i] = sc[mi];
-                        mze[i] = ze[mi];
-                    } else {
-                        const float sf = __half2float(__ushort_as_half(msc[i]));
-                        const float zf = __half2float(__ushort_as_half(mze[i]));
-                        const int row = idx / ngs, gl = idx - row * ngs;
-                        s_mf[row * mpitch + gl] = make_float2(sf, sf * zf);
-                    }
-                }
+        {
+            // (s, s*z) table: weights only, so it is filled before the wait on the previous kernel
+            const int nmeta = nseg * kTileRows * ngs;
+            const uint16_t *sc = reinterpret_cast<const uint16_t *>(p.scales);
+            const uint16_t *ze = reinterpret_cast<const uint16_t *>(p.zeros);
+#pragma unroll 4
+            for (int idx = tid; idx < nmeta; idx += nthr) {
+                const int row = idx / ngs, gl = idx - row * ngs;
+                const int n = min(tile_first * kTileRows + row, p.N - 1);
+                const size_t mi = (size_t)n * p.G + g0 + gl;
+                const float sf = __half2float(__ushort_as_half(sc[mi]));
+                const float zf = __half2float(__ushort_as_half(ze[mi]));
+                s_mf[row * mpitch + gl] = make_float2(sf, sf * zf);
             }
-        };
-        uint16_t msc0[MB], mze0[MB];
-        meta_batch(0, true, msc0, mze0);
+        }
 
         // From here on x may come from the previous kernel of the stream.
         pdl_wait();
@@ -593,12 +588,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                 xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
                 if (valid && (run & 3) == 0) s_px[(run >> 2) * mp + m] = make_float2(psum, xsum);
             }
-        }
-        meta_batch(0, false, msc0, mze0);
-        for (int mbase = MB * nthr; mbase < nmeta; mbase += MB * nthr) {
-            uint16_t msc[MB], mze[MB];
-            meta_batch(mbase, true, msc, mze);
-            meta_batch(mbase, false, msc, mze);
         }
         trace_mark(p, 4);
         bool dead = false;
@@ -737,7 +726,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     };
     // Finish `tile` from scratch slots (all contributions are there and visible).
     auto finish_from_slots = [&](int tile) {
-        finish_tile<T>(p, tile, lane, nullptr, 0, p.SK, s_t, own_b(tile));
+        finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
+                       static_cast<const T *>(p.B), p.M, p.N, p.rank, tile, lane, nullptr, 0, p.SK, s_t, own_b(tile));
         ++n_retired;
         if (p.rank == 0 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;   // nobody else will touch it again
     };
@@ -883,7 +873,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         if (cnt == 1 || others_in) {
             // This warp finishes the tile: straight from the staged sums if t is complete ...
             if (t_poll()) {
-                finish_tile<T>(p, tile, lane, s_stage, myslot, cnt, s_t, own_b(tile));
+                finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
+                               static_cast<const T *>(p.B), p.M, p.N, p.rank, tile, lane, s_stage, myslot, cnt, s_t,
+                               own_b(tile));
                 ++n_retired;
                 if (p.rank == 0 && cnt > 1 && lane == 0) p.ctr[kCtrFirstTile + tile] = 0;
                 __syncwarp();
@@ -923,31 +915,28 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         // t is normally complete within a microsecond or two of the first tiles: look a bounded
         // number of times before handing the tiles over (every CTA contributes to t before it
         // waits for anything, so this cannot block the contributors)
-        bool ready = t_poll();
+        bool ready = false;
 #pragma unroll 1
-        for (int spin = 0; spin < kTPolls && !ready; ++spin) ready = t_poll();
+        for (int spin = 0; spin <= kTPolls && !ready; ++spin) ready = t_poll();
 #pragma unroll 1
         for (int i = 0; i < n_def; ++i) {
             const int tile = s_def[i];
-            if (ready) {
-                finish_from_slots(tile);
-                continue;
-            }
-            int st = 0;
-            if (lane == 0) {
-                // park the tile, then look again: either we see the flag now, or the warp
-                // that raises it will see our entry (both sides fence in between)
-                const int idx = atomicAdd(p.ctr + kCtrPendingN, 1);
-                atomicExch(p.ctr + kCtrFirstTile + p.NT + idx, tile + 1);
+            if (!ready) {
+                int st = 0;
+                if (lane == 0) {
+                    // park the tile, then look again: either we see the flag now, or the warp
+                    // that raises it will see our entry (both sides fence in between)
+                    const int idx = atomicAdd(p.ctr + kCtrPendingN, 1);
+                    atomicExch(p.ctr + kCtrFirstTile + p.NT + idx, tile + 1);
+                    __threadfence();
+                    st = ld_acquire(p.ctr + kCtrReady);
+                }
+                st = __shfl_sync(0xffffffffu, st, 0);
+                if (!st || !tile_claim(p, tile, lane)) continue;     // parked (or already taken)
                 __threadfence();
-                st = ld_acquire(p.ctr + kCtrReady);
+                ready = t_poll();
             }
-            st = __shfl_sync(0xffffffffu, st, 0);
-            if (st && tile_claim(p, tile, lane)) {
-                __threadfence();
-                (void)t_poll();
-                finish_from_slots(tile);
-            }
+            finish_from_slots(tile);
         }
     }
     if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);

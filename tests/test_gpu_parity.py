@@ -248,6 +248,33 @@ def test_decode_many_back_to_back_launches(fbq, torch):
         assert rel <= REL_F_TOL and mx <= lim
 
 
+def test_decode_concurrent_streams(fbq, torch):
+    # Independent linears issued on several streams at once (each stream has its own scratch
+    # space), with the grid limited so that launches of different streams share the SMs: the
+    # launch configuration bench.py times.
+    inps = [make_linear(1, N, K, 3, 64, seed=600 + i) for i, (K, N) in enumerate(LLAMA2_7B_SHAPES)]
+    devs = [DeviceLinear(i, fbq) for i in inps]
+    streams = [torch.cuda.Stream() for _ in range(7)]
+    fbq.set_option("decode_ctas", 74)
+    try:
+        torch.cuda.synchronize()
+        ys = [None] * len(devs)
+        for rep in range(3):
+            for j, d in enumerate(devs):
+                i = d.inp
+                ys[j] = fbq.linear(d.x, d.qweight, d.scales, d.zeros, d.A, d.B, i.N, i.group, i.bits,
+                                   stream=streams[j % 7])
+        torch.cuda.synchronize()
+        for st in streams:
+            assert fbq.poll_status(st) == 0
+    finally:
+        fbq.set_option("decode_ctas", 0)
+    for inp, y in zip(inps, ys):
+        y_or = oracle.linear_inputs(inp, threads=8)
+        rel, mx, lim = compare(torch_to_f64(y, "f16"), y_or, inp.x_f64(), inp.K)
+        assert rel <= REL_F_TOL and mx <= lim
+
+
 # ---------------------------------------------------- workload-sized parity cases
 @pytest.mark.parametrize("shape_id", [0, 4, 6])
 def test_config1_llama7b_int3_rank64(fbq, shape_id):
