@@ -92,7 +92,7 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  * integer-valued zero points in [0, 127]; the generic kernel accepts any
  * fp16 value.  Accumulation is fp32; t = x.A^T stays fp32 in the decode and
  * generic kernels and is rounded once to the activation type in the prefill
- * kernel.  Summation order is fixed for a given shape (results are
+ * kernel (which also rounds the dequantised weights s*(q-z) once to that type).  Summation order is fixed for a given shape (results are
  * reproducible run to run) except for t in the decode kernel, which is
  * accumulated with floating-point atomics. */
 int fbq_linear(const void *x, const uint32_t *qweight, const void *scales, const void *zeros,

@@ -81,7 +81,7 @@ def test_e1_worked_example_on_gpu(fbq, torch):
 
 @pytest.mark.parametrize("bits,dtype,M,N,K,group,rank", [
     (4, "f16", 1, 40, 256, 64, 8), (3, "f16", 3, 33, 512, 32, 5), (4, "bf16", 9, 17, 128, 16, 2),
-    (3, "bf16", 20, 24, 256, 128, 0), (4, "f16", 5, 64, 512, 128, 12), (4, "f16", 1, 64, 1024, 128, 264)])
+    (3, "bf16", 20, 24, 256, 64, 0), (4, "f16", 5, 64, 512, 128, 12), (4, "f16", 1, 64, 1024, 128, 264)])
 def test_generic_kernel_parity(fbq, bits, dtype, M, N, K, group, rank):
     inp = make_linear(M, N, K, bits, rank, group=group, dtype=dtype, seed=40 + M)
     check_parity(inp, fbq, expect_kernel=fbq.KERNEL_GENERIC)
