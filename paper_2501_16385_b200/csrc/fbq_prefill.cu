@@ -4,43 +4,72 @@
 //   y = x.dequant(Q,s,z)^T + (x.A^T).B^T        (Algorithm 1 step 6 of the paper)
 //
 // At prefill the layer is a dense contraction, so it runs on the 5th-generation
-// tensor cores.  One CTA owns a 128-token x 128-row output tile.  Four producer
-// warps stream K in blocks of 64: each thread loads one token row of x and one
-// packed weight row, dequantises the codes to the activation type (s*(q-z),
-// q-z exact, one rounding) and writes both operands into shared memory in the
-// K-major core-matrix layout the MMA reads (8 rows x 16 bytes per core matrix,
-// no swizzle).  A fifth warp issues tcgen05.mma (128x128x16, fp32 accumulate in
-// 128 TMEM columns) and hands stages back through tcgen05.commit.  The low-rank
-// sub-branch is appended as extra K blocks of the same loop (Section 4.3 of the
-// paper adds the up-projection into the shared output): their "x" operand is
-// t = x.A^T, their "weight" operand is B as stored.  t itself comes from the
-// same kernel run in down-projection mode (plain fp16/bf16 rows of A as the
-// weight operand, K split over CTAs, fp32 atomics into scratch) one launch
-// earlier; it is rounded once to the activation type when it is fed to the MMA.
-// The producers' k order inside a block is permuted the same way for both
-// operands (so that one LOP3 yields a finished pair of codes); a contraction
-// does not care.  All waits are bounded.
+// tensor cores.  One CTA owns a tile of 128 weight rows x TOK tokens (TOK = 256,
+// or 128 for small M) and issues one 128 x TOK x 16 MMA per 16 elements of K:
+// the weight tile is the MMA's A operand (its rows become the 128 TMEM lanes),
+// the token tile the B operand (TOK fp32 columns).  Dequantising a weight tile
+// once per 256 tokens halves the unpack work per flop against a 128-token tile,
+// and the single wide MMA reads 96 bytes of shared memory per cycle, not 128.
+//
+// Every global read of the K loop is a TMA tensor copy (no multicast), so the
+// load/store units only see shared memory:
+//   * the token tile of a K block (64 elements of K) lands 128-byte swizzled,
+//     ready for the MMA;
+//   * the packed codes of the tile's 128 rows land, one quantisation group (two K
+//     blocks) per copy, in a small ring that runs several groups ahead;
+//   * in the sub-branch blocks the rows of B, and in down-projection mode the
+//     rows of A, land 128-byte swizzled as the weight operand itself.
+// Roles (20 warps):
+//   warps 0-15  producers of the weight operand: warps 0-7 take the even groups,
+//               warps 8-15 the odd ones; two threads per weight row, 32 codes of
+//               each of the group's two K blocks per thread.  A thread reads its
+//               words and (s, z) from the ring, dequantises to the activation type
+//               (q - z exact by the exponent trick, one rounding in the product
+//               with s), re-pairs the values into natural k order and stores them
+//               as 128-byte rows in the same 128-byte swizzle the TMA copies use
+//               (bank-conflict free for the stores and for the MMA's reads; the
+//               no-swizzle core-matrix layout halved the MMA rate).  Afterwards the same warps drain the
+//               accumulator: the tile is staged in shared memory and leaves with
+//               TMA tensor stores (epilogue).
+//   warp 16     one lane issues tcgen05.mma and hands stages back with
+//               tcgen05.commit.
+//   warp 17     one lane issues the operand-stage copies (token tile; B or A rows).
+//   warps 18-19 keep the ring full: one lane issues the copies of packed codes;
+//               all lanes read the tile's scales and zero points with 16-byte
+//               loads (one per row and eight groups), realign them and write each
+//               group's (s, z) words next to its ring slot.
+// The low-rank sub-branch is appended as extra K blocks of the same loop
+// (Section 4.3 of the paper adds the up-projection into the shared output):
+// their token operand is t = x.A^T (fp32 scratch, rounded once to the activation
+// type by the producers), their weight operand is B as stored.  t itself comes
+// from the same kernel in down-projection mode (K split over CTAs, fp32 atomics
+// into scratch) one launch earlier; the main launch may start while that one
+// drains and waits for it only before its sub-branch blocks.
+// All waits are bounded: a wait that runs out raises FBQ_ERR_TIMEOUT in the
+// status word and every role falls through to the common exit.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "fbq_common.cuh"
 
 namespace fbq {
 namespace {
 
-constexpr int kBM = 128, kBN = 128, kBK = 64;      // CTA tile (tokens, weight rows), K block
-constexpr int kStages = 4;
-constexpr int kProducers = 128;                    // threads 0..127: producers, then epilogue
-constexpr int kPfThreads = kProducers + 32;        // + the MMA warp
-constexpr uint32_t kStageBytes = 2u * kBM * kBK * 2u;          // x tile + weight tile, 16-bit elements
-constexpr uint32_t kLBO = (kBM / 8) * 128;         // bytes between the two 8-element K chunks of an MMA
-constexpr uint32_t kSBO = 128;                     // bytes between 8-row groups
+constexpr int kBN = 128;                           // weight rows per CTA tile (MMA M)
+constexpr int kBK = 64;                            // K block (one pipeline stage)
+constexpr int kStages = 4;                         // operand stages
+constexpr int kRing = 4;                           // groups of packed codes in flight
+constexpr int kProducers = 512;                    // threads 0..511: producers, then epilogue
+constexpr int kHalf = 256;                         // producers per group (two per weight row)
+constexpr int kMmaWarp = kProducers / 32, kTmaWarp = kMmaWarp + 1, kRawWarp = kMmaWarp + 2;
+constexpr int kPfThreads = kProducers + 128;         // + MMA warp, TMA warp, two ring warps
+constexpr uint32_t kWBytes = kBN * kBK * 2u;       // weight operand tile of a stage
+constexpr uint32_t kRawSlot = kBN * 64u;           // ring slot: 128 rows x one group of INT4 codes (INT3 uses 48 of 64)
 constexpr uint32_t kPfWaitLimit = 1u << 20;
-constexpr int kTmemCols = 128;
 
 struct PrefillParams {
-    const void *x;            // [M][K]
-    const uint32_t *qw;       // packed codes (mode 0)
-    const __half *scales;
+    const __half *scales;     // [N][K/128]
     const __half *zeros;
-    const void *Wplain;       // mode 1: A [rank][K];  mode 0: B [N][rank]
     float *t32;               // [M][rank] fp32: written (atomics) in mode 1, read in mode 0
     void *y;                  // [M][N] (mode 0)
     int *status;
@@ -80,13 +109,14 @@ __device__ __forceinline__ void pf_fence_proxy_async() { asm volatile("fence.pro
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Shared-memory operand descriptor: K-major, no swizzle, core matrices of 8 rows x 16 bytes.
+// Shared-memory operand descriptor: K-major tile with 128-byte rows (64 16-bit elements) in the
+// 128-byte swizzle (the 16-byte chunk c of row r is stored at chunk c ^ (r % 8)); groups of 8
+// rows are 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
 {
-    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)(kLBO >> 4) << 16) | ((uint64_t)(kSBO >> 4) << 32) |
-           (1ull << 46);
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
-// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 16, fp32 accumulate.
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, fp32 accumulate.
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
@@ -209,16 +239,16 @@ template <int BITS> __device__ __forceinline__ constexpr int pair_hi(int p)
     return 32 * r + (q == 15 ? 31 : 10 * (q / 5) + 5 + (q % 5));
 }
 
-// s*(q - z) for the 64 codes of one weight row and K block, as 32 packed pairs in the
-// order above.  q - z is exact (exponent trick, integer-valued z); the product is rounded
-// once to the activation type.  w: 8 words (INT4) or 6 words (INT3).
+// s*(q - z) for 32 consecutive codes of one weight row (half a K block), as 16 packed pairs
+// in the order above.  q - z is exact (exponent trick, integer-valued z); the product is
+// rounded once to the activation type.  w: 4 words (INT4) or one run of 3 words (INT3).
 template <int BITS, typename T> struct Dequant;
 template <> struct Dequant<4, __half> {
     static __device__ __forceinline__ void run(const uint32_t *w, float s, float z, uint32_t *out)
     {
         const uint32_t c0 = P2<__half>::splat(1024.f + z), c1 = P2<__half>::splat(-(64.f + z)), s2 = P2<__half>::splat(s);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
             const uint32_t a = w[i], b = w[i] >> 8;
             out[4 * i + 0] = P2<__half>::mul(P2<__half>::sub(pf_lop3(a, 0x000F000Fu, 0x64006400u), c0), s2);
             out[4 * i + 1] = P2<__half>::mul(P2<__half>::fma(pf_lop3(a, 0x00F000F0u, 0x64006400u), 0x2C002C00u, c1), s2);
@@ -233,7 +263,7 @@ template <> struct Dequant<4, __nv_bfloat16> {
         using P = P2<__nv_bfloat16>;
         const uint32_t c0 = P::splat(128.f + z), s2 = P::splat(s);   // 0x4300 | q is 128 + q in bf16
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int e = 0; e < 4; ++e)
                 out[4 * i + e] = P::mul(P::sub(pf_lop3(w[i] >> (4 * e), 0x000F000Fu, 0x43004300u), c0), s2);
@@ -244,10 +274,9 @@ template <> struct Dequant<3, __half> {
     {
         using P = P2<__half>;
         const uint32_t c0 = P::splat(1024.f + z), n1 = P::splat(-(128.f + z)), n2 = P::splat(-(16.f + z)), s2 = P::splat(s);
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const uint32_t *v = w + 3 * r;
-            uint32_t *o = out + 16 * r;
+        {
+            const uint32_t *v = w;
+            uint32_t *o = out;
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
                 const uint32_t a = v[i], b = v[i] >> 9;
@@ -269,10 +298,9 @@ template <> struct Dequant<3, __nv_bfloat16> {
     {
         using P = P2<__nv_bfloat16>;
         const uint32_t c0 = P::splat(128.f + z), n1 = P::splat(-(16.f + z)), s2 = P::splat(s);
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const uint32_t *v = w + 3 * r;
-            uint32_t *o = out + 16 * r;
+        {
+            const uint32_t *v = w;
+            uint32_t *o = out;
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
                 const uint32_t a = v[i], b = v[i] >> 6, c = v[i] >> 12;
@@ -290,43 +318,103 @@ template <> struct Dequant<3, __nv_bfloat16> {
     }
 };
 
-// The same pair order applied to 64 natural-order 16-bit elements (8 x uint4).
-template <int BITS> __device__ __forceinline__ void permute_pairs(const uint32_t *in /*32 words*/, uint32_t *out)
+// Where Dequant leaves element e (0..31, natural k order) of its 32 codes: register and half.
+template <int BITS> __device__ __forceinline__ constexpr int elem_reg(int e)
+{
+    if (BITS == 4) return 4 * (e / 8) + (e % 4);                       // word e/8: pairs (j, j+4)
+    const int r = e / 32, q = e % 32;                                  // run r of 32 codes
+    return 16 * r + (q >= 30 ? 15 : 5 * (q / 10) + (q % 10) % 5);
+}
+template <int BITS> __device__ __forceinline__ constexpr int elem_half(int e)
+{
+    if (BITS == 4) return (e % 8) / 4;
+    const int q = e % 32;
+    return q >= 30 ? q - 30 : (q % 10) / 5;
+}
+// Re-pair the 32 dequantised values into natural order: word p = elements (2p, 2p+1).
+template <int BITS> __device__ __forceinline__ void natural_pairs(const uint32_t *d /*16*/, uint32_t *out /*16*/)
 {
 #pragma unroll
-    for (int p = 0; p < 32; ++p) {
-        const int lo = pair_lo<BITS>(p), hi = pair_hi<BITS>(p);
-        const uint32_t sel = ((hi & 1) ? 0x7600u : 0x5400u) | ((lo & 1) ? 0x32u : 0x10u);
-        out[p] = pf_prmt(in[lo >> 1], in[hi >> 1], sel);
+    for (int p = 0; p < 16; ++p) {
+        const int a = elem_reg<BITS>(2 * p), ha = elem_half<BITS>(2 * p);
+        const int b = elem_reg<BITS>(2 * p + 1), hb = elem_half<BITS>(2 * p + 1);
+        out[p] = pf_prmt(d[a], d[b], (hb ? 0x7600u : 0x5400u) | (ha ? 0x32u : 0x10u));
     }
 }
 
-// One 64-element row of an operand tile goes to 8 core-matrix chunks of 16 bytes:
-// chunk kc of row r lives at  kc*kLBO + (r/8)*kSBO + (r%8)*16.
-__device__ __forceinline__ void store_row(uint8_t *tile, int r, const uint32_t *words /*32*/)
+template <typename T> __device__ __forceinline__ unsigned short to_bits16(float v)
 {
-    uint8_t *base = tile + (r >> 3) * kSBO + (r & 7) * 16;
-#pragma unroll
-    for (int kc = 0; kc < 8; ++kc)
-        *reinterpret_cast<uint4 *>(base + kc * kLBO) =
-            make_uint4(words[4 * kc], words[4 * kc + 1], words[4 * kc + 2], words[4 * kc + 3]);
+    return (unsigned short)(P2<T>::pack(v, 0.f) & 0xFFFFu);
 }
 
 // --------------------------------------------------------------------- kernel
-// MODE 0: y tile = x.dequant(W)^T + t.B^T  (grid: N tiles x M tiles)
-// MODE 1: t32 += x.A^T over this CTA's K range (grid: K splits x M tiles), fp32 atomics
-template <int MODE, int BITS, typename T>
-__global__ void __launch_bounds__(kPfThreads, 1) prefill_kernel(const PrefillParams p)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void pf_mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// Shared-memory map of a CTA (byte offsets from the 1024-byte aligned base)
+template <int MODE, int TOK> struct Smem {
+    static constexpr uint32_t kXBytes = (uint32_t)TOK * kBK * 2u;          // token operand tile of a stage
+    static constexpr uint32_t kStageBytes = kXBytes + kWBytes;
+    static constexpr uint32_t kRingOff = kStages * kStageBytes;
+    static constexpr uint32_t kTableOff = kRingOff + (MODE == 0 ? kRing * kRawSlot : 0u);
+    static constexpr uint32_t kBarOff = kTableOff + (MODE == 0 ? kRing * kBN * 4u : 0u);
+    static constexpr uint32_t kNumBars = 2 * kStages + 2 * kRing + 1 + 4;  // full, empty, ring full, ring empty, done, epilogue
+    static constexpr uint32_t kTotal = kBarOff + kNumBars * 8u + 16u;
+};
+
+// MODE 0: y tile = x.dequant(W)^T + t.B^T  (grid: N tiles x token tiles)
+// MODE 1: t32 += x.A^T over this CTA's K range (grid: K splits x token tiles x rank tiles), fp32 atomics
+// xmap: x [M][K], boxes of TOK rows x 64 elements, 128-byte swizzle
+// wmap: mode 0: packed codes [N][words per row], boxes of 128 rows x one group (64-byte swizzle for INT4);
+//       mode 1: A [rank][K], boxes of 128 rows x 64 elements, 128-byte swizzle
+// bmap: mode 0, rank > 0: B [N][rank], boxes of 128 rows x 64 elements, 128-byte swizzle
+// ymap: mode 0: y [M][N], boxes of TOK/4 rows x 128 elements, no swizzle (stores)
+template <int MODE, int BITS, typename T, int TOK>
+__global__ void __launch_bounds__(kPfThreads, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
+               const __grid_constant__ CUtensorMap bmap, const __grid_constant__ CUtensorMap ymap, const PrefillParams p)
+{
+    using L = Smem<MODE, TOK>;
+    constexpr uint32_t kXBytes = L::kXBytes, kStageBytes = L::kStageBytes;
+    constexpr int WPG = (BITS == 4) ? 16 : 12;                  // packed words per row and group
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint8_t *stages = smem;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kStages * kStageBytes);
-    const uint32_t full0 = pf_smem_u32(bars), empty0 = full0 + 8u * kStages, done_bar = empty0 + 8u * kStages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 1);
+    const uint32_t sbase = pf_smem_u32(smem);
+    if (sbase & 1023u) {                                        // swizzle atoms need a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicExch(p.status, (int)FBQ_ERR_CUDA);
+        return;
+    }
+    const uint32_t full0 = sbase + L::kBarOff, empty0 = full0 + 8u * kStages, rfull0 = empty0 + 8u * kStages,
+                   rempty0 = rfull0 + 8u * kRing, done_bar = rempty0 + 8u * kRing, epi0 = done_bar + 8u;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + L::kNumBars * 8u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.y * kBM;
+    const int m0 = blockIdx.y * TOK;
     const int n0 = (MODE == 0) ? blockIdx.x * kBN : blockIdx.z * kBN;   // mode 1: tile of rank rows of A
     int kb_begin = 0, kb_end = p.kb_main + p.kb_slab;
     if (MODE == 1) {
@@ -334,169 +422,201 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_kernel(const PrefillPar
         kb_end = (int)((long long)(blockIdx.x + 1) * p.kb_main / p.splitk);
     }
     const int nkb = kb_end - kb_begin;
+    const int kb_x = (MODE == 1) ? kb_end : p.kb_main;          // blocks below kb_x take their tokens from x
+    if (MODE == 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may start its K loop
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
-            pf_mbar_init(full0 + 8u * i, kProducers);
+            pf_mbar_init(full0 + 8u * i, (MODE == 0) ? kHalf + 1 : 1);   // 256 producers + the TMA lane
             pf_mbar_init(empty0 + 8u * i, 1);
         }
+        for (int i = 0; i < kRing; ++i) {
+            pf_mbar_init(rfull0 + 8u * i, 2);                   // the two ring warps
+            pf_mbar_init(rempty0 + 8u * i, kHalf);              // a group is consumed by one half of the producers
+        }
         pf_mbar_init(done_bar, 1);
+        for (int i = 0; i < 4; ++i) pf_mbar_init(epi0 + 8u * i, 128);     // the four warps of a column quarter
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kProducers / 32) {           // the MMA warp owns the tensor-memory allocation
+    if (warp == kMmaWarp) {                  // the MMA warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(pf_smem_u32(tmem_slot)),
-                     "r"((uint32_t)kTmemCols)
+                     "r"((uint32_t)TOK)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         tc_fence_before();
     }
+    if (warp == kTmaWarp && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&xmap)) : "memory");
+        if (MODE == 0 && p.rank > 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&bmap)) : "memory");
+        if (MODE == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ymap)) : "memory");
+    }
+    if (warp == kRawWarp && lane == 0)
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&wmap)) : "memory");
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp < kProducers / 32) {
-        // =================================================== producers
-        const int r = tid;                                  // row of both operand tiles
-        const T *x = static_cast<const T *>(p.x);
-        const int G = p.K / kGroupFast;
+    if (warp < kMmaWarp) {
         bool dead = false;
+        if (MODE == 0) {
+            // =================================================== producers
+            // Half h of the warps takes the groups g = h, h+2, ... (K blocks 2g and 2g+1, stages 2h
+            // and 2h+1); thread (row r, part) dequantises the codes [32*part, +32) of both blocks.
+            const int h = warp >> 3, part = (warp >> 2) & 1, r = tid & 127;
+            const bool row_ok = n0 + r < p.N;
+            const int groups = p.kb_main >> 1;
+            // this thread's words inside a ring slot: block b holds codes [64b, 64b+64) of the group
+            uint32_t roff0, roff1;
+            if (BITS == 4) {                                // 64-byte rows, 16-byte chunk c stored at c ^ ((row / 2) % 4)
+                const uint32_t sw = (uint32_t)(r >> 1) & 3u;
+                roff0 = (uint32_t)r * 64u + ((((uint32_t)part) ^ sw) << 4);
+                roff1 = (uint32_t)r * 64u + ((((uint32_t)part + 2u) ^ sw) << 4);
+            } else {                                        // 48-byte rows of four 12-byte runs
+                roff0 = (uint32_t)r * 48u + (uint32_t)part * 12u;
+                roff1 = roff0 + 24u;
+            }
+            const uint32_t ring0 = sbase + L::kRingOff, table0 = sbase + L::kTableOff + (uint32_t)r * 4u;
+            // weight tile rows are 128 bytes (64 elements); the 16-byte chunk c of row r sits at c ^ (r % 8)
+            const uint32_t wdst = sbase + kXBytes + (uint32_t)(2 * h) * kStageBytes + (uint32_t)r * 128u;
+            const uint32_t wsw = (uint32_t)r & 7u;
+            const uint32_t fullb = full0 + 16u * h, emptyb = empty0 + 16u * h;
+            uint32_t slot = (uint32_t)h, rphase = 0u, ephase = 0u;
 #pragma unroll 1
-        for (int i = 0; i < nkb && !dead; ++i) {
-            const int kb = kb_begin + i, s = i % kStages;
-            if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) {
-                dead = true;
-                break;
+            for (int g = h; g < groups; g += 2) {
+                if (!pf_mbar_wait(rfull0 + 8u * slot, rphase)) { dead = true; break; }
+                constexpr int NW = (BITS == 4) ? 4 : 3;
+                uint32_t w[2][NW];
+                const uint32_t rs = ring0 + slot * kRawSlot;
+                if (BITS == 4) {
+                    const uint4 a = lds128(rs + roff0), b = lds128(rs + roff1);
+                    w[0][0] = a.x; w[0][1] = a.y; w[0][2] = a.z; w[0][NW - 1] = a.w;
+                    w[1][0] = b.x; w[1][1] = b.y; w[1][2] = b.z; w[1][NW - 1] = b.w;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        w[0][c] = lds32(rs + roff0 + 4u * c);
+                        w[1][c] = lds32(rs + roff1 + 4u * c);
+                    }
+                }
+                const uint32_t sz = lds32(table0 + slot * (kBN * 4u));      // s | z << 16 of (row, group)
+                pf_mbar_arrive(rempty0 + 8u * slot);         // everything is in registers: the slot may be refilled
+                slot += 2u;
+                if (slot >= (uint32_t)kRing) { slot -= (uint32_t)kRing; rphase ^= 1u; }
+                const float sc = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
+                const float ze = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    if (g >= 2 && !pf_mbar_wait(emptyb + 8u * b, ephase)) { dead = true; break; }
+                    uint32_t wb[16];
+                    if (row_ok) {
+                        uint32_t d[16];
+                        Dequant<BITS, T>::run(w[b], sc, ze, d);
+                        natural_pairs<BITS>(d, wb);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) wb[c] = 0u;
+                    }
+#pragma unroll
+                    for (int kc = 0; kc < 4; ++kc)
+                        sts128(wdst + (uint32_t)b * kStageBytes + ((((uint32_t)(4 * part + kc)) ^ wsw) << 4), wb[4 * kc], wb[4 * kc + 1], wb[4 * kc + 2],
+                               wb[4 * kc + 3]);
+                    pf_fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
+                    pf_mbar_arrive(fullb + 8u * b);
+                }
+                if (dead) break;
+                if (g >= 2) ephase ^= 1u;
             }
-            if (*abort_flag) {
-                dead = true;
-                break;
-            }
-            uint32_t xa[32], wb[32];
-            const int m = m0 + r;
-            if (MODE == 1 || kb < p.kb_main) {
-                uint32_t in[32];
-                if (m < p.M) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + (size_t)kb * kBK);
+            // ---- sub-branch blocks: token operand = t (fp32 scratch, rounded once); B arrives by TMA.
+            // The halves take them in turn, one token row per thread.
+#pragma unroll 1
+            for (int i = p.kb_main + h; i < nkb && !dead; i += 2) {
+                const int s = i % kStages;
+                if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
+                asm volatile("griddepcontrol.wait;" ::: "memory");          // t is complete once the down-projection has ended
+                const int j0 = (i - p.kb_main) * kBK;
+                const int rr = tid & (kHalf - 1);            // token row of the tile
+                if (rr < TOK) {
+                    const int m = m0 + rr;
+                    uint32_t xa[32];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const uint4 v = __ldg(src + c);
-                        in[4 * c] = v.x; in[4 * c + 1] = v.y; in[4 * c + 2] = v.z; in[4 * c + 3] = v.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) in[c] = 0u;
-                }
-                if (MODE == 0) {
-                    permute_pairs<BITS>(in, xa);
-                    const int n = n0 + r;
-                    if (n < p.N) {
-                        constexpr int NW = (BITS == 4) ? 8 : 6;
-                        uint32_t w[NW];
-                        const uint32_t *src = p.qw + ((size_t)n * (p.K / kBK) + kb) * NW;
-                        if (BITS == 4) {
-                            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src)), b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
-                            w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[NW - 2] = b.z; w[NW - 1] = b.w;
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 3; ++c) {
-                                const uint2 a = __ldg(reinterpret_cast<const uint2 *>(src) + c);
-                                w[2 * c] = a.x; w[2 * c + 1] = a.y;
-                            }
-                        }
-                        const float sc = __half2float(p.scales[(size_t)n * G + kb / 2]);
-                        const float ze = __half2float(p.zeros[(size_t)n * G + kb / 2]);
-                        Dequant<BITS, T>::run(w, sc, ze, wb);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) wb[c] = 0u;
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) xa[c] = in[c];
-                    if (n0 + r < p.rank) {                  // rows of A are the "weight" rows
-                        const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const T *>(p.Wplain) + (size_t)(n0 + r) * p.K + (size_t)kb * kBK);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const uint4 v = __ldg(src + c);
-                            wb[4 * c] = v.x; wb[4 * c + 1] = v.y; wb[4 * c + 2] = v.z; wb[4 * c + 3] = v.w;
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) wb[c] = 0u;
-                    }
-                }
-            } else {
-                // sub-branch block: x operand = t (fp32 scratch, rounded once), weight operand = B as stored
-                const int j0 = (kb - p.kb_main) * kBK;
-                const int n = n0 + r;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int j = j0 + 8 * c;
-                    uint4 bv = make_uint4(0u, 0u, 0u, 0u);
-                    float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f), t1 = t0;
-                    if (j < p.rank) {                       // rank is a multiple of 8: whole chunks
-                        if (n < p.N) bv = __ldg(reinterpret_cast<const uint4 *>(static_cast<const T *>(p.Wplain) + (size_t)n * p.rank + j));
-                        if (m < p.M) {
-                            const float4 *ts = reinterpret_cast<const float4 *>(p.t32 + (size_t)m * p.rank + j);
+                        float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f), t1 = t0;
+                        if (m < p.M && j0 + 8 * c < p.rank) {              // rank is a multiple of 8: whole chunks
+                            const float4 *ts = reinterpret_cast<const float4 *>(p.t32 + (size_t)m * p.rank + j0 + 8 * c);
                             t0 = __ldcg(ts);
                             t1 = __ldcg(ts + 1);
                         }
+                        xa[4 * c] = P2<T>::pack(t0.x, t0.y); xa[4 * c + 1] = P2<T>::pack(t0.z, t0.w);
+                        xa[4 * c + 2] = P2<T>::pack(t1.x, t1.y); xa[4 * c + 3] = P2<T>::pack(t1.z, t1.w);
                     }
-                    wb[4 * c] = bv.x; wb[4 * c + 1] = bv.y; wb[4 * c + 2] = bv.z; wb[4 * c + 3] = bv.w;
-                    xa[4 * c] = P2<T>::pack(t0.x, t0.y); xa[4 * c + 1] = P2<T>::pack(t0.z, t0.w);
-                    xa[4 * c + 2] = P2<T>::pack(t1.x, t1.y); xa[4 * c + 3] = P2<T>::pack(t1.z, t1.w);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        sts128(sbase + (uint32_t)s * kStageBytes + (uint32_t)rr * 128u + ((((uint32_t)c) ^ ((uint32_t)rr & 7u)) << 4), xa[4 * c],
+                               xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
                 }
+                pf_fence_proxy_async();
+                pf_mbar_arrive(full0 + 8u * s);
             }
-            uint8_t *st = stages + (size_t)s * kStageBytes;
-            store_row(st, r, xa);
-            store_row(st + kBM * kBK * 2, r, wb);
-            pf_fence_proxy_async();                         // generic-proxy stores -> visible to the MMA's reads
-            pf_mbar_arrive(full0 + 8u * s);
-        }
-        if (dead) {
-            *abort_flag = 1;
-            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            if (dead) {
+                *abort_flag = 1;
+                atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            }
         }
 
-        // =================================================== epilogue (same four warps)
+        // =================================================== epilogue (same sixteen warps)
+        // TMEM lane = weight row of the tile, column = token.  Warp w reads lanes 32*(w%4)..+31
+        // (the only ones it may address) and the quarter w/4 of the columns.  Mode 0 stages the
+        // tile in shared memory as [token][128 features] (the operand stages are free by now) and
+        // each column quarter leaves with one TMA tensor store, which also clips the ragged edges.
         if (!dead && nkb > 0 && pf_mbar_wait(done_bar, 0)) {
             tc_fence_after();
-            const int m = m0 + 32 * warp + lane;            // TMEM lane = token row of the tile
+            const int q = warp & 3, cg = warp >> 2;
+            const int nn = n0 + 32 * q + lane;              // output feature (mode 0) / rank index (mode 1)
+            const int c_begin = cg * (TOK / 4);
+            if (m0 + c_begin < p.M) {                       // uniform over the four warps of a column quarter
 #pragma unroll 1
-            for (int c = 0; c < kBN / 32; ++c) {
-                uint32_t v[32];
-                tc_ld32(tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(32 * c), v);
-                tc_wait_ld();
-                if (m < p.M) {
+                for (int c = c_begin; c < c_begin + TOK / 4; c += 32) {
+                    if (m0 + c >= p.M) break;               // warp-uniform
+                    uint32_t v[32];
+                    tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+                    tc_wait_ld();
                     if (MODE == 0) {
-                        T *yrow = static_cast<T *>(p.y) + (size_t)m * p.N + n0 + 32 * c;
+                        unsigned short *sp = reinterpret_cast<unsigned short *>(smem + (size_t)c * (kBN * 2)) + 32 * q + lane;
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            if (n0 + 32 * c + 8 * q < p.N) {     // N is a multiple of 8
-                                uint4 o;
-                                o.x = P2<T>::pack(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
-                                o.y = P2<T>::pack(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
-                                o.z = P2<T>::pack(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
-                                o.w = P2<T>::pack(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
-                                *reinterpret_cast<uint4 *>(yrow + 8 * q) = o;
-                            }
-                        }
+                        for (int j = 0; j < 32; ++j) sp[j * kBN] = to_bits16<T>(__uint_as_float(v[j]));
                     } else {
+                        if (nn < p.rank) {
+                            float *tp = p.t32 + (size_t)(m0 + c) * p.rank + nn;
 #pragma unroll
-                        for (int q = 0; q < 32; ++q) {
-                            const int j = n0 + 32 * c + q;
-                            if (j < p.rank) atomicAdd(p.t32 + (size_t)m * p.rank + j, __uint_as_float(v[q]));
+                            for (int j = 0; j < 32; ++j)
+                                if (m0 + c + j < p.M) atomicAdd(tp + (size_t)j * p.rank, __uint_as_float(v[j]));
+                        }
+                    }
+                }
+                if (MODE == 0) {
+                    pf_fence_proxy_async();                 // staged tile -> visible to the TMA store
+                    pf_mbar_arrive(epi0 + 8u * cg);
+                    if (q == 0 && lane == 0) {
+                        if (pf_mbar_wait(epi0 + 8u * cg, 0)) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&ymap)), "r"(n0), "r"(m0 + c_begin),
+                                           "r"(sbase + (uint32_t)c_begin * (kBN * 2))
+                                         : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem may go once it has been read
+                        } else {
+                            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
                         }
                     }
                 }
             }
         }
         tc_fence_before();
-    } else {
+    } else if (warp == kMmaWarp) {
         // =================================================== MMA warp
-        constexpr uint32_t idesc = (1u << 4) | (P2<T>::kFmt << 7) | (P2<T>::kFmt << 10) | ((uint32_t)(kBN >> 3) << 17) |
-                                   ((uint32_t)(kBM >> 4) << 24);
+        constexpr uint32_t idesc = (1u << 4) | (P2<T>::kFmt << 7) | (P2<T>::kFmt << 10) | ((uint32_t)(TOK >> 3) << 17) |
+                                   ((uint32_t)(kBN >> 4) << 24);
         bool dead = false;
 #pragma unroll 1
         for (int i = 0; i < nkb && !dead; ++i) {
@@ -506,11 +626,12 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_kernel(const PrefillPar
                     dead = true;
                 } else {
                     tc_fence_after();
-                    const uint32_t a_base = pf_smem_u32(stages + (size_t)s * kStageBytes), b_base = a_base + kBM * kBK * 2;
+                    const uint32_t x_base = sbase + (uint32_t)s * kStageBytes, w_base = x_base + kXBytes;
+                    // every operand tile is K-major with 128-byte rows and the 128-byte swizzle, whether it
+                    // arrived by TMA or was written by the producers: 32 bytes per 16 elements of K inside a row
 #pragma unroll
                     for (int j = 0; j < kBK / 16; ++j)
-                        tc_mma(tmem_base, make_desc(a_base + j * 2 * kLBO), make_desc(b_base + j * 2 * kLBO), idesc,
-                               (i > 0 || j > 0) ? 1u : 0u);
+                        tc_mma(tmem_base, make_desc(w_base + j * 32), make_desc(x_base + j * 32), idesc, (i > 0 || j > 0) ? 1u : 0u);
                     tc_commit(empty0 + 8u * s);              // stage is free once these MMAs have read it
                 }
             }
@@ -526,36 +647,194 @@ __global__ void __launch_bounds__(kPfThreads, 1) prefill_kernel(const PrefillPar
         }
         __syncwarp();
         tc_fence_before();
+    } else if (warp == kTmaWarp) {
+        // =================================================== operand-stage copies
+        if (lane == 0) {
+            bool dead = false;
+#pragma unroll 1
+            for (int i = 0; i < nkb; ++i) {
+                const int kb = kb_begin + i, s = i % kStages;
+                if ((i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) || *abort_flag) {
+                    dead = true;
+                    break;
+                }
+                const uint32_t bar = full0 + 8u * s;
+                const uint32_t xt = sbase + (uint32_t)s * kStageBytes, wt = xt + kXBytes;
+                if (MODE == 1) {
+                    pf_mbar_expect_tx(bar, kXBytes + kWBytes);
+                    tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
+                    tma_load_2d(wt, &wmap, kb * kBK, n0, bar);      // rows of A
+                } else if (kb < kb_x) {
+                    pf_mbar_expect_tx(bar, kXBytes);
+                    tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
+                } else {
+                    pf_mbar_expect_tx(bar, kWBytes);
+                    tma_load_2d(wt, &bmap, (kb - p.kb_main) * kBK, n0, bar);   // rows of B
+                }
+            }
+            if (dead) {
+                *abort_flag = 1;
+                atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);   // let the copies in flight land before the CTA exits
+            }
+        }
+        __syncwarp();
+    } else if (MODE == 0) {
+        // =================================================== ring of packed codes and (s, z) table
+        // Two warps; lane l of ring warp v owns the tile rows 64v + l and 64v + l + 32.  Per chunk of
+        // eight groups it reads the rows' scales and zero points with 16-byte loads (two aligned chunks of the flat row-major arrays
+        // cover any eight consecutive values), realigns them in registers, and before each group's
+        // copy writes that group's (s | z << 16) words next to the ring slot.
+        const int G = p.K / kGroupFast, groups = p.kb_main >> 1;
+        const size_t n_chunks = (size_t)p.N * G / 8;        // N is a multiple of 8
+        const uint4 *s_arr = reinterpret_cast<const uint4 *>(p.scales), *z_arr = reinterpret_cast<const uint4 *>(p.zeros);
+        const int v = warp - kRawWarp;
+        size_t a0[2];                                       // aligned 16-byte chunk holding group 0 of the row
+        uint32_t off[2];                                    // position of group 0 inside that chunk (0..7)
+        bool ok[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int n = n0 + 64 * v + lane + 32 * k;
+            ok[k] = n < p.N;
+            const size_t f = (size_t)(ok[k] ? n : 0) * G;
+            a0[k] = f >> 3;
+            off[k] = (uint32_t)f & 7u;
+        }
+        uint4 raw[2][2][2];                                 // [row][s|z][low|high chunk] of the next eight groups
+        auto fetch = [&](int c) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const size_t a = a0[k] + (size_t)c;
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                raw[k][0][0] = (ok[k] && a < n_chunks) ? __ldg(s_arr + a) : zero;
+                raw[k][1][0] = (ok[k] && a < n_chunks) ? __ldg(z_arr + a) : zero;
+                raw[k][0][1] = (ok[k] && a + 1 < n_chunks) ? __ldg(s_arr + a + 1) : zero;
+                raw[k][1][1] = (ok[k] && a + 1 < n_chunks) ? __ldg(z_arr + a + 1) : zero;
+            }
+        };
+        // eight consecutive fp16 values starting `o` values into the 16-value window (lo, hi), as 4 pair-words
+        auto realign = [](const uint4 &lo, const uint4 &hi, uint32_t o, uint32_t (&out)[4]) {
+            uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            if (o & 2u) {
+#pragma unroll
+                for (int i = 0; i < 7; ++i) w[i] = w[i + 1];
+            }
+            if (o & 4u) {
+#pragma unroll
+                for (int i = 0; i < 5; ++i) w[i] = w[i + 2];
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) out[t] = __funnelshift_r(w[t], w[t + 1], (o & 1u) * 16u);
+        };
+        bool dead = false;
+        fetch(0);
+        const uint32_t ring0 = sbase + L::kRingOff, table0 = sbase + L::kTableOff + (uint32_t)(64 * v + lane) * 4u;
+#pragma unroll 1
+        for (int c = 0; 8 * c < groups && !dead; ++c) {
+            uint32_t sz[2][8];                              // (s | z << 16) of [row][group of this chunk]
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                uint32_t sp[4], zp[4];
+                realign(raw[k][0][0], raw[k][0][1], off[k], sp);
+                realign(raw[k][1][0], raw[k][1][1], off[k], zp);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    sz[k][2 * t] = pf_prmt(sp[t], zp[t], 0x5410u);
+                    sz[k][2 * t + 1] = pf_prmt(sp[t], zp[t], 0x7632u);
+                }
+            }
+            if (8 * (c + 1) < groups) fetch(c + 1);
+#pragma unroll
+            for (int g8 = 0; g8 < 8; ++g8) {
+                const int gi = 8 * c + g8;
+                if (gi < groups && !dead) {
+                    const uint32_t slot = (uint32_t)gi % kRing;
+                    if (lane == 0 && ((gi >= kRing && !pf_mbar_wait(rempty0 + 8u * slot, (uint32_t)(gi / kRing - 1) & 1u)) || *abort_flag))
+                        dead = true;
+                    dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;     // also orders the table writes after the wait
+                    if (!dead) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(table0 + slot * (kBN * 4u) + 128u * k), "r"(sz[k][g8]) : "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (v == 0) {
+                                pf_mbar_expect_tx(rfull0 + 8u * slot, (uint32_t)kBN * WPG * 4u);
+                                tma_load_2d(ring0 + slot * kRawSlot, &wmap, gi * WPG, n0, rfull0 + 8u * slot);
+                            } else {
+                                pf_mbar_arrive(rfull0 + 8u * slot);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if (dead && lane == 0) {
+            *abort_flag = 1;
+            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        }
+        __syncwarp();
     }
     __syncthreads();
-    if (warp == kProducers / 32) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TOK) : "memory");
     }
 }
 
-constexpr size_t kPfSmem = (size_t)kStages * kStageBytes + (2 * kStages + 1) * 8 + 16;
-
-template <int MODE, int BITS, typename T>
-cudaError_t launch_mode(const PrefillParams &p, dim3 grid, cudaStream_t s)
+template <int MODE, int BITS, typename T, int TOK>
+cudaError_t launch_mode(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &ymap, const PrefillParams &p,
+                        dim3 grid, cudaStream_t s, bool overlap_previous)
 {
-    auto kern = prefill_kernel<MODE, BITS, T>;
+    auto kern = prefill_kernel<MODE, BITS, T, TOK>;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPfSmem);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem<MODE, TOK>::kTotal);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    kern<<<grid, kPfThreads, kPfSmem, s>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kPfThreads);
+    cfg.dynamicSmemBytes = Smem<MODE, TOK>::kTotal;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = overlap_previous ? 1 : 0;       // may start while the previous kernel drains
+    return cudaLaunchKernelEx(&cfg, kern, xmap, wmap, bmap, ymap, p);
 }
 
-template <typename T>
+// 2-D tensor map of a row-major matrix: `cols` elements per row (16- or 32-bit), `rows` rows,
+// boxes of box_cols x box_rows.  Reads outside the matrix return zero.
+cudaError_t make_map(CUtensorMap *map, const void *base, bool elem32, size_t cols, size_t rows, int box_cols, int box_rows,
+                     CUtensorMapSwizzle swizzle)
+{
+    static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * (elem32 ? 4 : 2)};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(map, elem32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2,
+                              const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <typename T, int TOK>
 cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches)
 {
     PrefillParams p{};
-    p.x = a.x;
-    p.qw = a.qw;
     p.scales = a.scales;
     p.zeros = a.zeros;
     p.t32 = ws.t_gen;
@@ -564,37 +843,58 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
     p.M = a.M; p.N = a.N; p.K = a.K; p.rank = a.rank;
     p.kb_main = a.K / kBK;
     p.kb_slab = (a.rank + kBK - 1) / kBK;
-    const unsigned mt = (unsigned)((a.M + kBM - 1) / kBM), nt = (unsigned)((a.N + kBN - 1) / kBN);
+    CUtensorMap xmap, qmap, amap, bmap, ymap;
     cudaError_t e;
+    if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
+    const int wpg = (a.bits == 4) ? 16 : 12;
+    if ((e = make_map(&qmap, a.qw, true, (size_t)(a.K / kGroupFast) * wpg, (size_t)a.N, wpg, kBN,
+                      a.bits == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess)
+        return e;
+    if ((e = make_map(&ymap, a.y, false, (size_t)a.N, (size_t)a.M, kBN, TOK / 4, CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess) return e;
+    bmap = xmap;
+    const unsigned mt = (unsigned)((a.M + TOK - 1) / TOK), nt = (unsigned)((a.N + kBN - 1) / kBN);
     if (a.rank > 0) {
+        if ((e = make_map(&amap, a.A, false, (size_t)a.K, (size_t)a.rank, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
+        if ((e = make_map(&bmap, a.B, false, (size_t)a.rank, (size_t)a.N, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
         // t = x.A^T into fp32 scratch: K split so that about one CTA per SM is busy
         if ((e = cudaMemsetAsync(ws.t_gen, 0, sizeof(float) * (size_t)a.M * a.rank, s)) != cudaSuccess) return e;
-        p.Wplain = a.A;
-        p.splitk = (int)max(1u, min((unsigned)p.kb_main, 148u / mt));
-        e = launch_mode<1, 4, T>(p, dim3((unsigned)p.splitk, mt, (unsigned)((a.rank + kBN - 1) / kBN)), s);
+        const unsigned rt = (unsigned)((a.rank + kBN - 1) / kBN);
+        p.splitk = (int)max(1u, min((unsigned)p.kb_main, 148u / (mt * rt)));
+        e = launch_mode<1, 4, T, TOK>(xmap, amap, amap, amap, p, dim3((unsigned)p.splitk, mt, rt), s, false);
         if (e != cudaSuccess) return e;
         ++*launches;
     }
-    p.Wplain = a.B;
     p.splitk = 1;
-    e = (a.bits == 4) ? launch_mode<0, 4, T>(p, dim3(nt, mt), s) : launch_mode<0, 3, T>(p, dim3(nt, mt), s);
+    // The main launch may overlap the tail of the down-projection: it waits for t only before
+    // its sub-branch blocks.
+    const bool pdl = a.rank > 0;
+    e = (a.bits == 4) ? launch_mode<0, 4, T, TOK>(xmap, qmap, bmap, ymap, p, dim3(nt, mt), s, pdl)
+                      : launch_mode<0, 3, T, TOK>(xmap, qmap, bmap, ymap, p, dim3(nt, mt), s, pdl);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
+
+inline bool aligned16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
 
 }  // namespace
 
 bool prefill_supported(const LinearArgs &a)
 {
     return a.group == kGroupFast && a.K % kGroupFast == 0 && a.rank % 8 == 0 && a.rank <= kMaxRank && a.N % 8 == 0 &&
-           a.M >= 1 && a.M <= 65535 * kBM;
+           a.M >= 1 && a.M <= 65535 * 128;
 }
 
 // ws.t_gen must hold M x rank floats and ws.counters at least 8 ints (the caller grows them).
+// Operands that are not 16-byte aligned are refused (the caller then takes the generic kernel).
 cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches)
 {
     if (!prefill_supported(a)) return cudaErrorInvalidConfiguration;
-    return a.bf16 ? run_prefill<__nv_bfloat16>(a, ws, s, launches) : run_prefill<__half>(a, ws, s, launches);
+    if (!aligned16(a.x) || !aligned16(a.y) || !aligned16(a.qw) || !aligned16(a.scales) || !aligned16(a.zeros) ||
+        (a.rank > 0 && (!aligned16(a.A) || !aligned16(a.B))))
+        return cudaErrorInvalidConfiguration;
+    if (a.M <= 128)
+        return a.bf16 ? run_prefill<__nv_bfloat16, 128>(a, ws, s, launches) : run_prefill<__half, 128>(a, ws, s, launches);
+    return a.bf16 ? run_prefill<__nv_bfloat16, 256>(a, ws, s, launches) : run_prefill<__half, 256>(a, ws, s, launches);
 }
 
 }  // namespace fbq
