@@ -133,7 +133,7 @@ int run_linear(const LinearArgs &a, cudaStream_t s)
     }
     if (kernel == FBQ_KERNEL_PREFILL) {
         size_t have_c = (size_t)ws->n_counters;
-        if ((e = grow(ws->counters, have_c, (size_t)64, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->counters, have_c, (size_t)prefill_counters_need(a.M), sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         ws->n_counters = (int)have_c;
         if (a.rank > 0 &&
             (e = grow(ws->t_gen, ws->t_gen_floats, (size_t)a.M * a.rank, sizeof(float), s)) != cudaSuccess)

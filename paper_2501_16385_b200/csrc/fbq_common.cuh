@@ -74,6 +74,7 @@ void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t
                            int *counters);
 
 bool prefill_supported(const LinearArgs &a);
+int prefill_counters_need(int M);
 cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
 
 }  // namespace fbq

@@ -65,18 +65,24 @@ constexpr int kMmaWarp = kProducers / 32, kTmaWarp = kMmaWarp + 1, kRawWarp = kM
 constexpr int kPfThreads = kProducers + 128;         // + MMA warp, TMA warp, two ring warps
 constexpr uint32_t kWBytes = kBN * kBK * 2u;       // weight operand tile of a stage
 constexpr uint32_t kRawSlot = kBN * 64u;           // ring slot: 128 rows x one group of INT4 codes (INT3 uses 48 of 64)
+constexpr int kPfCtrBase = 8;                      // first int of the workspace counters used for the t flags
 constexpr uint32_t kPfWaitLimit = 1u << 20;
+constexpr uint32_t kPfFlagPolls = 1u << 21;        // polls (256 ns apart) of a token tile's t flag: about half a second
 
 struct PrefillParams {
     const __half *scales;     // [N][K/128]
     const __half *zeros;
-    float *t32;               // [M][rank] fp32: written (atomics) in mode 1, read in mode 0
-    void *y;                  // [M][N] (mode 0)
+    float *t32;               // [M][rank] fp32 scratch: written by the t CTAs, read by the main CTAs
+    void *y;                  // [M][N]
     int *status;
     int M, N, K, rank;
     int kb_main;              // K / 64
     int kb_slab;              // ceil(rank / 64) (mode 0)
-    int splitk;               // mode 1: number of K splits (grid.x)
+    int n_t;                  // number of t CTAs = token tiles x rank tiles (0 when rank == 0)
+    int rt;                   // rank tiles of 128
+    int nt;                   // feature tiles of 128
+    int *tflag;               // [token tiles] warps of t CTAs that have stored their part (self-clearing)
+    int *tdone;               // [token tiles] main CTAs that have consumed t (self-clearing)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -377,29 +383,35 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 }
 
 // Shared-memory map of a CTA (byte offsets from the 1024-byte aligned base)
-template <int MODE, int TOK> struct Smem {
+template <int TOK> struct Smem {
     static constexpr uint32_t kXBytes = (uint32_t)TOK * kBK * 2u;          // token operand tile of a stage
     static constexpr uint32_t kStageBytes = kXBytes + kWBytes;
     static constexpr uint32_t kRingOff = kStages * kStageBytes;
-    static constexpr uint32_t kTableOff = kRingOff + (MODE == 0 ? kRing * kRawSlot : 0u);
-    static constexpr uint32_t kBarOff = kTableOff + (MODE == 0 ? kRing * kBN * 4u : 0u);
+    static constexpr uint32_t kTableOff = kRingOff + kRing * kRawSlot;
+    static constexpr uint32_t kBarOff = kTableOff + kRing * kBN * 4u;
     static constexpr uint32_t kNumBars = 2 * kStages + 2 * kRing + 1 + 4;  // full, empty, ring full, ring empty, done, epilogue
     static constexpr uint32_t kTotal = kBarOff + kNumBars * 8u + 16u;
 };
 
-// MODE 0: y tile = x.dequant(W)^T + t.B^T  (grid: N tiles x token tiles)
-// MODE 1: t32 += x.A^T over this CTA's K range (grid: K splits x token tiles x rank tiles), fp32 atomics
+// One launch, 1-D grid.  The first n_t CTAs are "t CTAs": CTA (token tile, rank tile) computes
+// t = x.A^T for 256 tokens x 128 rank indices over all of K (both operands by TMA) and stores it as
+// fp32 to scratch, then raises the token tile's flag.  The other CTAs are main CTAs, one per
+// (feature tile, token tile): y tile = x.dequant(W)^T + t.B^T; they look at the flag only before
+// their sub-branch blocks, at the very end of the K loop, by which time the t CTAs (lowest block
+// indices, so dispatched first, and with no unpacking to do) have long finished.  The wait is
+// bounded like all others.  The last main CTA of a token tile to finish clears the flag again.
 // xmap: x [M][K], boxes of TOK rows x 64 elements, 128-byte swizzle
-// wmap: mode 0: packed codes [N][words per row], boxes of 128 rows x one group (64-byte swizzle for INT4);
-//       mode 1: A [rank][K], boxes of 128 rows x 64 elements, 128-byte swizzle
-// bmap: mode 0, rank > 0: B [N][rank], boxes of 128 rows x 64 elements, 128-byte swizzle
-// ymap: mode 0: y [M][N], boxes of TOK/4 rows x 128 elements, no swizzle (stores)
-template <int MODE, int BITS, typename T, int TOK>
+// wmap: packed codes [N][words per row], boxes of 128 rows x one group (64-byte swizzle for INT4)
+// amap: A [rank][K], boxes of 128 rows x 64 elements, 128-byte swizzle (t CTAs)
+// bmap: B [N][rank], boxes of 128 rows x 64 elements, 128-byte swizzle (main CTAs, rank > 0)
+// ymap: y [M][N], boxes of TOK/4 rows x 128 elements, no swizzle (stores)
+template <int BITS, typename T, int TOK>
 __global__ void __launch_bounds__(kPfThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
-               const __grid_constant__ CUtensorMap bmap, const __grid_constant__ CUtensorMap ymap, const PrefillParams p)
+               const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+               const __grid_constant__ CUtensorMap ymap, const PrefillParams p)
 {
-    using L = Smem<MODE, TOK>;
+    using L = Smem<TOK>;
     constexpr uint32_t kXBytes = L::kXBytes, kStageBytes = L::kStageBytes;
     constexpr int WPG = (BITS == 4) ? 16 : 12;                  // packed words per row and group
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -414,20 +426,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.y * TOK;
-    const int n0 = (MODE == 0) ? blockIdx.x * kBN : blockIdx.z * kBN;   // mode 1: tile of rank rows of A
-    int kb_begin = 0, kb_end = p.kb_main + p.kb_slab;
-    if (MODE == 1) {
-        kb_begin = (int)((long long)blockIdx.x * p.kb_main / p.splitk);
-        kb_end = (int)((long long)(blockIdx.x + 1) * p.kb_main / p.splitk);
+    const bool t_role = (int)blockIdx.x < p.n_t;                // t CTA or main CTA
+    int m_tile, n_tile;
+    if (t_role) {
+        m_tile = (int)blockIdx.x / p.rt;
+        n_tile = (int)blockIdx.x % p.rt;                        // tile of rank rows of A
+    } else {
+        m_tile = ((int)blockIdx.x - p.n_t) / p.nt;
+        n_tile = ((int)blockIdx.x - p.n_t) % p.nt;
     }
-    const int nkb = kb_end - kb_begin;
-    const int kb_x = (MODE == 1) ? kb_end : p.kb_main;          // blocks below kb_x take their tokens from x
-    if (MODE == 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may start its K loop
+    const int m0 = m_tile * TOK, n0 = n_tile * kBN;
+    const int nkb = t_role ? p.kb_main : p.kb_main + p.kb_slab;
+    const int kb_x = p.kb_main;                                 // blocks below kb_x take their tokens from x
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
-            pf_mbar_init(full0 + 8u * i, (MODE == 0) ? kHalf + 1 : 1);   // 256 producers + the TMA lane
+            pf_mbar_init(full0 + 8u * i, t_role ? 1 : kHalf + 1);        // 256 producers + the TMA lane
             pf_mbar_init(empty0 + 8u * i, 1);
         }
         for (int i = 0; i < kRing; ++i) {
@@ -448,8 +462,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
     if (warp == kTmaWarp && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&xmap)) : "memory");
-        if (MODE == 0 && p.rank > 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&bmap)) : "memory");
-        if (MODE == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ymap)) : "memory");
+        if (t_role) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&amap)) : "memory");
+        } else {
+            if (p.rank > 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&bmap)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ymap)) : "memory");
+        }
     }
     if (warp == kRawWarp && lane == 0)
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&wmap)) : "memory");
@@ -459,7 +477,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
 
     if (warp < kMmaWarp) {
         bool dead = false;
-        if (MODE == 0) {
+        if (!t_role) {
             // =================================================== producers
             // Half h of the warps takes the groups g = h, h+2, ... (K blocks 2g and 2g+1, stages 2h
             // and 2h+1); thread (row r, part) dequantises the codes [32*part, +32) of both blocks.
@@ -529,11 +547,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             }
             // ---- sub-branch blocks: token operand = t (fp32 scratch, rounded once); B arrives by TMA.
             // The halves take them in turn, one token row per thread.
+            bool t_ready = false;
 #pragma unroll 1
             for (int i = p.kb_main + h; i < nkb && !dead; i += 2) {
                 const int s = i % kStages;
                 if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
-                asm volatile("griddepcontrol.wait;" ::: "memory");          // t is complete once the down-projection has ended
+                if (!t_ready) {                              // every warp of every t CTA of this token tile has stored its part
+                    int seen = 0;
+                    if (lane == 0) {
+                        const int *flag = p.tflag + m_tile;
+                        const int target = 16 * p.rt;
+#pragma unroll 1
+                        for (uint32_t spin = 0; spin < kPfFlagPolls; ++spin) {
+                            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+                            if (seen >= target) break;
+                            __nanosleep(256);
+                        }
+                        seen = seen >= target;
+                    }
+                    t_ready = __shfl_sync(0xffffffffu, seen, 0) != 0;
+                    if (!t_ready) { dead = true; break; }
+                }
                 const int j0 = (i - p.kb_main) * kBK;
                 const int rr = tid & (kHalf - 1);            // token row of the tile
                 if (rr < TOK) {
@@ -581,20 +615,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     uint32_t v[32];
                     tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
                     tc_wait_ld();
-                    if (MODE == 0) {
+                    if (!t_role) {
                         unsigned short *sp = reinterpret_cast<unsigned short *>(smem + (size_t)c * (kBN * 2)) + 32 * q + lane;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) sp[j * kBN] = to_bits16<T>(__uint_as_float(v[j]));
                     } else {
-                        if (nn < p.rank) {
+                        if (nn < p.rank) {                   // 32 lanes = 32 consecutive rank indices: 128-byte stores
                             float *tp = p.t32 + (size_t)(m0 + c) * p.rank + nn;
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (m0 + c + j < p.M) atomicAdd(tp + (size_t)j * p.rank, __uint_as_float(v[j]));
+                                if (m0 + c + j < p.M) __stcg(tp + (size_t)j * p.rank, __uint_as_float(v[j]));
                         }
                     }
                 }
-                if (MODE == 0) {
+                if (!t_role) {
                     pf_fence_proxy_async();                 // staged tile -> visible to the TMA store
                     pf_mbar_arrive(epi0 + 8u * cg);
                     if (q == 0 && lane == 0) {
@@ -609,6 +643,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                             atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
                         }
                     }
+                }
+            }
+            if (t_role) {
+                // this warp's part of t is stored: make it visible, then count the warp in
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(p.tflag + m_tile, 1);
+            } else if (p.rank > 0 && tid == 0) {
+                // this CTA has consumed t (its MMAs are complete).  The last main CTA of the token
+                // tile leaves the flag and the count at zero for the next call.
+                if (atomicAdd(p.tdone + m_tile, 1) == p.nt - 1) {
+                    atomicExch(p.tflag + m_tile, 0);
+                    atomicExch(p.tdone + m_tile, 0);
                 }
             }
         }
@@ -653,17 +700,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             bool dead = false;
 #pragma unroll 1
             for (int i = 0; i < nkb; ++i) {
-                const int kb = kb_begin + i, s = i % kStages;
+                const int kb = i, s = i % kStages;
                 if ((i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) || *abort_flag) {
                     dead = true;
                     break;
                 }
                 const uint32_t bar = full0 + 8u * s;
                 const uint32_t xt = sbase + (uint32_t)s * kStageBytes, wt = xt + kXBytes;
-                if (MODE == 1) {
+                if (t_role) {
                     pf_mbar_expect_tx(bar, kXBytes + kWBytes);
                     tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
-                    tma_load_2d(wt, &wmap, kb * kBK, n0, bar);      // rows of A
+                    tma_load_2d(wt, &amap, kb * kBK, n0, bar);      // rows of A
                 } else if (kb < kb_x) {
                     pf_mbar_expect_tx(bar, kXBytes);
                     tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
@@ -679,7 +726,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             }
         }
         __syncwarp();
-    } else if (MODE == 0) {
+    } else if (!t_role) {
         // =================================================== ring of packed codes and (s, z) table
         // Two warps; lane l of ring warp v owns the tile rows 64v + l and 64v + l + 32.  Per chunk of
         // eight groups it reads the rows' scales and zero points with 16-byte loads (two aligned chunks of the flat row-major arrays
@@ -783,28 +830,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
 }
 
-template <int MODE, int BITS, typename T, int TOK>
-cudaError_t launch_mode(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &ymap, const PrefillParams &p,
-                        dim3 grid, cudaStream_t s, bool overlap_previous)
+template <int BITS, typename T, int TOK>
+cudaError_t launch_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &amap, const CUtensorMap &bmap,
+                          const CUtensorMap &ymap, const PrefillParams &p, unsigned grid, cudaStream_t s)
 {
-    auto kern = prefill_kernel<MODE, BITS, T, TOK>;
+    auto kern = prefill_kernel<BITS, T, TOK>;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem<MODE, TOK>::kTotal);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem<TOK>::kTotal);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(kPfThreads);
-    cfg.dynamicSmemBytes = Smem<MODE, TOK>::kTotal;
-    cfg.stream = s;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = overlap_previous ? 1 : 0;       // may start while the previous kernel drains
-    return cudaLaunchKernelEx(&cfg, kern, xmap, wmap, bmap, ymap, p);
+    kern<<<grid, kPfThreads, Smem<TOK>::kTotal, s>>>(xmap, wmap, amap, bmap, ymap, p);
+    return cudaGetLastError();
 }
 
 // 2-D tensor map of a row-major matrix: `cols` elements per row (16- or 32-bit), `rows` rows,
@@ -843,6 +881,12 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
     p.M = a.M; p.N = a.N; p.K = a.K; p.rank = a.rank;
     p.kb_main = a.K / kBK;
     p.kb_slab = (a.rank + kBK - 1) / kBK;
+    const int mt = (a.M + TOK - 1) / TOK;
+    p.nt = (a.N + kBN - 1) / kBN;
+    p.rt = (a.rank + kBN - 1) / kBN;
+    p.n_t = mt * p.rt;
+    p.tflag = ws.counters + kPfCtrBase;
+    p.tdone = p.tflag + mt;
     CUtensorMap xmap, qmap, amap, bmap, ymap;
     cudaError_t e;
     if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
@@ -851,25 +895,14 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
                       a.bits == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess)
         return e;
     if ((e = make_map(&ymap, a.y, false, (size_t)a.N, (size_t)a.M, kBN, TOK / 4, CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess) return e;
-    bmap = xmap;
-    const unsigned mt = (unsigned)((a.M + TOK - 1) / TOK), nt = (unsigned)((a.N + kBN - 1) / kBN);
+    amap = bmap = xmap;
     if (a.rank > 0) {
         if ((e = make_map(&amap, a.A, false, (size_t)a.K, (size_t)a.rank, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
         if ((e = make_map(&bmap, a.B, false, (size_t)a.rank, (size_t)a.N, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
-        // t = x.A^T into fp32 scratch: K split so that about one CTA per SM is busy
-        if ((e = cudaMemsetAsync(ws.t_gen, 0, sizeof(float) * (size_t)a.M * a.rank, s)) != cudaSuccess) return e;
-        const unsigned rt = (unsigned)((a.rank + kBN - 1) / kBN);
-        p.splitk = (int)max(1u, min((unsigned)p.kb_main, 148u / (mt * rt)));
-        e = launch_mode<1, 4, T, TOK>(xmap, amap, amap, amap, p, dim3((unsigned)p.splitk, mt, rt), s, false);
-        if (e != cudaSuccess) return e;
-        ++*launches;
     }
-    p.splitk = 1;
-    // The main launch may overlap the tail of the down-projection: it waits for t only before
-    // its sub-branch blocks.
-    const bool pdl = a.rank > 0;
-    e = (a.bits == 4) ? launch_mode<0, 4, T, TOK>(xmap, qmap, bmap, ymap, p, dim3(nt, mt), s, pdl)
-                      : launch_mode<0, 3, T, TOK>(xmap, qmap, bmap, ymap, p, dim3(nt, mt), s, pdl);
+    const unsigned grid = (unsigned)p.n_t + (unsigned)p.nt * (unsigned)mt;
+    e = (a.bits == 4) ? launch_kernel<4, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s)
+                      : launch_kernel<3, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -881,10 +914,14 @@ inline bool aligned16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 
 bool prefill_supported(const LinearArgs &a)
 {
     return a.group == kGroupFast && a.K % kGroupFast == 0 && a.rank % 8 == 0 && a.rank <= kMaxRank && a.N % 8 == 0 &&
-           a.M >= 1 && a.M <= 65535 * 128;
+           a.M >= 1 && a.M <= (1 << 22);
 }
 
-// ws.t_gen must hold M x rank floats and ws.counters at least 8 ints (the caller grows them).
+// Ints of ws.counters the prefill path uses for a call with M tokens (zero between calls).
+int prefill_counters_need(int M) { return kPfCtrBase + 2 * ((M + 127) / 128); }
+
+// ws.t_gen must hold M x rank floats and ws.counters prefill_counters_need(M) ints (the caller
+// grows them; new counters start at zero and the kernel leaves them at zero).
 // Operands that are not 16-byte aligned are refused (the caller then takes the generic kernel).
 cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches)
 {
