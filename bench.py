@@ -254,6 +254,44 @@ def time_e2e(fbq, torch, pool, steps: int, warmup: int):
     return dt, h2d, d2h
 
 
+def time_prefill(fbq, torch, peaks, steps: int = 20, warmup: int = 3):
+    """Secondary figure: the same seven linears at M = 1024, INT4, rank 64, bf16 with 1 % outlier
+    channels (the prefill configuration), through fbq_linear_bf16 on one stream.  Two layer instances
+    (2 x 118 MB) alternate, so operands come from HBM.  CUDA events on the launching stream."""
+    from paper_2501_16385_b200.accounting import algorithmic_flops
+    from paper_2501_16385_b200.microbench import make_instance
+    M, bits, rank = 1024, 4, RANK
+    pool = [[make_instance(M, N, K, bits, rank, "bf16", 7000 + 10 * li + sid, outlier_frac=0.01)
+             for sid, (K, N) in enumerate(layer_shapes())] for li in range(2)]
+    flops = sum(algorithmic_flops(M, N, K, rank) for K, N in layer_shapes())
+
+    def step(i):
+        for t in pool[i % 2]:
+            fbq.linear(t["x"], t["qweight"], t["scales"], t["zeros"], t["A"], t["B"], t["y"].shape[1], GROUP, bits, y=t["y"])
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    before = fbq.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    launches = (fbq.launch_count() - before) / steps
+    assert fbq.poll_status() == 0
+    del pool
+    torch.cuda.empty_cache()
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"workload": "llama2-7b decoder-layer linears, M=1024, INT4 g128, rank 64, bf16, 1% outlier channels",
+            "ms_per_step": ms, "tflops": tf, "steps": steps, "launches_per_step": launches,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": tf / peaks["bf16_tflops"], "kernel": "prefill_kernel<4,__nv_bfloat16,256>",
+                         "algorithmic_flops_per_step": flops}}
+
+
 def oracle_step_seconds(host0, reps: int):
     import oracle
     threads = oracle.max_threads()
@@ -313,6 +351,10 @@ def gpu_arm(args):
         dt, h2d, d2h = time_e2e(fbq, torch, pool, e2e_steps, 3)
         e2e_val = bytes_step * e2e_steps / dt / 1e9
         cpu_s, cores = oracle_step_seconds(host0, 3) if world == 1 else (None, None)
+        if world == 1:
+            del pool
+            torch.cuda.empty_cache()
+            extra["prefill"] = time_prefill(fbq, torch, peaks)
     barrier()
     if rank_id != 0:
         if world > 1:

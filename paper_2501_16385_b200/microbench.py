@@ -18,7 +18,9 @@ from .accounting import algorithmic_bytes, algorithmic_flops
 L2_BYTES = 126e6
 
 
-def make_instance(M, N, K, bits, rank, dtype, seed):
+def make_instance(M, N, K, bits, rank, dtype, seed, outlier_frac=0.0, outlier_scale=20.0):
+    """Device tensors of one synthetic linear.  outlier_frac > 0 scales that share of the input
+    channels of x by outlier_scale (the activation-outlier structure of LLM prefill inputs)."""
     g = torch.Generator(device="cuda")
     g.manual_seed(seed)
     G = K // 128
@@ -28,12 +30,17 @@ def make_instance(M, N, K, bits, rank, dtype, seed):
         "qweight": fbq.pack(codes, bits),
         "scales": (torch.rand((N, G), device="cuda", generator=g) * 0.015 + 0.005).half(),
         "zeros": torch.randint(2, (1 << bits) - 2, (N, G), device="cuda", generator=g).half(),
-        "x": torch.randn((M, K), device="cuda", generator=g).to(act),
+        "x": None,
         "A": (torch.randn((rank, K), device="cuda", generator=g) * 0.02).to(act) if rank else None,
         "B": (torch.randn((N, rank), device="cuda", generator=g) * 0.02).to(act) if rank else None,
         "y": torch.empty((M, N), device="cuda", dtype=act),
     }
     del codes
+    x = torch.randn((M, K), device="cuda", generator=g)
+    if outlier_frac > 0:
+        ch = torch.randperm(K, device="cuda", generator=g)[: max(1, int(outlier_frac * K))]
+        x[:, ch] *= outlier_scale
+    inst["x"] = x.to(act)
     return inst
 
 
