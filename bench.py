@@ -32,11 +32,14 @@ if ROOT not in sys.path:
 BITS, RANK, GROUP, M_TOKENS = 3, 64, 128, 1
 WORKLOAD = "llama2-7b decoder-layer linears, M=1, INT3 g128, rank 64 (7 linears per step)"
 GRAPH_STEPS = 100
-# The seven linears of a step are independent (each has its own x), so a step issues them
-# round-robin over N_STREAMS CUDA streams (fbq_linear keeps separate scratch per stream) with
-# the decode grid limited to DECODE_CTAS, which lets launches of different streams share the SMs.
+# The seven linears of a step are independent (each has its own x).  MODE "streams" (default): a
+# step issues seven fbq_linear calls round-robin over N_STREAMS CUDA streams of the bench, each with
+# its decode grid bounded by its share (by size) of DECODE_CTAS CTAs; the streams are joined once
+# per graph, so linears of consecutive steps overlap.  MODE "batch": a step is one fbq_linear_batch
+# call (the library runs the seven launches on its side streams and joins them every step).
+MODE = os.environ.get("FBQ_BENCH_MODE", "streams")
 N_STREAMS = int(os.environ.get("FBQ_BENCH_STREAMS", "7"))
-DECODE_CTAS = int(os.environ.get("FBQ_BENCH_CTAS", "74"))
+DECODE_CTAS = int(os.environ.get("FBQ_BENCH_CTAS", "400"))      # shared out among the 7 linears by size
 NVSMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                 "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                 "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -156,14 +159,33 @@ def run_step(fbq, layer, with_branch: bool = True, streams=None):
     """One step: the seven fbq_linear calls of one layer instance.  With `streams` (the
     current stream first), call j goes to stream j % len(streams)."""
     import torch
+    costs = [d.N * d.x.shape[1] for d in layer]
     for j, d in enumerate(layer):
         st = streams[j % len(streams)] if streams else None
+        fbq.set_option("decode_ctas", max(8, round(DECODE_CTAS * costs[j] / sum(costs))))
         fbq.linear(d.x, d.qweight, d.scales, d.zeros, d.A if with_branch else None,
                    d.B if with_branch else None, d.N, GROUP, BITS, y=d.y, stream=st)
 
 
+_BATCHES = {}
+
+
+def layer_batch(fbq, layer, with_branch: bool):
+    """Descriptor array of one layer instance for fbq_linear_batch (made once, reused)."""
+    key = (id(layer), with_branch)
+    if key not in _BATCHES:
+        _BATCHES[key] = fbq.make_batch([(d.x, d.qweight, d.scales, d.zeros, d.A if with_branch else None,
+                                         d.B if with_branch else None, d.y) for d in layer])
+    return _BATCHES[key]
+
+
 def run_steps_forked(fbq, torch, pool, n_steps: int, main, with_branch: bool):
-    """n_steps steps with the side streams forked from / joined to `main` once around them."""
+    """n_steps steps on `main`.  Batch mode: one fbq_linear_batch per step.  Streams mode: the side
+    streams are forked from / joined to `main` once around all the steps."""
+    if MODE == "batch":
+        for i in range(n_steps):
+            fbq.linear_batch(None, GROUP, BITS, stream=main, batch=layer_batch(fbq, pool[i % len(pool)], with_branch))
+        return
     sides = side_streams(torch)
     streams = [main] + sides
     for st in sides:
@@ -321,7 +343,8 @@ def gpu_arm(args):
             dist.barrier()
 
     import paper_2501_16385_b200 as fbq
-    fbq.set_option("decode_ctas", DECODE_CTAS)
+    if os.environ.get("FBQ_BATCH_CTAS"):
+        fbq.set_option("batch_ctas", int(os.environ["FBQ_BATCH_CTAS"]))
     peaks, peak_kind = measured_peaks()
     bytes_step = step_bytes()
     pool_layers = max(2, -(-3 * 126_000_000 // bytes_step))        # pool >= 3 x L2 (126 MB)
@@ -380,9 +403,12 @@ def gpu_arm(args):
                    "linears_per_step": n_linears, "pool_layers": pool_layers,
                    "cold": "pool of %d layer instances (%.0f MB) > 3x L2, visited round-robin" %
                            (pool_layers, pool_layers * bytes_step / 1e6),
-                   "launch": "CUDA graph replay of fbq_linear calls (programmatic dependent launch); the 7 "
-                             "independent linears of a step go round-robin over %d streams, decode grid <= %d CTAs"
-                             % (N_STREAMS, DECODE_CTAS),
+                   "launch": ("CUDA graph replay of one fbq_linear_batch call per step (7 concurrent decode launches on "
+                              "the library's side streams, %d CTAs shared out by size, joined every step)"
+                              % fbq.get_option("batch_ctas")) if MODE == "batch" else
+                             ("CUDA graph replay of fbq_linear calls (programmatic dependent launch); the 7 "
+                              "independent linears of a step go round-robin over %d streams, decode grids share %d CTAs by size"
+                              % (N_STREAMS, DECODE_CTAS)),
                    "parallelism": "replicas only (no collective on the path)" if world > 1 else "1 GPU"},
         "gpu_launches": args.steps * n_linears,       # one fused decode launch per linear per step
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -137,6 +137,40 @@ int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const void *scale
                        const void *zeros, const void *A, const void *B, void *y, int M, int N,
                        int K, int group, int bits, int rank, int act_is_bf16, void *stream);
 
+/* Several independent linears of the same kind in one call: the grouped decode of a decoder
+ * layer, where q, k, v (and gate, up) read the same x through different weights, or any set
+ * of layers whose inputs are ready (Algorithm 1 reconstructs each of the seven projections
+ * of a layer on its own; at inference those that do not depend on one another can run
+ * together).  Problem i computes
+ *     y_i = x_i . dequant(Q_i, s_i, z_i)^T + (x_i . A_i^T) . B_i^T
+ * exactly as fbq_linear / fbq_linear_bf16 would with the shared M, group, bits, rank and
+ * activation type; N and K are per problem.  No y_i may overlap another problem's inputs.
+ *   - `problems` is a HOST array of `count` (<= FBQ_BATCH_MAX) descriptors of DEVICE
+ *     pointers (layouts and alignment as for fbq_linear); it is read before the call returns.
+ *   - When every problem is decode sized (M <= 16 and the decode kernel's domain) the
+ *     problems run concurrently: each on a side stream of the library, forked from and
+ *     joined to `stream` with events, its grid bounded in proportion to its share of the
+ *     codes ("batch_ctas" CTAs in total), so that the whole batch is resident at once and
+ *     every CTA's start-up cost is paid once per batch instead of once per small launch.
+ *     Work queued on `stream` after the call sees every y_i.  The pattern is legal under
+ *     stream capture; make the first call on a device outside a capture (it creates the
+ *     side streams and events, which are kept until the process exits).
+ *   - Otherwise the problems run one after the other on `stream`.
+ * Returns the first error, or FBQ_OK. */
+#define FBQ_BATCH_MAX 16
+typedef struct fbq_problem {
+    const void *x;            /* [M][K] */
+    const uint32_t *qweight;  /* packed codes of [N][K] */
+    const void *scales;       /* fp16 [N][K/group] */
+    const void *zeros;        /* fp16 [N][K/group] */
+    const void *A;            /* [rank][K] or NULL when rank == 0 */
+    const void *B;            /* [N][rank] or NULL when rank == 0 */
+    void *y;                  /* [M][N] */
+    int N, K;
+} fbq_problem;
+int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, int bits, int rank,
+                     int act_is_bf16, void *stream);
+
 /* Which kernel fbq_linear / fbq_linear_bf16 would run for this shape, or
  * FBQ_KERNEL_NONE when the shape is rejected.  Pure host logic. */
 int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int act_is_bf16);
@@ -148,6 +182,7 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "decode_chunk"  0 = automatic, else quantisation groups per smem stage
  *   "decode_depth"  0 = automatic, else stages in flight per warp
  *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
+ *   "batch_ctas"    CTAs shared out among the problems of a decode-sized fbq_linear_batch (default 400)
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol

@@ -12,13 +12,16 @@ from .binding import (  # noqa: F401
     KERNEL_GENERIC,
     KERNEL_NONE,
     KERNEL_PREFILL,
+    Problem,
     STATUS,
     dequant,
     get_option,
     launch_count,
     lib,
     library_path,
+    make_batch,
     linear,
+    linear_batch,
     linear_hostio,
     linear_noalloc,
     pack,

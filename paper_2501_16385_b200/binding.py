@@ -28,6 +28,13 @@ def library_path() -> str:
     return _build.LIB
 
 
+class Problem(ctypes.Structure):
+    """struct fbq_problem of include/fbq.h."""
+    _fields_ = [("x", ctypes.c_void_p), ("qweight", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("zeros", ctypes.c_void_p), ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("N", ctypes.c_int), ("K", ctypes.c_int)]
+
+
 def lib() -> ctypes.CDLL:
     """Loads libfbq.so (building it with nvcc when absent).  Raises if the
     library cannot be had: there is no other implementation to run."""
@@ -48,6 +55,7 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_linear_noalloc.argtypes = [vp] * 7 + [i32] * 7 + [vp]
+        L.fbq_linear_batch.argtypes = [ctypes.POINTER(Problem), i32, i32, i32, i32, i32, i32, vp]
         L.fbq_select_kernel.argtypes = [i32] * 7
         L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
         L.fbq_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32)]
@@ -152,6 +160,31 @@ def linear_noalloc(x, qweight, scales, zeros, A, B, N: int, group: int, bits: in
                                     _ptr(y), M, N, K, group, bits, rank, bf16, _stream(stream)),
            "fbq_linear_noalloc")
     return y
+
+
+def make_batch(problems):
+    """Marshals a list of (x, qweight, scales, zeros, A, B, y) tensor tuples (A = B = None for
+    rank 0; every x [M, K], y [M, N]) into the descriptor array of fbq_linear_batch.  Returns
+    (array, count, M, rank, bf16); the array can be reused for as long as the tensors live."""
+    import torch
+    n = len(problems)
+    arr = (Problem * max(n, 1))()
+    M = rank = bf16 = None
+    for i, (x, qw, s, z, A, B, y) in enumerate(problems):
+        assert x.is_cuda and x.is_contiguous() and y.is_contiguous() and x.dtype == y.dtype
+        m, r, b = x.shape[0], (0 if A is None else A.shape[0]), (1 if x.dtype == torch.bfloat16 else 0)
+        if i == 0:
+            M, rank, bf16 = m, r, b
+        assert (m, r, b) == (M, rank, bf16), "the problems of a batch share M, rank and the activation type"
+        arr[i] = Problem(_ptr(x), _ptr(qw), _ptr(s), _ptr(z), _ptr(A), _ptr(B), _ptr(y), y.shape[1], x.shape[1])
+    return arr, n, M or 0, rank or 0, bf16 or 0
+
+
+def linear_batch(problems, group: int, bits: int, stream=None, batch=None):
+    """fbq_linear_batch over a list of (x, qweight, scales, zeros, A, B, y) tuples, or over a
+    descriptor array made earlier by make_batch (``batch``).  The y tensors are written."""
+    arr, n, M, rank, bf16 = batch if batch is not None else make_batch(problems)
+    _check(lib().fbq_linear_batch(arr, n, M, group, bits, rank, bf16, _stream(stream)), "fbq_linear_batch")
 
 
 def select_kernel(M, N, K, group, bits, rank, bf16=False) -> int:

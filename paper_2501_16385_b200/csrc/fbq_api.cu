@@ -22,6 +22,7 @@ struct Options {
     int force_kernel = -1;
     DecodeTuning decode;
     int decode_t_late = 0;
+    int batch_ctas = 400;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
@@ -87,8 +88,11 @@ Workspace *workspace_for(cudaStream_t s)
     return &g_ws[std::make_pair(dev, s)];
 }
 
-int run_linear(const LinearArgs &a, cudaStream_t s)
+// decode_ctas > 0 overrides the decode kernel's grid-size bound for this call.
+int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
 {
+    DecodeTuning tune = g_opt.decode;
+    if (decode_ctas > 0) tune.max_ctas = decode_ctas;
     if (!well_formed(a.M, a.N, a.K, a.group, a.bits, a.rank)) return FBQ_ERR_BADARG;
     if (a.M == 0) return FBQ_OK;
     if (!a.x || !a.qw || !a.scales || !a.zeros || !a.y) return FBQ_ERR_BADARG;
@@ -107,7 +111,7 @@ int run_linear(const LinearArgs &a, cudaStream_t s)
     if (kernel == FBQ_KERNEL_DECODE) {
         size_t pf = 0;
         int nc = 0;
-        decode_workspace_need(a, g_opt.decode, &pf, &nc);
+        decode_workspace_need(a, tune, &pf, &nc);
         size_t have_c = (size_t)ws->n_counters;
         if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         if ((e = grow(ws->t, ws->t_floats, (size_t)kDecodeMaxM * kMaxRank, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
@@ -123,7 +127,7 @@ int run_linear(const LinearArgs &a, cudaStream_t s)
                 ws->trace = nullptr;
             }
         }
-        e = launch_decode(a, *ws, g_opt.decode, s, &launches);
+        e = launch_decode(a, *ws, tune, s, &launches);
         if (e == cudaErrorInvalidConfiguration) {
             (void)cudaGetLastError();
             kernel = FBQ_KERNEL_GENERIC;          // plan does not fit shared memory
@@ -166,6 +170,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
+    if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
@@ -255,6 +260,85 @@ int fbq_linear_bf16(const void *x, const uint32_t *qweight, const void *scales, 
                     const void *B, void *y, int M, int N, int K, int group, int bits, int rank, void *stream)
 {
     return linear_common(x, qweight, scales, zeros, A, B, y, M, N, K, group, bits, rank, true, stream);
+}
+
+// Side streams and events of fbq_linear_batch, per device, created on first use and kept.
+struct BatchLanes {
+    cudaStream_t side[FBQ_BATCH_MAX] = {};
+    cudaEvent_t fork = nullptr, join[FBQ_BATCH_MAX] = {};
+    int n = 0;
+};
+static std::map<int, BatchLanes> g_lanes;
+
+static BatchLanes *lanes_for(int want)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lk(g_mu);
+    BatchLanes &b = g_lanes[dev];
+    if (!b.fork && cudaEventCreateWithFlags(&b.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    while (b.n < want) {
+        if (cudaStreamCreateWithFlags(&b.side[b.n], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&b.join[b.n], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ++b.n;
+    }
+    return &b;
+}
+
+int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, int bits, int rank, int act_is_bf16,
+                     void *stream)
+{
+    if (count < 0 || count > FBQ_BATCH_MAX || (count > 0 && !problems)) return FBQ_ERR_BADARG;
+    if (count == 0) return FBQ_OK;
+    cudaStream_t main = static_cast<cudaStream_t>(stream);
+    decode_set_test_switch(g_opt.decode_t_late);
+    LinearArgs a[FBQ_BATCH_MAX];
+    bool all_decode = count > 1;
+    double total_cost = 0.0;
+    for (int i = 0; i < count; ++i) {
+        const fbq_problem &q = problems[i];
+        a[i] = LinearArgs{};
+        a[i].x = q.x; a[i].qw = q.qweight;
+        a[i].scales = static_cast<const __half *>(q.scales);
+        a[i].zeros = static_cast<const __half *>(q.zeros);
+        a[i].A = rank > 0 ? q.A : nullptr;
+        a[i].B = rank > 0 ? q.B : nullptr;
+        a[i].y = q.y;
+        a[i].M = M; a[i].N = q.N; a[i].K = q.K; a[i].group = group; a[i].bits = bits; a[i].rank = rank;
+        a[i].bf16 = act_is_bf16 != 0;
+        if (!well_formed(M, q.N, q.K, group, bits, rank)) return FBQ_ERR_BADARG;
+        all_decode = all_decode && select_kernel(M, q.N, q.K, group, bits, rank, a[i].bf16) == FBQ_KERNEL_DECODE;
+        total_cost += (double)q.N * q.K;
+    }
+    if (!all_decode) {
+        // one after the other on the caller's stream (prefill-sized problems fill the GPU by themselves)
+        for (int i = 0; i < count; ++i) {
+            const int rc = run_linear(a[i], main);
+            if (rc != FBQ_OK) return rc;
+        }
+        return FBQ_OK;
+    }
+    // Decode-sized problems: all at once.  Problem i runs on side stream i, forked from and joined
+    // to the caller's stream by events, with a grid bound in proportion to its share of the codes,
+    // so that the CTAs of the whole batch are resident together and finish together.
+    BatchLanes *lanes = lanes_for(count);
+    if (!lanes) return FBQ_ERR_CUDA;
+    if (cudaEventRecord(lanes->fork, main) != cudaSuccess) return FBQ_ERR_CUDA;
+    int rc = FBQ_OK;
+    int forked = 0;
+    for (int i = 0; i < count; ++i) {
+        if (cudaStreamWaitEvent(lanes->side[i], lanes->fork, 0) != cudaSuccess) { rc = FBQ_ERR_CUDA; break; }
+        ++forked;
+        const int ctas = std::max(8, (int)(g_opt.batch_ctas * ((double)a[i].N * a[i].K / total_cost) + 0.5));
+        rc = run_linear(a[i], lanes->side[i], ctas);
+        if (rc != FBQ_OK) break;
+    }
+    for (int i = 0; i < forked; ++i) {              // always rejoin what was forked (also under stream capture)
+        if (cudaEventRecord(lanes->join[i], lanes->side[i]) != cudaSuccess ||
+            cudaStreamWaitEvent(main, lanes->join[i], 0) != cudaSuccess)
+            rc = (rc == FBQ_OK) ? FBQ_ERR_CUDA : rc;
+    }
+    return rc;
 }
 
 int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *scales, const void *zeros,

@@ -35,6 +35,9 @@
 // warps, and they are bounded.
 #include "fbq_common.cuh"
 
+#ifndef FBQ_NACC
+#define FBQ_NACC 2
+#endif
 namespace fbq {
 namespace {
 
@@ -394,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
     // for the 128-bit loads of INT4, 48-byte for the three 32-bit loads of INT3).
     constexpr int RP = (BITS == 4) ? 64 : 48;
     auto row_pitch = [](int ng) { const int b = ng * GB; return (b % 128 == 0) ? b + RP : b; };
-    constexpr int NACC = 2;                            // independent MMA accumulator chains
+    constexpr int NACC = FBQ_NACC;                     // independent MMA accumulator chains
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, tq = lane & 3;
@@ -457,13 +460,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             const int na = min(tu1 - tu0, p.a_cap);
             uint32_t total = 0;
             for (int i = 0; i < na; ++i) {
-                const int kc = (tu0 + i) % nkc;
+                const int kc = (tu0 + i) / p.rank;               // units are numbered k-chunk-major: u = kc*rank + j
                 total += (uint32_t)min(kTUnitK, kslice - kc * kTUnitK) * 2u;
             }
             if (lane == 0) mbar_expect_tx(a_full, total);
             __syncwarp();
             for (int i = lane; i < na; i += 32) {
-                const int u = tu0 + i, j = u / nkc, kc = u - j * nkc;
+                const int u = tu0 + i, kc = u / p.rank, j = u - kc * p.rank;
                 const int nk = min(kTUnitK, kslice - kc * kTUnitK);
                 bulk_g2s(smem_u32(s_A + (size_t)i * kTUnitK), A + (size_t)j * p.K + g0 * kGroupFast + kc * kTUnitK,
                          (uint32_t)nk * 2u, a_full);
@@ -639,9 +642,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
 
 #pragma unroll
                     for (int b = 0; b < MT; ++b) {
+                        // (P, X0) of tokens 8b+2tq and 8b+2tq+1 for this group; the chain starts at -P
+                        const float4 px = *reinterpret_cast<const float4 *>(s_px + (size_t)(pos + gi) * (8 * MT) + 8 * b + 2 * tq);
                         float tmp[NACC][4];
 #pragma unroll
                         for (int c = 0; c < NACC; ++c) tmp[c][0] = tmp[c][1] = tmp[c][2] = tmp[c][3] = 0.f;
+                        tmp[0][0] = tmp[0][2] = -px.x;
+                        tmp[0][1] = tmp[0][3] = -px.z;
                         const int token = 8 * b + g;
                         const uint4 *xg = reinterpret_cast<const uint4 *>(s_x + (size_t)token * p.x_pitch +
                                                                           (size_t)(pos + gi) * kGroupFast);
@@ -654,8 +661,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                             Pk<T>::mma(tmp[q4 % NACC], a0, xv.x, xv.y);
                             Pk<T>::mma(tmp[q4 % NACC], a1, xv.z, xv.w);
                         }
-                        // (P, X0) of tokens 8b+2tq and 8b+2tq+1 for this group
-                        const float4 px = *reinterpret_cast<const float4 *>(s_px + (size_t)(pos + gi) * (8 * MT) + 8 * b + 2 * tq);
                         float d[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
@@ -664,10 +669,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                             for (int c = 1; c < NACC; ++c) d[i] += tmp[c][i];
                         }
                         // s*(mma - P) - (s*z)*X0
-                        acc[b][0] = fmaf(-fa.y, px.y, fmaf(fa.x, d[0] - px.x, acc[b][0]));
-                        acc[b][1] = fmaf(-fa.y, px.w, fmaf(fa.x, d[1] - px.z, acc[b][1]));
-                        acc[b][2] = fmaf(-fb.y, px.y, fmaf(fb.x, d[2] - px.x, acc[b][2]));
-                        acc[b][3] = fmaf(-fb.y, px.w, fmaf(fb.x, d[3] - px.z, acc[b][3]));
+                        acc[b][0] = fmaf(-fa.y, px.y, fmaf(fa.x, d[0], acc[b][0]));
+                        acc[b][1] = fmaf(-fa.y, px.w, fmaf(fa.x, d[1], acc[b][1]));
+                        acc[b][2] = fmaf(-fb.y, px.y, fmaf(fb.x, d[2], acc[b][2]));
+                        acc[b][3] = fmaf(-fb.y, px.w, fmaf(fb.x, d[3], acc[b][3]));
                     }
                 }
                 // stage consumed by this warp
@@ -724,6 +729,49 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                    ? s_B + (size_t)(tile - tile_first) * kTileRows * p.rank
                    : nullptr;
     };
+    // Fast finish (rank <= 64, one K slice): lanes 2i and 2i+1 share row i of the tile; a lane holds
+    // every other 8-element chunk of that row of B in registers, requested before the wait for the
+    // segment, so that the up-projection costs no exposed load latency.
+    const bool fast_fin = (p.rank > 0) && (p.rank <= 64) && (p.SK == 1);
+    uint4 bq[4];
+    auto b_prefetch = [&](int tile) {
+        const int row = lane >> 1, n = tile * kTileRows + row;
+        const T *own = own_b(tile);
+        const T *src = own ? own + (size_t)row * p.rank : static_cast<const T *>(p.B) + (size_t)n * p.rank;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = (lane & 1) + 2 * i;
+            bq[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (8 * c < p.rank && n < p.N)
+                bq[i] = own ? *reinterpret_cast<const uint4 *>(src + 8 * c) : __ldg(reinterpret_cast<const uint4 *>(src + 8 * c));
+        }
+    };
+    // y rows of `tile` = staged main sums + t.B^T from the prefetched chunks
+    auto finish_fast = [&](int tile) {
+        const int row = lane >> 1, n = tile * kTileRows + row;
+#pragma unroll 1
+        for (int m = 0; m < p.M; ++m) {
+            float sub = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c = (lane & 1) + 2 * i;
+                if (8 * c < p.rank) {
+                    const float4 t0 = *reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank + 8 * c);
+                    const float4 t1 = *reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank + 8 * c + 4);
+                    const float2 b0 = Pk<T>::to_float2(bq[i].x), b1 = Pk<T>::to_float2(bq[i].y);
+                    const float2 b2 = Pk<T>::to_float2(bq[i].z), b3 = Pk<T>::to_float2(bq[i].w);
+                    sub = fmaf(t0.x, b0.x, sub); sub = fmaf(t0.y, b0.y, sub);
+                    sub = fmaf(t0.z, b1.x, sub); sub = fmaf(t0.w, b1.y, sub);
+                    sub = fmaf(t1.x, b2.x, sub); sub = fmaf(t1.y, b2.y, sub);
+                    sub = fmaf(t1.z, b3.x, sub); sub = fmaf(t1.w, b3.y, sub);
+                }
+            }
+            sub += __shfl_xor_sync(0xffffffffu, sub, 1);
+            if ((lane & 1) == 0 && n < p.N)
+                static_cast<T *>(p.y)[(size_t)m * p.N + n] = ActTraits<T>::from_float(s_stage[m * kTileRows + row] + sub);
+        }
+        ++n_retired;
+    };
     // Finish `tile` from scratch slots (all contributions are there and visible).
     auto finish_from_slots = [&](int tile) {
         finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
@@ -747,13 +795,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         }
         const T *A = static_cast<const T *>(p.A);
         const T *x = static_cast<const T *>(p.x) + g0 * kGroupFast;
-#pragma unroll 1
-        for (int u = tu0; u < tu1; ++u) {
-            const int j = u / nkc, kc = u - j * nkc;
-            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
+        // one unit = row j of A against one k chunk of 1024 (units are numbered k-chunk-major:
+        // u = kc*rank + j); a lane takes 8 elements out of every 256
+        auto load_a = [&](int u, int kbeg, int nk, uint4 (&av)[4]) {
+            const int j = u - (u / p.rank) * p.rank;
             const bool in_smem = (u - tu0) < p.a_cap;
             const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
-            uint4 av[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int k = lane * 8 + 256 * i;
@@ -761,30 +808,46 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                 if (k < nk) av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
                                             : __ldg(reinterpret_cast<const uint4 *>(arow + k));
             }
+        };
+#pragma unroll 1
+        for (int u0 = tu0; u0 < tu1;) {
+            // the units of one k chunk share x: it is read once per token and kept in registers
+            const int kc = u0 / p.rank, uend = min(tu1, (kc + 1) * p.rank);
+            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
 #pragma unroll 1
             for (int m = 0; m < p.M; ++m) {
-                uint4 xv[4];
+                uint4 xv[4], an[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int k = lane * 8 + 256 * i;
                     xv[i] = make_uint4(0u, 0u, 0u, 0u);
                     if (k < nk) xv[i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + kbeg + k));
                 }
-                float v = 0.f;
+                load_a(u0, kbeg, nk, an);
+#pragma unroll 1
+                for (int u = u0; u < uend; ++u) {
+                    uint4 av[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
-                    const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+                    for (int i = 0; i < 4; ++i) av[i] = an[i];
+                    if (u + 1 < uend) load_a(u + 1, kbeg, nk, an);     // next row of A is in flight during the sum
+                    float v0 = 0.f, v1 = 0.f;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
-                        v = fmaf(xf.x, af.x, v);
-                        v = fmaf(xf.y, af.y, v);
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
+                        const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
+                            v0 = fmaf(xf.x, af.x, v0);
+                            v1 = fmaf(xf.y, af.y, v1);
+                        }
                     }
+                    float v = v0 + v1;
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + (u - kc * p.rank), v);
                 }
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + j, v);
             }
+            u0 = uend;
         }
     };
     // After this CTA's share of t is in: count it; the warp that completes t publishes
@@ -841,6 +904,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             if (lane == 0) others_in = ((ld_acquire(p.ctr + kCtrFirstTile + tile) & 0xFFFF) == cnt - 1);
             others_in = __shfl_sync(0xffffffffu, others_in, 0);
         }
+        if (fast_fin) b_prefetch(tile);
         if (!mbar_wait(seg_full + 8u * buf, (uint32_t)(seg / kNBuf) & 1u)) {
             dead = true;
             break;
@@ -873,6 +937,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         if (cnt == 1 || others_in) {
             // This warp finishes the tile: straight from the staged sums if t is complete ...
             if (t_poll()) {
+                if (fast_fin) {
+                    finish_fast(tile);
+                    __syncwarp();
+                    continue;
+                }
                 finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
                                static_cast<const T *>(p.B), p.M, p.N, p.rank, tile, lane, s_stage, myslot, cnt, s_t,
                                own_b(tile));
