@@ -429,9 +429,9 @@ def gpu_arm(args):
 
 
 # DRAM bytes (read + write) per step measured with ncu (--set full) on the seven decode
-# launches of one step: 4 x 7.971 MB + 2 x 20.373 MB + 20.388 MB
+# launches of one step: 4 x 7.951 MB + 2 x 20.337 MB + 20.351 MB
 # (profiles/decode_int3_r64_m1_bench.md).
-TRAFFIC_BYTES_PER_STEP = 93_018_000
+TRAFFIC_BYTES_PER_STEP = 92_831_000
 
 
 # ---------------------------------------------------------------------- reference arm
