@@ -276,6 +276,57 @@ def time_e2e(fbq, torch, pool, steps: int, warmup: int):
     return dt, h2d, d2h
 
 
+def time_naive(fbq, torch, pool, steps: int, warmup: int):
+    """The paper's unfused sub-branch layer (Section 3.2 / Fig. kernel-fusion: quantised main path
+    plus two separate projections and an add) on the same inputs, as a comparator: per linear
+    fbq_linear at rank 0, then t = x.A^T, u = t.B^T and y += u as three library launches (torch.mm,
+    torch.mm, add_) on the same stream.  Same streams, same graph replay as the fused arm."""
+    sides = side_streams(torch)
+    L = len(pool)
+    ts = [[torch.empty((M_TOKENS, RANK), dtype=torch.float16, device="cuda") for _ in layer] for layer in pool]
+    us = [[torch.empty((M_TOKENS, d.N), dtype=torch.float16, device="cuda") for d in layer] for layer in pool]
+    ats = [[d.A.t() for d in layer] for layer in pool]
+    bts = [[d.B.t() for d in layer] for layer in pool]
+
+    def run(n_steps, main):
+        streams = [main] + sides
+        for st in sides:
+            st.wait_stream(main)
+        for i in range(n_steps):
+            li = i % L
+            layer = pool[li]
+            costs = [d.N * d.x.shape[1] for d in layer]
+            for j, d in enumerate(layer):
+                st = streams[j % len(streams)]
+                fbq.set_option("decode_ctas", max(8, round(DECODE_CTAS * costs[j] / sum(costs))))
+                fbq.linear(d.x, d.qweight, d.scales, d.zeros, None, None, d.N, GROUP, BITS, y=d.y, stream=st)
+                with torch.cuda.stream(st):
+                    torch.mm(d.x, ats[li][j], out=ts[li][j])
+                    torch.mm(ts[li][j], bts[li][j], out=us[li][j])
+                    d.y.add_(us[li][j])
+        for st in sides:
+            main.wait_stream(st)
+
+    chunk = max(1, min((GRAPH_STEPS // L) * L, steps))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        run(min(max(warmup, 3), 2 * L), stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            run(chunk, stream)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        reps = max(1, steps // chunk)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / (reps * chunk)
+
+
 def time_prefill(fbq, torch, peaks, steps: int = 20, warmup: int = 3):
     """Secondary figure: the same seven linears at M = 1024, INT4, rank 64, bf16 with 1 % outlier
     channels (the prefill configuration), through fbq_linear_bf16 on one stream.  Two layer instances
@@ -368,6 +419,14 @@ def gpu_arm(args):
         extra["rank0_GBs"] = step_bytes_rank0() * args.steps / (ms0 * 1e-3) / 1e9
         extra["sub_branch_overhead"] = (ms / ms0 - 1.0) if world == 1 else None
         extra["byte_floor_overhead"] = bytes_step / step_bytes_rank0() - 1.0
+        if world == 1 and MODE == "streams":
+            naive_ms = time_naive(fbq, torch, pool, min(args.steps, 4000), args.warmup)
+            fused_ms, r0_ms = ms / args.steps, ms0 / args.steps
+            extra["naive_sub_branch"] = {
+                "what": "rank-0 fbq_linear + torch.mm + torch.mm + add_ per linear (4 launches), same streams and graph replay",
+                "ms_per_step": naive_ms, "slowdown_vs_fused": naive_ms / fused_ms,
+                "overhead_vs_rank0": naive_ms / r0_ms - 1.0,
+                "extra_latency_removed_by_fusion": 1.0 - (fused_ms - r0_ms) / (naive_ms - r0_ms) if naive_ms > r0_ms else None}
         plain_steps = min(args.steps, 2000)
         extra["plain_launch_ms_per_step"] = time_plain_steps(fbq, torch, pool, plain_steps) / plain_steps
         e2e_steps = min(args.steps, 500)
