@@ -133,3 +133,38 @@ def linear_inputs(inp, *, n_list=None, threads=1, return_t=False, qweight=None):
     return linear(inp.x, qweight, inp.scales, inp.zeros, inp.A, inp.B, inp.M, inp.N, inp.K,
                   inp.group, inp.bits, inp.rank, dtype=inp.dtype, n_list=n_list,
                   threads=threads, return_t=return_t)
+
+
+def float_to_half(a: np.ndarray) -> np.ndarray:
+    """fp16 bit patterns (uint16) of float32 values, by the oracle's own rounding routine."""
+    _load()
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty(a.shape, dtype=np.uint16)
+    _lib.oracle_float_to_half(_p(a), _p(out), ctypes.c_int(a.size))
+    return out
+
+
+def quantize_feedback(W: np.ndarray, A, B, group: int, bits: int, *, dtype: str = "f16"):
+    """Feedback quantiser of Section 4.1 on W [N, K] float32 with Sigma = B.A (A [rank, K],
+    B [N, rank] as 16-bit patterns, or None for rank 0).  Returns codes (uint8 [N, K]),
+    scales, zeros (uint16 fp16 patterns [N, K/group]), r = W - Sigma and W_F (float32 [N, K])."""
+    _load()
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    rank = 0 if A is None else A.shape[0]
+    if K % group != 0:
+        raise ValueError("group must divide K")
+    codes = np.empty((N, K), dtype=np.uint8)
+    scales = np.empty((N, K // group), dtype=np.uint16)
+    zeros = np.empty((N, K // group), dtype=np.uint16)
+    r = np.empty((N, K), dtype=np.float32)
+    wf = np.empty((N, K), dtype=np.float32)
+    Ab = _u16(A) if rank else None
+    Bb = _u16(B) if rank else None
+    _lib.oracle_quantize_feedback.restype = ctypes.c_int
+    rc = _lib.oracle_quantize_feedback(_p(W), _p(Ab) if rank else None, _p(Bb) if rank else None, _p(codes), _p(scales),
+                                       _p(zeros), _p(r), _p(wf), ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                                       ctypes.c_int(bits), ctypes.c_int(rank), ctypes.c_int(1 if dtype == "bf16" else 0))
+    if rc != 0:
+        raise ValueError("oracle_quantize_feedback rejected the request")
+    return codes, scales, zeros, r, wf

@@ -21,6 +21,11 @@
  * one output row.  The paper does not fix a storage format for the codes; the
  * packed formats below are this project's (see the comments at each packer).
  *
+ * The feedback quantiser of Section 4.1 (oracle_quantize_feedback, below) is
+ * pinned by a hand-worked group with ties, exact recovery of weights that lie
+ * on a quantiser grid, the s/2 bound of Eq. "diff" in double precision, and
+ * numpy's float16 conversion.
+ *
  * Pins (tests/test_oracle_*.py): hand-worked 8x8 layer, literal packed words,
  * closed form for x = 1, numpy fp64 matmul special cases (rank 0, codes == zero
  * points), linearity, row permutation, token independence, MAC-count ratio
@@ -215,6 +220,120 @@ int oracle_linear(const uint16_t *x, const uint32_t *qweight, const uint16_t *sc
     free(xd);
     free(t);
     return 0;
+}
+
+/* ---- feedback quantiser (Section 4.1) --------------------------------------
+ * The main path of FBQuant stores Q(W - Sigma), Sigma = B.A, so that the
+ * reconstructed weight  W_F = Q(W - Sigma) + Sigma  stays within s/2 of W
+ * (Eq. "diff" and the bound below it, for a round-to-nearest Q).  The paper
+ * says only "linear quantizer", group size 128, round-to-nearest with scaling
+ * factor s; the reading taken here (asymmetric min-max per group) is:
+ *
+ *   r[n][k]   = W[n][k] - sum_j B[n][j]*A[j][k]          (the fed-back residual)
+ *   per group g of `group` consecutive k of one row, with maxq = 2^bits - 1:
+ *     mn = min r, mx = max r
+ *     s  = max((mx - mn)/maxq, 2^-14),  z = rint(-mn/s)                if mx > mn
+ *     s  = max(|mn|, 2^-14),            z = 1 if mn < 0 else 0         if mx == mn
+ *     s, z are stored as fp16 (round to nearest even); everything below uses
+ *     the STORED values, so that dequantisation inverts exactly what was coded
+ *   q[n][k]   = clamp(rint(r/s + z), 0, maxq)            (ties to even)
+ *   W_F[n][k] = s*(q - z) + Sigma[n][k]
+ *
+ * A rounding decides every code, so this function works in the arithmetic of
+ * the device kernel it checks, IEEE single precision with the operations in
+ * exactly this order: Sigma by fused multiply-adds over j ascending from 0,
+ * one subtraction for r, one division and one addition before rint, one
+ * multiplication and one addition for W_F.  (The bound itself is checked by
+ * the tests in double precision from the stored s, z and q.)
+ * W: N x K floats.  A: rank x K, B: N x rank (fp16 or bf16 bit patterns), may be
+ * NULL when rank == 0.  r_out, wf_out: N x K floats, may be NULL.
+ * Returns 0, or -1 on a malformed request. */
+static uint16_t float_to_half_bits(float f)
+{
+    /* round to nearest even, with subnormals, overflow to infinity */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    const uint32_t mag = u & 0x7FFFFFFFu;
+    if (mag >= 0x7F800000u) return (uint16_t)(sign | (mag > 0x7F800000u ? 0x7E00u : 0x7C00u));
+    if (mag >= 0x477FF000u) return (uint16_t)(sign | 0x7C00u);        /* >= 65520 rounds to infinity */
+    if (mag < 0x33000001u) return sign;                               /* <= 2^-25 rounds to zero     */
+    int e = (int)(mag >> 23) - 127;                                   /* unbiased exponent            */
+    uint32_t m = (mag & 0x7FFFFFu) | 0x800000u;                       /* 24-bit significand           */
+    int shift = (e < -14) ? (13 + (-14 - e)) : 13;                    /* bits dropped                 */
+    uint32_t kept = m >> shift, rem = m & ((1u << shift) - 1u), half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (kept & 1u))) ++kept;
+    if (e < -14) return (uint16_t)(sign | kept);                      /* subnormal (may carry to the first normal) */
+    return (uint16_t)(sign | (uint16_t)(((uint32_t)(e + 15) << 10) + (kept - 0x400u)));
+}
+
+static float bits_to_float(uint16_t bits, int act_is_bf16) { return (float)act_to_double(bits, act_is_bf16); }
+
+int oracle_quantize_feedback(const float *W, const uint16_t *A, const uint16_t *B, uint8_t *codes,
+                             uint16_t *scales, uint16_t *zeros, float *r_out, float *wf_out, int N,
+                             int K, int group, int bits, int rank, int act_is_bf16)
+{
+    if (N < 1 || K < 1 || group < 1 || K % group != 0 || rank < 0 || (bits != 3 && bits != 4)) return -1;
+    if (rank > 0 && (!A || !B)) return -1;
+    const int G = K / group;
+    const float maxq = (float)((1 << bits) - 1);
+    const float smin = ldexpf(1.0f, -14);
+    float *sig = (float *)malloc(sizeof(float) * (size_t)group);
+    float *r = (float *)malloc(sizeof(float) * (size_t)group);
+    if (!sig || !r) { free(sig); free(r); return -1; }
+    for (int n = 0; n < N; ++n)
+        for (int g = 0; g < G; ++g) {
+            float mn = INFINITY, mx = -INFINITY;
+            for (int i = 0; i < group; ++i) {
+                const int k = g * group + i;
+                float acc = 0.0f;
+                for (int j = 0; j < rank; ++j)
+                    acc = fmaf(bits_to_float(B[(size_t)n * rank + j], act_is_bf16),
+                               bits_to_float(A[(size_t)j * K + k], act_is_bf16), acc);
+                sig[i] = acc;
+                r[i] = W[(size_t)n * K + k] - acc;
+                if (r[i] < mn) mn = r[i];
+                if (r[i] > mx) mx = r[i];
+            }
+            float s, z;
+            if (mx > mn) {
+                s = (mx - mn) / maxq;
+                if (s < smin) s = smin;
+                const float sh = (float)half_bits_to_double(float_to_half_bits(s));
+                z = rintf(-mn / sh);
+            } else {
+                s = fabsf(mn);
+                if (s < smin) s = smin;
+                z = (mn < 0.0f) ? 1.0f : 0.0f;
+            }
+            const uint16_t s_bits = float_to_half_bits(s), z_bits = float_to_half_bits(z);
+            const float sh = (float)half_bits_to_double(s_bits), zh = (float)half_bits_to_double(z_bits);
+            scales[(size_t)n * G + g] = s_bits;
+            zeros[(size_t)n * G + g] = z_bits;
+            for (int i = 0; i < group; ++i) {
+                const size_t idx = (size_t)n * K + (size_t)g * group + i;
+                const float t = r[i] / sh;
+                float q = rintf(t + zh);
+                if (q < 0.0f) q = 0.0f;
+                if (q > maxq) q = maxq;
+                codes[idx] = (uint8_t)q;
+                if (r_out) r_out[idx] = r[i];
+                if (wf_out) {
+                    const float wq = sh * (q - zh);
+                    wf_out[idx] = wq + sig[i];
+                }
+            }
+        }
+    free(sig);
+    free(r);
+    return 0;
+}
+
+/* fp16 bit patterns (round to nearest even) of n floats: lets the tests pin the
+ * conversion above against numpy's. */
+void oracle_float_to_half(const float *in, uint16_t *out, int n)
+{
+    for (int i = 0; i < n; ++i) out[i] = float_to_half_bits(in[i]);
 }
 
 /* Widen n stored 16-bit values to double (lets the tests check the two
