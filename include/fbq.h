@@ -137,6 +137,28 @@ int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const void *scale
                        const void *zeros, const void *A, const void *B, void *y, int M, int N,
                        int K, int group, int bits, int rank, int act_is_bf16, void *stream);
 
+/* Feedback quantiser, the offline producer of (codes, s, z) for the main path (Section 4.1:
+ * the main path stores Q(W - Sigma) with Sigma = B.A, so that the reconstructed weight
+ * W_F = Q(W - Sigma) + Sigma stays within s/2 of W for a round-to-nearest Q).  Per group of
+ * `group` consecutive input channels of one output row, with r = W - B.A:
+ *     s = max((max r - min r) / (2^bits - 1), 2^-14),  z = rint(-min r / s),
+ *     q = clamp(rint(r / s + z), 0, 2^bits - 1),       ties to even
+ * (a constant group c gets s = max(|c|, 2^-14), z = 1 if c < 0 else 0).  s and z are rounded
+ * to fp16 and the stored values are the ones used for q.  All decisions are single-precision
+ * IEEE operations in this order, Sigma accumulated with fused multiply-adds over the rank
+ * index ascending.
+ *   W      device, [N][K] fp32 (the weights to be quantised)
+ *   A, B   device, [rank][K] and [N][rank], fp16 or bf16 (act_is_bf16); NULL when rank == 0
+ *   codes  device, [N][K] bytes, one code per byte (feed them to fbq_pack_int3 / fbq_pack_int4)
+ *   scales, zeros  device, fp16 [N][K/group]
+ *   WF     device, [N][K] fp32 or NULL: receives W_F = s*(q - z) + Sigma
+ * group: 1..1024 dividing K (a multiple of 8 (INT4) or 32 (INT3) if the codes are to be packed);
+ * K/group <= 65535.  Asynchronous on `stream`; nothing is allocated.  Returns FBQ_OK,
+ * FBQ_ERR_BADARG, FBQ_ERR_ALIGN or FBQ_ERR_CUDA. */
+int fbq_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes, void *scales,
+                          void *zeros, float *WF, int N, int K, int group, int bits, int rank,
+                          int act_is_bf16, void *stream);
+
 /* Several independent linears of the same kind in one call: the grouped decode of a decoder
  * layer, where q, k, v (and gate, up) read the same x through different weights, or any set
  * of layers whose inputs are ready (Algorithm 1 reconstructs each of the seven projections

@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     pack,
     packed_words,
     poll_status,
+    quantize_feedback,
     release_workspaces,
     select_kernel,
     set_option,

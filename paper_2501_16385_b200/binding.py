@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_linear_noalloc.argtypes = [vp] * 7 + [i32] * 7 + [vp]
+        L.fbq_quantize_feedback.argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_linear_batch.argtypes = [ctypes.POINTER(Problem), i32, i32, i32, i32, i32, i32, vp]
         L.fbq_select_kernel.argtypes = [i32] * 7
         L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
@@ -160,6 +161,23 @@ def linear_noalloc(x, qweight, scales, zeros, A, B, N: int, group: int, bits: in
                                     _ptr(y), M, N, K, group, bits, rank, bf16, _stream(stream)),
            "fbq_linear_noalloc")
     return y
+
+
+def quantize_feedback(W, A, B, group: int, bits: int, want_wf: bool = False, stream=None):
+    """fbq_quantize_feedback: W [N, K] float32 on the device, A [rank, K] / B [N, rank] (fp16 or
+    bf16, or None).  Returns (codes uint8 [N, K], scales, zeros fp16 [N, K/group], W_F or None)."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+    N, K = W.shape
+    rank = 0 if A is None else A.shape[0]
+    bf16 = 1 if (A is not None and A.dtype == torch.bfloat16) else 0
+    codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
+    scales = torch.empty((N, K // group), dtype=torch.float16, device=W.device)
+    zeros = torch.empty((N, K // group), dtype=torch.float16, device=W.device)
+    wf = torch.empty((N, K), dtype=torch.float32, device=W.device) if want_wf else None
+    _check(lib().fbq_quantize_feedback(_ptr(W), _ptr(A), _ptr(B), _ptr(codes), _ptr(scales), _ptr(zeros), _ptr(wf),
+                                       N, K, group, bits, rank, bf16, _stream(stream)), "fbq_quantize_feedback")
+    return codes, scales, zeros, wf
 
 
 def make_batch(problems):

@@ -234,6 +234,23 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
     return FBQ_OK;
 }
 
+int fbq_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes, void *scales, void *zeros,
+                          float *WF, int N, int K, int group, int bits, int rank, int act_is_bf16, void *stream)
+{
+    if (N < 1 || K < 1 || group < 1 || group > 1024 || K % group != 0 || K / group > 65535 || rank < 0) return FBQ_ERR_BADARG;
+    if (bits != 3 && bits != 4) return FBQ_ERR_BADARG;
+    if (!W || !codes || !scales || !zeros || (rank > 0 && (!A || !B))) return FBQ_ERR_BADARG;
+    if ((reinterpret_cast<uintptr_t>(W) & 3u) || (WF && (reinterpret_cast<uintptr_t>(WF) & 3u)) ||
+        (reinterpret_cast<uintptr_t>(scales) & 1u) || (reinterpret_cast<uintptr_t>(zeros) & 1u) ||
+        (rank > 0 && ((reinterpret_cast<uintptr_t>(A) & 1u) || (reinterpret_cast<uintptr_t>(B) & 1u))))
+        return FBQ_ERR_ALIGN;
+    if (launch_quantize_feedback(W, A, B, codes, static_cast<__half *>(scales), static_cast<__half *>(zeros), WF, N, K, group,
+                                 bits, rank, act_is_bf16 != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FBQ_ERR_CUDA;
+    ++g_launches;
+    return FBQ_OK;
+}
+
 static int linear_common(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
                          const void *B, void *y, int M, int N, int K, int group, int bits, int rank, bool bf16,
                          void *stream)

@@ -62,6 +62,9 @@ cudaError_t launch_unpack(const uint32_t *qw, uint8_t *codes, int N, int K, int 
 cudaError_t launch_dequant(const uint32_t *qw, const __half *sc, const __half *ze, float *W, int N,
                            int K, int group, int bits, cudaStream_t s);
 cudaError_t launch_generic(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
+cudaError_t launch_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes, __half *scales,
+                                     __half *zeros, float *WF, int N, int K, int group, int bits, int rank, bool bf16,
+                                     cudaStream_t s);
 
 struct DecodeTuning {
     int sk = 0, chunk = 0, depth = 0, max_ctas = 0, pdl = 1;
