@@ -146,7 +146,7 @@ def float_to_half(a: np.ndarray) -> np.ndarray:
 
 def quantize_feedback(W: np.ndarray, A, B, group: int, bits: int, *, dtype: str = "f16"):
     """Feedback quantiser of Section 4.1 on W [N, K] float32 with Sigma = B.A (A [rank, K],
-    B [N, rank] as 16-bit patterns, or None for rank 0).  Returns codes (uint8 [N, K]),
+    B [N, rank] as 16-bit patterns, or float32 with dtype="f32", or None for rank 0).  Returns codes (uint8 [N, K]),
     scales, zeros (uint16 fp16 patterns [N, K/group]), r = W - Sigma and W_F (float32 [N, K])."""
     _load()
     W = np.ascontiguousarray(W, dtype=np.float32)
@@ -159,12 +159,16 @@ def quantize_feedback(W: np.ndarray, A, B, group: int, bits: int, *, dtype: str 
     zeros = np.empty((N, K // group), dtype=np.uint16)
     r = np.empty((N, K), dtype=np.float32)
     wf = np.empty((N, K), dtype=np.float32)
-    Ab = _u16(A) if rank else None
-    Bb = _u16(B) if rank else None
+    if dtype == "f32":
+        Ab = np.ascontiguousarray(A, dtype=np.float32) if rank else None
+        Bb = np.ascontiguousarray(B, dtype=np.float32) if rank else None
+    else:
+        Ab = _u16(A) if rank else None
+        Bb = _u16(B) if rank else None
     _lib.oracle_quantize_feedback.restype = ctypes.c_int
     rc = _lib.oracle_quantize_feedback(_p(W), _p(Ab) if rank else None, _p(Bb) if rank else None, _p(codes), _p(scales),
                                        _p(zeros), _p(r), _p(wf), ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
-                                       ctypes.c_int(bits), ctypes.c_int(rank), ctypes.c_int(1 if dtype == "bf16" else 0))
+                                       ctypes.c_int(bits), ctypes.c_int(rank), ctypes.c_int({"f16": 0, "bf16": 1, "f32": 2}[dtype]))
     if rc != 0:
         raise ValueError("oracle_quantize_feedback rejected the request")
     return codes, scales, zeros, r, wf

@@ -245,8 +245,9 @@ int oracle_linear(const uint16_t *x, const uint32_t *qweight, const uint16_t *sc
  * one subtraction for r, one division and one addition before rint, one
  * multiplication and one addition for W_F.  (The bound itself is checked by
  * the tests in double precision from the stored s, z and q.)
- * W: N x K floats.  A: rank x K, B: N x rank (fp16 or bf16 bit patterns), may be
- * NULL when rank == 0.  r_out, wf_out: N x K floats, may be NULL.
+ * W: N x K floats.  A: rank x K, B: N x rank: fp16 bit patterns (ab_kind 0), bf16 bit
+ * patterns (1) or floats (2, the master copies of the reconstruction loop); may be NULL
+ * when rank == 0.  r_out, wf_out: N x K floats, may be NULL.
  * Returns 0, or -1 on a malformed request. */
 static uint16_t float_to_half_bits(float f)
 {
@@ -267,11 +268,16 @@ static uint16_t float_to_half_bits(float f)
     return (uint16_t)(sign | (uint16_t)(((uint32_t)(e + 15) << 10) + (kept - 0x400u)));
 }
 
-static float bits_to_float(uint16_t bits, int act_is_bf16) { return (float)act_to_double(bits, act_is_bf16); }
+/* element i of a sub-branch matrix: fp16 (kind 0) or bf16 (kind 1) bit patterns, or floats (kind 2) */
+static float ab_elem(const void *p, size_t i, int kind)
+{
+    if (kind == 2) return ((const float *)p)[i];
+    return (float)act_to_double(((const uint16_t *)p)[i], kind == 1);
+}
 
-int oracle_quantize_feedback(const float *W, const uint16_t *A, const uint16_t *B, uint8_t *codes,
+int oracle_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes,
                              uint16_t *scales, uint16_t *zeros, float *r_out, float *wf_out, int N,
-                             int K, int group, int bits, int rank, int act_is_bf16)
+                             int K, int group, int bits, int rank, int ab_kind)
 {
     if (N < 1 || K < 1 || group < 1 || K % group != 0 || rank < 0 || (bits != 3 && bits != 4)) return -1;
     if (rank > 0 && (!A || !B)) return -1;
@@ -288,8 +294,7 @@ int oracle_quantize_feedback(const float *W, const uint16_t *A, const uint16_t *
                 const int k = g * group + i;
                 float acc = 0.0f;
                 for (int j = 0; j < rank; ++j)
-                    acc = fmaf(bits_to_float(B[(size_t)n * rank + j], act_is_bf16),
-                               bits_to_float(A[(size_t)j * K + k], act_is_bf16), acc);
+                    acc = fmaf(ab_elem(B, (size_t)n * rank + j, ab_kind), ab_elem(A, (size_t)j * K + k, ab_kind), acc);
                 sig[i] = acc;
                 r[i] = W[(size_t)n * K + k] - acc;
                 if (r[i] < mn) mn = r[i];
