@@ -49,7 +49,7 @@ def test_printed_gradient_is_that_of_the_detached_objective():
         assert np.isclose(num, np.sum(G * V), rtol=1e-6)
     # with the straight-through surrogate Q(w) = w and nothing detached, Delta_F = W - (W - Sigma) - Sigma
     # vanishes identically, hence its gradient too: the reason the paper detaches the feedback signal
-    assert np.all(W.astype(np.float64) - (W.astype(np.float64) - S0) - S0 == 0)
+    assert np.abs(W.astype(np.float64) - (W.astype(np.float64) - S0) - S0).max() < 1e-15
 
 
 def test_chain_rule_through_the_low_rank_factors():
