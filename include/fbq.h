@@ -159,6 +159,25 @@ int fbq_quantize_feedback(const float *W, const void *A, const void *B, uint8_t 
                           void *zeros, float *WF, int N, int K, int group, int bits, int rank,
                           int act_is_bf16, void *stream);
 
+/* Layer-wise reconstruction (Algorithm 1, Section 4.2): the offline loop that fits the sub-branch.
+ * With H = X^T X of the layer's calibration activations X [T][K] (fbq_gram), one call of
+ * fbq_reconstruct_step performs lines 5-9 of Algorithm 1 once:
+ *     Delta_F = W - Q(W - B A) - B A          Q: the quantiser of fbq_quantize_feedback, detached
+ *     loss    = tr(Delta_F H Delta_F^T)       = ||W X^T - W_F X^T||_F^2, before the update
+ *     G       = -2 Delta_F H                  (the paper's dL/dSigma)
+ *     A      <- A - lr B^T G,   B <- B - lr G A^T      (both from the old A and B)
+ *   W [N][K], H [K][K], A [rank][K], B [N][rank]: device fp32 (A and B are the master copies and
+ *   are updated in place); loss: device float or NULL; workspace: device,
+ *   fbq_reconstruct_workspace_floats(N, K, rank) floats, contents meaningless afterwards.
+ * The three dense products are fp32 cuBLAS GEMMs (pedantic math); cuBLAS is loaded on first use
+ * (make that first call outside a stream capture), and FBQ_ERR_UNSUPPORTED is returned when it
+ * cannot be loaded.  Initialise as Algorithm 1 says (A ~ N(0, sigma^2), B = 0), iterate, then
+ * round A and B to the inference type and call fbq_quantize_feedback once more for (codes, s, z). */
+size_t fbq_reconstruct_workspace_floats(int N, int K, int rank);
+int fbq_gram(const float *X, float *H, int T, int K, void *stream);
+int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, float lr, float *loss,
+                         float *workspace, int N, int K, int group, int bits, int rank, void *stream);
+
 /* Several independent linears of the same kind in one call: the grouped decode of a decoder
  * layer, where q, k, v (and gate, up) read the same x through different weights, or any set
  * of layers whose inputs are ready (Algorithm 1 reconstructs each of the seven projections

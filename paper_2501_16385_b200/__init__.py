@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     STATUS,
     dequant,
     get_option,
+    gram,
     launch_count,
     lib,
     library_path,
@@ -28,6 +29,7 @@ from .binding import (  # noqa: F401
     packed_words,
     poll_status,
     quantize_feedback,
+    reconstruct_step,
     release_workspaces,
     select_kernel,
     set_option,

@@ -56,6 +56,10 @@ def lib() -> ctypes.CDLL:
         L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_linear_noalloc.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_quantize_feedback.argtypes = [vp] * 7 + [i32] * 6 + [vp]
+        L.fbq_reconstruct_workspace_floats.restype = ctypes.c_size_t
+        L.fbq_reconstruct_workspace_floats.argtypes = [i32, i32, i32]
+        L.fbq_gram.argtypes = [vp, vp, i32, i32, vp]
+        L.fbq_reconstruct_step.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, i32, vp]
         L.fbq_linear_batch.argtypes = [ctypes.POINTER(Problem), i32, i32, i32, i32, i32, i32, vp]
         L.fbq_select_kernel.argtypes = [i32] * 7
         L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
@@ -178,6 +182,34 @@ def quantize_feedback(W, A, B, group: int, bits: int, want_wf: bool = False, str
     _check(lib().fbq_quantize_feedback(_ptr(W), _ptr(A), _ptr(B), _ptr(codes), _ptr(scales), _ptr(zeros), _ptr(wf),
                                        N, K, group, bits, rank, bf16, _stream(stream)), "fbq_quantize_feedback")
     return codes, scales, zeros, wf
+
+
+def gram(X, stream=None):
+    """fbq_gram: H = X^T X (float32 [K, K]) of calibration activations X [T, K] float32."""
+    import torch
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous()
+    T, K = X.shape
+    H = torch.empty((K, K), dtype=torch.float32, device=X.device)
+    _check(lib().fbq_gram(_ptr(X), _ptr(H), T, K, _stream(stream)), "fbq_gram")
+    return H
+
+
+def reconstruct_step(W, H, A, B, lr: float, group: int, bits: int, workspace=None, loss=None, stream=None):
+    """fbq_reconstruct_step: one iteration of Algorithm 1 on float32 device tensors; A and B are
+    updated in place.  Returns (loss tensor [1], workspace) so that both can be reused."""
+    import torch
+    N, K = W.shape
+    rank = A.shape[0]
+    for t in (W, H, A, B):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+    need = int(lib().fbq_reconstruct_workspace_floats(N, K, rank))
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(need, dtype=torch.float32, device=W.device)
+    if loss is None:
+        loss = torch.zeros(1, dtype=torch.float32, device=W.device)
+    _check(lib().fbq_reconstruct_step(_ptr(W), _ptr(H), _ptr(A), _ptr(B), float(lr), _ptr(loss), _ptr(workspace), N, K,
+                                      group, bits, rank, _stream(stream)), "fbq_reconstruct_step")
+    return loss, workspace
 
 
 def make_batch(problems):

@@ -8,10 +8,11 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfbq.so")
-SOURCES = ["fbq_api.cu", "fbq_pack.cu", "fbq_generic.cu", "fbq_decode.cu", "fbq_prefill.cu", "fbq_noalloc.cu", "fbq_quant.cu"]
+SOURCES = ["fbq_api.cu", "fbq_pack.cu", "fbq_generic.cu", "fbq_decode.cu", "fbq_prefill.cu", "fbq_noalloc.cu", "fbq_quant.cu",
+           "fbq_reconstruct.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math" if False else "-Xptxas=-v", "-Xcompiler", "-fPIC", "-shared",
-              "-cudart", "static"]
+              "-cudart", "static", "-ldl"]
 
 
 def _stale() -> bool:

@@ -244,11 +244,36 @@ int fbq_quantize_feedback(const float *W, const void *A, const void *B, uint8_t 
         (reinterpret_cast<uintptr_t>(scales) & 1u) || (reinterpret_cast<uintptr_t>(zeros) & 1u) ||
         (rank > 0 && ((reinterpret_cast<uintptr_t>(A) & 1u) || (reinterpret_cast<uintptr_t>(B) & 1u))))
         return FBQ_ERR_ALIGN;
-    if (launch_quantize_feedback(W, A, B, codes, static_cast<__half *>(scales), static_cast<__half *>(zeros), WF, N, K, group,
-                                 bits, rank, act_is_bf16 != 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (launch_quantize_feedback(W, A, B, codes, static_cast<__half *>(scales), static_cast<__half *>(zeros), WF, nullptr, N, K,
+                                 group, bits, rank, act_is_bf16 ? 1 : 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return FBQ_ERR_CUDA;
     ++g_launches;
     return FBQ_OK;
+}
+
+size_t fbq_reconstruct_workspace_floats(int N, int K, int rank)
+{
+    if (N < 1 || K < 1 || rank < 1) return 0;
+    return reconstruct_workspace_floats(N, K, rank);
+}
+
+int fbq_gram(const float *X, float *H, int T, int K, void *stream)
+{
+    if (!X || !H || T < 1 || K < 1) return FBQ_ERR_BADARG;
+    const int rc = run_gram(X, H, T, K, static_cast<cudaStream_t>(stream));
+    if (rc == FBQ_OK) ++g_launches;
+    return rc;
+}
+
+int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, float lr, float *loss, float *workspace, int N,
+                         int K, int group, int bits, int rank, void *stream)
+{
+    if (N < 1 || K < 1 || rank < 1 || group < 1 || group > 1024 || K % group != 0 || K / group > 65535) return FBQ_ERR_BADARG;
+    if (bits != 3 && bits != 4) return FBQ_ERR_BADARG;
+    if (!W || !H || !A || !B || !workspace) return FBQ_ERR_BADARG;
+    const int rc = run_reconstruct_step(W, H, A, B, lr, loss, workspace, N, K, group, bits, rank, static_cast<cudaStream_t>(stream));
+    if (rc == FBQ_OK) g_launches += loss ? 5 : 3;       // own kernels: quantiser, (two-stage reduction), two updates
+    return rc;
 }
 
 static int linear_common(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,

@@ -63,8 +63,14 @@ cudaError_t launch_dequant(const uint32_t *qw, const __half *sc, const __half *z
                            int K, int group, int bits, cudaStream_t s);
 cudaError_t launch_generic(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
 cudaError_t launch_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes, __half *scales,
-                                     __half *zeros, float *WF, int N, int K, int group, int bits, int rank, bool bf16,
-                                     cudaStream_t s);
+                                     __half *zeros, float *WF, float *Delta, int N, int K, int group, int bits, int rank,
+                                     int ab_kind, cudaStream_t s);
+cudaError_t launch_scaled_dot(const float *a, const float *b, size_t n, float scale, float *partial, float *out, cudaStream_t s);
+cudaError_t launch_axpy(float *y, const float *x, float alpha, size_t n, cudaStream_t s);
+size_t reconstruct_workspace_floats(int N, int K, int rank);
+int run_gram(const float *X, float *H, int T, int K, cudaStream_t s);
+int run_reconstruct_step(const float *W, const float *H, float *A, float *B, float lr, float *loss, float *ws, int N, int K,
+                         int group, int bits, int rank, cudaStream_t s);
 
 struct DecodeTuning {
     int sk = 0, chunk = 0, depth = 0, max_ctas = 0, pdl = 1;
