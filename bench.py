@@ -248,20 +248,19 @@ def time_plain_steps(fbq, torch, pool, steps: int):
 
 
 def time_e2e(fbq, torch, pool, steps: int, warmup: int):
-    """Same steps through fbq_linear_hostio: x from pinned host memory, y read back, every step."""
+    """Same steps end to end through the C ABI with HOST buffers: one fbq_linear_batch_hostio call per
+    step (x of the seven linears from pinned host memory, y read back to pinned host memory), then a
+    stream synchronise so that the step's results are on the host.  Wall clock."""
     L = len(pool)
     xs = [[d.x.cpu().pin_memory() for d in layer] for layer in pool]
     ys = [[torch.empty((M_TOKENS, d.N), dtype=torch.float16).pin_memory() for d in layer] for layer in pool]
-
-    streams = [torch.cuda.current_stream()] + side_streams(torch)
+    batches = [fbq.make_batch([(xs[li][j], d.qweight, d.scales, d.zeros, d.A, d.B, ys[li][j]) for j, d in enumerate(layer)])
+               for li, layer in enumerate(pool)]
+    main = torch.cuda.current_stream()
 
     def one(i):
-        layer = pool[i % L]
-        for j, d in enumerate(layer):
-            fbq.linear_hostio(xs[i % L][j], d.qweight, d.scales, d.zeros, d.A, d.B, ys[i % L][j], d.N, GROUP, BITS,
-                              stream=streams[j % len(streams)])
-        for st in streams:
-            st.synchronize()                          # the step's results are read on the host
+        fbq.linear_batch(None, GROUP, BITS, stream=main, batch=batches[i % L], host_io=True)
+        main.synchronize()                            # the step's results are read on the host
 
     for i in range(max(3, warmup)):
         one(i)

@@ -211,6 +211,13 @@ typedef struct fbq_problem {
 } fbq_problem;
 int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, int bits, int rank,
                      int act_is_bf16, void *stream);
+/* The same with every problem's x and y in HOST memory (pinned for asynchronous copies), the
+ * weights on the device as before: per problem the library copies x to a staging buffer it
+ * keeps per stream, runs the linear, and copies y back, all on the stream the problem runs on.
+ * y is complete once work queued on `stream` after the call has run (synchronise `stream`
+ * before reading it).  The end-to-end path of the benchmark. */
+int fbq_linear_batch_hostio(const fbq_problem *problems, int count, int M, int group, int bits, int rank,
+                            int act_is_bf16, void *stream);
 
 /* Which kernel fbq_linear / fbq_linear_bf16 would run for this shape, or
  * FBQ_KERNEL_NONE when the shape is rejected.  Pure host logic. */

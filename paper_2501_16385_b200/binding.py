@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.fbq_gram.argtypes = [vp, vp, i32, i32, vp]
         L.fbq_reconstruct_step.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, i32, vp]
         L.fbq_linear_batch.argtypes = [ctypes.POINTER(Problem), i32, i32, i32, i32, i32, i32, vp]
+        L.fbq_linear_batch_hostio.argtypes = [ctypes.POINTER(Problem), i32, i32, i32, i32, i32, i32, vp]
         L.fbq_select_kernel.argtypes = [i32] * 7
         L.fbq_set_option.argtypes = [ctypes.c_char_p, i32]
         L.fbq_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(i32)]
@@ -221,7 +222,7 @@ def make_batch(problems):
     arr = (Problem * max(n, 1))()
     M = rank = bf16 = None
     for i, (x, qw, s, z, A, B, y) in enumerate(problems):
-        assert x.is_cuda and x.is_contiguous() and y.is_contiguous() and x.dtype == y.dtype
+        assert x.is_contiguous() and y.is_contiguous() and x.dtype == y.dtype and x.is_cuda == y.is_cuda
         m, r, b = x.shape[0], (0 if A is None else A.shape[0]), (1 if x.dtype == torch.bfloat16 else 0)
         if i == 0:
             M, rank, bf16 = m, r, b
@@ -230,11 +231,13 @@ def make_batch(problems):
     return arr, n, M or 0, rank or 0, bf16 or 0
 
 
-def linear_batch(problems, group: int, bits: int, stream=None, batch=None):
+def linear_batch(problems, group: int, bits: int, stream=None, batch=None, host_io: bool = False):
     """fbq_linear_batch over a list of (x, qweight, scales, zeros, A, B, y) tuples, or over a
-    descriptor array made earlier by make_batch (``batch``).  The y tensors are written."""
+    descriptor array made earlier by make_batch (``batch``).  The y tensors are written.  With
+    host_io the x and y tensors are (pinned) CPU tensors: fbq_linear_batch_hostio."""
     arr, n, M, rank, bf16 = batch if batch is not None else make_batch(problems)
-    _check(lib().fbq_linear_batch(arr, n, M, group, bits, rank, bf16, _stream(stream)), "fbq_linear_batch")
+    fn = lib().fbq_linear_batch_hostio if host_io else lib().fbq_linear_batch
+    _check(fn(arr, n, M, group, bits, rank, bf16, _stream(stream)), "fbq_linear_batch")
 
 
 def select_kernel(M, N, K, group, bits, rank, bf16=False) -> int:

@@ -327,8 +327,8 @@ static BatchLanes *lanes_for(int want)
     return &b;
 }
 
-int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, int bits, int rank, int act_is_bf16,
-                     void *stream)
+static int linear_batch_common(const fbq_problem *problems, int count, int M, int group, int bits, int rank, int act_is_bf16,
+                               void *stream, bool host_io)
 {
     if (count < 0 || count > FBQ_BATCH_MAX || (count > 0 && !problems)) return FBQ_ERR_BADARG;
     if (count == 0) return FBQ_OK;
@@ -352,10 +352,33 @@ int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, i
         all_decode = all_decode && select_kernel(M, q.N, q.K, group, bits, rank, a[i].bf16) == FBQ_KERNEL_DECODE;
         total_cost += (double)q.N * q.K;
     }
+    // With host_io, x and y of every problem are host buffers: x is copied to, and y back from,
+    // staging buffers kept per stream, on the stream the problem runs on.
+    auto stage_in = [&](LinearArgs &la, cudaStream_t st) -> int {
+        if (!host_io) return FBQ_OK;
+        Workspace *ws = workspace_for(st);
+        if (!ws || !la.x || !la.y) return ws ? FBQ_ERR_BADARG : FBQ_ERR_CUDA;
+        const size_t xb = (size_t)M * la.K * 2, yb = (size_t)M * la.N * 2;
+        char *sx = static_cast<char *>(ws->stage_x), *sy = static_cast<char *>(ws->stage_y);
+        if (grow(sx, ws->stage_x_bytes, xb, 1, st) != cudaSuccess) return FBQ_ERR_CUDA;
+        if (grow(sy, ws->stage_y_bytes, yb, 1, st) != cudaSuccess) return FBQ_ERR_CUDA;
+        ws->stage_x = sx;
+        ws->stage_y = sy;
+        if (cudaMemcpyAsync(sx, la.x, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FBQ_ERR_CUDA;
+        la.x = sx;
+        la.y = sy;
+        return FBQ_OK;
+    };
+    auto stage_out = [&](const LinearArgs &la, void *y_host, cudaStream_t st) -> int {
+        if (!host_io) return FBQ_OK;
+        return cudaMemcpyAsync(y_host, la.y, (size_t)M * la.N * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess ? FBQ_OK : FBQ_ERR_CUDA;
+    };
     if (!all_decode) {
         // one after the other on the caller's stream (prefill-sized problems fill the GPU by themselves)
         for (int i = 0; i < count; ++i) {
-            const int rc = run_linear(a[i], main);
+            int rc = stage_in(a[i], main);
+            if (rc == FBQ_OK) rc = run_linear(a[i], main);
+            if (rc == FBQ_OK) rc = stage_out(a[i], problems[i].y, main);
             if (rc != FBQ_OK) return rc;
         }
         return FBQ_OK;
@@ -372,7 +395,9 @@ int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, i
         if (cudaStreamWaitEvent(lanes->side[i], lanes->fork, 0) != cudaSuccess) { rc = FBQ_ERR_CUDA; break; }
         ++forked;
         const int ctas = std::max(8, (int)(g_opt.batch_ctas * ((double)a[i].N * a[i].K / total_cost) + 0.5));
-        rc = run_linear(a[i], lanes->side[i], ctas);
+        rc = stage_in(a[i], lanes->side[i]);
+        if (rc == FBQ_OK) rc = run_linear(a[i], lanes->side[i], ctas);
+        if (rc == FBQ_OK) rc = stage_out(a[i], problems[i].y, lanes->side[i]);
         if (rc != FBQ_OK) break;
     }
     for (int i = 0; i < forked; ++i) {              // always rejoin what was forked (also under stream capture)
@@ -381,6 +406,18 @@ int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, i
             rc = (rc == FBQ_OK) ? FBQ_ERR_CUDA : rc;
     }
     return rc;
+}
+
+int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, int bits, int rank, int act_is_bf16,
+                     void *stream)
+{
+    return linear_batch_common(problems, count, M, group, bits, rank, act_is_bf16, stream, false);
+}
+
+int fbq_linear_batch_hostio(const fbq_problem *problems, int count, int M, int group, int bits, int rank, int act_is_bf16,
+                            void *stream)
+{
+    return linear_batch_common(problems, count, M, group, bits, rank, act_is_bf16, stream, true);
 }
 
 int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *scales, const void *zeros,

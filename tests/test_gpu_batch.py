@@ -85,6 +85,25 @@ def test_batch_under_graph_replay(fbq):
         assert torch.allclose(r.float(), p[6].float(), rtol=2e-2, atol=2e-3)
 
 
+def test_batch_hostio_reads_and_writes_host_buffers(fbq):
+    import torch
+    inps, devs, probs = _problems(fbq, 1, 3, 64, "f16", 4700)
+    host = [(p[0].cpu().pin_memory(), p[1], p[2], p[3], p[4], p[5], torch.zeros(p[6].shape, dtype=p[6].dtype).pin_memory())
+            for p in probs]
+    fbq.linear_batch(probs, 128, 3)
+    fbq.linear_batch(host, 128, 3, host_io=True)
+    torch.cuda.synchronize()
+    assert fbq.poll_status() == 0
+    for p, h in zip(probs, host):
+        assert torch.allclose(p[6].cpu().float(), h[6].float(), rtol=2e-2, atol=2e-3)
+        assert h[6].abs().max() > 0
+    one = host[:1]                                        # a single problem goes the sequential way
+    one[0][6].zero_()
+    fbq.linear_batch(one, 128, 3, host_io=True)
+    torch.cuda.synchronize()
+    assert torch.allclose(probs[0][6].cpu().float(), one[0][6].float(), rtol=2e-2, atol=2e-3)
+
+
 def test_batch_falls_back_for_prefill_sized_problems(fbq):
     import torch
     inps = [make_linear(40, 256, 256, 4, 8, seed=4600 + i) for i in range(2)]
