@@ -189,13 +189,14 @@ int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, flo
  *   - `problems` is a HOST array of `count` (<= FBQ_BATCH_MAX) descriptors of DEVICE
  *     pointers (layouts and alignment as for fbq_linear); it is read before the call returns.
  *   - When every problem is decode sized (M <= 16 and the decode kernel's domain) the
- *     problems run concurrently: each on a side stream of the library, forked from and
- *     joined to `stream` with events, its grid bounded in proportion to its share of the
- *     codes ("batch_ctas" CTAs in total), so that the whole batch is resident at once and
- *     every CTA's start-up cost is paid once per batch instead of once per small launch.
- *     Work queued on `stream` after the call sees every y_i.  The pattern is legal under
- *     stream capture; make the first call on a device outside a capture (it creates the
- *     side streams and events, which are kept until the process exits).
+ *     problems run concurrently, each with a share of "batch_ctas" CTAs in proportion to its
+ *     share of the codes, so that the whole batch is resident at once.  Up to 8 problems run
+ *     as ONE launch of the decode kernel over a problem list, on `stream` ("batch_single" = 1,
+ *     the default); more problems, or "batch_single" = 0, run one launch per problem on side
+ *     streams of the library, forked from and joined to `stream` with events (legal under
+ *     stream capture; make the first such call on a device outside a capture: it creates the
+ *     side streams and events, which are kept until the process exits).  Either way work
+ *     queued on `stream` after the call sees every y_i.
  *   - Otherwise the problems run one after the other on `stream`.
  * Returns the first error, or FBQ_OK. */
 #define FBQ_BATCH_MAX 16
@@ -231,6 +232,7 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "decode_depth"  0 = automatic, else stages in flight per warp
  *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
  *   "batch_ctas"    CTAs shared out among the problems of a decode-sized fbq_linear_batch (default 400)
+ *   "batch_single"  1 = such a batch of up to 8 problems is one launch (default), 0 = one launch per problem
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol

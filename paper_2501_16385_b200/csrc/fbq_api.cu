@@ -23,6 +23,7 @@ struct Options {
     DecodeTuning decode;
     int decode_t_late = 0;
     int batch_ctas = 400;
+    int batch_single = 1;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
@@ -171,6 +172,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
     if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;
+    if (!strcmp(name, "batch_single")) return &g_opt.batch_single;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
@@ -383,9 +385,41 @@ static int linear_batch_common(const fbq_problem *problems, int count, int M, in
         }
         return FBQ_OK;
     }
-    // Decode-sized problems: all at once.  Problem i runs on side stream i, forked from and joined
-    // to the caller's stream by events, with a grid bound in proportion to its share of the codes,
-    // so that the CTAs of the whole batch are resident together and finish together.
+    // Decode-sized problems: all at once, grids in proportion to the problems' share of the codes so
+    // that the CTAs of the whole batch are resident together and finish together.
+    int ctas[FBQ_BATCH_MAX];
+    for (int i = 0; i < count; ++i)
+        ctas[i] = std::max(8, (int)(g_opt.batch_ctas * ((double)a[i].N * a[i].K / total_cost) + 0.5));
+    if (g_opt.batch_single && !host_io && count <= decode_batch_max()) {
+        // One launch: the decode kernel over a problem list, on the caller's stream.  (With host
+        // buffers the per-problem streams below are faster: their small copies overlap.)
+        for (int i = 0; i < count; ++i) {
+            if (!a[i].x || !a[i].qw || !a[i].scales || !a[i].zeros || !a[i].y || (rank > 0 && (!a[i].A || !a[i].B)))
+                return FBQ_ERR_BADARG;
+            if (misaligned16(a[i].qw) || (rank > 0 && (misaligned16(a[i].A) || misaligned16(a[i].B))) || misaligned16(a[i].x) ||
+                misaligned16(a[i].y))
+                return FBQ_ERR_ALIGN;
+        }
+        Workspace *ws = workspace_for(main);
+        if (!ws) return FBQ_ERR_CUDA;
+        size_t pf = 0, tf = 0;
+        int nc = 0;
+        if (decode_batch_need(a, count, ctas, g_opt.decode, &pf, &tf, &nc)) {
+            size_t have_c = (size_t)ws->n_counters;
+            if (grow(ws->partial, ws->partial_floats, pf, sizeof(float), main) != cudaSuccess) return FBQ_ERR_CUDA;
+            if (grow(ws->t, ws->t_floats, tf, sizeof(float), main) != cudaSuccess) return FBQ_ERR_CUDA;
+            if (grow(ws->counters, have_c, (size_t)nc, sizeof(int), main) != cudaSuccess) return FBQ_ERR_CUDA;
+            ws->n_counters = (int)have_c;
+            int launches = 0;
+            const cudaError_t e = launch_decode_batch(a, count, ctas, *ws, g_opt.decode, main, &launches);
+            if (e != cudaSuccess) return FBQ_ERR_CUDA;
+            g_launches += launches;
+            return FBQ_OK;
+        }
+        // a problem has no decode plan: fall through to one launch per problem
+    }
+    // One launch per problem: problem i runs on side stream i, forked from and joined to the caller's
+    // stream by events.
     BatchLanes *lanes = lanes_for(count);
     if (!lanes) return FBQ_ERR_CUDA;
     if (cudaEventRecord(lanes->fork, main) != cudaSuccess) return FBQ_ERR_CUDA;
@@ -394,9 +428,8 @@ static int linear_batch_common(const fbq_problem *problems, int count, int M, in
     for (int i = 0; i < count; ++i) {
         if (cudaStreamWaitEvent(lanes->side[i], lanes->fork, 0) != cudaSuccess) { rc = FBQ_ERR_CUDA; break; }
         ++forked;
-        const int ctas = std::max(8, (int)(g_opt.batch_ctas * ((double)a[i].N * a[i].K / total_cost) + 0.5));
         rc = stage_in(a[i], lanes->side[i]);
-        if (rc == FBQ_OK) rc = run_linear(a[i], lanes->side[i], ctas);
+        if (rc == FBQ_OK) rc = run_linear(a[i], lanes->side[i], ctas[i]);
         if (rc == FBQ_OK) rc = stage_out(a[i], problems[i].y, lanes->side[i]);
         if (rc != FBQ_OK) break;
     }

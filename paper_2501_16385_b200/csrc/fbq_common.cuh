@@ -82,6 +82,11 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
 void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t *partial_floats,
                            int *counters);
 
+int decode_batch_max();
+bool decode_batch_need(const LinearArgs *a, int count, const int *ctas, const DecodeTuning &tune, size_t *partial_floats,
+                       size_t *t_floats, int *counters);
+cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas, Workspace &ws, const DecodeTuning &tune,
+                                cudaStream_t s, int *launches);
 bool prefill_supported(const LinearArgs &a);
 int prefill_counters_need(int M);
 cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);

@@ -67,6 +67,7 @@ struct DecodeParams {
     float *partial;     // [NT][maxslots][M][16]
     float *t;           // [M][rank], zero on entry, zero again on exit
     int *ctr;           // counters, see above; all zero on entry and on exit
+    int *status;        // word that receives FBQ_ERR_TIMEOUT when a bounded wait runs out
     int M, N, K, G, rank;
     int SK, R, NT, CHG, NS;
     int maxslots;
@@ -386,8 +387,9 @@ __device__ __forceinline__ bool tile_claim(const DecodeParams &p, int tile, int 
 }
 
 // --------------------------------------------------------------------- kernel
+// The whole CTA program; `cta` is the CTA's index among the p.R * p.SK CTAs of its problem.
 template <int BITS, typename T, int MT>
-__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams p)
+__device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int GB = (BITS == 4) ? 64 : 48;          // packed bytes of one group of one row
@@ -401,7 +403,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, tq = lane & 3;
-    const int s = blockIdx.x % p.SK, r = blockIdx.x / p.SK;
+    const int s = cta % p.SK, r = cta / p.SK;
     const int g0 = (int)((long long)s * p.G / p.SK), g1 = (int)((long long)(s + 1) * p.G / p.SK);
     const int ngs = g1 - g0;
     // whole 16-row tiles, dealt out in contiguous ranges; a "segment" is one tile of the range
@@ -507,7 +509,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
                 }
             }
         }
-        if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+        if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
         trace_mark(p, 9);
         return;
     }
@@ -698,7 +700,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             trace_mark(p, seg == 0 ? 7 : 8);
         }
         trace_mark(p, 9);
-        if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+        if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
         return;
     }
 
@@ -1008,7 +1010,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
             finish_from_slots(tile);
         }
     }
-    if (dead && lane == 0) atomicExch(p.ctr + kCtrStatus, (int)FBQ_ERR_TIMEOUT);
+    if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
 
     // ---- retire: whoever brings the count to NT + 1 (every tile finished, and the t-completing
     // warp out of its parked-tile loop) restores the scratch invariants for the next call ----
@@ -1032,6 +1034,29 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
         }
     }
     trace_mark(p, 9);
+}
+
+template <int BITS, typename T, int MT>
+__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams p)
+{
+    decode_body<BITS, T, MT>(p, (int)blockIdx.x);
+}
+
+// Several independent problems in one grid: CTAs first[i] .. first[i+1]-1 run problem i exactly as
+// a launch of its own would (its own scratch, counters and shared-memory plan); the CTAs of all
+// problems are resident together and nothing synchronises across problems.
+constexpr int kBatchMax = 8;
+struct DecodeBatch {
+    DecodeParams prob[kBatchMax];
+    int first[kBatchMax + 1];
+    int count;
+};
+template <int BITS, typename T, int MT>
+__global__ void __launch_bounds__(kThreads, 2) decode_batch_kernel(const __grid_constant__ DecodeBatch b)
+{
+    int pi = 0;
+    while (pi + 1 < b.count && (int)blockIdx.x >= b.first[pi + 1]) ++pi;
+    decode_body<BITS, T, MT>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
 }
 
 // ------------------------------------------------------------------ host side
@@ -1175,10 +1200,9 @@ void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t
     *counters = kCtrFirstTile + 2 * pl.NT;
 }
 
-cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning &tune, cudaStream_t s, int *launches)
+namespace {
+DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, float *t, int *ctr, int *status, void *trace)
 {
-    const Plan pl = make_plan(a, tune);
-    if (!pl.ok) return cudaErrorInvalidConfiguration;
     DecodeParams p{};
     p.x = a.x;
     p.qw = reinterpret_cast<const uint8_t *>(a.qw);
@@ -1187,9 +1211,10 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     p.A = a.A;
     p.B = a.B;
     p.y = a.y;
-    p.partial = ws.partial;
-    p.t = ws.t;
-    p.ctr = ws.counters;
+    p.partial = partial;
+    p.t = t;
+    p.ctr = ctr;
+    p.status = status;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.K / kGroupFast; p.rank = a.rank;
     p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CHG = pl.CHG; p.NS = pl.NS;
     p.maxslots = pl.maxslots;
@@ -1201,7 +1226,39 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     p.meta_rows = pl.meta_rows;
     p.off_tab = pl.off_tab; p.off_def = pl.off_def; p.off_meta = pl.off_meta; p.off_x = pl.off_x; p.off_px = pl.off_px;
     p.off_segbuf = pl.off_segbuf; p.off_A = pl.off_A; p.off_B = pl.off_B; p.off_t = pl.off_t; p.off_ring = pl.off_ring;
-    p.trace = reinterpret_cast<unsigned long long *>(ws.trace);
+    p.trace = reinterpret_cast<unsigned long long *>(trace);
+    return p;
+}
+
+template <int BITS, typename T, int MT>
+cudaError_t launch_batch_variant(const DecodeBatch &b, size_t smem, bool pdl, cudaStream_t s)
+{
+    auto kern = decode_batch_kernel<BITS, T, MT>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)b.first[b.count]);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, b);
+}
+}  // namespace
+
+cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning &tune, cudaStream_t s, int *launches)
+{
+    const Plan pl = make_plan(a, tune);
+    if (!pl.ok) return cudaErrorInvalidConfiguration;
+    const DecodeParams p = fill_params(a, pl, ws.partial, ws.t, ws.counters, ws.counters + kCtrStatus, ws.trace);
     const bool pdl = tune.pdl != 0;
     cudaError_t e;
     const int mt = (a.M <= 8) ? 1 : 2;
@@ -1211,6 +1268,66 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     } else {
         if (a.bits == 4) e = (mt == 1) ? launch_variant<4, __half, 1>(p, pl, pdl, s) : launch_variant<4, __half, 2>(p, pl, pdl, s);
         else             e = (mt == 1) ? launch_variant<3, __half, 1>(p, pl, pdl, s) : launch_variant<3, __half, 2>(p, pl, pdl, s);
+    }
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
+
+// ---- several problems in one launch ---------------------------------------------------------
+int decode_batch_max() { return kBatchMax; }
+
+// Scratch the batch needs in one workspace: partial floats, t floats and counters, summed over the
+// problems (problem i is planned with at most ctas[i] CTAs).  false if a problem has no plan.
+bool decode_batch_need(const LinearArgs *a, int count, const int *ctas, const DecodeTuning &tune, size_t *partial_floats,
+                       size_t *t_floats, int *counters)
+{
+    *partial_floats = 0;
+    *t_floats = 0;
+    *counters = kCtrFirstTile;                      // the shared head (status word) comes first
+    for (int i = 0; i < count; ++i) {
+        DecodeTuning tn = tune;
+        tn.max_ctas = ctas[i];
+        const Plan pl = make_plan(a[i], tn);
+        if (!pl.ok) return false;
+        *partial_floats += (size_t)pl.NT * pl.maxslots * a[i].M * kTileRows;
+        *t_floats += (size_t)kDecodeMaxM * kMaxRank;
+        *counters += kCtrFirstTile + 2 * pl.NT;
+    }
+    return true;
+}
+
+// All problems share M, bits, rank and the activation type.  ws must hold decode_batch_need().
+cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas, Workspace &ws, const DecodeTuning &tune,
+                                cudaStream_t s, int *launches)
+{
+    if (count < 1 || count > kBatchMax) return cudaErrorInvalidConfiguration;
+    DecodeBatch b{};
+    b.count = count;
+    size_t smem = 0, off_p = 0, off_t = 0;
+    int off_c = kCtrFirstTile;
+    for (int i = 0; i < count; ++i) {
+        DecodeTuning tn = tune;
+        tn.max_ctas = ctas[i];
+        const Plan pl = make_plan(a[i], tn);
+        if (!pl.ok) return cudaErrorInvalidConfiguration;
+        b.prob[i] = fill_params(a[i], pl, ws.partial + off_p, ws.t + off_t, ws.counters + off_c, ws.counters + kCtrStatus, nullptr);
+        b.first[i] = (i == 0) ? 0 : b.first[i];
+        b.first[i + 1] = b.first[i] + pl.R * pl.SK;
+        off_p += (size_t)pl.NT * pl.maxslots * a[i].M * kTileRows;
+        off_t += (size_t)kDecodeMaxM * kMaxRank;
+        off_c += kCtrFirstTile + 2 * pl.NT;
+        smem = pl.smem > smem ? pl.smem : smem;
+    }
+    const bool pdl = tune.pdl != 0;
+    const LinearArgs &a0 = a[0];
+    cudaError_t e;
+    const int mt = (a0.M <= 8) ? 1 : 2;
+    if (a0.bf16) {
+        if (a0.bits == 4) e = (mt == 1) ? launch_batch_variant<4, __nv_bfloat16, 1>(b, smem, pdl, s) : launch_batch_variant<4, __nv_bfloat16, 2>(b, smem, pdl, s);
+        else              e = (mt == 1) ? launch_batch_variant<3, __nv_bfloat16, 1>(b, smem, pdl, s) : launch_batch_variant<3, __nv_bfloat16, 2>(b, smem, pdl, s);
+    } else {
+        if (a0.bits == 4) e = (mt == 1) ? launch_batch_variant<4, __half, 1>(b, smem, pdl, s) : launch_batch_variant<4, __half, 2>(b, smem, pdl, s);
+        else              e = (mt == 1) ? launch_batch_variant<3, __half, 1>(b, smem, pdl, s) : launch_batch_variant<3, __half, 2>(b, smem, pdl, s);
     }
     if (e == cudaSuccess) ++*launches;
     return e;

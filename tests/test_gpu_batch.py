@@ -35,17 +35,20 @@ def _problems(fbq, M, bits, rank, dtype, seed0):
     return inps, devs, probs
 
 
+@pytest.mark.parametrize("single", [1, 0])
 @pytest.mark.parametrize("bits,rank,dtype,M", [(3, 64, "f16", 1), (4, 64, "bf16", 1), (3, 0, "f16", 1), (3, 16, "f16", 5),
                                               (4, 64, "f16", 16)])
-def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M):
+def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M, single):
     import torch
+    fbq.set_option("batch_single", single)       # 1: the decode kernel over a problem list; 0: one launch per problem
     inps, devs, probs = _problems(fbq, M, bits, rank, dtype, 4000 + 10 * bits + rank)
     for N, K in [(inp.N, inp.K) for inp in inps]:
         assert fbq.select_kernel(M, N, K, 128, bits, rank, dtype == "bf16") == fbq.KERNEL_DECODE
     before = fbq.launch_count()
     fbq.linear_batch(probs, 128, bits)
     torch.cuda.synchronize()
-    assert fbq.launch_count() - before == len(probs)        # one fused decode launch per problem
+    assert fbq.launch_count() - before == (1 if single else len(probs))
+    fbq.set_option("batch_single", 1)
     assert fbq.poll_status() == 0
     for inp, d, pr in zip(inps, devs, probs):
         want = oracle.linear_inputs(inp, threads=8)
