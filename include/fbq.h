@@ -56,8 +56,8 @@ typedef enum {
 typedef enum {
     FBQ_KERNEL_NONE = -1,
     FBQ_KERNEL_GENERIC = 0,   /* any supported shape, CUDA cores, two launches if rank>0 */
-    FBQ_KERNEL_DECODE = 1,    /* M <= 16: fused split-K streaming kernel, one launch      */
-    FBQ_KERNEL_PREFILL = 2    /* M > 16: tcgen05 / TMEM tensor-core kernel                */
+    FBQ_KERNEL_DECODE = 1,    /* M <= 16 (chosen for M <= 6): fused streaming kernel, one launch */
+    FBQ_KERNEL_PREFILL = 2    /* tcgen05 / TMEM tensor-core kernel, one launch (chosen from M = 7) */
 } fbq_kernel;
 
 /* Number of uint32 words of a packed N x K code matrix: N*K/8 (4 bits) or

@@ -51,8 +51,10 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     if (g_opt.force_kernel == FBQ_KERNEL_DECODE && decode_ok) return FBQ_KERNEL_DECODE;
     if (g_opt.force_kernel == FBQ_KERNEL_PREFILL && prefill_ok) return FBQ_KERNEL_PREFILL;
     if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
-    if (decode_ok) return FBQ_KERNEL_DECODE;
-    if (prefill_ok && M > kDecodeMaxM) return FBQ_KERNEL_PREFILL;
+    // Measured on B200 (7B shapes): the decode kernel wins up to M = 6; from M = 7 on the tensor-core
+    // kernel is faster even though few of its token rows are real.
+    if (decode_ok && (M <= kDecodePreferM || !prefill_ok)) return FBQ_KERNEL_DECODE;
+    if (prefill_ok) return FBQ_KERNEL_PREFILL;
     return FBQ_KERNEL_GENERIC;
 }
 

@@ -12,7 +12,7 @@ namespace fbq {
 
 constexpr int kGroupFast = 128;   // group size of the decode / prefill kernels (Section 5.1)
 constexpr int kMaxRank = 256;
-constexpr int kDecodeMaxM = 16;
+constexpr int kDecodeMaxM = 16, kDecodePreferM = 6;
 
 // Activation-type helpers ---------------------------------------------------
 template <typename T> struct ActTraits;

@@ -70,10 +70,19 @@ def check_parity(inp, fbq, *, expect_kernel=None, n_list=None, threads=8, floor=
     """Runs the CUDA path and the oracle on `inp` and asserts the tolerances."""
     import torch
     dev = DeviceLinear(inp, fbq)
-    if expect_kernel is not None:
-        assert fbq.select_kernel(inp.M, inp.N, inp.K, inp.group, inp.bits, inp.rank,
-                                 inp.dtype == "bf16") == expect_kernel
-    y = dev.run(fbq)
+    # a test that names the decode kernel means that kernel, also for token counts at which the
+    # dispatcher would by now prefer the tensor-core kernel
+    forced = expect_kernel == fbq.KERNEL_DECODE and fbq.get_option("force_kernel") == -1
+    if forced:
+        fbq.set_option("force_kernel", fbq.KERNEL_DECODE)
+    try:
+        if expect_kernel is not None:
+            assert fbq.select_kernel(inp.M, inp.N, inp.K, inp.group, inp.bits, inp.rank,
+                                     inp.dtype == "bf16") == expect_kernel
+        y = dev.run(fbq)
+    finally:
+        if forced:
+            fbq.set_option("force_kernel", -1)
     torch.cuda.synchronize()
     assert fbq.poll_status() == 0
     y64 = torch_to_f64(y, inp.dtype)

@@ -23,7 +23,11 @@ def test_noalloc_matches_allocating_entry_point_twice():
              make_linear(16, 528, 1024, 4, 16, dtype="bf16", seed=502), make_linear(2, 272, 1024, 3, 0, seed=503)]
     for inp in cases:
         dev = DeviceLinear(inp, fbq)
-        want = dev.run(fbq)                                   # existing entry point
+        fbq.set_option("force_kernel", fbq.KERNEL_DECODE)     # the same kernel, whatever the dispatcher prefers at this M
+        try:
+            want = dev.run(fbq)                               # existing entry point
+        finally:
+            fbq.set_option("force_kernel", -1)
         torch.cuda.synchronize()
         want64 = torch_to_f64(want, inp.dtype)
         for call in range(2):                                 # two calls in a row share the array
