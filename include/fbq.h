@@ -85,14 +85,16 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  *   rank == 0: A and B are ignored (may be NULL); y is the main path alone.
  *   M == 0: nothing is done.
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128
- * and rank a multiple of 8 not above 256 -> decode kernel for M <= 16, prefill
- * kernel for M > 16; everything else that is well formed -> generic kernel.
+ * and rank a multiple of 8 not above 256 -> decode kernel for M <= 6, prefill
+ * kernel from M = 7 (N a multiple of 8 and 16-byte aligned operands; otherwise the decode
+ * kernel up to M = 16); everything else that is well formed -> generic kernel.
  * Well formed means bits in {3,4}, group a multiple of 8 (4 bits) or 32
  * (3 bits) dividing K, rank >= 0.  The decode and prefill kernels assume
  * integer-valued zero points in [0, 127]; the generic kernel accepts any
  * fp16 value.  Accumulation is fp32; t = x.A^T stays fp32 in the decode and
  * generic kernels and is rounded once to the activation type in the prefill
- * kernel (which also rounds the dequantised weights s*(q-z) once to that type).  Summation order is fixed for a given shape (results are
+ * kernel (which also rounds the dequantised weights s*(q-z) once to that type).
+ * Summation order is fixed for a given shape (results are
  * reproducible run to run) except for t in the decode kernel, which is
  * accumulated with floating-point atomics. */
 int fbq_linear(const void *x, const uint32_t *qweight, const void *scales, const void *zeros,
