@@ -234,6 +234,9 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "decode_depth"  0 = automatic, else stages in flight per warp
  *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
  *   "batch_ctas"    CTAs shared out among the problems of a decode-sized fbq_linear_batch (default 400)
+ *   "prefill_pair"  1 = token tiles of 256 of the prefill kernel run on CTA pairs (cta_group::2 MMAs,
+ *                   each CTA staging half of the token tile); 0 (default) = one CTA per tile, which
+ *                   measured faster
  *   "batch_single"  1 = such a batch of up to 8 problems is one launch (default), 0 = one launch per problem
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives

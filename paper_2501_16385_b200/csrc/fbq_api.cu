@@ -11,6 +11,7 @@
 
 namespace fbq {
 void decode_set_test_switch(int t_late);
+void prefill_set_pair(int on);
 
 namespace {
 
@@ -24,6 +25,7 @@ struct Options {
     int decode_t_late = 0;
     int batch_ctas = 400;
     int batch_single = 1;
+    int prefill_pair = 0;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
@@ -175,6 +177,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
     if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;
     if (!strcmp(name, "batch_single")) return &g_opt.batch_single;
+    if (!strcmp(name, "prefill_pair")) return &g_opt.prefill_pair;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
@@ -293,6 +296,7 @@ static int linear_common(const void *x, const uint32_t *qweight, const void *sca
     a.y = y;
     a.M = M; a.N = N; a.K = K; a.group = group; a.bits = bits; a.rank = rank; a.bf16 = bf16;
     decode_set_test_switch(g_opt.decode_t_late);
+    prefill_set_pair(g_opt.prefill_pair);
     return run_linear(a, static_cast<cudaStream_t>(stream));
 }
 

@@ -830,6 +830,531 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
 }
 
+// ---------------------------------------------------------------- CTA-pair variant
+// Two CTAs of a cluster (two SMs) share one MMA of 256 weight rows x 256 tokens x 16
+// (tcgen05 cta_group::2): each CTA dequantises its own 128 weight rows and stages only HALF of
+// the token tile (128 tokens); the tensor cores of both SMs read both halves.  Per CTA and K
+// block that is 16 KB less written by TMA and 16 KB less read by the MMA than in the single-CTA
+// kernel, and it leaves room for six stages.  MEASURED SLOWER than the single-CTA kernel on B200
+// (M = 1024, 4096 -> 4096, INT4, bf16: 47.8 us against 39.8 us; 1120 against 880 cycles per K
+// block), so it is off by default ("prefill_pair" option) and kept as a checked alternative.
+// The leader CTA (cluster rank 0) issues every MMA; all arrivals that say "stage full" (the
+// producer warps of both CTAs, the byte counts of both CTAs' TMA copies) go to the leader's
+// barriers; tcgen05.commit with a cluster multicast frees the stage in both CTAs.
+constexpr int kPairStages = 6;
+struct PairSmem {
+    static constexpr uint32_t kXBytes = 128u * kBK * 2u;                   // this CTA's half of the token tile
+    static constexpr uint32_t kStageBytes = kXBytes + kWBytes;
+    static constexpr uint32_t kRingOff = kPairStages * kStageBytes;
+    static constexpr uint32_t kTableOff = kRingOff + kRing * kRawSlot;
+    static constexpr uint32_t kBarOff = kTableOff + kRing * kBN * 4u;
+    static constexpr uint32_t kNumBars = 2 * kPairStages + 2 * kRing + 1 + 4;
+    static constexpr uint32_t kTotal = kBarOff + kNumBars * 8u + 16u;
+};
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool pf_mbar_wait_cluster(uint32_t bar, uint32_t parity)     // sees arrivals from the peer CTA
+{
+#pragma unroll 1
+    for (uint32_t i = 0; i < kPfWaitLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive, in BOTH CTAs of the pair, on the barrier at this shared-memory offset once every MMA issued so far is complete.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    const unsigned short mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(mask)
+                 : "memory");
+}
+// TMA tensor copy into this CTA's shared memory that completes on a barrier of either CTA of the pair (no multicast)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t cluster_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(cluster_bar)
+        : "memory");
+}
+
+// Grid: 1-D, clusters of two consecutive CTAs.  t CTAs first (pairs: 256 tokens x 256 rank rows),
+// then main CTAs (pairs: 256 tokens x 256 features; a padding CTA past the last feature tile
+// computes zeros and stores nothing).  Maps as for prefill_kernel, except that the boxes of xmap
+// hold 128 token rows.
+template <int BITS, typename T>
+__global__ void __launch_bounds__(kPfThreads, 1)
+prefill_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
+               const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+               const __grid_constant__ CUtensorMap ymap, const PrefillParams p)
+{
+    using L = PairSmem;
+    constexpr int TOK = 256;                                    // tokens of the pair's tile; this CTA stages 128 of them
+    constexpr int kStages = kPairStages;                        // (shadows the single-CTA kernel's depth)
+    constexpr uint32_t kXBytes = L::kXBytes, kStageBytes = L::kStageBytes;
+    const uint32_t cr = cluster_ctarank();                      // 0: leader (issues the MMAs), 1: peer
+    constexpr int WPG = (BITS == 4) ? 16 : 12;                  // packed words per row and group
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = pf_smem_u32(smem);
+    if (sbase & 1023u) {                                        // swizzle atoms need a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicExch(p.status, (int)FBQ_ERR_CUDA);
+        return;
+    }
+    const uint32_t full0 = sbase + L::kBarOff, empty0 = full0 + 8u * kStages, rfull0 = empty0 + 8u * kStages,
+                   rempty0 = rfull0 + 8u * kRing, done_bar = rempty0 + 8u * kRing, epi0 = done_bar + 8u;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + L::kNumBars * 8u);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool t_role = (int)blockIdx.x < p.n_t;                // t CTA or main CTA
+    int m_tile, n_tile;
+    if (t_role) {
+        m_tile = (int)blockIdx.x / p.rt;
+        n_tile = (int)blockIdx.x % p.rt;                        // tile of rank rows of A
+    } else {
+        m_tile = ((int)blockIdx.x - p.n_t) / p.nt;
+        n_tile = ((int)blockIdx.x - p.n_t) % p.nt;
+    }
+    const int m0 = m_tile * TOK, n0 = n_tile * kBN;
+    const int mh = m0 + 128 * (int)cr;                          // first token of the half this CTA stages
+    const int nkb = t_role ? p.kb_main : p.kb_main + p.kb_slab;
+    const int kb_x = p.kb_main;                                 // blocks below kb_x take their tokens from x
+
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            pf_mbar_init(full0 + 8u * i, t_role ? 1 : 17);      // leader's TMA lane + 8 producer warps of each CTA
+            pf_mbar_init(empty0 + 8u * i, 1);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            pf_mbar_init(rfull0 + 8u * i, 2);                   // the two ring warps
+            pf_mbar_init(rempty0 + 8u * i, kHalf);              // a group is consumed by one half of the producers
+        }
+        pf_mbar_init(done_bar, 1);
+        for (int i = 0; i < 4; ++i) pf_mbar_init(epi0 + 8u * i, 128);     // the four warps of a column quarter
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {                  // the MMA warp owns the tensor-memory allocation
+        // the MMA warps of both CTAs of the pair allocate together (same columns in both)
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(pf_smem_u32(tmem_slot)),
+                     "r"((uint32_t)TOK)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        tc_fence_before();
+    }
+    if (warp == kTmaWarp && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&xmap)) : "memory");
+        if (t_role) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&amap)) : "memory");
+        } else {
+            if (p.rank > 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&bmap)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ymap)) : "memory");
+        }
+    }
+    if (warp == kRawWarp && lane == 0)
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&wmap)) : "memory");
+    cluster_sync();                          // barriers of both CTAs are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < kMmaWarp) {
+        bool dead = false;
+        if (!t_role) {
+            // =================================================== producers
+            // Half h of the warps takes the groups g = h, h+2, ... (K blocks 2g and 2g+1, stages 2h
+            // and 2h+1); thread (row r, part) dequantises the codes [32*part, +32) of both blocks.
+            const int h = warp >> 3, part = (warp >> 2) & 1, r = tid & 127;
+            const bool row_ok = n0 + r < p.N;
+            const int groups = p.kb_main >> 1;
+            // this thread's words inside a ring slot: block b holds codes [64b, 64b+64) of the group
+            uint32_t roff0, roff1;
+            if (BITS == 4) {                                // 64-byte rows, 16-byte chunk c stored at c ^ ((row / 2) % 4)
+                const uint32_t sw = (uint32_t)(r >> 1) & 3u;
+                roff0 = (uint32_t)r * 64u + ((((uint32_t)part) ^ sw) << 4);
+                roff1 = (uint32_t)r * 64u + ((((uint32_t)part + 2u) ^ sw) << 4);
+            } else {                                        // 48-byte rows of four 12-byte runs
+                roff0 = (uint32_t)r * 48u + (uint32_t)part * 12u;
+                roff1 = roff0 + 24u;
+            }
+            const uint32_t ring0 = sbase + L::kRingOff, table0 = sbase + L::kTableOff + (uint32_t)r * 4u;
+            // weight tile rows are 128 bytes (64 elements); the 16-byte chunk c of row r sits at c ^ (r % 8)
+            const uint32_t wdst = sbase + kXBytes + (uint32_t)r * 128u;
+            const uint32_t wsw = (uint32_t)r & 7u;
+            const uint32_t lfull0 = mapa_shared(full0, 0);     // the leader's "full" barriers, as seen from this CTA
+            uint32_t slot = (uint32_t)h, rphase = 0u;
+#pragma unroll 1
+            for (int g = h; g < groups; g += 2) {
+                if (!pf_mbar_wait(rfull0 + 8u * slot, rphase)) { dead = true; break; }
+                constexpr int NW = (BITS == 4) ? 4 : 3;
+                uint32_t w[2][NW];
+                const uint32_t rs = ring0 + slot * kRawSlot;
+                if (BITS == 4) {
+                    const uint4 a = lds128(rs + roff0), b = lds128(rs + roff1);
+                    w[0][0] = a.x; w[0][1] = a.y; w[0][2] = a.z; w[0][NW - 1] = a.w;
+                    w[1][0] = b.x; w[1][1] = b.y; w[1][2] = b.z; w[1][NW - 1] = b.w;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        w[0][c] = lds32(rs + roff0 + 4u * c);
+                        w[1][c] = lds32(rs + roff1 + 4u * c);
+                    }
+                }
+                const uint32_t sz = lds32(table0 + slot * (kBN * 4u));      // s | z << 16 of (row, group)
+                pf_mbar_arrive(rempty0 + 8u * slot);         // everything is in registers: the slot may be refilled
+                slot += 2u;
+                if (slot >= (uint32_t)kRing) { slot -= (uint32_t)kRing; rphase ^= 1u; }
+                const float sc = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
+                const float ze = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int i = 2 * g + b, s = i % kStages;
+                    if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
+                    uint32_t wb[16];
+                    if (row_ok) {
+                        uint32_t d[16];
+                        Dequant<BITS, T>::run(w[b], sc, ze, d);
+                        natural_pairs<BITS>(d, wb);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) wb[c] = 0u;
+                    }
+#pragma unroll
+                    for (int kc = 0; kc < 4; ++kc)
+                        sts128(wdst + (uint32_t)s * kStageBytes + ((((uint32_t)(4 * part + kc)) ^ wsw) << 4), wb[4 * kc], wb[4 * kc + 1], wb[4 * kc + 2],
+                               wb[4 * kc + 3]);
+                    pf_fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(lfull0 + 8u * s);       // one arrival per warp, on the leader's barrier
+                }
+                if (dead) break;
+            }
+            // ---- sub-branch blocks: token operand = t (fp32 scratch, rounded once); B arrives by TMA.
+            // The halves take them in turn, one token row per thread.
+            bool t_ready = false;
+#pragma unroll 1
+            for (int i = p.kb_main + h; i < nkb && !dead; i += 2) {
+                const int s = i % kStages;
+                if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
+                if (!t_ready) {                              // every warp of every t CTA of this token tile has stored its part
+                    int seen = 0;
+                    if (lane == 0) {
+                        const int *flag = p.tflag + m_tile;
+                        const int target = 16 * p.rt;
+#pragma unroll 1
+                        for (uint32_t spin = 0; spin < kPfFlagPolls; ++spin) {
+                            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+                            if (seen >= target) break;
+                            __nanosleep(256);
+                        }
+                        seen = seen >= target;
+                    }
+                    t_ready = __shfl_sync(0xffffffffu, seen, 0) != 0;
+                    if (!t_ready) { dead = true; break; }
+                }
+                const int j0 = (i - p.kb_main) * kBK;
+                const int rr = tid & (kHalf - 1);            // token row of this CTA's half of the tile
+                if (rr < 128) {
+                    const int m = mh + rr;
+                    uint32_t xa[32];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f), t1 = t0;
+                        if (m < p.M && j0 + 8 * c < p.rank) {              // rank is a multiple of 8: whole chunks
+                            const float4 *ts = reinterpret_cast<const float4 *>(p.t32 + (size_t)m * p.rank + j0 + 8 * c);
+                            t0 = __ldcg(ts);
+                            t1 = __ldcg(ts + 1);
+                        }
+                        xa[4 * c] = P2<T>::pack(t0.x, t0.y); xa[4 * c + 1] = P2<T>::pack(t0.z, t0.w);
+                        xa[4 * c + 2] = P2<T>::pack(t1.x, t1.y); xa[4 * c + 3] = P2<T>::pack(t1.z, t1.w);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        sts128(sbase + (uint32_t)s * kStageBytes + (uint32_t)rr * 128u + ((((uint32_t)c) ^ ((uint32_t)rr & 7u)) << 4), xa[4 * c],
+                               xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
+                }
+                pf_fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(lfull0 + 8u * s);
+            }
+            if (dead) {
+                *abort_flag = 1;
+                atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            }
+        }
+
+        // =================================================== epilogue (same sixteen warps)
+        // TMEM lane = weight row of the tile, column = token.  Warp w reads lanes 32*(w%4)..+31
+        // (the only ones it may address) and the quarter w/4 of the columns.  Mode 0 stages the
+        // tile in shared memory as [token][128 features] (the operand stages are free by now) and
+        // each column quarter leaves with one TMA tensor store, which also clips the ragged edges.
+        if (!dead && nkb > 0 && pf_mbar_wait(done_bar, 0)) {
+            tc_fence_after();
+            const int q = warp & 3, cg = warp >> 2;
+            const int nn = n0 + 32 * q + lane;              // output feature (mode 0) / rank index (mode 1)
+            const int c_begin = cg * (TOK / 4);
+            if (m0 + c_begin < p.M) {                       // uniform over the four warps of a column quarter
+#pragma unroll 1
+                for (int c = c_begin; c < c_begin + TOK / 4; c += 32) {
+                    if (m0 + c >= p.M) break;               // warp-uniform
+                    uint32_t v[32];
+                    tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+                    tc_wait_ld();
+                    if (!t_role) {
+                        unsigned short *sp = reinterpret_cast<unsigned short *>(smem + (size_t)c * (kBN * 2)) + 32 * q + lane;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sp[j * kBN] = to_bits16<T>(__uint_as_float(v[j]));
+                    } else {
+                        if (nn < p.rank) {                   // 32 lanes = 32 consecutive rank indices: 128-byte stores
+                            float *tp = p.t32 + (size_t)(m0 + c) * p.rank + nn;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (m0 + c + j < p.M) __stcg(tp + (size_t)j * p.rank, __uint_as_float(v[j]));
+                        }
+                    }
+                }
+                if (!t_role) {
+                    pf_fence_proxy_async();                 // staged tile -> visible to the TMA store
+                    pf_mbar_arrive(epi0 + 8u * cg);
+                    if (q == 0 && lane == 0 && n0 < p.N) {   // (a padding CTA past the last feature tile stores nothing)
+                        if (pf_mbar_wait(epi0 + 8u * cg, 0)) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&ymap)), "r"(n0), "r"(m0 + c_begin),
+                                           "r"(sbase + (uint32_t)c_begin * (kBN * 2))
+                                         : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem may go once it has been read
+                        } else {
+                            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+                        }
+                    }
+                }
+            }
+            if (t_role) {
+                // this warp's part of t is stored: make it visible, then count the warp in
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(p.tflag + m_tile, 1);
+            } else if (p.rank > 0 && tid == 0) {
+                // this CTA has consumed t (its MMAs are complete).  The last main CTA of the token
+                // tile leaves the flag and the count at zero for the next call.
+                if (atomicAdd(p.tdone + m_tile, 1) == p.nt - 1) {
+                    atomicExch(p.tflag + m_tile, 0);
+                    atomicExch(p.tdone + m_tile, 0);
+                }
+            }
+        }
+        tc_fence_before();
+    } else if (warp == kMmaWarp) {
+        // =================================================== MMA warp
+        // one MMA of the pair: 256 weight rows (128 per CTA) x 256 tokens (128 staged by each CTA) x 16
+        constexpr uint32_t idesc = (1u << 4) | (P2<T>::kFmt << 7) | (P2<T>::kFmt << 10) | ((uint32_t)(TOK >> 3) << 17) |
+                                   ((uint32_t)((2 * kBN) >> 4) << 24);
+        bool dead = false;
+#pragma unroll 1
+        for (int i = 0; i < nkb && !dead && cr == 0; ++i) {     // only the leader CTA issues
+            const int s = i % kStages;
+            if (lane == 0) {
+                if (!pf_mbar_wait_cluster(full0 + 8u * s, (uint32_t)(i / kStages) & 1u) || *abort_flag) {
+                    dead = true;
+                } else {
+                    tc_fence_after();
+                    const uint32_t x_base = sbase + (uint32_t)s * kStageBytes, w_base = x_base + kXBytes;
+                    // every operand tile is K-major with 128-byte rows and the 128-byte swizzle, whether it
+                    // arrived by TMA or was written by the producers: 32 bytes per 16 elements of K inside a row
+#pragma unroll
+                    for (int j = 0; j < kBK / 16; ++j)
+                        tc_mma_pair(tmem_base, make_desc(w_base + j * 32), make_desc(x_base + j * 32), idesc, (i > 0 || j > 0) ? 1u : 0u);
+                    tc_commit_pair(empty0 + 8u * s);         // the stage is free, in both CTAs, once these MMAs have read it
+                }
+            }
+            dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+        }
+        if (lane == 0) {
+            if (dead) {
+                *abort_flag = 1;
+                atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            } else if (nkb > 0 && cr == 0) {
+                tc_commit_pair(done_bar);                    // accumulators complete in both CTAs
+            }
+        }
+        __syncwarp();
+        tc_fence_before();
+    } else if (warp == kTmaWarp) {
+        // =================================================== operand-stage copies
+        if (lane == 0) {
+            bool dead = false;
+#pragma unroll 1
+            for (int i = 0; i < nkb; ++i) {
+                const int kb = i, s = i % kStages;
+                if ((i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) || *abort_flag) {
+                    dead = true;
+                    break;
+                }
+                const uint32_t bar = full0 + 8u * s;
+                const uint32_t xt = sbase + (uint32_t)s * kStageBytes, wt = xt + kXBytes;
+                // every copy of the pair completes on the LEADER's barrier; the leader announces the bytes of both
+                const uint32_t lbar = mapa_shared(bar, 0);
+                if (t_role) {
+                    if (cr == 0) pf_mbar_expect_tx(bar, 2u * (kXBytes + kWBytes));
+                    tma_load_2d_pair(xt, &xmap, kb * kBK, mh, lbar);
+                    tma_load_2d_pair(wt, &amap, kb * kBK, n0, lbar);      // rows of A
+                } else if (kb < kb_x) {
+                    if (cr == 0) pf_mbar_expect_tx(bar, 2u * kXBytes);
+                    tma_load_2d_pair(xt, &xmap, kb * kBK, mh, lbar);
+                } else {
+                    if (cr == 0) pf_mbar_expect_tx(bar, 2u * kWBytes);
+                    tma_load_2d_pair(wt, &bmap, (kb - p.kb_main) * kBK, n0, lbar);   // rows of B
+                }
+            }
+            if (dead) {
+                *abort_flag = 1;
+                atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);   // let the copies in flight land before the CTA exits
+            }
+        }
+        __syncwarp();
+    } else if (!t_role) {
+        // =================================================== ring of packed codes and (s, z) table
+        // Two warps; lane l of ring warp v owns the tile rows 64v + l and 64v + l + 32.  Per chunk of
+        // eight groups it reads the rows' scales and zero points with 16-byte loads (two aligned chunks of the flat row-major arrays
+        // cover any eight consecutive values), realigns them in registers, and before each group's
+        // copy writes that group's (s | z << 16) words next to the ring slot.
+        const int G = p.K / kGroupFast, groups = p.kb_main >> 1;
+        const size_t n_chunks = (size_t)p.N * G / 8;        // N is a multiple of 8
+        const uint4 *s_arr = reinterpret_cast<const uint4 *>(p.scales), *z_arr = reinterpret_cast<const uint4 *>(p.zeros);
+        const int v = warp - kRawWarp;
+        size_t a0[2];                                       // aligned 16-byte chunk holding group 0 of the row
+        uint32_t off[2];                                    // position of group 0 inside that chunk (0..7)
+        bool ok[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int n = n0 + 64 * v + lane + 32 * k;
+            ok[k] = n < p.N;
+            const size_t f = (size_t)(ok[k] ? n : 0) * G;
+            a0[k] = f >> 3;
+            off[k] = (uint32_t)f & 7u;
+        }
+        uint4 raw[2][2][2];                                 // [row][s|z][low|high chunk] of the next eight groups
+        auto fetch = [&](int c) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const size_t a = a0[k] + (size_t)c;
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                raw[k][0][0] = (ok[k] && a < n_chunks) ? __ldg(s_arr + a) : zero;
+                raw[k][1][0] = (ok[k] && a < n_chunks) ? __ldg(z_arr + a) : zero;
+                raw[k][0][1] = (ok[k] && a + 1 < n_chunks) ? __ldg(s_arr + a + 1) : zero;
+                raw[k][1][1] = (ok[k] && a + 1 < n_chunks) ? __ldg(z_arr + a + 1) : zero;
+            }
+        };
+        // eight consecutive fp16 values starting `o` values into the 16-value window (lo, hi), as 4 pair-words
+        auto realign = [](const uint4 &lo, const uint4 &hi, uint32_t o, uint32_t (&out)[4]) {
+            uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            if (o & 2u) {
+#pragma unroll
+                for (int i = 0; i < 7; ++i) w[i] = w[i + 1];
+            }
+            if (o & 4u) {
+#pragma unroll
+                for (int i = 0; i < 5; ++i) w[i] = w[i + 2];
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) out[t] = __funnelshift_r(w[t], w[t + 1], (o & 1u) * 16u);
+        };
+        bool dead = false;
+        fetch(0);
+        const uint32_t ring0 = sbase + L::kRingOff, table0 = sbase + L::kTableOff + (uint32_t)(64 * v + lane) * 4u;
+#pragma unroll 1
+        for (int c = 0; 8 * c < groups && !dead; ++c) {
+            uint32_t sz[2][8];                              // (s | z << 16) of [row][group of this chunk]
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                uint32_t sp[4], zp[4];
+                realign(raw[k][0][0], raw[k][0][1], off[k], sp);
+                realign(raw[k][1][0], raw[k][1][1], off[k], zp);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    sz[k][2 * t] = pf_prmt(sp[t], zp[t], 0x5410u);
+                    sz[k][2 * t + 1] = pf_prmt(sp[t], zp[t], 0x7632u);
+                }
+            }
+            if (8 * (c + 1) < groups) fetch(c + 1);
+#pragma unroll
+            for (int g8 = 0; g8 < 8; ++g8) {
+                const int gi = 8 * c + g8;
+                if (gi < groups && !dead) {
+                    const uint32_t slot = (uint32_t)gi % kRing;
+                    if (lane == 0 && ((gi >= kRing && !pf_mbar_wait(rempty0 + 8u * slot, (uint32_t)(gi / kRing - 1) & 1u)) || *abort_flag))
+                        dead = true;
+                    dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;     // also orders the table writes after the wait
+                    if (!dead) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(table0 + slot * (kBN * 4u) + 128u * k), "r"(sz[k][g8]) : "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (v == 0) {
+                                pf_mbar_expect_tx(rfull0 + 8u * slot, (uint32_t)kBN * WPG * 4u);
+                                tma_load_2d(ring0 + slot * kRawSlot, &wmap, gi * WPG, n0, rfull0 + 8u * slot);
+                            } else {
+                                pf_mbar_arrive(rfull0 + 8u * slot);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if (dead && lane == 0) {
+            *abort_flag = 1;
+            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+            for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        }
+        __syncwarp();
+    }
+    cluster_sync();                          // both CTAs are done with their tensor memory and with each other's barriers
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TOK) : "memory");
+    }
+}
+
+
 template <int BITS, typename T, int TOK>
 cudaError_t launch_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &amap, const CUtensorMap &bmap,
                           const CUtensorMap &ymap, const PrefillParams &p, unsigned grid, cudaStream_t s)
@@ -844,6 +1369,34 @@ cudaError_t launch_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, cons
     kern<<<grid, kPfThreads, Smem<TOK>::kTotal, s>>>(xmap, wmap, amap, bmap, ymap, p);
     return cudaGetLastError();
 }
+
+template <int BITS, typename T>
+cudaError_t launch_pair_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &amap, const CUtensorMap &bmap,
+                               const CUtensorMap &ymap, const PrefillParams &p, unsigned grid, cudaStream_t s)
+{
+    auto kern = prefill_pair_kernel<BITS, T>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairSmem::kTotal);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kPfThreads);
+    cfg.dynamicSmemBytes = PairSmem::kTotal;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, xmap, wmap, amap, bmap, ymap, p);
+}
+
+int g_pair = 0;
 
 // 2-D tensor map of a row-major matrix: `cols` elements per row (16- or 32-bit), `rows` rows,
 // boxes of box_cols x box_rows.  Reads outside the matrix return zero.
@@ -869,7 +1422,7 @@ cudaError_t make_map(CUtensorMap *map, const void *base, bool elem32, size_t col
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <typename T, int TOK>
+template <typename T, int TOK, bool PAIR>
 cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches)
 {
     PrefillParams p{};
@@ -884,12 +1437,17 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
     const int mt = (a.M + TOK - 1) / TOK;
     p.nt = (a.N + kBN - 1) / kBN;
     p.rt = (a.rank + kBN - 1) / kBN;
+    if (PAIR) {                                     // CTAs come in pairs: feature tiles and rank tiles padded to even counts
+        p.nt = (p.nt + 1) & ~1;
+        p.rt = (p.rt + 1) & ~1;
+    }
     p.n_t = mt * p.rt;
     p.tflag = ws.counters + kPfCtrBase;
     p.tdone = p.tflag + mt;
     CUtensorMap xmap, qmap, amap, bmap, ymap;
     cudaError_t e;
-    if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
+    if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, PAIR ? 128 : TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess)
+        return e;
     const int wpg = (a.bits == 4) ? 16 : 12;
     if ((e = make_map(&qmap, a.qw, true, (size_t)(a.K / kGroupFast) * wpg, (size_t)a.N, wpg, kBN,
                       a.bits == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess)
@@ -901,8 +1459,12 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
         if ((e = make_map(&bmap, a.B, false, (size_t)a.rank, (size_t)a.N, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
     }
     const unsigned grid = (unsigned)p.n_t + (unsigned)p.nt * (unsigned)mt;
-    e = (a.bits == 4) ? launch_kernel<4, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s)
-                      : launch_kernel<3, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s);
+    if (PAIR)
+        e = (a.bits == 4) ? launch_pair_kernel<4, T>(xmap, qmap, amap, bmap, ymap, p, grid, s)
+                          : launch_pair_kernel<3, T>(xmap, qmap, amap, bmap, ymap, p, grid, s);
+    else
+        e = (a.bits == 4) ? launch_kernel<4, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s)
+                          : launch_kernel<3, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -910,6 +1472,9 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
 inline bool aligned16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
 
 }  // namespace
+
+// 1: token tiles of 256 run on CTA pairs (cta_group::2); 0: single-CTA kernel
+void prefill_set_pair(int on) { g_pair = on ? 1 : 0; }
 
 bool prefill_supported(const LinearArgs &a)
 {
@@ -930,8 +1495,10 @@ cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, i
         (a.rank > 0 && (!aligned16(a.A) || !aligned16(a.B))))
         return cudaErrorInvalidConfiguration;
     if (a.M <= 128)
-        return a.bf16 ? run_prefill<__nv_bfloat16, 128>(a, ws, s, launches) : run_prefill<__half, 128>(a, ws, s, launches);
-    return a.bf16 ? run_prefill<__nv_bfloat16, 256>(a, ws, s, launches) : run_prefill<__half, 256>(a, ws, s, launches);
+        return a.bf16 ? run_prefill<__nv_bfloat16, 128, false>(a, ws, s, launches) : run_prefill<__half, 128, false>(a, ws, s, launches);
+    if (g_pair)
+        return a.bf16 ? run_prefill<__nv_bfloat16, 256, true>(a, ws, s, launches) : run_prefill<__half, 256, true>(a, ws, s, launches);
+    return a.bf16 ? run_prefill<__nv_bfloat16, 256, false>(a, ws, s, launches) : run_prefill<__half, 256, false>(a, ws, s, launches);
 }
 
 }  // namespace fbq

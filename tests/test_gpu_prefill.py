@@ -77,3 +77,19 @@ def test_prefill_fp16_full_size(fbq):
     rows = np.sort(np.random.default_rng(5).choice(4096, size=128, replace=False))
     rel, _, _, _ = check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, n_list=rows, threads=16, floor=2e-5)
     assert rel < 1e-3
+
+
+@pytest.mark.parametrize("bits,dtype,M,N,K,rank", [(4, "bf16", 1024, 1160, 1024, 64), (3, "f16", 300, 264, 1024, 256),
+                                                   (4, "f16", 513, 136, 512, 0)])
+def test_prefill_cta_pair_variant(fbq, bits, dtype, M, N, K, rank):
+    # the cta_group::2 kernel (two CTAs share one 256 x 256 x 16 MMA; odd tile counts get a padding CTA)
+    fbq.set_option("prefill_pair", 1)
+    try:
+        inp = make_linear(M, N, K, bits, rank, dtype=dtype, seed=2200 + M, outlier_frac=0.01 if dtype == "bf16" else 0.0)
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, floor=2e-5 if dtype == "f16" else 5e-4)
+        exact = make_exact_class(260, 392, 1024, bits, 64, seed=2300 + bits, x_nnz=32, x_max=2)
+        dev = DeviceLinear(exact, fbq)
+        assert np.array_equal(torch_to_f64(dev.run(fbq), "f16"), oracle.linear_inputs(exact, threads=8))
+        assert fbq.poll_status() == 0
+    finally:
+        fbq.set_option("prefill_pair", 0)
