@@ -837,7 +837,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
 // block that is 16 KB less written by TMA and 16 KB less read by the MMA than in the single-CTA
 // kernel, and it leaves room for six stages.  MEASURED SLOWER than the single-CTA kernel on B200
 // (M = 1024, 4096 -> 4096, INT4, bf16: 47.8 us against 39.8 us; 1120 against 880 cycles per K
-// block), so it is off by default ("prefill_pair" option) and kept as a checked alternative.
+// block; with dequantisation, copies and MMAs all switched off the bare hand-shake still takes 760
+// cycles per block: the round trip peer arrival -> leader -> multicast commit -> peer is about
+// 4500 cycles, more than six stages of MMA time cover), so it is off by default ("prefill_pair"
+// option) and kept as a checked alternative.
 // The leader CTA (cluster rank 0) issues every MMA; all arrivals that say "stage full" (the
 // producer warps of both CTAs, the byte counts of both CTAs' TMA copies) go to the leader's
 // barriers; tcgen05.commit with a cluster multicast frees the stage in both CTAs.
