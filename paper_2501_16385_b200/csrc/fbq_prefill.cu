@@ -441,12 +441,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
-            pf_mbar_init(full0 + 8u * i, t_role ? 1 : kHalf + 1);        // 256 producers + the TMA lane
+            pf_mbar_init(full0 + 8u * i, t_role ? 1 : kHalf / 32 + 1);   // 8 producer warps + the TMA lane
             pf_mbar_init(empty0 + 8u * i, 1);
         }
         for (int i = 0; i < kRing; ++i) {
             pf_mbar_init(rfull0 + 8u * i, 2);                   // the two ring warps
-            pf_mbar_init(rempty0 + 8u * i, kHalf);              // a group is consumed by one half of the producers
+            pf_mbar_init(rempty0 + 8u * i, kHalf / 32);         // a group is consumed by one half of the producers (8 warps)
         }
         pf_mbar_init(done_bar, 1);
         for (int i = 0; i < 4; ++i) pf_mbar_init(epi0 + 8u * i, 128);     // the four warps of a column quarter
@@ -518,7 +518,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     }
                 }
                 const uint32_t sz = lds32(table0 + slot * (kBN * 4u));      // s | z << 16 of (row, group)
-                pf_mbar_arrive(rempty0 + 8u * slot);         // everything is in registers: the slot may be refilled
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(rempty0 + 8u * slot);   // the warp's words are in registers: the slot may be refilled
                 slot += 2u;
                 if (slot >= (uint32_t)kRing) { slot -= (uint32_t)kRing; rphase ^= 1u; }
                 const float sc = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
@@ -540,7 +541,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         sts128(wdst + (uint32_t)b * kStageBytes + ((((uint32_t)(4 * part + kc)) ^ wsw) << 4), wb[4 * kc], wb[4 * kc + 1], wb[4 * kc + 2],
                                wb[4 * kc + 3]);
                     pf_fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
-                    pf_mbar_arrive(fullb + 8u * b);
+                    __syncwarp();
+                    if (lane == 0) pf_mbar_arrive(fullb + 8u * b);          // one arrival per warp
                 }
                 if (dead) break;
                 if (g >= 2) ephase ^= 1u;
@@ -590,7 +592,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                                xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
                 }
                 pf_fence_proxy_async();
-                pf_mbar_arrive(full0 + 8u * s);
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(full0 + 8u * s);
             }
             if (dead) {
                 *abort_flag = 1;
@@ -967,7 +970,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_const
         }
         for (int i = 0; i < kRing; ++i) {
             pf_mbar_init(rfull0 + 8u * i, 2);                   // the two ring warps
-            pf_mbar_init(rempty0 + 8u * i, kHalf);              // a group is consumed by one half of the producers
+            pf_mbar_init(rempty0 + 8u * i, kHalf / 32);         // a group is consumed by one half of the producers (8 warps)
         }
         pf_mbar_init(done_bar, 1);
         for (int i = 0; i < 4; ++i) pf_mbar_init(epi0 + 8u * i, 128);     // the four warps of a column quarter
@@ -1040,7 +1043,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_const
                     }
                 }
                 const uint32_t sz = lds32(table0 + slot * (kBN * 4u));      // s | z << 16 of (row, group)
-                pf_mbar_arrive(rempty0 + 8u * slot);         // everything is in registers: the slot may be refilled
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(rempty0 + 8u * slot);   // the warp's words are in registers: the slot may be refilled
                 slot += 2u;
                 if (slot >= (uint32_t)kRing) { slot -= (uint32_t)kRing; rphase ^= 1u; }
                 const float sc = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
