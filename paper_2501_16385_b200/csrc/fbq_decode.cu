@@ -33,6 +33,8 @@
 // is complete before t is waits in a local list and, at worst, is handed to
 // the warp that completes t.  The only waits are on this CTA's own copies and
 // warps, and they are bounded.
+#include <type_traits>
+
 #include "fbq_common.cuh"
 
 #ifndef FBQ_NACC
@@ -51,6 +53,7 @@ constexpr int kNBuf = 4;                     // segment partial buffers in fligh
 constexpr int kTUnitK = 1024;                // k extent of one unit of the down-projection
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kEarlyStages = 1;                // weight stages prefetched before x has been requested
+constexpr int kTUnitsOneWarp = 10;             // (token, unit) pairs of the down-projection one warp takes by itself
 constexpr int kTPolls = 64;                  // looks at the "t complete" flag before a finished tile is parked
 
 // counters[] layout (ints) inside the per-stream scratch
@@ -388,7 +391,10 @@ __device__ __forceinline__ bool tile_claim(const DecodeParams &p, int tile, int 
 
 // --------------------------------------------------------------------- kernel
 // The whole CTA program; `cta` is the CTA's index among the p.R * p.SK CTAs of its problem.
-template <int BITS, typename T, int MT>
+// HEAVY selects the variant for a heavy sub-branch (rank above 64, or many (token, unit) pairs of the
+// down-projection per CTA): its units are shared by the eight compute warps and the tile finish
+// keeps twice as many chunks of B in registers.  The light variant keeps both out of its code.
+template <int BITS, typename T, int MT, bool HEAVY>
 __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -423,7 +429,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     const uint32_t st_full = smem_u32(bars), st_empty = st_full + 8u * p.NS;
     const uint32_t seg_full = st_empty + 8u * p.NS, seg_free = seg_full + 8u * kNBuf;
-    const uint32_t a_full = seg_free + 8u * kNBuf, b_full = a_full + 8u, x_req = b_full + 8u;
+    const uint32_t a_full = seg_free + 8u * kNBuf, b_full = a_full + 8u, x_req = b_full + 8u, t_done = x_req + 8u;
     int *s_def = reinterpret_cast<int *>(smem + p.off_def);
     float2 *s_mf = reinterpret_cast<float2 *>(smem + p.off_meta);         // (s, s*z) [segment row][slice group]
     float2 *s_px = reinterpret_cast<float2 *>(smem + p.off_px);           // (P, X0)  [slice group][token]
@@ -446,6 +452,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         mbar_init(a_full, 1);
         mbar_init(b_full, 1);
         mbar_init(x_req, kCW);
+        mbar_init(t_done, kCW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -453,6 +460,75 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
 
     const int b_rows = min(p.N, (tile_first + nseg) * kTileRows) - tile_first * kTileRows;   // weight rows of our tiles
     const bool b_in_smem = (p.rank > 0) && nseg > 0 && b_rows <= p.b_cap_rows;
+
+    // This CTA's share of t = x.A^T:  t[m][j] += sum over its units (row j of A, k chunk of 1024);
+    // units are numbered k-chunk-major (u = kc*rank + j).  A warp takes the units first, first +
+    // stride, ...; a lane takes 8 elements out of every 256.  A comes from shared memory (bulk
+    // copy) for the CTA's first a_cap units, else from global memory one unit ahead of use; x of a
+    // (token, k chunk) is read from global memory once and kept in registers.  false = a wait ran out.
+    auto t_units = [&](int first, int stride) -> bool {
+        if (!mbar_wait(a_full, 0)) return false;
+        const T *A = static_cast<const T *>(p.A);
+        const T *x = static_cast<const T *>(p.x) + g0 * kGroupFast;
+        auto load_a = [&](int u, uint4 (&av)[4]) {
+            const int kc = u / p.rank, j = u - kc * p.rank;
+            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
+            const bool in_smem = (u - tu0) < p.a_cap;
+            const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = lane * 8 + 256 * i;
+                av[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (k < nk) av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
+                                            : __ldg(reinterpret_cast<const uint4 *>(arow + k));
+            }
+        };
+#pragma unroll 1
+        for (int m = 0; m < p.M; ++m) {
+            uint4 xv[4], an[4];
+            int cur_kc = -1;
+            if (first < tu1) load_a(first, an);
+#pragma unroll 1
+            for (int u = first; u < tu1; u += stride) {
+                const int kc = u / p.rank;
+                if (kc != cur_kc) {
+                    cur_kc = kc;
+                    const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = lane * 8 + 256 * i;
+                        xv[i] = make_uint4(0u, 0u, 0u, 0u);
+                        if (k < nk) xv[i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + kbeg + k));
+                    }
+                }
+                uint4 av[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) av[i] = an[i];
+                if (u + stride < tu1) load_a(u + stride, an);       // the next row of A is in flight during the sum
+                float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
+                    const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
+                        v0 = fmaf(xf.x, af.x, v0);
+                        v1 = fmaf(xf.y, af.y, v1);
+                    }
+                }
+                float v = v0 + v1;
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + (u - kc * p.rank), v);
+            }
+        }
+        return true;
+    };
+
+    // Who works the units off: the epilogue warp alone while there are few (token, unit) pairs (it has
+    // nothing else to do until the first tile is through: light variant), all eight compute warps before
+    // they turn to the weights when there are many (heavy variant: one warp would hold up the tiles).
+    const bool t_by_compute = HEAVY && has_t && !p.t_late;
 
     if (warp == kProdWarp) {
         // =================================================== producer warp
@@ -598,6 +674,12 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         bool dead = false;
         named_barrier_sync(1, kCW * 32);
         trace_mark(p, 5);
+        if (t_by_compute) {
+            if (!t_units(tu0 + warp, kCW)) dead = true;
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(t_done);
+        }
 
         // ---- consumer: every stage is shared; this warp takes an eighth of its groups ----
         const uint8_t *ring_ptr = smem + p.off_ring;
@@ -731,17 +813,18 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                    ? s_B + (size_t)(tile - tile_first) * kTileRows * p.rank
                    : nullptr;
     };
-    // Fast finish (rank <= 64, one K slice): lanes 2i and 2i+1 share row i of the tile; a lane holds
+    // Fast finish (rank <= 64, heavy variant 128; one K slice): lanes 2i and 2i+1 share row i of the tile; a lane holds
     // every other 8-element chunk of that row of B in registers, requested before the wait for the
     // segment, so that the up-projection costs no exposed load latency.
-    const bool fast_fin = (p.rank > 0) && (p.rank <= 64) && (p.SK == 1);
-    uint4 bq[4];
+    constexpr int NBQ = HEAVY ? 8 : 4;               // 8-element chunks of a row of B held per lane
+    const bool fast_fin = (p.rank > 0) && (p.rank <= 16 * NBQ) && (p.SK == 1);
+    uint4 bq[NBQ];
     auto b_prefetch = [&](int tile) {
         const int row = lane >> 1, n = tile * kTileRows + row;
         const T *own = own_b(tile);
         const T *src = own ? own + (size_t)row * p.rank : static_cast<const T *>(p.B) + (size_t)n * p.rank;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < NBQ; ++i) {
             const int c = (lane & 1) + 2 * i;
             bq[i] = make_uint4(0u, 0u, 0u, 0u);
             if (8 * c < p.rank && n < p.N)
@@ -755,7 +838,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         for (int m = 0; m < p.M; ++m) {
             float sub = 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < NBQ; ++i) {
                 const int c = (lane & 1) + 2 * i;
                 if (8 * c < p.rank) {
                     const float4 t0 = *reinterpret_cast<const float4 *>(s_t + (size_t)m * p.rank + 8 * c);
@@ -788,70 +871,6 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         __syncwarp();
     };
 
-    // This CTA's share of t = x.A^T:  t[m][j] += sum over its units (row j of A, k chunk).
-    // A comes from shared memory (bulk copy) for the first a_cap units, x from global memory.
-    auto t_share = [&]() {
-        if (!mbar_wait(a_full, 0)) {
-            dead = true;
-            return;
-        }
-        const T *A = static_cast<const T *>(p.A);
-        const T *x = static_cast<const T *>(p.x) + g0 * kGroupFast;
-        // one unit = row j of A against one k chunk of 1024 (units are numbered k-chunk-major:
-        // u = kc*rank + j); a lane takes 8 elements out of every 256
-        auto load_a = [&](int u, int kbeg, int nk, uint4 (&av)[4]) {
-            const int j = u - (u / p.rank) * p.rank;
-            const bool in_smem = (u - tu0) < p.a_cap;
-            const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int k = lane * 8 + 256 * i;
-                av[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (k < nk) av[i] = in_smem ? *reinterpret_cast<const uint4 *>(arow + k)
-                                            : __ldg(reinterpret_cast<const uint4 *>(arow + k));
-            }
-        };
-#pragma unroll 1
-        for (int u0 = tu0; u0 < tu1;) {
-            // the units of one k chunk share x: it is read once per token and kept in registers
-            const int kc = u0 / p.rank, uend = min(tu1, (kc + 1) * p.rank);
-            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
-#pragma unroll 1
-            for (int m = 0; m < p.M; ++m) {
-                uint4 xv[4], an[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int k = lane * 8 + 256 * i;
-                    xv[i] = make_uint4(0u, 0u, 0u, 0u);
-                    if (k < nk) xv[i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + kbeg + k));
-                }
-                load_a(u0, kbeg, nk, an);
-#pragma unroll 1
-                for (int u = u0; u < uend; ++u) {
-                    uint4 av[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) av[i] = an[i];
-                    if (u + 1 < uend) load_a(u + 1, kbeg, nk, an);     // next row of A is in flight during the sum
-                    float v0 = 0.f, v1 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t aw[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
-                        const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float2 af = Pk<T>::to_float2(aw[q]), xf = Pk<T>::to_float2(xw[q]);
-                            v0 = fmaf(xf.x, af.x, v0);
-                            v1 = fmaf(xf.y, af.y, v1);
-                        }
-                    }
-                    float v = v0 + v1;
-                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (lane == 0) atomicAdd(p.t + (size_t)m * p.rank + (u - kc * p.rank), v);
-                }
-            }
-            u0 = uend;
-        }
-    };
     // After this CTA's share of t is in: count it; the warp that completes t publishes
     // the flag and finishes every tile that was parked (by any CTA) before the flag was up.
     auto t_arrive = [&]() {
@@ -887,7 +906,11 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     };
 
     if (has_t && !p.t_late) {
-        t_share();
+        if (t_by_compute) {
+            if (!mbar_wait(t_done, 0)) dead = true;     // the compute warps' units are in
+        } else if (!t_units(tu0, 1)) {
+            dead = true;
+        }
         trace_mark(p, 3);
         t_arrive();
     }
@@ -976,7 +999,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     trace_mark(p, 8);
 
     if (has_t && p.t_late) {
-        t_share();
+        if (!t_units(tu0, 1)) dead = true;
         t_arrive();
     }
     // ---- tiles this warp still owes: finish them once t is complete, else park them
@@ -1036,10 +1059,10 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     trace_mark(p, 9);
 }
 
-template <int BITS, typename T, int MT>
+template <int BITS, typename T, int MT, bool HEAVY>
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams p)
 {
-    decode_body<BITS, T, MT>(p, (int)blockIdx.x);
+    decode_body<BITS, T, MT, HEAVY>(p, (int)blockIdx.x);
 }
 
 // Several independent problems in one grid: CTAs first[i] .. first[i+1]-1 run problem i exactly as
@@ -1051,12 +1074,12 @@ struct DecodeBatch {
     int first[kBatchMax + 1];
     int count;
 };
-template <int BITS, typename T, int MT>
+template <int BITS, typename T, int MT, bool HEAVY>
 __global__ void __launch_bounds__(kThreads, 2) decode_batch_kernel(const __grid_constant__ DecodeBatch b)
 {
     int pi = 0;
     while (pi + 1 < b.count && (int)blockIdx.x >= b.first[pi + 1]) ++pi;
-    decode_body<BITS, T, MT>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
+    decode_body<BITS, T, MT, HEAVY>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
 }
 
 // ------------------------------------------------------------------ host side
@@ -1103,7 +1126,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         const int nkc = (ngs_max * kGroupFast + kTUnitK - 1) / kTUnitK;
         const long long tu_max = ((long long)a.rank * nkc + pl.R - 1) / pl.R;
         pl.a_cap = (int)min(tu_max, 8LL);
-        size_t off = (size_t)(2 * 8 + 2 * kNBuf + 3) * 8;      // room for up to 8 stages' barriers
+        size_t off = (size_t)(2 * 8 + 2 * kNBuf + 4) * 8;      // room for up to 8 stages' barriers
         off = (off + 15) & ~(size_t)15;
         pl.off_tab = (int)off;
         pl.off_def = (int)off;
@@ -1164,10 +1187,10 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     return pl;
 }
 
-template <int BITS, typename T, int MT>
+template <int BITS, typename T, int MT, bool HEAVY>
 cudaError_t launch_variant(const DecodeParams &p, const Plan &pl, bool pdl, cudaStream_t s)
 {
-    auto kern = decode_kernel<BITS, T, MT>;
+    auto kern = decode_kernel<BITS, T, MT, HEAVY>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -1201,6 +1224,33 @@ void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t
 }
 
 namespace {
+template <typename X> struct TypeTag { using type = X; };
+
+// Calls f(bits, activation type, MT, HEAVY) with compile-time tags for this problem.
+template <typename F>
+cudaError_t dispatch_variant(const LinearArgs &a, F f, bool heavy)
+{
+    auto with_heavy = [&](auto bits, auto type, auto mt) {
+        return heavy ? f(bits, type, mt, std::true_type{}) : f(bits, type, mt, std::false_type{});
+    };
+    auto with_mt = [&](auto bits, auto type) {
+        return (a.M <= 8) ? with_heavy(bits, type, std::integral_constant<int, 1>{}) : with_heavy(bits, type, std::integral_constant<int, 2>{});
+    };
+    auto with_type = [&](auto bits) { return a.bf16 ? with_mt(bits, TypeTag<__nv_bfloat16>{}) : with_mt(bits, TypeTag<__half>{}); };
+    return (a.bits == 4) ? with_type(std::integral_constant<int, 4>{}) : with_type(std::integral_constant<int, 3>{});
+}
+
+// Heavy sub-branch: rank above what the light tile finish holds, or more (token, unit) pairs of the
+// down-projection per CTA than one warp should take by itself.
+bool heavy_sub_branch(const LinearArgs &a, const Plan &pl)
+{
+    if (a.rank == 0) return false;
+    if (a.rank > 64) return true;
+    const int G = a.K / kGroupFast, ngs = (G + pl.SK - 1) / pl.SK;
+    const long long tu = (long long)a.rank * ((ngs * kGroupFast + kTUnitK - 1) / kTUnitK);
+    return (tu + pl.R - 1) / pl.R * a.M > kTUnitsOneWarp;
+}
+
 DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, float *t, int *ctr, int *status, void *trace)
 {
     DecodeParams p{};
@@ -1230,10 +1280,10 @@ DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, fl
     return p;
 }
 
-template <int BITS, typename T, int MT>
+template <int BITS, typename T, int MT, bool HEAVY>
 cudaError_t launch_batch_variant(const DecodeBatch &b, size_t smem, bool pdl, cudaStream_t s)
 {
-    auto kern = decode_batch_kernel<BITS, T, MT>;
+    auto kern = decode_batch_kernel<BITS, T, MT, HEAVY>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -1260,15 +1310,10 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     if (!pl.ok) return cudaErrorInvalidConfiguration;
     const DecodeParams p = fill_params(a, pl, ws.partial, ws.t, ws.counters, ws.counters + kCtrStatus, ws.trace);
     const bool pdl = tune.pdl != 0;
-    cudaError_t e;
-    const int mt = (a.M <= 8) ? 1 : 2;
-    if (a.bf16) {
-        if (a.bits == 4) e = (mt == 1) ? launch_variant<4, __nv_bfloat16, 1>(p, pl, pdl, s) : launch_variant<4, __nv_bfloat16, 2>(p, pl, pdl, s);
-        else             e = (mt == 1) ? launch_variant<3, __nv_bfloat16, 1>(p, pl, pdl, s) : launch_variant<3, __nv_bfloat16, 2>(p, pl, pdl, s);
-    } else {
-        if (a.bits == 4) e = (mt == 1) ? launch_variant<4, __half, 1>(p, pl, pdl, s) : launch_variant<4, __half, 2>(p, pl, pdl, s);
-        else             e = (mt == 1) ? launch_variant<3, __half, 1>(p, pl, pdl, s) : launch_variant<3, __half, 2>(p, pl, pdl, s);
-    }
+    const bool heavy = heavy_sub_branch(a, pl);
+    cudaError_t e = dispatch_variant(a, [&](auto bits, auto type, auto mt, auto hv) {
+        return launch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value>(p, pl, pdl, s);
+    }, heavy);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -1305,6 +1350,7 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
     b.count = count;
     size_t smem = 0, off_p = 0, off_t = 0;
     int off_c = kCtrFirstTile;
+    bool heavy = false;
     for (int i = 0; i < count; ++i) {
         DecodeTuning tn = tune;
         tn.max_ctas = ctas[i];
@@ -1317,18 +1363,12 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
         off_t += (size_t)kDecodeMaxM * kMaxRank;
         off_c += kCtrFirstTile + 2 * pl.NT;
         smem = pl.smem > smem ? pl.smem : smem;
+        heavy = heavy || heavy_sub_branch(a[i], pl);
     }
     const bool pdl = tune.pdl != 0;
-    const LinearArgs &a0 = a[0];
-    cudaError_t e;
-    const int mt = (a0.M <= 8) ? 1 : 2;
-    if (a0.bf16) {
-        if (a0.bits == 4) e = (mt == 1) ? launch_batch_variant<4, __nv_bfloat16, 1>(b, smem, pdl, s) : launch_batch_variant<4, __nv_bfloat16, 2>(b, smem, pdl, s);
-        else              e = (mt == 1) ? launch_batch_variant<3, __nv_bfloat16, 1>(b, smem, pdl, s) : launch_batch_variant<3, __nv_bfloat16, 2>(b, smem, pdl, s);
-    } else {
-        if (a0.bits == 4) e = (mt == 1) ? launch_batch_variant<4, __half, 1>(b, smem, pdl, s) : launch_batch_variant<4, __half, 2>(b, smem, pdl, s);
-        else              e = (mt == 1) ? launch_batch_variant<3, __half, 1>(b, smem, pdl, s) : launch_batch_variant<3, __half, 2>(b, smem, pdl, s);
-    }
+    cudaError_t e = dispatch_variant(a[0], [&](auto bits, auto type, auto mt, auto hv) {
+        return launch_batch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value>(b, smem, pdl, s);
+    }, heavy);
     if (e == cudaSuccess) ++*launches;
     return e;
 }

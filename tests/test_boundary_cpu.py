@@ -37,9 +37,12 @@ def test_packed_words():
 def test_dispatch_rules():
     G, D, P = fbq.KERNEL_GENERIC, fbq.KERNEL_DECODE, fbq.KERNEL_PREFILL
     sel = fbq.select_kernel
-    for M in (1, 2, 6):
+    for M in (1, 2):
         assert sel(M, 4096, 4096, 128, 4, 32) == D
         assert sel(M, 11008, 4096, 128, 3, 64, bf16=True) == D
+    assert sel(6, 4096, 4096, 128, 4, 16) == D and sel(6, 4096, 4096, 128, 4, 0) == D
+    assert sel(4, 4096, 4096, 128, 4, 64) == P and sel(4, 4096, 4096, 128, 4, 32) == D    # M * rank above 128 from M = 3
+    assert sel(2, 4096, 4096, 128, 4, 128) == D
     for M in (7, 8, 15, 16):                        # measured crossover: the tensor-core kernel wins from M = 7
         assert sel(M, 4096, 4096, 128, 4, 32) == P
         assert sel(M, 4100, 4096, 128, 4, 32) == D  # N not a multiple of 8: outside the prefill kernel's domain

@@ -37,7 +37,7 @@ def _problems(fbq, M, bits, rank, dtype, seed0):
 
 @pytest.mark.parametrize("single", [1, 0])
 @pytest.mark.parametrize("bits,rank,dtype,M", [(3, 64, "f16", 1), (4, 64, "bf16", 1), (3, 0, "f16", 1), (3, 16, "f16", 5),
-                                              (4, 64, "f16", 6)])
+                                              (4, 64, "f16", 2), (3, 16, "bf16", 6)])
 def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M, single):
     import torch
     fbq.set_option("batch_single", single)       # 1: the decode kernel over a problem list; 0: one launch per problem
