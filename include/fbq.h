@@ -237,6 +237,11 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "prefill_pair"  1 = token tiles of 256 of the prefill kernel run on CTA pairs (cta_group::2 MMAs,
  *                   each CTA staging half of the token tile); 0 (default) = one CTA per tile, which
  *                   measured faster
+ *   "prefill_split" the prefill kernel at M <= 128, where a shape has fewer 128-row tiles than SMs: K is cut
+ *                   into up to 8 slices, one CTA each, which store fp32 partial tiles to the stream's scratch;
+ *                   the CTA that finishes last adds them in slice order and writes y (results do not depend
+ *                   on timing).  0 = never, 1 (default) = only for K >= 8192, 2 = whenever the tiles are
+ *                   few (faster for a linear that runs alone, slower when several run side by side)
  *   "batch_single"  1 = such a batch of up to 8 problems is one launch (default), 0 = one launch per problem
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives

@@ -12,6 +12,7 @@
 namespace fbq {
 void decode_set_test_switch(int t_late);
 void prefill_set_pair(int on);
+void prefill_set_split(int mode);
 
 namespace {
 
@@ -26,6 +27,7 @@ struct Options {
     int batch_ctas = 400;
     int batch_single = 1;
     int prefill_pair = 0;
+    int prefill_split = 1;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
@@ -145,12 +147,13 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         }
     }
     if (kernel == FBQ_KERNEL_PREFILL) {
-        size_t have_c = (size_t)ws->n_counters;
-        if ((e = grow(ws->counters, have_c, (size_t)prefill_counters_need(a.M), sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        size_t have_c = (size_t)ws->n_counters, need_t = 0, need_p = 0;
+        int need_c = 0;
+        prefill_workspace_need(a, &need_c, &need_t, &need_p);
+        if ((e = grow(ws->counters, have_c, (size_t)need_c, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         ws->n_counters = (int)have_c;
-        if (a.rank > 0 &&
-            (e = grow(ws->t_gen, ws->t_gen_floats, (size_t)a.M * a.rank, sizeof(float), s)) != cudaSuccess)
-            return FBQ_ERR_CUDA;
+        if (need_t > 0 && (e = grow(ws->t_gen, ws->t_gen_floats, need_t, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if (need_p > 0 && (e = grow(ws->partial, ws->partial_floats, need_p, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         e = launch_prefill(a, *ws, s, &launches);
         if (e == cudaErrorInvalidConfiguration) {
             (void)cudaGetLastError();
@@ -182,6 +185,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;
     if (!strcmp(name, "batch_single")) return &g_opt.batch_single;
     if (!strcmp(name, "prefill_pair")) return &g_opt.prefill_pair;
+    if (!strcmp(name, "prefill_split")) return &g_opt.prefill_split;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
@@ -287,6 +291,14 @@ int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, flo
     return rc;
 }
 
+// Hands the process-wide switches to the kernel files before a launch.
+static void apply_kernel_options()
+{
+    decode_set_test_switch(g_opt.decode_t_late);
+    prefill_set_pair(g_opt.prefill_pair);
+    prefill_set_split(g_opt.prefill_split);
+}
+
 static int linear_common(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
                          const void *B, void *y, int M, int N, int K, int group, int bits, int rank, bool bf16,
                          void *stream)
@@ -299,8 +311,7 @@ static int linear_common(const void *x, const uint32_t *qweight, const void *sca
     a.B = rank > 0 ? B : nullptr;
     a.y = y;
     a.M = M; a.N = N; a.K = K; a.group = group; a.bits = bits; a.rank = rank; a.bf16 = bf16;
-    decode_set_test_switch(g_opt.decode_t_late);
-    prefill_set_pair(g_opt.prefill_pair);
+    apply_kernel_options();
     return run_linear(a, static_cast<cudaStream_t>(stream));
 }
 
@@ -345,7 +356,7 @@ static int linear_batch_common(const fbq_problem *problems, int count, int M, in
     if (count < 0 || count > FBQ_BATCH_MAX || (count > 0 && !problems)) return FBQ_ERR_BADARG;
     if (count == 0) return FBQ_OK;
     cudaStream_t main = static_cast<cudaStream_t>(stream);
-    decode_set_test_switch(g_opt.decode_t_late);
+    apply_kernel_options();
     LinearArgs a[FBQ_BATCH_MAX];
     bool all_decode = count > 1;
     double total_cost = 0.0;

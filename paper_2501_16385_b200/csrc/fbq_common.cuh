@@ -88,7 +88,7 @@ bool decode_batch_need(const LinearArgs *a, int count, const int *ctas, const De
 cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas, Workspace &ws, const DecodeTuning &tune,
                                 cudaStream_t s, int *launches);
 bool prefill_supported(const LinearArgs &a);
-int prefill_counters_need(int M);
+void prefill_workspace_need(const LinearArgs &a, int *counters, size_t *t_floats, size_t *partial_floats);
 cudaError_t launch_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
 
 }  // namespace fbq

@@ -83,6 +83,9 @@ struct PrefillParams {
     int nt;                   // feature tiles of 128
     int *tflag;               // [token tiles] warps of t CTAs that have stored their part (self-clearing)
     int *tdone;               // [token tiles] main CTAs that have consumed t (self-clearing)
+    int splitk, splitt;       // K splits of a main tile / of a t tile (1 unless there are few tokens)
+    float *part;              // [tile][split][128 rows][TOK] fp32 partial tiles (splitk > 1)
+    int *split_ctr;           // [tile] splits that have stored their partial (self-clearing)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -389,7 +392,7 @@ template <int TOK> struct Smem {
     static constexpr uint32_t kRingOff = kStages * kStageBytes;
     static constexpr uint32_t kTableOff = kRingOff + kRing * kRawSlot;
     static constexpr uint32_t kBarOff = kTableOff + kRing * kBN * 4u;
-    static constexpr uint32_t kNumBars = 2 * kStages + 2 * kRing + 1 + 4;  // full, empty, ring full, ring empty, done, epilogue
+    static constexpr uint32_t kNumBars = 2 * kStages + 2 * kRing + 1 + 4 + 2;  // full, empty, ring full, ring empty, done, epilogue, split
     static constexpr uint32_t kTotal = kBarOff + kNumBars * 8u + 16u;
 };
 
@@ -421,23 +424,33 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         return;
     }
     const uint32_t full0 = sbase + L::kBarOff, empty0 = full0 + 8u * kStages, rfull0 = empty0 + 8u * kStages,
-                   rempty0 = rfull0 + 8u * kRing, done_bar = rempty0 + 8u * kRing, epi0 = done_bar + 8u;
+                   rempty0 = rfull0 + 8u * kRing, done_bar = rempty0 + 8u * kRing, epi0 = done_bar + 8u,
+                   split_bar = epi0 + 32u, split_bar2 = split_bar + 8u;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + L::kNumBars * 8u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    volatile int *split_last = abort_flag + 1;                  // 1: this CTA adds up the K splits of its tile
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool t_role = (int)blockIdx.x < p.n_t;                // t CTA or main CTA
-    int m_tile, n_tile;
-    if (t_role) {
-        m_tile = (int)blockIdx.x / p.rt;
-        n_tile = (int)blockIdx.x % p.rt;                        // tile of rank rows of A
-    } else {
-        m_tile = ((int)blockIdx.x - p.n_t) / p.nt;
-        n_tile = ((int)blockIdx.x - p.n_t) % p.nt;
+    // (token tile, feature or rank tile, K split): with few tokens there are few tiles, so K is split over
+    // several CTAs per tile (splitk main CTAs whose fp32 partial tiles the last one to finish adds up,
+    // splitt t CTAs that each store their own partial t)
+    int m_tile, n_tile, split;
+    const int S = t_role ? p.splitt : p.splitk;
+    {
+        int b = t_role ? (int)blockIdx.x : (int)blockIdx.x - p.n_t;
+        split = b % S;
+        b /= S;
+        const int tiles = t_role ? p.rt : p.nt;
+        m_tile = b / tiles;
+        n_tile = b % tiles;
     }
     const int m0 = m_tile * TOK, n0 = n_tile * kBN;
-    const int nkb = t_role ? p.kb_main : p.kb_main + p.kb_slab;
-    const int kb_x = p.kb_main;                                 // blocks below kb_x take their tokens from x
+    const int G_all = p.kb_main >> 1;
+    const int g_begin = (int)((long long)split * G_all / S), g_end = (int)((long long)(split + 1) * G_all / S);
+    const int kb_begin = 2 * g_begin;                           // first K block of this CTA's range
+    const int kb_x = 2 * (g_end - g_begin);                     // blocks [0, kb_x) of the CTA take their tokens from x
+    const int nkb = kb_x + ((t_role || split != 0) ? 0 : p.kb_slab);     // the sub-branch blocks go to split 0
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -450,7 +463,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         }
         pf_mbar_init(done_bar, 1);
         for (int i = 0; i < 4; ++i) pf_mbar_init(epi0 + 8u * i, 128);     // the four warps of a column quarter
+        pf_mbar_init(split_bar, kProducers / 32);               // every epilogue warp has stored its partial chunk
+        pf_mbar_init(split_bar2, 1);                            // warp 0 has counted the CTA in
         *abort_flag = 0;
+        *split_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {                  // the MMA warp owns the tensor-memory allocation
@@ -483,7 +499,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             // and 2h+1); thread (row r, part) dequantises the codes [32*part, +32) of both blocks.
             const int h = warp >> 3, part = (warp >> 2) & 1, r = tid & 127;
             const bool row_ok = n0 + r < p.N;
-            const int groups = p.kb_main >> 1;
+            const int groups = kb_x >> 1;
             // this thread's words inside a ring slot: block b holds codes [64b, 64b+64) of the group
             uint32_t roff0, roff1;
             if (BITS == 4) {                                // 64-byte rows, 16-byte chunk c stored at c ^ ((row / 2) % 4)
@@ -551,14 +567,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             // The halves take them in turn, one token row per thread.
             bool t_ready = false;
 #pragma unroll 1
-            for (int i = p.kb_main + h; i < nkb && !dead; i += 2) {
+            for (int i = kb_x + h; i < nkb && !dead; i += 2) {
                 const int s = i % kStages;
                 if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
                 if (!t_ready) {                              // every warp of every t CTA of this token tile has stored its part
                     int seen = 0;
                     if (lane == 0) {
                         const int *flag = p.tflag + m_tile;
-                        const int target = 16 * p.rt;
+                        const int target = 16 * p.rt * p.splitt;
 #pragma unroll 1
                         for (uint32_t spin = 0; spin < kPfFlagPolls; ++spin) {
                             asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
@@ -570,7 +586,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     t_ready = __shfl_sync(0xffffffffu, seen, 0) != 0;
                     if (!t_ready) { dead = true; break; }
                 }
-                const int j0 = (i - p.kb_main) * kBK;
+                const int j0 = (i - kb_x) * kBK;
                 const int rr = tid & (kHalf - 1);            // token row of the tile
                 if (rr < TOK) {
                     const int m = m0 + rr;
@@ -582,6 +598,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                             const float4 *ts = reinterpret_cast<const float4 *>(p.t32 + (size_t)m * p.rank + j0 + 8 * c);
                             t0 = __ldcg(ts);
                             t1 = __ldcg(ts + 1);
+                            for (int sp = 1; sp < p.splitt; ++sp) {         // partial t of the other K splits, in order
+                                const float4 *us = ts + (size_t)sp * p.M * p.rank / 4;
+                                const float4 u0 = __ldcg(us), u1 = __ldcg(us + 1);
+                                t0.x += u0.x; t0.y += u0.y; t0.z += u0.z; t0.w += u0.w;
+                                t1.x += u1.x; t1.y += u1.y; t1.z += u1.z; t1.w += u1.w;
+                            }
                         }
                         xa[4 * c] = P2<T>::pack(t0.x, t0.y); xa[4 * c + 1] = P2<T>::pack(t0.z, t0.w);
                         xa[4 * c + 2] = P2<T>::pack(t1.x, t1.y); xa[4 * c + 3] = P2<T>::pack(t1.z, t1.w);
@@ -611,7 +633,73 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             const int q = warp & 3, cg = warp >> 2;
             const int nn = n0 + 32 * q + lane;              // output feature (mode 0) / rank index (mode 1)
             const int c_begin = cg * (TOK / 4);
-            if (m0 + c_begin < p.M) {                       // uniform over the four warps of a column quarter
+            if (!t_role && S > 1) {
+                // ---- K split over S CTAs (TOK = 128: one 32-column chunk per warp).  Every CTA stores its
+                // fp32 partial tile; the CTA that counts in last adds the S partials in split order (the
+                // result does not depend on which CTA that is) and is the one that writes y.
+                const bool mine = m0 + c_begin < p.M;       // uniform over the four warps of a column quarter
+                const size_t slice = (size_t)kBN * TOK;
+                float *pt = p.part + ((size_t)(m_tile * p.nt + n_tile) * S) * slice + (size_t)(32 * q + lane) * TOK + c_begin;
+                uint32_t v[32];
+                if (mine) {
+                    tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c_begin, v);
+                    tc_wait_ld();
+                    float4 *dst = reinterpret_cast<float4 *>(pt + (size_t)split * slice);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        __stcg(dst + j, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                    __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+                }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(split_bar);
+                if (warp == 0 && lane == 0) {
+                    int last = 0;
+                    if (pf_mbar_wait(split_bar, 0)) {
+                        int *ctr = p.split_ctr + m_tile * p.nt + n_tile;
+                        last = (atomicAdd(ctr, 1) == S - 1);
+                        if (last) atomicExch(ctr, 0);       // left at zero for the next call
+                    } else {
+                        atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+                    }
+                    *split_last = last;
+                    __threadfence_block();
+                    pf_mbar_arrive(split_bar2);
+                }
+                const bool last = pf_mbar_wait(split_bar2, 0) && *split_last != 0;
+                if (last && mine) {
+                    __threadfence();
+                    float acc[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+#pragma unroll 1
+                    for (int sp = 0; sp < S; ++sp) {
+                        const float4 *src = reinterpret_cast<const float4 *>(pt + (size_t)sp * slice);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 u = __ldcg(src + j);
+                            acc[4 * j] += u.x; acc[4 * j + 1] += u.y; acc[4 * j + 2] += u.z; acc[4 * j + 3] += u.w;
+                        }
+                    }
+                    unsigned short *sp16 = reinterpret_cast<unsigned short *>(smem + (size_t)c_begin * (kBN * 2)) + 32 * q + lane;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sp16[j * kBN] = to_bits16<T>(acc[j]);
+                    pf_fence_proxy_async();                 // staged tile -> visible to the TMA store
+                    pf_mbar_arrive(epi0 + 8u * cg);
+                    if (q == 0 && lane == 0) {
+                        if (pf_mbar_wait(epi0 + 8u * cg, 0)) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&ymap)), "r"(n0), "r"(m0 + c_begin),
+                                           "r"(sbase + (uint32_t)c_begin * (kBN * 2))
+                                         : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        } else {
+                            atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+                        }
+                    }
+                }
+            } else if (m0 + c_begin < p.M) {                // uniform over the four warps of a column quarter
 #pragma unroll 1
                 for (int c = c_begin; c < c_begin + TOK / 4; c += 32) {
                     if (m0 + c >= p.M) break;               // warp-uniform
@@ -624,7 +712,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         for (int j = 0; j < 32; ++j) sp[j * kBN] = to_bits16<T>(__uint_as_float(v[j]));
                     } else {
                         if (nn < p.rank) {                   // 32 lanes = 32 consecutive rank indices: 128-byte stores
-                            float *tp = p.t32 + (size_t)(m0 + c) * p.rank + nn;
+                            float *tp = p.t32 + (size_t)split * p.M * p.rank + (size_t)(m0 + c) * p.rank + nn;
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (m0 + c + j < p.M) __stcg(tp + (size_t)j * p.rank, __uint_as_float(v[j]));
@@ -653,7 +741,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 __threadfence();
                 __syncwarp();
                 if (lane == 0) atomicAdd(p.tflag + m_tile, 1);
-            } else if (p.rank > 0 && tid == 0) {
+            } else if (p.rank > 0 && tid == 0 && split == 0) {
                 // this CTA has consumed t (its MMAs are complete).  The last main CTA of the token
                 // tile leaves the flag and the count at zero for the next call.
                 if (atomicAdd(p.tdone + m_tile, 1) == p.nt - 1) {
@@ -712,14 +800,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const uint32_t xt = sbase + (uint32_t)s * kStageBytes, wt = xt + kXBytes;
                 if (t_role) {
                     pf_mbar_expect_tx(bar, kXBytes + kWBytes);
-                    tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
-                    tma_load_2d(wt, &amap, kb * kBK, n0, bar);      // rows of A
+                    tma_load_2d(xt, &xmap, (kb_begin + kb) * kBK, m0, bar);
+                    tma_load_2d(wt, &amap, (kb_begin + kb) * kBK, n0, bar);      // rows of A
                 } else if (kb < kb_x) {
                     pf_mbar_expect_tx(bar, kXBytes);
-                    tma_load_2d(xt, &xmap, kb * kBK, m0, bar);
+                    tma_load_2d(xt, &xmap, (kb_begin + kb) * kBK, m0, bar);
                 } else {
                     pf_mbar_expect_tx(bar, kWBytes);
-                    tma_load_2d(wt, &bmap, (kb - p.kb_main) * kBK, n0, bar);   // rows of B
+                    tma_load_2d(wt, &bmap, (kb - kb_x) * kBK, n0, bar);   // rows of B
                 }
             }
             if (dead) {
@@ -735,7 +823,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         // eight groups it reads the rows' scales and zero points with 16-byte loads (two aligned chunks of the flat row-major arrays
         // cover any eight consecutive values), realigns them in registers, and before each group's
         // copy writes that group's (s | z << 16) words next to the ring slot.
-        const int G = p.K / kGroupFast, groups = p.kb_main >> 1;
+        const int G = p.K / kGroupFast, groups = kb_x >> 1;     // all groups of a row; groups of this CTA's K range
         const size_t n_chunks = (size_t)p.N * G / 8;        // N is a multiple of 8
         const uint4 *s_arr = reinterpret_cast<const uint4 *>(p.scales), *z_arr = reinterpret_cast<const uint4 *>(p.zeros);
         const int v = warp - kRawWarp;
@@ -746,7 +834,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         for (int k = 0; k < 2; ++k) {
             const int n = n0 + 64 * v + lane + 32 * k;
             ok[k] = n < p.N;
-            const size_t f = (size_t)(ok[k] ? n : 0) * G;
+            const size_t f = (size_t)(ok[k] ? n : 0) * G + g_begin;      // first group of this CTA's range
             a0[k] = f >> 3;
             off[k] = (uint32_t)f & 7u;
         }
@@ -810,7 +898,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         if (lane == 0) {
                             if (v == 0) {
                                 pf_mbar_expect_tx(rfull0 + 8u * slot, (uint32_t)kBN * WPG * 4u);
-                                tma_load_2d(ring0 + slot * kRawSlot, &wmap, gi * WPG, n0, rfull0 + 8u * slot);
+                                tma_load_2d(ring0 + slot * kRawSlot, &wmap, (g_begin + gi) * WPG, n0, rfull0 + 8u * slot);
                             } else {
                                 pf_mbar_arrive(rfull0 + 8u * slot);
                             }
@@ -1429,6 +1517,19 @@ cudaError_t make_map(CUtensorMap *map, const void *base, bool elem32, size_t col
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// K splits of a main tile when all tokens fit one tile of 128: as many as keep the CTA count near the
+// number of SMs, at most 8, at least 2 groups of K per split.
+int g_split_mode = 1;     // 0: never split K, 1: only deep K (>= 8192), 2: whenever tiles are few
+int prefill_splits(int N, int K)
+{
+    if (g_split_mode == 0 || (g_split_mode == 1 && K < 8192)) return 1;
+    const int nt = (N + kBN - 1) / kBN, G = K / kGroupFast;
+    int s = 148 / nt;
+    if (s > 8) s = 8;
+    if (s > G / 2) s = G / 2;
+    return s < 1 ? 1 : s;
+}
+
 template <typename T, int TOK, bool PAIR>
 cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches)
 {
@@ -1448,9 +1549,19 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
         p.nt = (p.nt + 1) & ~1;
         p.rt = (p.rt + 1) & ~1;
     }
-    p.n_t = mt * p.rt;
+    // Few tokens mean few tiles: split K so that about one CTA per SM has work (single-CTA kernel, one
+    // token tile).  The same number of splits goes to the t CTAs, which are cheap.
+    p.splitk = p.splitt = 1;
+    if (!PAIR && TOK == 128 && mt == 1) {             // (the split epilogue is written for one 32-column chunk per warp)
+        const int want = prefill_splits(a.N, a.K);
+        p.splitk = want;
+        p.splitt = (a.rank > 0) ? want : 1;
+    }
+    p.n_t = mt * p.rt * p.splitt;
     p.tflag = ws.counters + kPfCtrBase;
     p.tdone = p.tflag + mt;
+    p.split_ctr = p.tdone + mt;
+    p.part = ws.partial;
     CUtensorMap xmap, qmap, amap, bmap, ymap;
     cudaError_t e;
     if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, PAIR ? 128 : TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess)
@@ -1465,7 +1576,7 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
         if ((e = make_map(&amap, a.A, false, (size_t)a.K, (size_t)a.rank, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
         if ((e = make_map(&bmap, a.B, false, (size_t)a.rank, (size_t)a.N, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
     }
-    const unsigned grid = (unsigned)p.n_t + (unsigned)p.nt * (unsigned)mt;
+    const unsigned grid = (unsigned)p.n_t + (unsigned)p.nt * (unsigned)mt * (unsigned)p.splitk;
     if (PAIR)
         e = (a.bits == 4) ? launch_pair_kernel<4, T>(xmap, qmap, amap, bmap, ymap, p, grid, s)
                           : launch_pair_kernel<3, T>(xmap, qmap, amap, bmap, ymap, p, grid, s);
@@ -1482,6 +1593,7 @@ inline bool aligned16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 
 
 // 1: token tiles of 256 run on CTA pairs (cta_group::2); 0: single-CTA kernel
 void prefill_set_pair(int on) { g_pair = on ? 1 : 0; }
+void prefill_set_split(int mode) { g_split_mode = mode; }
 
 bool prefill_supported(const LinearArgs &a)
 {
@@ -1489,8 +1601,17 @@ bool prefill_supported(const LinearArgs &a)
            a.M >= 1 && a.M <= (1 << 22);
 }
 
-// Ints of ws.counters the prefill path uses for a call with M tokens (zero between calls).
-int prefill_counters_need(int M) { return kPfCtrBase + 2 * ((M + 127) / 128); }
+// Scratch the prefill path needs in the workspace for this call: counters (zero between calls), floats
+// of t (one slice per K split), floats of fp32 partial tiles (K split only).
+void prefill_workspace_need(const LinearArgs &a, int *counters, size_t *t_floats, size_t *partial_floats)
+{
+    const int nt = (a.N + kBN - 1) / kBN;
+    const int mt128 = (a.M + 127) / 128;
+    const int splits = (a.M <= 128) ? prefill_splits(a.N, a.K) : 1;
+    *counters = kPfCtrBase + 2 * mt128 + nt * mt128 + 2;
+    *t_floats = (size_t)a.M * a.rank * splits;
+    *partial_floats = (splits > 1) ? (size_t)nt * splits * kBN * 128 : 0;
+}
 
 // ws.t_gen must hold M x rank floats and ws.counters prefill_counters_need(M) ints (the caller
 // grows them; new counters start at zero and the kernel leaves them at zero).

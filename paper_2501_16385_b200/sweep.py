@@ -69,8 +69,13 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--tokens", type=int, nargs="*", default=[1, 2, 4, 8, 16])
+    ap.add_argument("--opt", nargs="*", default=[], help="library options as name=value (fbq_set_option)")
     a = ap.parse_args()
-    for M in (1, 2, 4, 8, 16):
+    for kv in a.opt:
+        name, value = kv.split("=")
+        fbq.set_option(name, int(value))
+    for M in a.tokens:
         base = None
         for rank in (0, 16, 32, 64, 128):
             us = time_layer(M, a.bits, rank, a.steps)

@@ -93,3 +93,26 @@ def test_prefill_cta_pair_variant(fbq, bits, dtype, M, N, K, rank):
         assert fbq.poll_status() == 0
     finally:
         fbq.set_option("prefill_pair", 0)
+
+
+@pytest.mark.parametrize("bits,dtype,M,N,K,rank", [(3, "f16", 16, 512, 4096, 64), (4, "bf16", 8, 1160, 2048, 128),
+                                                   (4, "f16", 100, 384, 1408, 0), (3, "f16", 7, 136, 1024, 8)])
+def test_prefill_few_tokens_split_k(fbq, bits, dtype, M, N, K, rank):
+    # M <= 128: K is split over several CTAs per tile (fp32 partial tiles, the last CTA adds them up;
+    # partial t per split); called three times in a row: the counters must be back at zero each time
+    import torch
+    inp = make_linear(M, N, K, bits, rank, dtype=dtype, seed=2400 + M, outlier_frac=0.01 if dtype == "bf16" else 0.0)
+    fbq.set_option("force_kernel", fbq.KERNEL_PREFILL)
+    fbq.set_option("prefill_split", 2)                                      # split whenever the tiles are few
+    try:
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, floor=2e-5 if dtype == "f16" else 5e-4)
+        dev = DeviceLinear(inp, fbq)
+        ys = [dev.run(fbq).clone() for _ in range(3)]
+        torch.cuda.synchronize()
+        assert fbq.poll_status() == 0
+        assert torch.equal(ys[0], ys[1]) and torch.equal(ys[1], ys[2])      # partials are added in split order
+        fbq.set_option("prefill_split", 0)                                  # and the unsplit kernel on the same input
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, floor=2e-5 if dtype == "f16" else 5e-4)
+    finally:
+        fbq.set_option("force_kernel", -1)
+        fbq.set_option("prefill_split", 1)
