@@ -180,6 +180,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_chunk")) return &g_opt.decode.chunk;
     if (!strcmp(name, "decode_depth")) return &g_opt.decode.depth;
     if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
+    if (!strcmp(name, "decode_i8")) return &g_opt.decode.i8;
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
     if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;

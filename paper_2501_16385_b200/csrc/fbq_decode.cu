@@ -54,6 +54,7 @@ constexpr int kTUnitK = 1024;                // k extent of one unit of the down
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kEarlyStages = 1;                // weight stages prefetched before x has been requested
 constexpr int kTUnitsOneWarp = 10;             // (token, unit) pairs of the down-projection one warp takes by itself
+constexpr int kI8MaxM = 2;                     // tokens of the integer form: 3 digits (and a spare column) each fill the MMA's 8 columns
 constexpr int kTPolls = 64;                  // looks at the "t complete" flag before a finished tile is parked
 
 // counters[] layout (ints) inside the per-stream scratch
@@ -119,6 +120,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 #pragma unroll 1
     for (uint32_t i = 0; i < kWaitLimit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// The same for the warps that wait most of the time (producer, epilogue): they back off between
+// looks so that their polling does not take issue slots from the compute warps of their SM.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity)
+{
+#pragma unroll 1
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(100);
+    }
     return false;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
@@ -306,6 +318,71 @@ template <int BITS> __device__ __forceinline__ int frag_pos(int c)
     const int i = c / 10, f = c - 10 * i;
     return (f < 5) ? 2 * (5 * i + f) : 2 * (5 * i + f - 5) + 1;
 }
+// ------------------------------------------------- integer form (M <= 2)
+// A 3- or 4-bit code masked out of its word where it sits is already an unsigned
+// byte q * 2^j (j = the field's offset inside its byte): an operand of the 8-bit
+// integer MMA (m16n8k32, u8 x s8 -> s32) as it stands, four codes per register,
+// with no magic constant, no zero-point arithmetic and at most one shift per word:
+//   INT4 word i:  r[2i]   = w & 0x0F0F0F0F          codes 8i+0, 8i+2, 8i+4, 8i+6
+//                 r[2i+1] = w & 0xF0F0F0F0          codes 8i+1, 8i+3, 8i+5, 8i+7   (x 16)
+//   INT3 word i:  r[3i]   = w & 0x0E070E07          codes 10i+0, 10i+3 (x 2), 10i+5, 10i+8 (x 2)
+//                 r[3i+1] = w & 0x70387038          codes 10i+1 (x 8), 10i+4 (x 16), 10i+6 (x 8), 10i+9 (x 16)
+//                 r[3i+2] = (w >> 6) & 0x02070207   codes 10i+2, bit i of code 30 (x 2), 10i+7, bit i of code 31 (x 2)
+// The three bits of the bit-sliced codes 30 and 31 are three operands of their
+// own, so a lane's 32 codes of INT3 take 36 slots (9 registers, 4.5 MMAs).
+// x becomes fixed point: per group the power of two 2^e that puts the group's
+// largest |x| into [2^20, 2^21) (the slots of the bit-sliced codes take up to 2x, and
+// three signed digits hold |X| < 2^23 - 2^15), per slot X = rint(x 2^e 2^-j) (the slot's
+// factor undone), and X is written with three signed base-256 digits, X = d0 2^16 +
+// d1 2^8 + d2 (the bytes of (X + 0x808080) ^ 0x808080).  At M <= 2 the MMA has
+// columns to spare: column 4m + i carries digit i of token m, the int32 sums of
+// the three columns are exact, and they are added with the weights 2^16, 2^8, 1
+// (times 2^-e) in fp32.  An fp16 or bf16 x is represented to 2^-17 of the
+// group's maximum or better, far below the rounding of the fp16 product path.
+template <int BITS> struct SlotsI8 {
+    static constexpr int kRegs = (BITS == 4) ? 8 : 9;
+    // code (0..31) of a lane's run whose value sits in byte j of register R
+    static __host__ __device__ constexpr int code(int R, int j)
+    {
+        if (BITS == 4) return 8 * (R >> 1) + 2 * j + (R & 1);
+        const int i = R / 3, f = R % 3;
+        if (f == 2 && (j & 1)) return 30 + (j >> 1);
+        return 10 * i + 5 * (j >> 1) + f + 3 * (j & 1);
+    }
+    // log2 of the factor x is stored with in that slot
+    static __host__ __device__ constexpr int scale_log2(int R, int j)
+    {
+        if (BITS == 4) return (R & 1) ? -4 : 0;
+        const int i = R / 3, f = R % 3;
+        if (f == 2) return (j & 1) ? i - 1 : 0;
+        if (f == 1) return (j & 1) ? -4 : -3;
+        return (j & 1) ? -1 : 0;
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *r)
+    {
+        if (BITS == 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                r[2 * i] = w[i] & 0x0F0F0F0Fu;
+                r[2 * i + 1] = w[i] & 0xF0F0F0F0u;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                r[3 * i] = w[i] & 0x0E070E07u;
+                r[3 * i + 1] = w[i] & 0x70387038u;
+                r[3 * i + 2] = (w[i] >> 6) & 0x02070207u;
+            }
+        }
+    }
+};
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // x in shared memory: per token and 128-element group, 16-byte units are laid out
 // [h_index / 4][lane t][h_index % 4], so that one 128-bit load per lane fetches the
 // operands of two MMAs, conflict free.
@@ -394,7 +471,7 @@ __device__ __forceinline__ bool tile_claim(const DecodeParams &p, int tile, int 
 // HEAVY selects the variant for a heavy sub-branch (rank above 64, or many (token, unit) pairs of the
 // down-projection per CTA): its units are shared by the eight compute warps and the tile finish
 // keeps twice as many chunks of B in registers.  The light variant keeps both out of its code.
-template <int BITS, typename T, int MT, bool HEAVY>
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -557,13 +634,17 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         }
         // the weight stream
         const uint32_t ring = smem_u32(smem + p.off_ring);
-        int it = 0;
+        int it = 0, slot = -1;
+        uint32_t lap = 1u;                       // parity of the ring lap before the current one
         bool dead = false;
         for (int seg = 0; seg < nseg && !dead; ++seg) {
             const int tile = tile_first + seg;
             for (int pos = 0; pos < ngs; pos += p.CHG, ++it) {
                 const int ng = min(p.CHG, ngs - pos);
-                const int slot = it % p.NS;
+                if (++slot == p.NS) {
+                    slot = 0;
+                    lap ^= 1u;
+                }
                 // Until the compute warps have put their loads of x (which everything waits for)
                 // into the memory system, keep the prefetch shallow: x must not queue behind
                 // megabytes of weights that cannot be used before it arrives.
@@ -571,7 +652,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                     dead = true;
                     break;
                 }
-                if (it >= p.NS && !mbar_wait(st_empty + 8u * slot, (uint32_t)(it / p.NS - 1) & 1u)) {
+                if (it >= p.NS && !mbar_wait_idle(st_empty + 8u * slot, lap)) {
                     dead = true;
                     break;
                 }
@@ -618,7 +699,85 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         pdl_wait();
         pdl_launch_dependents();
         trace_mark(p, 3);
-        {
+        if constexpr (I8) {
+            // One lane takes one 32-element run of x (the k range of lane tq of one group), an even warp
+            // the run's registers 0..3, an odd warp the rest.  Per group: 2^e puts the largest |x| into
+            // [2^20, 2^21); per slot X = rint(x 2^e 2^-j) and its three signed base-256 digits.
+            constexpr int NR = SlotsI8<BITS>::kRegs;
+            const T *x = static_cast<const T *>(p.x);
+            const int ncol = 4 * p.M;
+            float2 *s_ux = reinterpret_cast<float2 *>(smem + p.off_px);               // (2^-e, X0) [slice group][token slot]
+            uint4 *s_x8 = reinterpret_cast<uint4 *>(smem + p.off_x);                  // [slice group][chunk][column][lane tq]
+            uint32_t *s_xt = reinterpret_cast<uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16;   // register 8
+            if (p.M == 1)
+                for (int i = tid; i < ngs; i += nthr) s_ux[2 * i + 1] = make_float2(0.f, 0.f);
+            const int runs_per_tok = kslice / 32, nruns = p.M * runs_per_tok;         // multiples of 4
+            const int upper = warp & 1;
+            for (int base = 0; base < nruns; base += (kCW / 2) * 32) {
+                const int idx = base + (warp >> 1) * 32 + lane;                       // whole quads are valid or not
+                const bool valid = idx < nruns;
+                const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+                uint4 xv[4];
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + g0 * kGroupFast + run * 32);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+                if (base == 0) {                                  // our loads of x are on their way
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(x_req);
+                }
+                const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
+                float xf[32];
+                float amax = 0.f, xsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    T xe;
+                    *reinterpret_cast<uint16_t *>(&xe) = e[c];
+                    xf[c] = ActTraits<T>::to_float(xe);
+                    amax = fmaxf(amax, fabsf(xf[c]));
+                    xsum += xf[c];
+                }
+                // the four runs of one (token, group) sit in four consecutive lanes
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+                const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 32u), 230u);          // biased exponent of the maximum
+                const float xs = __uint_as_float((274u - ex) << 23);                         // 2^(20 - floor(log2 max))
+                if (valid && !upper && (run & 3) == 0)
+                    s_ux[(run >> 2) * 2 + m] = make_float2(__uint_as_float((ex - 20u) << 23), xsum);   // 1 / xs
+                auto make = [&](auto rbeg, auto rend) {
+                    constexpr int R0 = decltype(rbeg)::value, R1 = decltype(rend)::value;
+                    uint32_t dg[R1 - R0][3];
+#pragma unroll
+                    for (int R = R0; R < R1; ++R) {
+                        uint32_t y[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            constexpr float kPow[7] = {1.f / 16.f, 1.f / 8.f, 1.f / 4.f, 1.f / 2.f, 1.f, 2.f, 4.f};
+                            const float f = xs * kPow[SlotsI8<BITS>::scale_log2(R, j) + 4];
+                            const int X = __float2int_rn(xf[SlotsI8<BITS>::code(R, j)] * f);
+                            y[j] = ((uint32_t)X + 0x00808080u) ^ 0x00808080u;
+                        }
+                        // digit i of the four slots -> one register (byte j = slot j)
+                        const uint32_t lo01 = __byte_perm(y[0], y[1], 0x5140), lo23 = __byte_perm(y[2], y[3], 0x5140);   // b0 b0' b1 b1'
+                        dg[R - R0][2] = __byte_perm(lo01, lo23, 0x5410);
+                        dg[R - R0][1] = __byte_perm(lo01, lo23, 0x7632);
+                        dg[R - R0][0] = __byte_perm(__byte_perm(y[0], y[1], 0x0062), __byte_perm(y[2], y[3], 0x0062), 0x5410);
+                    }
+                    if (valid) {
+                        const int gl = run >> 2, lq = run & 3;
+#pragma unroll
+                        for (int k = 0; k < 3; ++k) {
+                            const int col = 4 * m + k;
+                            s_x8[(size_t)((gl * 2 + R0 / 4) * ncol + col) * 4 + lq] = make_uint4(dg[0][k], dg[1][k], dg[2][k], dg[3][k]);
+                            if constexpr (R1 - R0 == 5) s_xt[(size_t)(gl * ncol + col) * 4 + lq] = dg[4][k];
+                        }
+                    }
+                };
+                if (!upper) make(std::integral_constant<int, 0>{}, std::integral_constant<int, 4>{});
+                else make(std::integral_constant<int, 4>{}, std::integral_constant<int, NR>{});
+            }
+        } else {
             // One thread prepares one 32-element run of x: 64 contiguous bytes in, the run's 16
             // fragment-order pairs (four 16-byte units) out, with compile-time positions.
             const T *x = static_cast<const T *>(p.x);
@@ -683,20 +842,28 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
 
         // ---- consumer: every stage is shared; this warp takes an eighth of its groups ----
         const uint8_t *ring_ptr = smem + p.off_ring;
-        int it = 0;
+        int it = 0, slot = -1;
+        uint32_t lap = 1u;                       // parity of the current lap around the ring, inverted
+        long long t_wait = 0;                    // trace: cycles spent waiting for weight stages
         for (int seg = 0; seg < nseg && !dead; ++seg) {
             float acc[MT][4];
+            float accz[2] = {0.f, 0.f};          // integer form: sum of (s z) X0 of rows g and g + 8
 #pragma unroll
             for (int b = 0; b < MT; ++b)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[b][i] = 0.f;
             for (int pos = 0; pos < ngs; pos += p.CHG, ++it) {
                 const int ng = min(p.CHG, ngs - pos);
-                const int slot = it % p.NS;
-                if (!mbar_wait(st_full + 8u * slot, (uint32_t)(it / p.NS) & 1u)) {
+                if (++slot == p.NS) {
+                    slot = 0;
+                    lap ^= 1u;
+                }
+                const long long c_wait = p.trace ? clock64() : 0;
+                if (!mbar_wait(st_full + 8u * slot, lap ^ 1u)) {
                     dead = true;
                     break;
                 }
+                if (p.trace) t_wait += clock64() - c_wait;
                 if (it == 0) trace_mark(p, 6);
                 const uint8_t *slot_ptr = ring_ptr + (size_t)slot * p.stage_bytes;
                 const uint32_t bytes_row = (uint32_t)row_pitch(ng);
@@ -719,6 +886,39 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                             wa[i] = reinterpret_cast<const uint32_t *>(pa)[i];
                             wb[i] = reinterpret_cast<const uint32_t *>(pb)[i];
                         }
+                    }
+                    if constexpr (I8) {
+                        constexpr int NR = SlotsI8<BITS>::kRegs;
+                        uint32_t ra[NR], rb[NR];
+                        SlotsI8<BITS>::run(wa, ra);
+                        SlotsI8<BITS>::run(wb, rb);
+                        // this lane's column (token g / 4, digit g % 4) of the group, and (2^-e, X0) of the
+                        // token whose columns its accumulators hold
+                        const int ncol = 4 * p.M;
+                        const uint4 *xg = reinterpret_cast<const uint4 *>(smem + p.off_x) + (size_t)((pos + gi) * 2 * ncol + g) * 4 + tq;
+                        uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
+                        uint32_t xt = 0u;
+                        if (g < ncol && (g & 3) != 3) {
+                            x0 = xg[0];
+                            x1 = xg[ncol * 4];
+                            if (BITS == 3)
+                                xt = (reinterpret_cast<const uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16)[((pos + gi) * ncol + g) * 4 + tq];
+                        }
+                        const float2 ux = reinterpret_cast<const float2 *>(smem + p.off_px)[(pos + gi) * 2 + (tq >> 1)];
+                        int d[4] = {0, 0, 0, 0};
+                        mma_u8s8(d, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
+                        mma_u8s8(d, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
+                        mma_u8s8(d, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
+                        mma_u8s8(d, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
+                        if constexpr (BITS == 3) mma_u8s8(d, ra[NR - 1], rb[NR - 1], 0u, 0u, xt, 0u);
+                        const float sa = fa.x * ux.x, sb = fb.x * ux.x;
+                        acc[0][0] = fmaf(sa, (float)d[0], acc[0][0]);
+                        acc[0][1] = fmaf(sa, (float)d[1], acc[0][1]);
+                        acc[0][2] = fmaf(sb, (float)d[2], acc[0][2]);
+                        acc[0][3] = fmaf(sb, (float)d[3], acc[0][3]);
+                        accz[0] = fmaf(fa.y, ux.y, accz[0]);
+                        accz[1] = fmaf(fb.y, ux.y, accz[1]);
+                        continue;
                     }
                     uint32_t ha[16], hb[16];
                     Unpack<BITS, T>::run(wa, ha);
@@ -764,6 +964,21 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                 if (lane == 0) mbar_arrive(st_empty + 8u * slot);
             }
             if (dead) break;
+            if constexpr (I8) {
+                // Columns 4m, 4m+1, 4m+2 are the digits of token m (weights 2^16, 2^8, 1), column 4m+3 is empty;
+                // lane tq = 2m holds the first two, 2m + 1 the rest; afterwards lane tq = 0 holds (token 0,
+                // token 1) of rows g and g + 8.
+                const float w0 = (tq & 1) ? 1.f : 65536.f, w1 = (tq & 1) ? 0.f : 256.f;
+                float vg = fmaf(acc[0][1], w1, acc[0][0] * w0), vh = fmaf(acc[0][3], w1, acc[0][2] * w0);
+                vg += __shfl_xor_sync(0xffffffffu, vg, 1);
+                vh += __shfl_xor_sync(0xffffffffu, vh, 1);
+                vg -= accz[0];
+                vh -= accz[1];
+                acc[0][0] = vg;
+                acc[0][1] = __shfl_xor_sync(0xffffffffu, vg, 2);
+                acc[0][2] = vh;
+                acc[0][3] = __shfl_xor_sync(0xffffffffu, vh, 2);
+            }
 
             // ---- deposit this warp's partial tile for the epilogue warp ---------------
             const int buf = seg % kNBuf;
@@ -782,6 +997,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             trace_mark(p, seg == 0 ? 7 : 8);
         }
         trace_mark(p, 9);
+        if (p.trace && lane == 0) p.trace[((size_t)blockIdx.x * kWarps + warp) * 16 + 12] = (unsigned long long)t_wait;
         if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
         return;
     }
@@ -930,7 +1146,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             others_in = __shfl_sync(0xffffffffu, others_in, 0);
         }
         if (fast_fin) b_prefetch(tile);
-        if (!mbar_wait(seg_full + 8u * buf, (uint32_t)(seg / kNBuf) & 1u)) {
+        if (!mbar_wait_idle(seg_full + 8u * buf, (uint32_t)(seg / kNBuf) & 1u)) {
             dead = true;
             break;
         }
@@ -1059,10 +1275,10 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     trace_mark(p, 9);
 }
 
-template <int BITS, typename T, int MT, bool HEAVY>
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams p)
 {
-    decode_body<BITS, T, MT, HEAVY>(p, (int)blockIdx.x);
+    decode_body<BITS, T, MT, HEAVY, I8>(p, (int)blockIdx.x);
 }
 
 // Several independent problems in one grid: CTAs first[i] .. first[i+1]-1 run problem i exactly as
@@ -1074,12 +1290,12 @@ struct DecodeBatch {
     int first[kBatchMax + 1];
     int count;
 };
-template <int BITS, typename T, int MT, bool HEAVY>
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 __global__ void __launch_bounds__(kThreads, 2) decode_batch_kernel(const __grid_constant__ DecodeBatch b)
 {
     int pi = 0;
     while (pi + 1 < b.count && (int)blockIdx.x >= b.first[pi + 1]) ++pi;
-    decode_body<BITS, T, MT, HEAVY>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
+    decode_body<BITS, T, MT, HEAVY, I8>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
 }
 
 // ------------------------------------------------------------------ host side
@@ -1089,6 +1305,7 @@ struct Plan {
     int off_tab, off_def, off_meta, off_x, off_px, off_segbuf, off_A, off_B, off_t, off_ring;
     size_t smem;
     bool ok;
+    bool i8;            // codes and x go to the tensor cores as 8-bit integers (M <= 2)
 };
 
 int g_sm_count = 0;
@@ -1111,6 +1328,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     int max_ctas = 2 * g_sm_count;            // two CTAs per SM: one streams while the other starts or ends
     if (tune.max_ctas > 0) max_ctas = min(max_ctas, tune.max_ctas);
     pl.vt = (mt == 2) ? 4 : min(4, (a.M + 1) / 2);
+    pl.i8 = tune.i8 != 0 && a.M <= kI8MaxM;
     // K slices: one, unless the x slice and the other tables do not fit next to the ring.
     // First try to stay within half an SM's shared memory (so that this launch and the next
     // one can be resident together) with few slices; otherwise take the whole SM.
@@ -1137,7 +1355,8 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         off += (size_t)pl.meta_rows * (ngs_max | 1) * 8;
         off = (off + 127) & ~(size_t)127;
         pl.off_x = (int)off;
-        off += (size_t)a.M * pl.x_pitch * 2;
+        // x of the slice: 16-bit values per token, or (integer form) four one-byte columns per value, 36 slots per 32 values
+        off += pl.i8 ? (size_t)ngs_max * (4 * a.M) * 144 : (size_t)a.M * pl.x_pitch * 2;
         off = (off + 127) & ~(size_t)127;
         pl.off_px = (int)off;
         off += (size_t)ngs_max * 8 * mt * 8;
@@ -1187,10 +1406,10 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     return pl;
 }
 
-template <int BITS, typename T, int MT, bool HEAVY>
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 cudaError_t launch_variant(const DecodeParams &p, const Plan &pl, bool pdl, cudaStream_t s)
 {
-    auto kern = decode_kernel<BITS, T, MT, HEAVY>;
+    auto kern = decode_kernel<BITS, T, MT, HEAVY, I8>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -1226,15 +1445,18 @@ void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t
 namespace {
 template <typename X> struct TypeTag { using type = X; };
 
-// Calls f(bits, activation type, MT, HEAVY) with compile-time tags for this problem.
+// Calls f(bits, activation type, MT, HEAVY, I8) with compile-time tags for this problem (the integer
+// form exists for one token block only).
 template <typename F>
-cudaError_t dispatch_variant(const LinearArgs &a, F f, bool heavy)
+cudaError_t dispatch_variant(const LinearArgs &a, F f, bool heavy, bool i8)
 {
-    auto with_heavy = [&](auto bits, auto type, auto mt) {
-        return heavy ? f(bits, type, mt, std::true_type{}) : f(bits, type, mt, std::false_type{});
+    auto with_heavy = [&](auto bits, auto type, auto mt, auto e4) {
+        return heavy ? f(bits, type, mt, std::true_type{}, e4) : f(bits, type, mt, std::false_type{}, e4);
     };
     auto with_mt = [&](auto bits, auto type) {
-        return (a.M <= 8) ? with_heavy(bits, type, std::integral_constant<int, 1>{}) : with_heavy(bits, type, std::integral_constant<int, 2>{});
+        if (i8) return with_heavy(bits, type, std::integral_constant<int, 1>{}, std::true_type{});
+        return (a.M <= 8) ? with_heavy(bits, type, std::integral_constant<int, 1>{}, std::false_type{})
+                          : with_heavy(bits, type, std::integral_constant<int, 2>{}, std::false_type{});
     };
     auto with_type = [&](auto bits) { return a.bf16 ? with_mt(bits, TypeTag<__nv_bfloat16>{}) : with_mt(bits, TypeTag<__half>{}); };
     return (a.bits == 4) ? with_type(std::integral_constant<int, 4>{}) : with_type(std::integral_constant<int, 3>{});
@@ -1280,10 +1502,10 @@ DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, fl
     return p;
 }
 
-template <int BITS, typename T, int MT, bool HEAVY>
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 cudaError_t launch_batch_variant(const DecodeBatch &b, size_t smem, bool pdl, cudaStream_t s)
 {
-    auto kern = decode_batch_kernel<BITS, T, MT, HEAVY>;
+    auto kern = decode_batch_kernel<BITS, T, MT, HEAVY, I8>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -1311,9 +1533,10 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     const DecodeParams p = fill_params(a, pl, ws.partial, ws.t, ws.counters, ws.counters + kCtrStatus, ws.trace);
     const bool pdl = tune.pdl != 0;
     const bool heavy = heavy_sub_branch(a, pl);
-    cudaError_t e = dispatch_variant(a, [&](auto bits, auto type, auto mt, auto hv) {
-        return launch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value>(p, pl, pdl, s);
-    }, heavy);
+    cudaError_t e = dispatch_variant(a, [&](auto bits, auto type, auto mt, auto hv, auto e4) {
+        return launch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value,
+                              decltype(e4)::value>(p, pl, pdl, s);
+    }, heavy, pl.i8);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -1350,12 +1573,13 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
     b.count = count;
     size_t smem = 0, off_p = 0, off_t = 0;
     int off_c = kCtrFirstTile;
-    bool heavy = false;
+    bool heavy = false, i8 = false;
     for (int i = 0; i < count; ++i) {
         DecodeTuning tn = tune;
         tn.max_ctas = ctas[i];
         const Plan pl = make_plan(a[i], tn);
         if (!pl.ok) return cudaErrorInvalidConfiguration;
+        i8 = pl.i8;                                   // the same for all problems: they share M
         b.prob[i] = fill_params(a[i], pl, ws.partial + off_p, ws.t + off_t, ws.counters + off_c, ws.counters + kCtrStatus, nullptr);
         b.first[i] = (i == 0) ? 0 : b.first[i];
         b.first[i + 1] = b.first[i] + pl.R * pl.SK;
@@ -1366,9 +1590,10 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
         heavy = heavy || heavy_sub_branch(a[i], pl);
     }
     const bool pdl = tune.pdl != 0;
-    cudaError_t e = dispatch_variant(a[0], [&](auto bits, auto type, auto mt, auto hv) {
-        return launch_batch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value>(b, smem, pdl, s);
-    }, heavy);
+    cudaError_t e = dispatch_variant(a[0], [&](auto bits, auto type, auto mt, auto hv, auto e4) {
+        return launch_batch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value,
+                                    decltype(e4)::value>(b, smem, pdl, s);
+    }, heavy, i8);
     if (e == cudaSuccess) ++*launches;
     return e;
 }

@@ -55,7 +55,11 @@ def main():
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--hot", action="store_true", help="reuse one instance (operands stay in L2)")
+    ap.add_argument("--opt", nargs="*", default=[], help="library options as name=value (fbq_set_option)")
     a = ap.parse_args()
+    for kv in a.opt:
+        name, value = kv.split("=")
+        fbq.set_option(name, int(value))
 
     by = algorithmic_bytes(a.M, a.N, a.K, a.bits, a.rank)
     n_inst = 1 if a.hot else max(2, int(2 * L2_BYTES / by) + 1)
