@@ -11,6 +11,7 @@
 
 namespace fbq {
 void decode_set_test_switch(int t_late);
+void decode_set_t_wait(int on);
 void prefill_set_pair(int on);
 void prefill_set_split(int mode);
 
@@ -24,6 +25,7 @@ struct Options {
     int force_kernel = -1;
     DecodeTuning decode;
     int decode_t_late = 0;
+    int decode_t_wait = 1;
     int batch_ctas = 400;
     int batch_single = 1;
     int prefill_pair = 0;
@@ -181,6 +183,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_depth")) return &g_opt.decode.depth;
     if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
     if (!strcmp(name, "decode_i8")) return &g_opt.decode.i8;
+    if (!strcmp(name, "decode_t_wait")) return &g_opt.decode_t_wait;
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;
     if (!strcmp(name, "batch_ctas")) return &g_opt.batch_ctas;
@@ -296,6 +299,7 @@ int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, flo
 static void apply_kernel_options()
 {
     decode_set_test_switch(g_opt.decode_t_late);
+    decode_set_t_wait(g_opt.decode_t_wait);
     prefill_set_pair(g_opt.prefill_pair);
     prefill_set_split(g_opt.prefill_split);
 }

@@ -33,7 +33,14 @@
 // is complete before t is waits in a local list and, at worst, is handed to
 // the warp that completes t.  The only waits are on this CTA's own copies and
 // warps, and they are bounded.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <mutex>
 #include <type_traits>
+#include <vector>
 
 #include "fbq_common.cuh"
 
@@ -49,8 +56,11 @@ constexpr int kWarps = kCW + 2;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 16;
 constexpr int kMaxSeg = 64;                  // segments (tiles touched) per CTA
-constexpr int kNBuf = 4;                     // segment partial buffers in flight
+constexpr int kNBufMax = 8;                  // segment partial buffers in flight, at most (p.nbuf of them are used)
 constexpr int kTUnitK = 1024;                // k extent of one unit of the down-projection
+constexpr int kTMmaMaxM = 4;                   // tokens up to which the down-projection of the light variant runs on tensor cores
+constexpr int kAPitch = kTUnitK + 8;         // elements between units of A in shared memory: 16 bytes past a multiple of 128, so
+                                             // that eight units read at the same k fall into different banks
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kEarlyStages = 1;                // weight stages prefetched before x has been requested
 constexpr int kTUnitsOneWarp = 10;             // (token, unit) pairs of the down-projection one warp takes by itself
@@ -73,7 +83,7 @@ struct DecodeParams {
     int *ctr;           // counters, see above; all zero on entry and on exit
     int *status;        // word that receives FBQ_ERR_TIMEOUT when a bounded wait runs out
     int M, N, K, G, rank;
-    int SK, R, NT, CHG, NS;
+    int SK, R, NT, CHG, NS, nbuf;
     int maxslots;
     int t_target;       // number of CTAs that contribute to t
     int t_late;         // test switch: contribute to t after the main loop
@@ -83,6 +93,8 @@ struct DecodeParams {
     int meta_rows;      // rows of the shared-memory scale / zero tables
     int a_cap;          // units of A held in shared memory
     int b_cap_rows;     // rows of B held in shared memory (0: read B from global memory)
+    int t_wait;         // 1: a finished tile may wait in its segment buffer for t (as long as nobody is held up)
+    int ab_alias;       // 1: B takes the place of A (and of the staged x) once the epilogue warp has used them; it issues the copy
     int off_tab, off_def, off_meta, off_x, off_px, off_segbuf, off_A, off_B, off_t, off_ring;
     unsigned long long *trace;   // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
@@ -114,6 +126,19 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
+// Completed or not, without waiting at all.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
 // Bounded wait: returns false when the limit is hit (never spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
@@ -137,6 +162,13 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// One box of a 3-D tensor map (coordinates: word in group, weight row, group) into shared memory.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+                 "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
                  : "memory");
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -472,16 +504,15 @@ __device__ __forceinline__ bool tile_claim(const DecodeParams &p, int tile, int 
 // down-projection per CTA): its units are shared by the eight compute warps and the tile finish
 // keeps twice as many chunks of B in registers.  The light variant keeps both out of its code.
 template <int BITS, typename T, int MT, bool HEAVY, bool I8>
-__device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta)
+__device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtensorMap *wmap, const int cta)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int GB = (BITS == 4) ? 64 : 48;          // packed bytes of one group of one row
     constexpr int NWORDS = Unpack<BITS, T>::kWords;    // words per lane per group
-    // Row pitch of a stage in shared memory: the packed bytes of the row, padded so that the
-    // eight rows a warp reads at once start in different banks (64-byte offset per row pair
-    // for the 128-bit loads of INT4, 48-byte for the three 32-bit loads of INT3).
-    constexpr int RP = (BITS == 4) ? 64 : 48;
-    auto row_pitch = [](int ng) { const int b = ng * GB; return (b % 128 == 0) ? b + RP : b; };
+    // A stage in shared memory is [group][row][GB bytes], dense, as the tensor copy writes it: the
+    // eight rows a warp reads at once are GB bytes apart, which spreads them over all banks (48 B:
+    // 12 words, every lane of a 32-bit load in a bank of its own; 64 B: 128-bit loads, a quarter
+    // warp covers 128 contiguous bytes).
     constexpr int NACC = FBQ_NACC;                     // independent MMA accumulator chains
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -492,7 +523,6 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     // whole 16-row tiles, dealt out in contiguous ranges; a "segment" is one tile of the range
     const int tile_first = (int)((long long)r * p.NT / p.R);
     const int nseg = (int)((long long)(r + 1) * p.NT / p.R) - tile_first;
-    const size_t row_bytes = (size_t)p.G * GB;
 
     // units of the down-projection owned by this CTA: (row j of A, 1024-wide k chunk of the slice)
     const int kslice = ngs * kGroupFast;
@@ -505,8 +535,8 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     trace_mark(p, 0);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     const uint32_t st_full = smem_u32(bars), st_empty = st_full + 8u * p.NS;
-    const uint32_t seg_full = st_empty + 8u * p.NS, seg_free = seg_full + 8u * kNBuf;
-    const uint32_t a_full = seg_free + 8u * kNBuf, b_full = a_full + 8u, x_req = b_full + 8u, t_done = x_req + 8u;
+    const uint32_t seg_full = st_empty + 8u * p.NS, seg_free = seg_full + 8u * kNBufMax;
+    const uint32_t a_full = seg_free + 8u * kNBufMax, b_full = a_full + 8u, x_req = b_full + 8u, t_done = x_req + 8u;
     int *s_def = reinterpret_cast<int *>(smem + p.off_def);
     float2 *s_mf = reinterpret_cast<float2 *>(smem + p.off_meta);         // (s, s*z) [segment row][slice group]
     float2 *s_px = reinterpret_cast<float2 *>(smem + p.off_px);           // (P, X0)  [slice group][token]
@@ -522,7 +552,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             mbar_init(st_full + 8u * i, 1);
             mbar_init(st_empty + 8u * i, kCW);
         }
-        for (int i = 0; i < kNBuf; ++i) {
+        for (int i = 0; i < kNBufMax; ++i) {
             mbar_init(seg_full + 8u * i, kCW);
             mbar_init(seg_free + 8u * i, 1);
         }
@@ -551,7 +581,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             const int kc = u / p.rank, j = u - kc * p.rank;
             const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);
             const bool in_smem = (u - tu0) < p.a_cap;
-            const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kTUnitK : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
+            const T *arow = in_smem ? s_A + (size_t)(u - tu0) * kAPitch : A + (size_t)j * p.K + g0 * kGroupFast + kbeg;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int k = lane * 8 + 256 * i;
@@ -602,6 +632,82 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         return true;
     };
 
+    // The same for the units of A that sit in shared memory, on the tensor cores: up to eight units of one
+    // k chunk are the eight columns of m16n8k16 MMAs whose rows are the tokens (the chunk of x is staged
+    // in shared memory first), four accumulators in turn.  One warp; far fewer
+    // instructions and no long dependent chain, so t is complete soon after x is.
+    auto t_units_mma = [&]() -> bool {
+        if (p.M > kTMmaMaxM) return t_units(tu0, 1);
+        if (!mbar_wait(a_full, 0)) return false;
+        const int u_end = min(tu1, tu0 + p.a_cap);
+        const T *x = static_cast<const T *>(p.x) + g0 * kGroupFast;
+        T *s_xt = s_A + (size_t)p.a_cap * kAPitch;                              // x of the current k chunk, [token][kAPitch]
+        int cur_kc = -1;
+#pragma unroll 1
+        for (int ub = tu0; ub < u_end;) {
+            const int kc = ub / p.rank, j0 = ub - kc * p.rank;
+            const int ue = min(min(ub + 8, u_end), (kc + 1) * p.rank);
+            const int kbeg = kc * kTUnitK, nk = min(kTUnitK, kslice - kbeg);      // a multiple of 128
+            if (kc != cur_kc) {
+                // the chunk of x, coalesced and all loads in flight at once (two tokens at a time)
+                cur_kc = kc;
+                __syncwarp();
+#pragma unroll 1
+                for (int m = 0; m < p.M; m += 2) {
+                    uint4 v[2][4];
+#pragma unroll
+                    for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int k = lane * 8 + 256 * i;
+                            v[mm][i] = make_uint4(0u, 0u, 0u, 0u);
+                            if (k < nk && m + mm < p.M) v[mm][i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)(m + mm) * p.K + kbeg + k));
+                        }
+#pragma unroll
+                    for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (m + mm < p.M) *reinterpret_cast<uint4 *>(s_xt + (size_t)(m + mm) * kAPitch + lane * 8 + 256 * i) = v[mm][i];
+                }
+                __syncwarp();
+            }
+            const uint32_t *arow = reinterpret_cast<const uint32_t *>(s_A + (size_t)(ub - tu0 + g) * kAPitch);
+            const uint32_t *xa = reinterpret_cast<const uint32_t *>(s_xt + (size_t)g * kAPitch);
+            const bool col_ok = g < ue - ub, ra_ok = g < p.M;
+            float d[4][4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) d[c][0] = d[c][1] = d[c][2] = d[c][3] = 0.f;
+#pragma unroll 2
+            for (int s16 = 0; s16 < nk / 16; s16 += 4) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int w = (s16 + c) * 8 + tq;                          // word index of k = 16 s + 2 tq
+                    uint32_t a[4] = {0u, 0u, 0u, 0u}, b0 = 0u, b1 = 0u;
+                    if (ra_ok) {
+                        a[0] = xa[w];
+                        a[2] = xa[w + 4];
+                    }
+                    if (col_ok) {
+                        b0 = arow[w];
+                        b1 = arow[w + 4];
+                    }
+                    Pk<T>::mma(d[c], a, b0, b1);
+                }
+            }
+            // d[.][0], d[.][1]: (token g, units 2 tq, 2 tq + 1) of the block (tokens 8.. do not occur here)
+            const float v0 = (d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), v1 = (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]);
+            const int c0 = 2 * tq, nb = ue - ub;
+            if (ra_ok) {
+                if (c0 < nb) atomicAdd(p.t + (size_t)g * p.rank + j0 + c0, v0);
+                if (c0 + 1 < nb) atomicAdd(p.t + (size_t)g * p.rank + j0 + c0 + 1, v1);
+            }
+            ub = ue;
+        }
+        // units beyond the ones held in shared memory: the plain way
+        if (u_end < tu1) return t_units(u_end, 1);
+        return true;
+    };
+
     // Who works the units off: the epilogue warp alone while there are few (token, unit) pairs (it has
     // nothing else to do until the first tile is through: light variant), all eight compute warps before
     // they turn to the weights when there are many (heavy variant: one warp would hold up the tiles).
@@ -623,11 +729,11 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             for (int i = lane; i < na; i += 32) {
                 const int u = tu0 + i, kc = u / p.rank, j = u - kc * p.rank;
                 const int nk = min(kTUnitK, kslice - kc * kTUnitK);
-                bulk_g2s(smem_u32(s_A + (size_t)i * kTUnitK), A + (size_t)j * p.K + g0 * kGroupFast + kc * kTUnitK,
+                bulk_g2s(smem_u32(s_A + (size_t)i * kAPitch), A + (size_t)j * p.K + g0 * kGroupFast + kc * kTUnitK,
                          (uint32_t)nk * 2u, a_full);
             }
         }
-        if (b_in_smem && lane == 0) {
+        if (b_in_smem && !p.ab_alias && lane == 0) {
             const uint32_t bytes = (uint32_t)b_rows * p.rank * 2u;
             mbar_expect_tx(b_full, bytes);
             bulk_g2s(smem_u32(s_B), static_cast<const T *>(p.B) + (size_t)tile_first * kTileRows * p.rank, bytes, b_full);
@@ -656,14 +762,13 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                     dead = true;
                     break;
                 }
-                const uint32_t bytes_row = (uint32_t)ng * GB;
-                if (lane == 0) mbar_expect_tx(st_full + 8u * slot, bytes_row * kTileRows);
-                __syncwarp();
-                if (lane < kTileRows) {
-                    const int n = min(tile * kTileRows + lane, p.N - 1);
-                    bulk_g2s(ring + slot * p.stage_bytes + lane * row_pitch(ng),
-                             p.qw + (size_t)n * row_bytes + (size_t)(g0 + pos) * GB, bytes_row, st_full + 8u * slot);
+                // one box of CHG groups x 16 rows (rows past N and groups past G arrive as zeros; the
+                // groups of a short last stage beyond ng are not used)
+                if (lane == 0) {
+                    mbar_expect_tx(st_full + 8u * slot, (uint32_t)p.stage_bytes);
+                    tma_load_3d(ring + slot * p.stage_bytes, wmap, 0, tile * kTileRows, g0 + pos, st_full + 8u * slot);
                 }
+                __syncwarp();
             }
         }
         if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
@@ -705,7 +810,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             // [2^20, 2^21); per slot X = rint(x 2^e 2^-j) and its three signed base-256 digits.
             constexpr int NR = SlotsI8<BITS>::kRegs;
             const T *x = static_cast<const T *>(p.x);
-            const int ncol = 4 * p.M;
+            const int ncol = 3 * p.M;                                                 // three digit columns per token
             float2 *s_ux = reinterpret_cast<float2 *>(smem + p.off_px);               // (2^-e, X0) [slice group][token slot]
             uint4 *s_x8 = reinterpret_cast<uint4 *>(smem + p.off_x);                  // [slice group][chunk][column][lane tq]
             uint32_t *s_xt = reinterpret_cast<uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16;   // register 8
@@ -768,7 +873,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                         const int gl = run >> 2, lq = run & 3;
 #pragma unroll
                         for (int k = 0; k < 3; ++k) {
-                            const int col = 4 * m + k;
+                            const int col = 3 * m + k;
                             s_x8[(size_t)((gl * 2 + R0 / 4) * ncol + col) * 4 + lq] = make_uint4(dg[0][k], dg[1][k], dg[2][k], dg[3][k]);
                             if constexpr (R1 - R0 == 5) s_xt[(size_t)(gl * ncol + col) * 4 + lq] = dg[4][k];
                         }
@@ -866,7 +971,6 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                 if (p.trace) t_wait += clock64() - c_wait;
                 if (it == 0) trace_mark(p, 6);
                 const uint8_t *slot_ptr = ring_ptr + (size_t)slot * p.stage_bytes;
-                const uint32_t bytes_row = (uint32_t)row_pitch(ng);
                 const int gbeg = warp * ng / kCW, gend = (warp + 1) * ng / kCW;     // this warp's groups of the stage
                 const float2 *meta_a = s_mf + (size_t)(seg * kTileRows + g) * mpitch + pos;   // row g; row g+8 is 8 rows on
                 const float2 *meta_b = meta_a + 8 * mpitch;
@@ -874,8 +978,8 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                 for (int gi = gbeg; gi < gend; ++gi) {
                     const float2 fa = meta_a[gi], fb = meta_b[gi];          // (s, s*z) of rows g and g+8
                     uint32_t wa[NWORDS], wb[NWORDS];
-                    const uint8_t *pa = slot_ptr + (size_t)g * bytes_row + gi * GB + tq * (GB / 4);
-                    const uint8_t *pb = pa + (size_t)8 * bytes_row;
+                    const uint8_t *pa = slot_ptr + gi * (kTileRows * GB) + g * GB + tq * (GB / 4);
+                    const uint8_t *pb = pa + 8 * GB;
                     if constexpr (BITS == 4) {
                         const uint4 va = *reinterpret_cast<const uint4 *>(pa), vb = *reinterpret_cast<const uint4 *>(pb);
                         wa[0] = va.x; wa[1] = va.y; wa[2] = va.z; wa[3] = va.w;
@@ -894,15 +998,15 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
                         SlotsI8<BITS>::run(wb, rb);
                         // this lane's column (token g / 4, digit g % 4) of the group, and (2^-e, X0) of the
                         // token whose columns its accumulators hold
-                        const int ncol = 4 * p.M;
-                        const uint4 *xg = reinterpret_cast<const uint4 *>(smem + p.off_x) + (size_t)((pos + gi) * 2 * ncol + g) * 4 + tq;
+                        const int ncol = 3 * p.M, cc = g - (g >> 2);                 // stored columns; MMA column g = 4 m + digit
+                        const uint4 *xg = reinterpret_cast<const uint4 *>(smem + p.off_x) + (size_t)((pos + gi) * 2 * ncol + cc) * 4 + tq;
                         uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
                         uint32_t xt = 0u;
-                        if (g < ncol && (g & 3) != 3) {
+                        if (g < 4 * p.M && (g & 3) != 3) {
                             x0 = xg[0];
                             x1 = xg[ncol * 4];
                             if (BITS == 3)
-                                xt = (reinterpret_cast<const uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16)[((pos + gi) * ncol + g) * 4 + tq];
+                                xt = (reinterpret_cast<const uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16)[((pos + gi) * ncol + cc) * 4 + tq];
                         }
                         const float2 ux = reinterpret_cast<const float2 *>(smem + p.off_px)[(pos + gi) * 2 + (tq >> 1)];
                         int d[4] = {0, 0, 0, 0};
@@ -981,8 +1085,8 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             }
 
             // ---- deposit this warp's partial tile for the epilogue warp ---------------
-            const int buf = seg % kNBuf;
-            if (seg >= kNBuf && !mbar_wait(seg_free + 8u * buf, (uint32_t)(seg / kNBuf - 1) & 1u)) {
+            const int buf = seg % p.nbuf;
+            if (seg >= p.nbuf && !mbar_wait(seg_free + 8u * buf, (uint32_t)(seg / p.nbuf - 1) & 1u)) {
                 dead = true;
                 break;
             }
@@ -1073,6 +1177,91 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         }
         ++n_retired;
     };
+    // Up-projection of all rows of this CTA at once (light variant, one K slice, B of the own tiles in
+    // shared memory, M <= 4, rank a multiple of 16): once t is complete it becomes eight 16-bit columns
+    // (tokens 0..3 rounded, then the remainders of that rounding), and per tile rank / 16 MMAs
+    // (rows of B x columns of t) give t.B^T for its 16 rows.  A tile is then finished by adding
+    // two numbers per output.  Tiles that are done before t is wait in their segment buffers for
+    // as long as that holds nobody up.
+    T *s_th = reinterpret_cast<T *>(s_stage + kTileRows * kDecodeMaxM);       // [8 columns][rank]
+    float *s_sub = reinterpret_cast<float *>(s_th + 8 * p.rank);             // [segment][row][4 tokens]
+    const bool sub_at_once = !HEAVY && fast_fin && b_in_smem && p.M <= 4 && (p.rank % 16) == 0 && !p.t_late;
+    bool sub_done = false;
+    auto make_sub = [&]() {
+        // fp16 columns: a power of two keeps a large t inside the format (exact, undone below)
+        float sc = 1.f, isc = 1.f;
+        if (std::is_same<T, __half>::value) {
+            float tmax = 0.f;
+            for (int i = lane; i < p.M * p.rank; i += 32) tmax = fmaxf(tmax, fabsf(s_t[i]));
+            for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+            if (tmax >= 16384.f) {
+                int e = 0;
+                (void)frexpf(tmax, &e);
+                sc = ldexpf(1.f, 14 - e);
+                isc = ldexpf(1.f, e - 14);
+            }
+        }
+        for (int j = lane; j < p.rank; j += 32)
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                float hi = 0.f, lo = 0.f;
+                if (m < p.M) {
+                    const float tv = s_t[m * p.rank + j] * sc;
+                    hi = tv;
+                    lo = tv - ActTraits<T>::to_float(ActTraits<T>::from_float(tv));
+                }
+                s_th[m * p.rank + j] = ActTraits<T>::from_float(hi);
+                s_th[(4 + m) * p.rank + j] = ActTraits<T>::from_float(lo);
+            }
+        __syncwarp();
+        const uint32_t *tcol = reinterpret_cast<const uint32_t *>(s_th + (size_t)g * p.rank);
+#pragma unroll 1
+        for (int i = 0; i < nseg; ++i) {
+            const uint32_t *ba = reinterpret_cast<const uint32_t *>(s_B + (size_t)(i * kTileRows + g) * p.rank);
+            const uint32_t *bb = ba + 4 * p.rank;                                // row g + 8
+            float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+            for (int k16 = 0; k16 < p.rank / 16; ++k16) {
+                const int w = k16 * 8 + tq;
+                const uint32_t a[4] = {ba[w], bb[w], ba[w + 4], bb[w + 4]};
+                Pk<T>::mma(d, a, tcol[w], tcol[w + 4]);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) d[q] = (d[q] + __shfl_xor_sync(0xffffffffu, d[q], 2)) * isc;   // rounded part + remainder
+            if (tq < 2) {
+                float *o = s_sub + (size_t)(i * kTileRows + g) * 4 + 2 * tq;
+                o[0] = d[0];
+                o[1] = d[1];
+                o[8 * 4] = d[2];
+                o[8 * 4 + 1] = d[3];
+            }
+        }
+        __syncwarp();
+        sub_done = true;
+    };
+    auto finish_sub = [&](int tile, int seg) {
+        for (int idx = lane; idx < kTileRows * p.M; idx += 32) {
+            const int row = idx & (kTileRows - 1), m = idx >> 4, n = tile * kTileRows + row;
+            if (n < p.N)
+                static_cast<T *>(p.y)[(size_t)m * p.N + n] =
+                    ActTraits<T>::from_float(s_stage[m * kTileRows + row] + s_sub[(size_t)(seg * kTileRows + row) * 4 + m]);
+        }
+        ++n_retired;
+    };
+    // Waits for t while that costs nothing: until it is complete, or the compute warps are about to
+    // run out of segment buffers, or they are through with all segments (then the tile is parked as
+    // before: a CTA never holds its SM just to wait for other CTAs).
+    auto wait_t_with_slack = [&](int seg) {
+        const int last = min(seg + p.nbuf, nseg - 1);
+        if (last <= seg) return;
+        const uint32_t bar = seg_full + 8u * (uint32_t)(last % p.nbuf), par = (uint32_t)(last / p.nbuf) & 1u;
+#pragma unroll 1
+        for (uint32_t i = 0; i < kWaitLimit; ++i) {
+            if (t_poll()) return;
+            if (mbar_test(bar, par)) return;
+            __nanosleep(200);
+        }
+    };
     // Finish `tile` from scratch slots (all contributions are there and visible).
     auto finish_from_slots = [&](int tile) {
         finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
@@ -1124,18 +1313,29 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
     if (has_t && !p.t_late) {
         if (t_by_compute) {
             if (!mbar_wait(t_done, 0)) dead = true;     // the compute warps' units are in
-        } else if (!t_units(tu0, 1)) {
+        } else if (!t_units_mma()) {
             dead = true;
         }
         trace_mark(p, 3);
-        t_arrive();
     }
+    if (!HEAVY && p.ab_alias && b_in_smem) {
+        // A and the staged x are used up: their place goes to B of the own tiles (needed once t is complete)
+        __syncwarp();
+        if (lane == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const uint32_t bytes = (uint32_t)b_rows * p.rank * 2u;
+            mbar_expect_tx(b_full, bytes);
+            bulk_g2s(smem_u32(s_B), static_cast<const T *>(p.B) + (size_t)tile_first * kTileRows * p.rank, bytes, b_full);
+        }
+    }
+    if (has_t && !p.t_late) t_arrive();
     trace_mark(p, 4);
     if (b_in_smem && !mbar_wait(b_full, 0)) dead = true;
 
+    long long e_wait = 0, e_sum = 0, e_fin = 0;      // trace: cycles waiting for segments, adding partials, finishing (fast path)
 #pragma unroll 1
     for (int seg = 0; seg < nseg && !dead; ++seg) {
-        const int buf = seg % kNBuf;
+        const int buf = seg % p.nbuf;
         const int tile = tile_first + seg;
         const int cnt = p.SK, myslot = s;       // one contribution per K slice
         // While the compute warps still work on the segment, look whether every other
@@ -1145,11 +1345,14 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
             if (lane == 0) others_in = ((ld_acquire(p.ctr + kCtrFirstTile + tile) & 0xFFFF) == cnt - 1);
             others_in = __shfl_sync(0xffffffffu, others_in, 0);
         }
-        if (fast_fin) b_prefetch(tile);
-        if (!mbar_wait_idle(seg_full + 8u * buf, (uint32_t)(seg / kNBuf) & 1u)) {
+        if (fast_fin && !sub_at_once) b_prefetch(tile);
+        const long long c_w0 = p.trace ? clock64() : 0;
+        if (!mbar_wait_idle(seg_full + 8u * buf, (uint32_t)(seg / p.nbuf) & 1u)) {
             dead = true;
             break;
         }
+        const long long c_w1 = p.trace ? clock64() : 0;
+        e_wait += c_w1 - c_w0;
         trace_mark(p, seg == 0 ? 5 : 7);
         // add the eight warps' partial tiles in warp order and stage the result as [token][row]
         if (tq < p.vt) {
@@ -1174,13 +1377,24 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(seg_free + 8u * buf);
+        const long long c_w2 = p.trace ? clock64() : 0;
+        e_sum += c_w2 - c_w1;
 
         if (cnt == 1 || others_in) {
             // This warp finishes the tile: straight from the staged sums if t is complete ...
+            if (sub_at_once && p.t_wait && !t_local) wait_t_with_slack(seg);
             if (t_poll()) {
+                if (sub_at_once) {
+                    if (!sub_done) make_sub();
+                    finish_sub(tile, seg);
+                    __syncwarp();
+                    if (p.trace) e_fin += clock64() - c_w2;
+                    continue;
+                }
                 if (fast_fin) {
                     finish_fast(tile);
                     __syncwarp();
+                    if (p.trace) e_fin += clock64() - c_w2;
                     continue;
                 }
                 finish_tile<T>(static_cast<T *>(p.y), p.partial + (size_t)tile * p.maxslots * p.M * kTileRows,
@@ -1273,12 +1487,20 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const int cta
         }
     }
     trace_mark(p, 9);
+    if (p.trace && lane == 0) {
+        unsigned long long *row = p.trace + ((size_t)blockIdx.x * kWarps + warp) * 16;
+        row[10] = (unsigned long long)e_wait;
+        row[11] = (unsigned long long)e_sum;
+        row[12] = (unsigned long long)e_fin;
+        row[13] = (unsigned long long)n_def;
+    }
 }
 
 template <int BITS, typename T, int MT, bool HEAVY, bool I8>
-__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams p)
+__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeParams p,
+                                                             const __grid_constant__ CUtensorMap wmap)
 {
-    decode_body<BITS, T, MT, HEAVY, I8>(p, (int)blockIdx.x);
+    decode_body<BITS, T, MT, HEAVY, I8>(p, &wmap, (int)blockIdx.x);
 }
 
 // Several independent problems in one grid: CTAs first[i] .. first[i+1]-1 run problem i exactly as
@@ -1286,6 +1508,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const DecodeParams 
 // problems are resident together and nothing synchronises across problems.
 constexpr int kBatchMax = 8;
 struct DecodeBatch {
+    CUtensorMap wmap[kBatchMax];
     DecodeParams prob[kBatchMax];
     int first[kBatchMax + 1];
     int count;
@@ -1295,21 +1518,24 @@ __global__ void __launch_bounds__(kThreads, 2) decode_batch_kernel(const __grid_
 {
     int pi = 0;
     while (pi + 1 < b.count && (int)blockIdx.x >= b.first[pi + 1]) ++pi;
-    decode_body<BITS, T, MT, HEAVY, I8>(b.prob[pi], (int)blockIdx.x - b.first[pi]);
+    decode_body<BITS, T, MT, HEAVY, I8>(b.prob[pi], &b.wmap[pi], (int)blockIdx.x - b.first[pi]);
 }
 
 // ------------------------------------------------------------------ host side
 struct Plan {
-    int SK, R, NT, CHG, NS, t_target, maxslots, vt, a_cap, b_cap_rows, meta_rows;
+    int SK, R, NT, CHG, NS, nbuf, t_target, maxslots, vt, a_cap, b_cap_rows, meta_rows;
     int x_pitch, stage_bytes;
     int off_tab, off_def, off_meta, off_x, off_px, off_segbuf, off_A, off_B, off_t, off_ring;
     size_t smem;
     bool ok;
     bool i8;            // codes and x go to the tensor cores as 8-bit integers (M <= 2)
+    bool heavy;         // the compute warps take the units of the down-projection
+    int ab_alias;
 };
 
 int g_sm_count = 0;
-constexpr size_t kSmemBudget = 110 * 1024;   // two CTAs (this launch and the next one) fit on an SM
+int g_t_late = 0, g_t_wait = 1;
+constexpr size_t kSmemBudget = 112 * 1024;   // two CTAs (this launch and the next one) fit on an SM (228 KB, 1 KB reserved per CTA)
 constexpr size_t kSmemMax = 227 * 1024;      // everything an SM has
 
 Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
@@ -1332,19 +1558,24 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     // K slices: one, unless the x slice and the other tables do not fit next to the ring.
     // First try to stay within half an SM's shared memory (so that this launch and the next
     // one can be resident together) with few slices; otherwise take the whole SM.
-    auto layout = [&](int sk, size_t budget) {
+    auto layout = [&](int sk, size_t budget, bool many_buffers) {
         pl.SK = sk;
         const int ngs_max = (G + sk - 1) / sk;
         pl.R = max(1, min(max_ctas / sk, pl.NT));
         const int nseg_max = (pl.NT + pl.R - 1) / pl.R;
         pl.maxslots = sk;
         pl.CHG = max(1, min(tune.chunk > 0 ? tune.chunk : 16, ngs_max));
-        pl.stage_bytes = kTileRows * (pl.CHG * GB + 64);      // rows are padded by up to 64 bytes
+        pl.stage_bytes = kTileRows * pl.CHG * GB;             // [group][row][GB], dense
         pl.x_pitch = ngs_max * kGroupFast + 32;    // +64 bytes: tokens 2j, 2j+1 land in different bank halves
         const int nkc = (ngs_max * kGroupFast + kTUnitK - 1) / kTUnitK;
         const long long tu_max = ((long long)a.rank * nkc + pl.R - 1) / pl.R;
         pl.a_cap = (int)min(tu_max, 8LL);
-        size_t off = (size_t)(2 * 8 + 2 * kNBuf + 4) * 8;      // room for up to 8 stages' barriers
+        // Heavy sub-branch: rank above what the light tile finish holds, or more units of the down-projection
+        // per CTA than its epilogue warp should take by itself (tensor-core form: what fits its staging
+        // area; plain form: (token, unit) pairs).
+        pl.heavy = a.rank > 64 || (a.rank > 0 && (a.M <= kTMmaMaxM ? tu_max > 8 : tu_max * a.M > kTUnitsOneWarp));
+        pl.ab_alias = (a.rank > 0 && !pl.heavy && !g_t_late) ? 1 : 0;
+        size_t off = (size_t)(2 * 8 + 2 * kNBufMax + 4) * 8;      // room for up to 8 stages' barriers
         off = (off + 15) & ~(size_t)15;
         pl.off_tab = (int)off;
         pl.off_def = (int)off;
@@ -1355,28 +1586,34 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         off += (size_t)pl.meta_rows * (ngs_max | 1) * 8;
         off = (off + 127) & ~(size_t)127;
         pl.off_x = (int)off;
-        // x of the slice: 16-bit values per token, or (integer form) four one-byte columns per value, 36 slots per 32 values
-        off += pl.i8 ? (size_t)ngs_max * (4 * a.M) * 144 : (size_t)a.M * pl.x_pitch * 2;
+        // x of the slice: 16-bit values per token, or (integer form) three one-byte columns per value, 36 slots per 32 values
+        off += pl.i8 ? (size_t)ngs_max * (3 * a.M) * 144 : (size_t)a.M * pl.x_pitch * 2;
         off = (off + 127) & ~(size_t)127;
         pl.off_px = (int)off;
         off += (size_t)ngs_max * 8 * mt * 8;
         off = (off + 127) & ~(size_t)127;
         pl.off_segbuf = (int)off;
-        off += (size_t)kNBuf * kCW * 8 * pl.vt * 4 * mt * 4;
+        pl.nbuf = (many_buffers && (size_t)kCW * 8 * pl.vt * 4 * mt * 4 <= 1024) ? kNBufMax : 4;   // small tiles (M <= 2): more of them may wait for t
+        off += (size_t)pl.nbuf * kCW * 8 * pl.vt * 4 * mt * 4;
         off = (off + 127) & ~(size_t)127;
         pl.off_A = (int)off;
-        off += (size_t)pl.a_cap * kTUnitK * 2;
+        const size_t b_bytes = (size_t)nseg_max * kTileRows * a.rank * 2;
+        const size_t a_bytes = (size_t)(pl.a_cap + (a.rank > 0 && a.M <= kTMmaMaxM ? a.M : 0)) * kAPitch * 2;   // units of A, then x of one k chunk
+        off += pl.ab_alias ? max(a_bytes, b_bytes) : a_bytes;
         off = (off + 127) & ~(size_t)127;
         pl.off_t = (int)off;
         off += (size_t)a.M * a.rank * 4 + (size_t)kTileRows * kDecodeMaxM * 4;   // t, then the epilogue warp's staging tile
+        off += (size_t)8 * a.rank * 2 + (size_t)nseg_max * kTileRows * 4 * 4;      // t as 16-bit columns, up-projection of all own rows
         off = (off + 127) & ~(size_t)127;
-        // what is left goes to the ring first (at least 2 stages), then to B
+        // what is left: two stages of the ring, then B of the own tiles, then more stages
         pl.off_B = (int)off;
-        const size_t b_bytes = (size_t)nseg_max * kTileRows * a.rank * 2;
         int ns_want = tune.depth > 0 ? tune.depth : 4;
         ns_want = max(2, min(ns_want, 8));
         pl.b_cap_rows = 0;
-        if (off + b_bytes + (size_t)ns_want * pl.stage_bytes <= budget) {
+        if (pl.ab_alias) {
+            pl.off_B = pl.off_A;
+            pl.b_cap_rows = nseg_max * kTileRows;
+        } else if (off + b_bytes + (size_t)2 * pl.stage_bytes <= budget) {      // B of the own tiles before a third and fourth stage
             pl.b_cap_rows = nseg_max * kTileRows;
             off += b_bytes;
             off = (off + 127) & ~(size_t)127;
@@ -1388,12 +1625,25 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         pl.smem = off;
         return nseg_max <= kMaxSeg && pl.smem <= budget;
     };
+    // the integer form first; where its larger x does not fit, the 16-bit form before more K slices
+    const bool want_i8 = pl.i8;
+    auto either = [&](int sk, size_t budget) {
+        for (int form = 0; form < (want_i8 ? 2 : 1); ++form) {
+            pl.i8 = want_i8 && form == 0;
+            if (layout(sk, budget, true) || layout(sk, budget, false)) return true;
+        }
+        return false;
+    };
     if (tune.sk > 0) {
-        pl.ok = layout(min(tune.sk, G), kSmemMax);
+        pl.ok = either(min(tune.sk, G), kSmemMax);
     } else {
-        for (int sk = 1; sk <= min(G, 4) && !pl.ok; ++sk) pl.ok = layout(sk, kSmemBudget);
-        for (int sk = 1; sk <= G && !pl.ok; ++sk) pl.ok = layout(sk, kSmemMax);
+        for (int sk = 1; sk <= min(G, 4) && !pl.ok; ++sk) pl.ok = either(sk, kSmemBudget);
+        for (int sk = 1; sk <= G && !pl.ok; ++sk) pl.ok = either(sk, kSmemMax);
     }
+    if (getenv("FBQ_PLAN"))
+        fprintf(stderr, "plan M %d N %d K %d r %d: ok %d SK %d R %d CHG %d NS %d nbuf %d a_cap %d b_rows %d smem %zu (meta %d x %d ring@%d) i8 %d heavy %d alias %d\n", a.M, a.N, a.K,
+                a.rank, (int)pl.ok, pl.SK, pl.R, pl.CHG, pl.NS, pl.nbuf, pl.a_cap, pl.b_cap_rows, pl.smem, pl.off_x - pl.off_meta,
+                pl.off_px - pl.off_x, pl.off_ring, (int)pl.i8, (int)pl.heavy, pl.ab_alias);
     // CTAs that own at least one unit of the down-projection
     pl.t_target = 0;
     if (a.rank > 0) {
@@ -1406,8 +1656,55 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     return pl;
 }
 
+// 3-D tensor map of the packed codes for the weight stream: (word in group, weight row, group), boxes of
+// one group's words x 16 rows x CHG groups, which land in shared memory as [group][row][GB bytes].
+// Encoding takes a microsecond or two on the host, so the last maps are kept (they depend on the
+// weights' address and the plan only).
+struct MapKey {
+    const void *qw;
+    int N, G, bits, chg;
+    bool operator==(const MapKey &o) const { return qw == o.qw && N == o.N && G == o.G && bits == o.bits && chg == o.chg; }
+};
+cudaError_t weight_map(CUtensorMap *map, const LinearArgs &a, const Plan &pl)
+{
+    static std::mutex mu;
+    static std::vector<std::pair<MapKey, CUtensorMap>> cache;
+    static size_t next = 0;
+    static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    const MapKey key{a.qw, a.N, a.K / kGroupFast, a.bits, pl.CHG};
+    std::lock_guard<std::mutex> lk(mu);
+    for (const auto &e : cache)
+        if (e.first == key) {
+            *map = e.second;
+            return cudaSuccess;
+        }
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    const cuuint32_t wpg = (a.bits == 4) ? 16 : 12;
+    const cuuint64_t dims[3] = {wpg, (cuuint64_t)a.N, (cuuint64_t)key.G};
+    const cuuint64_t strides[2] = {(cuuint64_t)key.G * wpg * 4, (cuuint64_t)wpg * 4};
+    const cuuint32_t box[3] = {wpg, (cuuint32_t)kTileRows, (cuuint32_t)pl.CHG};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t *>(a.qw), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    constexpr size_t kKeep = 256;
+    if (cache.size() < kKeep)
+        cache.emplace_back(key, *map);
+    else
+        cache[next++ % kKeep] = std::make_pair(key, *map);
+    return cudaSuccess;
+}
+
 template <int BITS, typename T, int MT, bool HEAVY, bool I8>
-cudaError_t launch_variant(const DecodeParams &p, const Plan &pl, bool pdl, cudaStream_t s)
+cudaError_t launch_variant(const DecodeParams &p, const CUtensorMap &wmap, const Plan &pl, bool pdl, cudaStream_t s)
 {
     auto kern = decode_kernel<BITS, T, MT, HEAVY, I8>;
     static bool attr_set = false;
@@ -1426,14 +1723,13 @@ cudaError_t launch_variant(const DecodeParams &p, const Plan &pl, bool pdl, cuda
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, p);
+    return cudaLaunchKernelEx(&cfg, kern, p, wmap);
 }
-
-int g_t_late = 0;
 
 }  // namespace
 
 void decode_set_test_switch(int t_late) { g_t_late = t_late; }
+void decode_set_t_wait(int on) { g_t_wait = on; }
 
 void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t *partial_floats, int *counters)
 {
@@ -1462,17 +1758,6 @@ cudaError_t dispatch_variant(const LinearArgs &a, F f, bool heavy, bool i8)
     return (a.bits == 4) ? with_type(std::integral_constant<int, 4>{}) : with_type(std::integral_constant<int, 3>{});
 }
 
-// Heavy sub-branch: rank above what the light tile finish holds, or more (token, unit) pairs of the
-// down-projection per CTA than one warp should take by itself.
-bool heavy_sub_branch(const LinearArgs &a, const Plan &pl)
-{
-    if (a.rank == 0) return false;
-    if (a.rank > 64) return true;
-    const int G = a.K / kGroupFast, ngs = (G + pl.SK - 1) / pl.SK;
-    const long long tu = (long long)a.rank * ((ngs * kGroupFast + kTUnitK - 1) / kTUnitK);
-    return (tu + pl.R - 1) / pl.R * a.M > kTUnitsOneWarp;
-}
-
 DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, float *t, int *ctr, int *status, void *trace)
 {
     DecodeParams p{};
@@ -1488,13 +1773,13 @@ DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, fl
     p.ctr = ctr;
     p.status = status;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.K / kGroupFast; p.rank = a.rank;
-    p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CHG = pl.CHG; p.NS = pl.NS;
+    p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CHG = pl.CHG; p.NS = pl.NS; p.nbuf = pl.nbuf;
     p.maxslots = pl.maxslots;
     p.t_target = pl.t_target;
     p.t_late = g_t_late;
     p.vt = pl.vt;
     p.x_pitch = pl.x_pitch; p.stage_bytes = pl.stage_bytes;
-    p.a_cap = pl.a_cap; p.b_cap_rows = pl.b_cap_rows;
+    p.a_cap = pl.a_cap; p.b_cap_rows = pl.b_cap_rows; p.ab_alias = pl.ab_alias; p.t_wait = g_t_wait;
     p.meta_rows = pl.meta_rows;
     p.off_tab = pl.off_tab; p.off_def = pl.off_def; p.off_meta = pl.off_meta; p.off_x = pl.off_x; p.off_px = pl.off_px;
     p.off_segbuf = pl.off_segbuf; p.off_A = pl.off_A; p.off_B = pl.off_B; p.off_t = pl.off_t; p.off_ring = pl.off_ring;
@@ -1531,11 +1816,13 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
     const Plan pl = make_plan(a, tune);
     if (!pl.ok) return cudaErrorInvalidConfiguration;
     const DecodeParams p = fill_params(a, pl, ws.partial, ws.t, ws.counters, ws.counters + kCtrStatus, ws.trace);
+    CUtensorMap wmap;
+    if (cudaError_t me = weight_map(&wmap, a, pl); me != cudaSuccess) return me;
     const bool pdl = tune.pdl != 0;
-    const bool heavy = heavy_sub_branch(a, pl);
+    const bool heavy = pl.heavy;
     cudaError_t e = dispatch_variant(a, [&](auto bits, auto type, auto mt, auto hv, auto e4) {
         return launch_variant<decltype(bits)::value, typename decltype(type)::type, decltype(mt)::value, decltype(hv)::value,
-                              decltype(e4)::value>(p, pl, pdl, s);
+                              decltype(e4)::value>(p, wmap, pl, pdl, s);
     }, heavy, pl.i8);
     if (e == cudaSuccess) ++*launches;
     return e;
@@ -1580,6 +1867,7 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
         const Plan pl = make_plan(a[i], tn);
         if (!pl.ok) return cudaErrorInvalidConfiguration;
         i8 = pl.i8;                                   // the same for all problems: they share M
+        if (cudaError_t me = weight_map(&b.wmap[i], a[i], pl); me != cudaSuccess) return me;
         b.prob[i] = fill_params(a[i], pl, ws.partial + off_p, ws.t + off_t, ws.counters + off_c, ws.counters + kCtrStatus, nullptr);
         b.first[i] = (i == 0) ? 0 : b.first[i];
         b.first[i + 1] = b.first[i] + pl.R * pl.SK;
@@ -1587,7 +1875,7 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
         off_t += (size_t)kDecodeMaxM * kMaxRank;
         off_c += kCtrFirstTile + 2 * pl.NT;
         smem = pl.smem > smem ? pl.smem : smem;
-        heavy = heavy || heavy_sub_branch(a[i], pl);
+        heavy = heavy || pl.heavy;
     }
     const bool pdl = tune.pdl != 0;
     cudaError_t e = dispatch_variant(a[0], [&](auto bits, auto type, auto mt, auto hv, auto e4) {
