@@ -1558,13 +1558,13 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     // K slices: one, unless the x slice and the other tables do not fit next to the ring.
     // First try to stay within half an SM's shared memory (so that this launch and the next
     // one can be resident together) with few slices; otherwise take the whole SM.
-    auto layout = [&](int sk, size_t budget, bool many_buffers) {
+    auto layout = [&](int sk, size_t budget, bool many_buffers, int chg_cap) {
         pl.SK = sk;
         const int ngs_max = (G + sk - 1) / sk;
         pl.R = max(1, min(max_ctas / sk, pl.NT));
         const int nseg_max = (pl.NT + pl.R - 1) / pl.R;
         pl.maxslots = sk;
-        pl.CHG = max(1, min(tune.chunk > 0 ? tune.chunk : 16, ngs_max));
+        pl.CHG = max(1, min(min(tune.chunk > 0 ? tune.chunk : 16, chg_cap), ngs_max));
         pl.stage_bytes = kTileRows * pl.CHG * GB;             // [group][row][GB], dense
         pl.x_pitch = ngs_max * kGroupFast + 32;    // +64 bytes: tokens 2j, 2j+1 land in different bank halves
         const int nkc = (ngs_max * kGroupFast + kTUnitK - 1) / kTUnitK;
@@ -1630,7 +1630,9 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     auto either = [&](int sk, size_t budget) {
         for (int form = 0; form < (want_i8 ? 2 : 1); ++form) {
             pl.i8 = want_i8 && form == 0;
-            if (layout(sk, budget, true) || layout(sk, budget, false)) return true;
+            // stages of 16 groups, else of 8 (more hand-overs per byte, but still one K slice)
+            for (int chg = 16; chg >= 8; chg -= 8)
+                if (layout(sk, budget, true, chg) || layout(sk, budget, false, chg)) return true;
         }
         return false;
     };
