@@ -139,6 +139,25 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
+// Loads through 32-bit shared-window addresses (no 64-bit address arithmetic in the inner loops).
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f2(uint32_t a)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+    return v;
+}
 // Bounded wait: returns false when the limit is hit (never spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
@@ -957,6 +976,82 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
             for (int b = 0; b < MT; ++b)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[b][i] = 0.f;
+            if constexpr (I8) {
+                // Integer form, written lean: everything that does not change per unit sits in registers as
+                // 32-bit shared-memory addresses and strides, and nothing in the unit loop is conditional.
+                // Lanes whose MMA column carries no digit (column 3 of a token, tokens >= M) read a column
+                // that exists instead: their sums land in output columns nobody looks at.
+                constexpr int NR = SlotsI8<BITS>::kRegs;
+                const int ncol = 3 * p.M, CHG = p.CHG, NS = p.NS;
+                const int cc = (g < 4 * p.M && (g & 3) != 3) ? g - (g >> 2) : 0;
+                const uint32_t sbase = smem_u32(smem);
+                const uint32_t x_gstride = (uint32_t)ncol * 128u, x_chunk1 = (uint32_t)ncol * 64u;
+                const uint32_t x_lane = sbase + p.off_x + (uint32_t)(cc * 4 + tq) * 16u;
+                const uint32_t xt_lane = sbase + p.off_x + (uint32_t)ngs * x_gstride + (uint32_t)(cc * 4 + tq) * 4u;
+                const uint32_t xt_gstride = (uint32_t)ncol * 16u;
+                const uint32_t ux_lane = sbase + p.off_px + (uint32_t)(tq >> 1) * 8u;
+                const uint32_t w_lane = sbase + p.off_ring + (uint32_t)(g * GB + tq * (GB / 4));
+                const uint32_t m_lane = sbase + p.off_meta + (uint32_t)((seg * kTileRows + g) * mpitch) * 8u;
+                const uint32_t stage_bytes = (uint32_t)p.stage_bytes;
+                for (int pos = 0; pos < ngs; pos += CHG, ++it) {
+                    const int ng = min(CHG, ngs - pos);
+                    if (++slot == NS) {
+                        slot = 0;
+                        lap ^= 1u;
+                    }
+                    if (!mbar_wait(st_full + 8u * slot, lap ^ 1u)) {
+                        dead = true;
+                        break;
+                    }
+                    const int gbeg = (warp * ng) >> 3, gend = ((warp + 1) * ng) >> 3;      // this warp's groups of the stage
+                    uint32_t wa = w_lane + (uint32_t)slot * stage_bytes + (uint32_t)gbeg * (kTileRows * GB);
+                    uint32_t xa = x_lane + (uint32_t)(pos + gbeg) * x_gstride;
+                    uint32_t xta = xt_lane + (uint32_t)(pos + gbeg) * xt_gstride;
+                    uint32_t ua = ux_lane + (uint32_t)(pos + gbeg) * 16u;
+                    uint32_t ma = m_lane + (uint32_t)(pos + gbeg) * 8u;
+#pragma unroll 1
+                    for (int gi = gbeg; gi < gend; ++gi) {
+                        uint32_t wra[NWORDS], wrb[NWORDS];
+                        if constexpr (BITS == 4) {
+                            const uint4 va = lds_v4(wa), vb = lds_v4(wa + 8 * GB);
+                            wra[0] = va.x; wra[1] = va.y; wra[2] = va.z; wra[3] = va.w;
+                            wrb[0] = vb.x; wrb[1] = vb.y; wrb[2] = vb.z; wrb[3] = vb.w;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < NWORDS; ++i) {
+                                wra[i] = lds_u32(wa + 4 * i);
+                                wrb[i] = lds_u32(wa + 8 * GB + 4 * i);
+                            }
+                        }
+                        const uint4 x0 = lds_v4(xa), x1 = lds_v4(xa + x_chunk1);
+                        const float2 fa = lds_f2(ma), fb = lds_f2(ma + 8u * (uint32_t)mpitch * 8u), ux = lds_f2(ua);
+                        uint32_t ra[NR], rb[NR];
+                        SlotsI8<BITS>::run(wra, ra);
+                        SlotsI8<BITS>::run(wrb, rb);
+                        int d[4] = {0, 0, 0, 0};
+                        mma_u8s8(d, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
+                        mma_u8s8(d, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
+                        mma_u8s8(d, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
+                        mma_u8s8(d, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
+                        if constexpr (BITS == 3) mma_u8s8(d, ra[NR - 1], rb[NR - 1], 0u, 0u, lds_u32(xta), 0u);
+                        const float sa = fa.x * ux.x, sb = fb.x * ux.x;
+                        acc[0][0] = fmaf(sa, (float)d[0], acc[0][0]);
+                        acc[0][1] = fmaf(sa, (float)d[1], acc[0][1]);
+                        acc[0][2] = fmaf(sb, (float)d[2], acc[0][2]);
+                        acc[0][3] = fmaf(sb, (float)d[3], acc[0][3]);
+                        accz[0] = fmaf(fa.y, ux.y, accz[0]);
+                        accz[1] = fmaf(fb.y, ux.y, accz[1]);
+                        wa += kTileRows * GB;
+                        xa += x_gstride;
+                        xta += xt_gstride;
+                        ua += 16u;
+                        ma += 8u;
+                    }
+                    // stage consumed by this warp
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(st_empty + 8u * slot);
+                }
+            } else
             for (int pos = 0; pos < ngs; pos += p.CHG, ++it) {
                 const int ng = min(p.CHG, ngs - pos);
                 if (++slot == p.NS) {
@@ -990,39 +1085,6 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
                             wa[i] = reinterpret_cast<const uint32_t *>(pa)[i];
                             wb[i] = reinterpret_cast<const uint32_t *>(pb)[i];
                         }
-                    }
-                    if constexpr (I8) {
-                        constexpr int NR = SlotsI8<BITS>::kRegs;
-                        uint32_t ra[NR], rb[NR];
-                        SlotsI8<BITS>::run(wa, ra);
-                        SlotsI8<BITS>::run(wb, rb);
-                        // this lane's column (token g / 4, digit g % 4) of the group, and (2^-e, X0) of the
-                        // token whose columns its accumulators hold
-                        const int ncol = 3 * p.M, cc = g - (g >> 2);                 // stored columns; MMA column g = 4 m + digit
-                        const uint4 *xg = reinterpret_cast<const uint4 *>(smem + p.off_x) + (size_t)((pos + gi) * 2 * ncol + cc) * 4 + tq;
-                        uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
-                        uint32_t xt = 0u;
-                        if (g < 4 * p.M && (g & 3) != 3) {
-                            x0 = xg[0];
-                            x1 = xg[ncol * 4];
-                            if (BITS == 3)
-                                xt = (reinterpret_cast<const uint32_t *>(smem + p.off_x) + (size_t)ngs * 2 * ncol * 16)[((pos + gi) * ncol + cc) * 4 + tq];
-                        }
-                        const float2 ux = reinterpret_cast<const float2 *>(smem + p.off_px)[(pos + gi) * 2 + (tq >> 1)];
-                        int d[4] = {0, 0, 0, 0};
-                        mma_u8s8(d, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
-                        mma_u8s8(d, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
-                        mma_u8s8(d, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
-                        mma_u8s8(d, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
-                        if constexpr (BITS == 3) mma_u8s8(d, ra[NR - 1], rb[NR - 1], 0u, 0u, xt, 0u);
-                        const float sa = fa.x * ux.x, sb = fb.x * ux.x;
-                        acc[0][0] = fmaf(sa, (float)d[0], acc[0][0]);
-                        acc[0][1] = fmaf(sa, (float)d[1], acc[0][1]);
-                        acc[0][2] = fmaf(sb, (float)d[2], acc[0][2]);
-                        acc[0][3] = fmaf(sb, (float)d[3], acc[0][3]);
-                        accz[0] = fmaf(fa.y, ux.y, accz[0]);
-                        accz[1] = fmaf(fb.y, ux.y, accz[1]);
-                        continue;
                     }
                     uint32_t ha[16], hb[16];
                     Unpack<BITS, T>::run(wa, ha);
