@@ -522,6 +522,27 @@ __device__ __forceinline__ bool tile_claim(const DecodeParams &p, int tile, int 
 // HEAVY selects the variant for a heavy sub-branch (rank above 64, or many (token, unit) pairs of the
 // down-projection per CTA): its units are shared by the eight compute warps and the tile finish
 // keeps twice as many chunks of B in registers.  The light variant keeps both out of its code.
+// Units of the down-projection (u = k chunk * rank + row of A) of CTA r out of R, for nkc chunks.  With
+// at least as many CTAs as chunks, CTA r works on chunk r % nkc only (so it needs one chunk of x) and
+// shares the chunk's rows evenly with the other CTAs of that chunk; with fewer CTAs the units are
+// dealt out in contiguous ranges.  Host and device use the same function.
+__host__ __device__ inline void unit_range(int r, int R, int rank, int nkc, int *u0, int *u1)
+{
+    if (rank <= 0 || nkc <= 0) {
+        *u0 = *u1 = 0;
+        return;
+    }
+    if (R >= nkc) {
+        const int c = r % nkc, i = r / nkc, n_c = (R - c + nkc - 1) / nkc;      // CTAs of chunk c
+        *u0 = c * rank + (int)((long long)i * rank / n_c);
+        *u1 = c * rank + (int)((long long)(i + 1) * rank / n_c);
+    } else {
+        const long long TU = (long long)rank * nkc;
+        *u0 = (int)((long long)r * TU / R);
+        *u1 = (int)((long long)(r + 1) * TU / R);
+    }
+}
+
 template <int BITS, typename T, int MT, bool HEAVY, bool I8>
 __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtensorMap *wmap, const int cta)
 {
@@ -546,8 +567,8 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
     // units of the down-projection owned by this CTA: (row j of A, 1024-wide k chunk of the slice)
     const int kslice = ngs * kGroupFast;
     const int nkc = (kslice + kTUnitK - 1) / kTUnitK;
-    const long long TU = (long long)p.rank * nkc;
-    const int tu0 = (int)((long long)r * TU / p.R), tu1 = (int)((long long)(r + 1) * TU / p.R);
+    int tu0, tu1;
+    unit_range(r, p.R, p.rank, nkc, &tu0, &tu1);
     const bool has_t = (p.rank > 0) && (tu1 > tu0);
 
     // shared memory: barriers | table | deferred list | meta | x | segbuf | A | B | t | ring
@@ -1630,7 +1651,13 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         pl.stage_bytes = kTileRows * pl.CHG * GB;             // [group][row][GB], dense
         pl.x_pitch = ngs_max * kGroupFast + 32;    // +64 bytes: tokens 2j, 2j+1 land in different bank halves
         const int nkc = (ngs_max * kGroupFast + kTUnitK - 1) / kTUnitK;
-        const long long tu_max = ((long long)a.rank * nkc + pl.R - 1) / pl.R;
+        long long tu_max = 0;                                 // most units any CTA gets
+        for (int r = 0; r < pl.R && r < 2 * nkc + 2; ++r) {   // the ranges repeat with period nkc; the first CTAs have the largest
+            int u0, u1;
+            unit_range(r, pl.R, a.rank, nkc, &u0, &u1);
+            tu_max = max(tu_max, (long long)(u1 - u0));
+        }
+        if (pl.R < nkc) tu_max = ((long long)a.rank * nkc + pl.R - 1) / pl.R;
         pl.a_cap = (int)min(tu_max, 8LL);
         // Heavy sub-branch: rank above what the light tile finish holds, or more units of the down-projection
         // per CTA than its epilogue warp should take by itself (tensor-core form: what fits its staging
@@ -1713,8 +1740,12 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
     if (a.rank > 0) {
         for (int s = 0; s < pl.SK; ++s) {
             const int ngs = (int)((long long)(s + 1) * G / pl.SK) - (int)((long long)s * G / pl.SK);
-            const long long TU = (long long)a.rank * ((ngs * kGroupFast + kTUnitK - 1) / kTUnitK);
-            pl.t_target += (int)min((long long)pl.R, TU);
+            const int nkc = (ngs * kGroupFast + kTUnitK - 1) / kTUnitK;
+            for (int r = 0; r < pl.R; ++r) {
+                int u0, u1;
+                unit_range(r, pl.R, a.rank, nkc, &u0, &u1);
+                pl.t_target += (u1 > u0) ? 1 : 0;
+            }
         }
     }
     return pl;

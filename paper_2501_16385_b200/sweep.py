@@ -23,7 +23,7 @@ SHAPES = [(4096, 4096)] * 4 + [(4096, 11008), (4096, 11008), (11008, 4096)]     
 TOTAL_CTAS = 400
 
 
-def time_layer(M, bits, rank, steps, pool_layers=3):
+def time_layer(M, bits, rank, steps, pool_layers=3, total_ctas=TOTAL_CTAS):
     pool = [[make_instance(M, N, K, bits, rank, "f16", 50 * li + j) for j, (K, N) in enumerate(SHAPES)]
             for li in range(pool_layers)]
     costs = [K * N for K, N in SHAPES]
@@ -36,7 +36,7 @@ def time_layer(M, bits, rank, steps, pool_layers=3):
             st.wait_stream(main)
         for i in range(n):
             for j, t in enumerate(pool[i % pool_layers]):
-                fbq.set_option("decode_ctas", max(8, round(TOTAL_CTAS * costs[j] / sum(costs))))
+                fbq.set_option("decode_ctas", max(8, round(total_ctas * costs[j] / sum(costs))))
                 fbq.linear(t["x"], t["qweight"], t["scales"], t["zeros"], t["A"], t["B"], t["y"].shape[1], 128, bits,
                            y=t["y"], stream=streams[j])
         for st in sides:
@@ -69,6 +69,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--ctas", type=int, default=TOTAL_CTAS, help="decode CTAs shared out among the seven linears")
     ap.add_argument("--tokens", type=int, nargs="*", default=[1, 2, 4, 8, 16])
     ap.add_argument("--opt", nargs="*", default=[], help="library options as name=value (fbq_set_option)")
     a = ap.parse_args()
@@ -78,7 +79,7 @@ def main():
     for M in a.tokens:
         base = None
         for rank in (0, 16, 32, 64, 128):
-            us = time_layer(M, a.bits, rank, a.steps)
+            us = time_layer(M, a.bits, rank, a.steps, total_ctas=a.ctas)
             by = sum(algorithmic_bytes(M, N, K, a.bits, rank) for K, N in SHAPES)
             by0 = sum(algorithmic_bytes(M, N, K, a.bits, 0) for K, N in SHAPES)
             if rank == 0:
