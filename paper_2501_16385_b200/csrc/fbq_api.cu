@@ -183,6 +183,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "decode_depth")) return &g_opt.decode.depth;
     if (!strcmp(name, "decode_ctas")) return &g_opt.decode.max_ctas;
     if (!strcmp(name, "decode_i8")) return &g_opt.decode.i8;
+    if (!strcmp(name, "decode_t_ctas")) return &g_opt.decode.t_ctas;
     if (!strcmp(name, "decode_t_wait")) return &g_opt.decode_t_wait;
     if (!strcmp(name, "pdl")) return &g_opt.decode.pdl;
     if (!strcmp(name, "decode_t_late")) return &g_opt.decode_t_late;

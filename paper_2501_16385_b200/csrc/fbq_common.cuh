@@ -74,6 +74,7 @@ int run_reconstruct_step(const float *W, const float *H, float *A, float *B, flo
 
 struct DecodeTuning {
     int sk = 0, chunk = 0, depth = 0, max_ctas = 0, pdl = 1;
+    int t_ctas = 1;  // 1: t = x.A^T comes from a few CTAs at the head of the grid (M <= 4, one K slice)
     int i8 = 1;      // 1: M <= 2 runs the form whose MMAs take the codes and x as 8-bit integers
 };
 // Returns cudaErrorInvalidConfiguration when no plan fits (caller falls back).

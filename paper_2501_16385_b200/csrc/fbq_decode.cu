@@ -86,6 +86,7 @@ struct DecodeParams {
     int SK, R, NT, CHG, NS, nbuf;
     int maxslots;
     int t_target;       // number of CTAs that contribute to t
+    int n_t;            // > 0: the first n_t CTAs of the grid compute t and nothing else; the others only read it
     int t_late;         // test switch: contribute to t after the main loop
     int vt;             // lanes per quad whose accumulators are exchanged (tokens 2tq, 2tq+1 valid)
     int x_pitch;        // elements per token in shared memory
@@ -543,9 +544,140 @@ __host__ __device__ inline void unit_range(int r, int R, int rank, int nkc, int 
     }
 }
 
-template <int BITS, typename T, int MT, bool HEAVY, bool I8>
-__device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtensorMap *wmap, const int cta)
+// A CTA that only computes t = x.A^T (the first n_t CTAs of a grid when the plan says so).  The main CTAs
+// of one launch start over a span of time (they take SM slots as these become free), and a t that every
+// CTA contributes to is complete only some microseconds after the LAST of them has started; these few
+// CTAs are dispatched first, depend on nothing but x, and are done a few microseconds after the first.
+// kTWarps warps each take blocks of up to eight rows of A of one 1024-wide k chunk: rows by bulk copies
+// (requested before the wait on the previous kernel), the chunk of x by coalesced loads, then m16n8k16 MMAs
+// whose rows are the tokens; fp32 atomics into t, and the last of these CTAs raises the "t complete" flag.
+constexpr int kTWarps = 4;
+template <typename T>
+__device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
 {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    const uint32_t bar0 = smem_u32(smem);
+    if (tid == 0) {
+        for (int i = 0; i < kTWarps; ++i) mbar_init(bar0 + 8u * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp >= kTWarps) {
+        pdl_wait();
+        pdl_launch_dependents();
+        return;
+    }
+    const int area = (8 + p.M) * kAPitch;                                     // elements per warp: 8 rows of A, M rows of x
+    T *s_Aw = reinterpret_cast<T *>(smem + 1024) + (size_t)warp * area, *s_xw = s_Aw + 8 * kAPitch;
+    const uint32_t bar = bar0 + 8u * warp;
+    const int bpr = (p.rank + 7) / 8, nkc = (p.K + kTUnitK - 1) / kTUnitK, nblocks = nkc * bpr;
+    const T *A = static_cast<const T *>(p.A), *x = static_cast<const T *>(p.x);
+    bool waited = false, dead = false;
+    int round = 0;
+#pragma unroll 1
+    for (int b = cta * kTWarps + warp; b < nblocks; b += p.n_t * kTWarps, ++round) {
+        const int kc = b / bpr, j0 = (b - kc * bpr) * 8, nrows = min(8, p.rank - j0);
+        const int kbeg = kc * kTUnitK, nk = min(kTUnitK, p.K - kbeg);            // a multiple of 128
+        __syncwarp();
+        if (lane == 0) {
+            if (round > 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the last block's reads are done
+            mbar_expect_tx(bar, (uint32_t)(nrows * nk * 2));
+        }
+        __syncwarp();
+        if (lane < nrows)
+            bulk_g2s(smem_u32(s_Aw + (size_t)lane * kAPitch), A + (size_t)(j0 + lane) * p.K + kbeg, (uint32_t)nk * 2u, bar);
+        if (!waited) {                                                         // x may come from the previous kernel
+            pdl_wait();
+            pdl_launch_dependents();
+            waited = true;
+        }
+#pragma unroll 1
+        for (int m = 0; m < p.M; m += 2) {
+            uint4 v[2][4];
+#pragma unroll
+            for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int k = lane * 8 + 256 * i;
+                    v[mm][i] = make_uint4(0u, 0u, 0u, 0u);
+                    if (k < nk && m + mm < p.M) v[mm][i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)(m + mm) * p.K + kbeg + k));
+                }
+#pragma unroll
+            for (int mm = 0; mm < 2; ++mm)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (m + mm < p.M) *reinterpret_cast<uint4 *>(s_xw + (size_t)(m + mm) * kAPitch + lane * 8 + 256 * i) = v[mm][i];
+        }
+        __syncwarp();
+        if (!mbar_wait(bar, (uint32_t)round & 1u)) {
+            dead = true;
+            break;
+        }
+        const uint32_t *arow = reinterpret_cast<const uint32_t *>(s_Aw + (size_t)g * kAPitch);
+        const uint32_t *xa = reinterpret_cast<const uint32_t *>(s_xw + (size_t)g * kAPitch);
+        const bool col_ok = g < nrows, ra_ok = g < p.M;
+        float d[4][4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) d[c][0] = d[c][1] = d[c][2] = d[c][3] = 0.f;
+#pragma unroll 2
+        for (int s16 = 0; s16 < nk / 16; s16 += 4) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int w = (s16 + c) * 8 + tq;                              // word index of k = 16 s + 2 tq
+                uint32_t a[4] = {0u, 0u, 0u, 0u}, b0 = 0u, b1 = 0u;
+                if (ra_ok) {
+                    a[0] = xa[w];
+                    a[2] = xa[w + 4];
+                }
+                if (col_ok) {
+                    b0 = arow[w];
+                    b1 = arow[w + 4];
+                }
+                Pk<T>::mma(d[c], a, b0, b1);
+            }
+        }
+        const float v0 = (d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), v1 = (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]);
+        const int c0 = 2 * tq;
+        if (ra_ok) {
+            if (c0 < nrows) atomicAdd(p.t + (size_t)g * p.rank + j0 + c0, v0);
+            if (c0 + 1 < nrows) atomicAdd(p.t + (size_t)g * p.rank + j0 + c0 + 1, v1);
+        }
+    }
+    if (!waited) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
+    if (dead && lane == 0) atomicExch(p.status, (int)FBQ_ERR_TIMEOUT);
+    named_barrier_sync(2, kTWarps * 32);
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(p.ctr + kCtrT, 1) == p.n_t - 1) {
+            // all of t is in: publish it, then take part in the retire count like a finished tile would
+            p.ctr[kCtrT] = 0;
+            __threadfence();
+            atomicExch(p.ctr + kCtrReady, 1);
+            __threadfence();
+            if (atomicAdd(p.ctr + kCtrDone, 1) + 1 == p.NT + 1) {
+                __threadfence();
+                for (int i = 0; i < 2 * p.NT; ++i) p.ctr[kCtrFirstTile + i] = 0;
+                for (int i = 0; i < p.M * p.rank; ++i) p.t[i] = 0.f;
+                p.ctr[kCtrDone] = 0;
+                p.ctr[kCtrReady] = 0;
+                p.ctr[kCtrPendingN] = 0;
+            }
+        }
+    }
+}
+
+template <int BITS, typename T, int MT, bool HEAVY, bool I8>
+__device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtensorMap *wmap, const int cta_in_grid)
+{
+    if (cta_in_grid < p.n_t) {
+        t_cta_body<T>(p, cta_in_grid);
+        return;
+    }
+    const int cta = cta_in_grid - p.n_t;
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int GB = (BITS == 4) ? 64 : 48;          // packed bytes of one group of one row
     constexpr int NWORDS = Unpack<BITS, T>::kWords;    // words per lane per group
@@ -569,7 +701,7 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
     const int nkc = (kslice + kTUnitK - 1) / kTUnitK;
     int tu0, tu1;
     unit_range(r, p.R, p.rank, nkc, &tu0, &tu1);
-    const bool has_t = (p.rank > 0) && (tu1 > tu0);
+    const bool has_t = (p.n_t == 0) && (p.rank > 0) && (tu1 > tu0);
 
     // shared memory: barriers | table | deferred list | meta | x | segbuf | A | B | t | ring
     trace_mark(p, 0);
@@ -1267,12 +1399,12 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
     // two numbers per output.  Tiles that are done before t is wait in their segment buffers for
     // as long as that holds nobody up.
     T *s_th = reinterpret_cast<T *>(s_stage + kTileRows * kDecodeMaxM);       // [8 columns][rank]
-    float *s_sub = reinterpret_cast<float *>(s_th + 8 * p.rank);             // [segment][row][4 tokens]
     const bool sub_at_once = !HEAVY && fast_fin && b_in_smem && p.M <= 4 && (p.rank % 16) == 0 && !p.t_late;
-    bool sub_done = false;
+    bool sub_done = false;          // t is there as 16-bit columns
+    float isc = 1.f;
     auto make_sub = [&]() {
-        // fp16 columns: a power of two keeps a large t inside the format (exact, undone below)
-        float sc = 1.f, isc = 1.f;
+        // fp16 columns: a power of two keeps a large t inside the format (exact, undone in the finish)
+        float sc = 1.f;
         if (std::is_same<T, __half>::value) {
             float tmax = 0.f;
             for (int i = lane; i < p.M * p.rank; i += 32) tmax = fmaxf(tmax, fabsf(s_t[i]));
@@ -1297,37 +1429,39 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
                 s_th[(4 + m) * p.rank + j] = ActTraits<T>::from_float(lo);
             }
         __syncwarp();
-        const uint32_t *tcol = reinterpret_cast<const uint32_t *>(s_th + (size_t)g * p.rank);
-#pragma unroll 1
-        for (int i = 0; i < nseg; ++i) {
-            const uint32_t *ba = reinterpret_cast<const uint32_t *>(s_B + (size_t)(i * kTileRows + g) * p.rank);
-            const uint32_t *bb = ba + 4 * p.rank;                                // row g + 8
-            float d[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-            for (int k16 = 0; k16 < p.rank / 16; ++k16) {
-                const int w = k16 * 8 + tq;
-                const uint32_t a[4] = {ba[w], bb[w], ba[w + 4], bb[w + 4]};
-                Pk<T>::mma(d, a, tcol[w], tcol[w + 4]);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) d[q] = (d[q] + __shfl_xor_sync(0xffffffffu, d[q], 2)) * isc;   // rounded part + remainder
-            if (tq < 2) {
-                float *o = s_sub + (size_t)(i * kTileRows + g) * 4 + 2 * tq;
-                o[0] = d[0];
-                o[1] = d[1];
-                o[8 * 4] = d[2];
-                o[8 * 4 + 1] = d[3];
-            }
-        }
-        __syncwarp();
         sub_done = true;
     };
-    auto finish_sub = [&](int tile, int seg) {
-        for (int idx = lane; idx < kTileRows * p.M; idx += 32) {
-            const int row = idx & (kTileRows - 1), m = idx >> 4, n = tile * kTileRows + row;
-            if (n < p.N)
-                static_cast<T *>(p.y)[(size_t)m * p.N + n] =
-                    ActTraits<T>::from_float(s_stage[m * kTileRows + row] + s_sub[(size_t)(seg * kTileRows + row) * 4 + m]);
+    // One tile: t.B^T of its 16 rows by rank / 16 MMAs (the result has the layout of the main sums: lane
+    // (g, tq < 2) holds tokens 2 tq, 2 tq + 1 of rows g and g + 8), added to the main sums in registers,
+    // rounded and stored.
+    auto finish_sub = [&](int tile, int seg, const float (&main)[4]) {
+        const uint32_t *tcol = reinterpret_cast<const uint32_t *>(s_th + (size_t)g * p.rank);
+        const uint32_t *ba = reinterpret_cast<const uint32_t *>(s_B + (size_t)(seg * kTileRows + g) * p.rank);
+        const uint32_t *bb = ba + 4 * p.rank;                                // row g + 8
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+        const int nk16 = p.rank / 16;                                        // at most 4 here (rank <= 64): all loads go out first
+        uint32_t a[4][4], tb[4][2];
+#pragma unroll
+        for (int k16 = 0; k16 < 4; ++k16) {
+            const int w = k16 * 8 + tq;
+            const bool on = k16 < nk16;
+            a[k16][0] = on ? ba[w] : 0u;
+            a[k16][1] = on ? bb[w] : 0u;
+            a[k16][2] = on ? ba[w + 4] : 0u;
+            a[k16][3] = on ? bb[w + 4] : 0u;
+            tb[k16][0] = on ? tcol[w] : 0u;
+            tb[k16][1] = on ? tcol[w + 4] : 0u;
+        }
+#pragma unroll
+        for (int k16 = 0; k16 < 4; ++k16) Pk<T>::mma(d, a[k16], tb[k16][0], tb[k16][1]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) d[q] = (d[q] + __shfl_xor_sync(0xffffffffu, d[q], 2)) * isc;   // rounded part + remainder
+        if (tq < p.vt) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int n = tile * kTileRows + g + 8 * (i >> 1), m = 2 * tq + (i & 1);
+                if (m < p.M && n < p.N) static_cast<T *>(p.y)[(size_t)m * p.N + n] = ActTraits<T>::from_float(main[i] + d[i]);
+            }
         }
         ++n_retired;
     };
@@ -1438,10 +1572,10 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
         e_wait += c_w1 - c_w0;
         trace_mark(p, seg == 0 ? 5 : 7);
         // add the eight warps' partial tiles in warp order and stage the result as [token][row]
-        if (tq < p.vt) {
-            float acc[MT][4];
+        float acc[MT][4];
 #pragma unroll
-            for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+        for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+        if (tq < p.vt) {
             const float4 *src = reinterpret_cast<const float4 *>(s_seg + (size_t)buf * segbuf_floats);
 #pragma unroll
             for (int w = 0; w < kCW; ++w)
@@ -1466,10 +1600,27 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
         if (cnt == 1 || others_in) {
             // This warp finishes the tile: straight from the staged sums if t is complete ...
             if (sub_at_once && p.t_wait && !t_local) wait_t_with_slack(seg);
+            if (p.n_t > 0 && !t_local) {
+                // t comes from the CTAs at the head of this grid, which wait for nothing: wait for it (bounded)
+                bool ok = false;
+#pragma unroll 1
+                for (uint32_t i = 0; i < kWaitLimit && !ok; ++i) {
+                    ok = t_poll();
+                    if (!ok) __nanosleep(200);
+                }
+                if (!ok) {
+                    dead = true;
+                    break;
+                }
+            }
             if (t_poll()) {
                 if (sub_at_once) {
-                    if (!sub_done) make_sub();
-                    finish_sub(tile, seg);
+                    if (!sub_done) {
+                        trace_mark(p, 3);
+                        make_sub();
+                        trace_mark(p, 14);
+                    }
+                    finish_sub(tile, seg, acc[0]);
                     __syncwarp();
                     if (p.trace) e_fin += clock64() - c_w2;
                     continue;
@@ -1614,6 +1765,7 @@ struct Plan {
     bool i8;            // codes and x go to the tensor cores as 8-bit integers (M <= 2)
     bool heavy;         // the compute warps take the units of the down-projection
     int ab_alias;
+    int n_t;            // CTAs at the head of the grid that compute t (0: every CTA contributes)
 };
 
 int g_sm_count = 0;
@@ -1662,8 +1814,16 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         // Heavy sub-branch: rank above what the light tile finish holds, or more units of the down-projection
         // per CTA than its epilogue warp should take by itself (tensor-core form: what fits its staging
         // area; plain form: (token, unit) pairs).
+        // t from a few CTAs at the head of the grid (one K slice, M <= 4): then the others hold no A
+        pl.n_t = 0;
+        if (a.rank > 0 && sk == 1 && a.M <= kTMmaMaxM && !g_t_late && tune.t_ctas != 0) {
+            const int nblocks = nkc * ((a.rank + 7) / 8);
+            pl.n_t = min(12, (nblocks + kTWarps - 1) / kTWarps);
+            pl.a_cap = 0;
+            tu_max = 0;
+        }
         pl.heavy = a.rank > 64 || (a.rank > 0 && (a.M <= kTMmaMaxM ? tu_max > 8 : tu_max * a.M > kTUnitsOneWarp));
-        pl.ab_alias = (a.rank > 0 && !pl.heavy && !g_t_late) ? 1 : 0;
+        pl.ab_alias = (a.rank > 0 && !pl.heavy && !g_t_late && pl.n_t == 0) ? 1 : 0;
         size_t off = (size_t)(2 * 8 + 2 * kNBufMax + 4) * 8;      // room for up to 8 stages' barriers
         off = (off + 15) & ~(size_t)15;
         pl.off_tab = (int)off;
@@ -1687,12 +1847,12 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         off = (off + 127) & ~(size_t)127;
         pl.off_A = (int)off;
         const size_t b_bytes = (size_t)nseg_max * kTileRows * a.rank * 2;
-        const size_t a_bytes = (size_t)(pl.a_cap + (a.rank > 0 && a.M <= kTMmaMaxM ? a.M : 0)) * kAPitch * 2;   // units of A, then x of one k chunk
+        const size_t a_bytes = pl.n_t > 0 ? 0 : (size_t)(pl.a_cap + (a.rank > 0 && a.M <= kTMmaMaxM ? a.M : 0)) * kAPitch * 2;   // units of A, then x of one k chunk
         off += pl.ab_alias ? max(a_bytes, b_bytes) : a_bytes;
         off = (off + 127) & ~(size_t)127;
         pl.off_t = (int)off;
         off += (size_t)a.M * a.rank * 4 + (size_t)kTileRows * kDecodeMaxM * 4;   // t, then the epilogue warp's staging tile
-        off += (size_t)8 * a.rank * 2 + (size_t)nseg_max * kTileRows * 4 * 4;      // t as 16-bit columns, up-projection of all own rows
+        off += (size_t)8 * a.rank * 2;                                            // t as 16-bit columns
         off = (off + 127) & ~(size_t)127;
         // what is left: two stages of the ring, then B of the own tiles, then more stages
         pl.off_B = (int)off;
@@ -1711,6 +1871,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         pl.NS = ns_want;
         while (pl.NS > 2 && off + (size_t)pl.NS * pl.stage_bytes > budget) --pl.NS;
         off += (size_t)pl.NS * pl.stage_bytes;
+        if (pl.n_t > 0) off = max(off, (size_t)1024 + (size_t)kTWarps * (8 + a.M) * kAPitch * 2);   // what a t CTA needs
         pl.smem = off;
         return nseg_max <= kMaxSeg && pl.smem <= budget;
     };
@@ -1732,12 +1893,14 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         for (int sk = 1; sk <= G && !pl.ok; ++sk) pl.ok = either(sk, kSmemMax);
     }
     if (getenv("FBQ_PLAN"))
-        fprintf(stderr, "plan M %d N %d K %d r %d: ok %d SK %d R %d CHG %d NS %d nbuf %d a_cap %d b_rows %d smem %zu (meta %d x %d ring@%d) i8 %d heavy %d alias %d\n", a.M, a.N, a.K,
+        fprintf(stderr, "plan M %d N %d K %d r %d: ok %d SK %d R %d CHG %d NS %d nbuf %d a_cap %d b_rows %d smem %zu (meta %d x %d ring@%d) i8 %d heavy %d alias %d n_t %d\n", a.M, a.N, a.K,
                 a.rank, (int)pl.ok, pl.SK, pl.R, pl.CHG, pl.NS, pl.nbuf, pl.a_cap, pl.b_cap_rows, pl.smem, pl.off_x - pl.off_meta,
-                pl.off_px - pl.off_x, pl.off_ring, (int)pl.i8, (int)pl.heavy, pl.ab_alias);
+                pl.off_px - pl.off_x, pl.off_ring, (int)pl.i8, (int)pl.heavy, pl.ab_alias, pl.n_t);
     // CTAs that own at least one unit of the down-projection
     pl.t_target = 0;
-    if (a.rank > 0) {
+    if (pl.n_t > 0) {
+        pl.t_target = pl.n_t;
+    } else if (a.rank > 0) {
         for (int s = 0; s < pl.SK; ++s) {
             const int ngs = (int)((long long)(s + 1) * G / pl.SK) - (int)((long long)s * G / pl.SK);
             const int nkc = (ngs * kGroupFast + kTUnitK - 1) / kTUnitK;
@@ -1809,7 +1972,7 @@ cudaError_t launch_variant(const DecodeParams &p, const CUtensorMap &wmap, const
         attr_set = true;
     }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)(pl.R * pl.SK));
+    cfg.gridDim = dim3((unsigned)(pl.n_t + pl.R * pl.SK));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = s;
@@ -1871,6 +2034,7 @@ DecodeParams fill_params(const LinearArgs &a, const Plan &pl, float *partial, fl
     p.SK = pl.SK; p.R = pl.R; p.NT = pl.NT; p.CHG = pl.CHG; p.NS = pl.NS; p.nbuf = pl.nbuf;
     p.maxslots = pl.maxslots;
     p.t_target = pl.t_target;
+    p.n_t = pl.n_t;
     p.t_late = g_t_late;
     p.vt = pl.vt;
     p.x_pitch = pl.x_pitch; p.stage_bytes = pl.stage_bytes;
@@ -1965,7 +2129,7 @@ cudaError_t launch_decode_batch(const LinearArgs *a, int count, const int *ctas,
         if (cudaError_t me = weight_map(&b.wmap[i], a[i], pl); me != cudaSuccess) return me;
         b.prob[i] = fill_params(a[i], pl, ws.partial + off_p, ws.t + off_t, ws.counters + off_c, ws.counters + kCtrStatus, nullptr);
         b.first[i] = (i == 0) ? 0 : b.first[i];
-        b.first[i + 1] = b.first[i] + pl.R * pl.SK;
+        b.first[i + 1] = b.first[i] + pl.n_t + pl.R * pl.SK;
         off_p += (size_t)pl.NT * pl.maxslots * a[i].M * kTileRows;
         off_t += (size_t)kDecodeMaxM * kMaxRank;
         off_c += kCtrFirstTile + 2 * pl.NT;

@@ -125,19 +125,23 @@ def test_integer_form_rows_of_codes_at_the_ends(fbq):
         check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE)
 
 
-@pytest.mark.parametrize("M,rank", [(1, 16), (2, 64), (3, 32), (4, 64), (4, 48)])
-def test_sub_branch_paths_of_the_light_variant(fbq, M, rank):
-    # tensor-core down-projection (M <= 4), up-projection of all own rows at once (rank a multiple of 16) and
-    # the plain tile finish (rank 48), each against the oracle; three calls in a row leave the scratch clean
+@pytest.mark.parametrize("t_ctas", [1, 0])
+@pytest.mark.parametrize("M,rank", [(1, 16), (2, 64), (3, 32), (4, 64), (4, 48), (2, 128), (1, 200)])
+def test_sub_branch_paths(fbq, M, rank, t_ctas):
+    # t from the CTAs at the head of the grid (t_ctas = 1) or from every CTA's epilogue warp (0); tensor-core
+    # up-projection per tile (rank a multiple of 16, at most 64), the plain tile finish (rank 48) and the heavy
+    # variant (rank > 64), each against the oracle; three calls in a row leave the scratch clean
     import torch
     inp = make_linear(M, 1160, 2048, 4, rank, seed=7400 + M + rank)
-    check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE)
-    dev = DeviceLinear(inp, fbq)
-    fbq.set_option("force_kernel", fbq.KERNEL_DECODE)
+    fbq.set_option("decode_t_ctas", t_ctas)
     try:
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE)
+        dev = DeviceLinear(inp, fbq)
+        fbq.set_option("force_kernel", fbq.KERNEL_DECODE)
         ys = [dev.run(fbq).clone() for _ in range(3)]
     finally:
         fbq.set_option("force_kernel", -1)
+        fbq.set_option("decode_t_ctas", 1)
     torch.cuda.synchronize()
     assert fbq.poll_status() == 0
     for y in ys[1:]:
@@ -147,10 +151,12 @@ def test_sub_branch_paths_of_the_light_variant(fbq, M, rank):
 @pytest.mark.parametrize("t_wait", [0, 1])
 def test_tiles_wait_for_t_or_are_parked(fbq, t_wait):
     fbq.set_option("decode_t_wait", t_wait)
+    fbq.set_option("decode_t_ctas", 0)                     # every CTA contributes to t: it is complete late
     try:
         inp = make_linear(1, 2048, 4096, 3, 64, seed=7500)
         fbq.set_option("decode_ctas", 16)                  # eight tiles per CTA: some are done before t is
         check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE)
     finally:
         fbq.set_option("decode_t_wait", 1)
+        fbq.set_option("decode_t_ctas", 1)
         fbq.set_option("decode_ctas", 0)
