@@ -471,7 +471,7 @@ def gpu_arm(args):
         "gpu_launches": args.steps * n_linears,       # one fused decode launch per linear per step
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": value / world / peaks["hbm_gbs"], "of": peak_kind,
-                     "kernel": "decode_kernel<3,__half,1>",
+                     "kernel": "decode_kernel<3,__half,1,light,int8>",
                      "algorithmic_bytes_per_step": bytes_step, "traffic": TRAFFIC_BYTES_PER_STEP},
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -487,9 +487,9 @@ def gpu_arm(args):
 
 
 # DRAM bytes (read + write) per step measured with ncu (--set full) on the seven decode
-# launches of one step: 4 x 7.951 MB + 2 x 20.337 MB + 20.351 MB
+# launches of one step: 4 x 7.970 MB + 2 x 20.356 MB + 20.367 MB
 # (profiles/decode_int3_r64_m1_bench.md).
-TRAFFIC_BYTES_PER_STEP = 92_831_000
+TRAFFIC_BYTES_PER_STEP = 92_958_000
 
 
 # ---------------------------------------------------------------------- reference arm

@@ -92,8 +92,11 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  * (3 bits) dividing K, rank >= 0.  The decode and prefill kernels assume
  * integer-valued zero points in [0, 127]; the generic kernel accepts any
  * fp16 value.  Accumulation is fp32; t = x.A^T stays fp32 in the decode and
- * generic kernels and is rounded once to the activation type in the prefill
- * kernel (which also rounds the dequantised weights s*(q-z) once to that type).
+ * generic kernels (where the decode kernel multiplies it with B on tensor cores it enters as
+ * two 16-bit terms, the rounded value and the remainder) and is rounded once to the activation
+ * type in the prefill kernel (which also rounds the dequantised weights s*(q-z) once to that
+ * type).  At M <= 2 the decode kernel reads x in fixed point per group of 128, exact to 2^-17
+ * of the group's largest element ("decode_i8").
  * Summation order is fixed for a given shape (results are
  * reproducible run to run) except for t in the decode kernel, which is
  * accumulated with floating-point atomics. */
@@ -233,6 +236,13 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "decode_chunk"  0 = automatic, else quantisation groups per smem stage
  *   "decode_depth"  0 = automatic, else stages in flight per warp
  *   "decode_ctas"   0 = automatic, else an upper bound on the decode grid size
+ *   "decode_i8"     1 (default) = at M <= 2 the decode kernel takes the codes as unsigned bytes and x as three
+ *                   signed base-256 digits per group scale through 8-bit integer MMAs (x exact to 2^-17 of its
+ *                   group's largest element); 0 = the 16-bit form (x exact) at every M
+ *   "decode_t_ctas" 1 (default) = at M <= 4 (one K slice) t = x.A^T is computed by a few CTAs at the head of the
+ *                   grid and the others wait for it (bounded); 0 = every CTA contributes its share
+ *   "decode_t_wait" 1 (default) = a finished tile may wait for t in shared memory while that holds nobody up,
+ *                   0 = it is parked in scratch at once (only matters without t CTAs)
  *   "batch_ctas"    CTAs shared out among the problems of a decode-sized fbq_linear_batch (default 400)
  *   "prefill_pair"  1 = token tiles of 256 of the prefill kernel run on CTA pairs (cta_group::2 MMAs,
  *                   each CTA staging half of the token tile); 0 (default) = one CTA per tile, which
