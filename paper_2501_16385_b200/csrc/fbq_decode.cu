@@ -958,17 +958,32 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
         const int mpitch = ngs | 1;                  // odd pitch: the eight rows of a warp hit different banks
         {
             // (s, s*z) table: weights only, so it is filled before the wait on the previous kernel
-            const int nmeta = nseg * kTileRows * ngs;
+            // (a warp per row, lanes over the row's groups: coalesced, and no division per entry)
             const uint16_t *sc = reinterpret_cast<const uint16_t *>(p.scales);
             const uint16_t *ze = reinterpret_cast<const uint16_t *>(p.zeros);
-#pragma unroll 4
-            for (int idx = tid; idx < nmeta; idx += nthr) {
-                const int row = idx / ngs, gl = idx - row * ngs;
-                const int n = min(tile_first * kTileRows + row, p.N - 1);
-                const size_t mi = (size_t)n * p.G + g0 + gl;
-                const float sf = __half2float(__ushort_as_half(sc[mi]));
-                const float zf = __half2float(__ushort_as_half(ze[mi]));
-                s_mf[row * mpitch + gl] = make_float2(sf, sf * zf);
+            const int nrows = nseg * kTileRows;
+            // sixteen rows at a time, all their loads in flight before the first conversion
+            constexpr int kRowsAtOnce = 16;
+            for (int gl = lane; gl < ngs; gl += 32) {
+#pragma unroll 1
+                for (int row0 = warp; row0 < nrows; row0 += kRowsAtOnce * kCW) {
+                    uint16_t sv[kRowsAtOnce], zv[kRowsAtOnce];
+#pragma unroll
+                    for (int u = 0; u < kRowsAtOnce; ++u) {
+                        const int row = row0 + u * kCW;
+                        const int n = min(tile_first * kTileRows + min(row, nrows - 1), p.N - 1);
+                        const size_t mi = (size_t)n * p.G + g0 + gl;
+                        sv[u] = sc[mi];
+                        zv[u] = ze[mi];
+                    }
+#pragma unroll
+                    for (int u = 0; u < kRowsAtOnce; ++u) {
+                        const int row = row0 + u * kCW;
+                        const float sf = __half2float(__ushort_as_half(sv[u]));
+                        const float zf = __half2float(__ushort_as_half(zv[u]));
+                        if (row < nrows) s_mf[row * mpitch + gl] = make_float2(sf, sf * zf);
+                    }
+                }
             }
         }
 
