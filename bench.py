@@ -487,9 +487,9 @@ def gpu_arm(args):
 
 
 # DRAM bytes (read + write) per step measured with ncu (--set full) on the seven decode
-# launches of one step: 4 x 7.970 MB + 2 x 20.356 MB + 20.367 MB
+# launches of one step: 4 x 7.971 MB + 2 x 20.357 MB + 20.369 MB
 # (profiles/decode_int3_r64_m1_bench.md).
-TRAFFIC_BYTES_PER_STEP = 92_958_000
+TRAFFIC_BYTES_PER_STEP = 92_969_000
 
 
 # ---------------------------------------------------------------------- reference arm

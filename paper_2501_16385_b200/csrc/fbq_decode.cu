@@ -1896,8 +1896,15 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         for (int form = 0; form < (want_i8 ? 2 : 1); ++form) {
             pl.i8 = want_i8 && form == 0;
             // stages of 16 groups, else of 8 (more hand-overs per byte, but still one K slice)
-            for (int chg = 16; chg >= 8; chg -= 8)
-                if (layout(sk, budget, true, chg) || layout(sk, budget, false, chg)) return true;
+            // B of the own tiles in shared memory (tensor-core tile finish) is worth more than eight segment
+            // buffers: a layout without it is taken only if none with it fits
+            for (int chg = 16; chg >= 8; chg -= 8) {
+                const bool with_many = layout(sk, budget, true, chg);
+                if (with_many && (a.rank == 0 || pl.b_cap_rows > 0)) return true;
+                if (layout(sk, budget, false, chg) && (a.rank == 0 || pl.b_cap_rows > 0)) return true;
+                if (with_many) return layout(sk, budget, true, chg);
+                if (layout(sk, budget, false, chg)) return true;
+            }
         }
         return false;
     };
