@@ -258,7 +258,9 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *                   every tile through the parked-tile branch of the combine protocol
  *   "decode_trace"  tuning aid: 1 = the decode kernel records, per CTA and warp, the SM cycle
  *                   counter at its phases, read with fbq_debug_read_trace
- * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name. */
+ * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name.
+ * (Tuning aid outside this interface: with the environment variable FBQ_PLAN set, every plan of the
+ * decode kernel is printed to stderr: K slices, CTAs, stage size and count, shared-memory layout, form.) */
 int fbq_set_option(const char *name, int value);
 int fbq_get_option(const char *name, int *value);
 
