@@ -71,6 +71,18 @@ def test_force_kernel_option_roundtrip():
         fbq.set_option("no_such_option", 1)
 
 
+def test_documented_options_exist_with_their_defaults():
+    # every switch named in include/fbq.h is known to the library and starts at the documented value
+    defaults = {"force_kernel": -1, "decode_sk": 0, "decode_chunk": 0, "decode_depth": 0, "decode_ctas": 0,
+                "decode_i8": 1, "decode_t_ctas": 1, "decode_t_wait": 1, "batch_ctas": 400, "batch_single": 1,
+                "prefill_pair": 0, "prefill_split": 1, "pdl": 1, "decode_t_late": 0, "decode_trace": 0}
+    header = open(os.path.join(os.path.dirname(__file__), "..", "include", "fbq.h")).read()
+    for name, value in defaults.items():
+        assert '"%s"' % name in header, name
+        assert fbq.get_option(name) == value, name
+        fbq.set_option(name, value)
+
+
 def test_argument_validation_happens_before_any_cuda_call():
     L = fbq.lib()
     buf = (ctypes.c_char * 4096)()
