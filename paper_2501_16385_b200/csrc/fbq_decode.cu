@@ -6,33 +6,33 @@
 // a second launch; here t is produced by the same launch, so a decode step costs
 // one launch per linear and y is written exactly once.
 //
-// Work split (stream-K).  The grid is R x SK CTAs, about one per SM.  K is cut
-// into SK slices (SK = 1 unless x is too large for shared memory); inside a
-// slice the (16-row tile, quantisation group) units are dealt out tile-major in
-// equal contiguous ranges, so every CTA streams the same number of bytes and at
-// most its first and last tile are shared with a neighbour.  A CTA walks its
-// range tile by tile ("segments").
+// Work split.  The grid is n_t + R x SK CTAs, about two per SM.  K is cut into SK
+// slices (SK = 1 unless the tables do not fit shared memory); the 16-row tiles
+// are dealt out in equal contiguous ranges, and a CTA walks its range tile by
+// tile ("segments").
 //
-// Warp roles.  A producer warp streams the packed codes of the range with bulk
-// asynchronous copies (one per weight row and stage, 1-2 KB each, mbarrier
-// completion) into a ring of shared-memory stages, and also fetches this CTA's
-// rows of A and B once.  Eight compute warps share every stage: each takes an
-// eighth of its groups, expands the codes with the exponent trick ((w & mask) |
-// 0x6400 is 1024+q in fp16), subtracts the zero point exactly and contracts the
-// integers q-z with x by warp-level m16n8k16 tensor-core MMAs (16 weight rows x
-// 8 tokens, fp32 accumulation); the group scale multiplies the fp32 partial sum
-// once per group.  The k order inside an MMA is a fixed permutation chosen so
-// that a lane's packed word IS its operand fragment; x is kept in shared memory
-// in the matching order.  An epilogue warp owns everything else: it computes
-// this CTA's share of t = x.A^T, and for every segment adds the eight warps'
-// partial tiles (fixed order), then finishes the tile (adds t.B^T, rounds,
-// stores y) or, for a tile shared with other CTAs, combines through scratch:
-// whoever finds all other contributions already there finishes the tile
-// directly; otherwise it leaves its partial and an arrival count, and the last
-// arrival finishes.  Nothing in the kernel spins on another CTA: a tile that
-// is complete before t is waits in a local list and, at worst, is handed to
-// the warp that completes t.  The only waits are on this CTA's own copies and
-// warps, and they are bounded.
+// Warp roles of a main CTA.  A producer warp streams the packed codes of the
+// range: one TMA tensor copy per stage (16 groups x 16 rows, landing as
+// [group][row][48 or 64 bytes]; mbarrier completion) into a ring of stages.
+// Eight compute warps share every stage, two groups each.  At M <= 2 (integer
+// form) a code masked out of its word is an unsigned byte operand of the 8-bit
+// integer MMA as it stands and x is held as three signed base-256 digits per
+// group scale, one digit per spare MMA column; above that (16-bit form) the codes
+// are expanded with the exponent trick ((w & mask) | 0x6400 is 1024+q in fp16) and
+// contracted with x by m16n8k16 MMAs.  In both forms the group scale multiplies
+// the partial sum once per group and the zero point enters as s*z*sum(x).  An
+// epilogue warp adds the eight warps' partial tiles of every segment (fixed
+// order), adds t.B^T (per tile on tensor cores where the rank allows), rounds
+// and stores y.
+//
+// t = x.A^T is computed by the first n_t CTAs of the grid (tensor-core blocks of
+// eight rows of A), which raise a flag when it is complete; the main CTAs wait
+// for the flag (bounded) where they need t.  Without such CTAs (M > 4, several
+// K slices) every CTA's epilogue warp contributes a share of t, tiles shared
+// between K slices are combined through scratch (whoever arrives last
+// finishes), and a tile that is complete before t is waits in a list and is, at
+// worst, handed to the warp that completes t: then nothing spins on another
+// CTA.  All waits are bounded.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
