@@ -85,8 +85,8 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  *   rank == 0: A and B are ignored (may be NULL); y is the main path alone.
  *   M == 0: nothing is done.
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128
- * and rank a multiple of 8 not above 256 -> decode kernel for M <= 6 (and M * rank <= 128
- * once M >= 3), else prefill kernel (N a multiple of 8 and 16-byte aligned operands; otherwise the decode
+ * and rank a multiple of 8 not above 256 -> decode kernel for M <= 4 with rank <= 128 and for
+ * M = 5, 6 with M * rank <= 128, else prefill kernel (N a multiple of 8 and 16-byte aligned operands; otherwise the decode
  * kernel up to M = 16); everything else that is well formed -> generic kernel.
  * Well formed means bits in {3,4}, group a multiple of 8 (4 bits) or 32
  * (3 bits) dividing K, rank >= 0.  The decode and prefill kernels assume

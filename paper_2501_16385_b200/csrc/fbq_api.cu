@@ -59,10 +59,11 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
     // Measured on B200 (7B shapes): the decode kernel wins up to M = 6; from M = 7 on the tensor-core
     // kernel is faster even though few of its token rows are real.
-    // The decode kernel's sub-branch work grows with M * rank (one t for the whole grid, tiles wait for
-    // it): from M = 3 on, M * rank above 128 also goes to the tensor-core kernel (M = 4, rank 64, seven
-    // streams: 494 us per layer against 105 us).
-    const bool decode_pays = M <= kDecodePreferM && !(M >= 3 && M * rank > 128);
+    // Up to M = 4 the decode kernel gets t from CTAs at the head of its grid and wins at every rank up to
+    // 128 (M = 4, rank 64, seven streams: 57 us per layer against 100 us).  At M = 5 and 6 every CTA
+    // contributes to t and the tiles wait for it, work that grows with M * rank: there M * rank above 128
+    // goes to the tensor-core kernel (M = 6, rank 64: 614 us per layer against 101 us).
+    const bool decode_pays = M <= kDecodePreferM && (M <= 4 ? rank <= 128 : M * rank <= 128);
     if (decode_ok && (decode_pays || !prefill_ok)) return FBQ_KERNEL_DECODE;
     if (prefill_ok) return FBQ_KERNEL_PREFILL;
     return FBQ_KERNEL_GENERIC;

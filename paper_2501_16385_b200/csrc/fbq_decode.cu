@@ -1691,6 +1691,18 @@ __device__ __forceinline__ void decode_body(const DecodeParams &p, const CUtenso
         bool ready = false;
 #pragma unroll 1
         for (int spin = 0; spin <= kTPolls && !ready; ++spin) ready = t_poll();
+        if (p.n_t > 0 && !ready) {
+            // t comes from the CTAs at the head of the grid, and nobody would pick parked tiles up: wait (bounded)
+#pragma unroll 1
+            for (uint32_t i = 0; i < kWaitLimit && !ready; ++i) {
+                ready = t_poll();
+                if (!ready) __nanosleep(200);
+            }
+            if (!ready) {
+                dead = true;
+                n_def = 0;
+            }
+        }
 #pragma unroll 1
         for (int i = 0; i < n_def; ++i) {
             const int tile = s_def[i];
@@ -1829,10 +1841,10 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         // Heavy sub-branch: rank above what the light tile finish holds, or more units of the down-projection
         // per CTA than its epilogue warp should take by itself (tensor-core form: what fits its staging
         // area; plain form: (token, unit) pairs).
-        // t from a few CTAs at the head of the grid (one K slice, M <= 4): then the others hold no A
+        // t from a few CTAs at the head of the grid (M <= 4; over all of K, whatever the K slices): then the others hold no A
         pl.n_t = 0;
-        if (a.rank > 0 && sk == 1 && a.M <= kTMmaMaxM && !g_t_late && tune.t_ctas != 0) {
-            const int nblocks = nkc * ((a.rank + 7) / 8);
+        if (a.rank > 0 && a.M <= kTMmaMaxM && !g_t_late && tune.t_ctas != 0) {
+            const int nblocks = ((a.K + kTUnitK - 1) / kTUnitK) * ((a.rank + 7) / 8);      // over all of K
             pl.n_t = min(12, (nblocks + kTWarps - 1) / kTWarps);
             pl.a_cap = 0;
             tu_max = 0;

@@ -41,7 +41,8 @@ def test_dispatch_rules():
         assert sel(M, 4096, 4096, 128, 4, 32) == D
         assert sel(M, 11008, 4096, 128, 3, 64, bf16=True) == D
     assert sel(6, 4096, 4096, 128, 4, 16) == D and sel(6, 4096, 4096, 128, 4, 0) == D
-    assert sel(4, 4096, 4096, 128, 4, 64) == P and sel(4, 4096, 4096, 128, 4, 32) == D    # M * rank above 128 from M = 3
+    assert sel(4, 4096, 4096, 128, 4, 64) == D and sel(4, 4096, 4096, 128, 4, 128) == D and sel(4, 4096, 4096, 128, 4, 256) == P
+    assert sel(5, 4096, 4096, 128, 4, 64) == P and sel(5, 4096, 4096, 128, 4, 24) == D    # M * rank above 128 at M = 5, 6
     assert sel(2, 4096, 4096, 128, 4, 128) == D
     for M in (7, 8, 15, 16):                        # measured crossover: the tensor-core kernel wins from M = 7
         assert sel(M, 4096, 4096, 128, 4, 32) == P
