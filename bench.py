@@ -39,7 +39,9 @@ GRAPH_STEPS = 100
 # call (the library runs the seven launches on its side streams and joins them every step).
 MODE = os.environ.get("FBQ_BENCH_MODE", "streams")
 N_STREAMS = int(os.environ.get("FBQ_BENCH_STREAMS", "7"))
-DECODE_CTAS = int(os.environ.get("FBQ_BENCH_CTAS", "400"))      # shared out among the 7 linears by size
+# main CTAs shared out among the 7 linears by size: 386 gives the 4096-wide linears 32 CTAs and the 11008-wide ones
+# 86, i.e. exactly eight 16-row tiles per CTA for both (256 and 688 tiles)
+DECODE_CTAS = int(os.environ.get("FBQ_BENCH_CTAS", "386"))
 NVSMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                 "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                 "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")

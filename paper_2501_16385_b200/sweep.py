@@ -4,7 +4,7 @@ M in {1, 2, 4, 8, 16} tokens x rank in {0, 16, 32, 64, 128}, INT4 (or --bits 3),
     python -m paper_2501_16385_b200.sweep [--bits 4] [--steps 300]
 
 Same launch scheme as bench.py's headline arm: the seven independent linears of a step go to seven
-CUDA streams (joined once per graph), decode grids share 400 CTAs by size, CUDA-graph replay, a pool
+CUDA streams (joined once per graph), decode grids share 386 main CTAs by size (eight 16-row tiles per CTA for N = 4096 and 11008), CUDA-graph replay, a pool
 of layer instances larger than L2, CUDA events on the launching stream.  Prints one JSON line per
 (M, rank): microseconds per step, effective GB/s, and the overhead against rank 0 at the same M
 beside the byte floor (extra bytes the sub-branch adds).  Inputs are random device tensors
@@ -20,7 +20,7 @@ from .accounting import algorithmic_bytes
 from .microbench import make_instance
 
 SHAPES = [(4096, 4096)] * 4 + [(4096, 11008), (4096, 11008), (11008, 4096)]       # (K, N): q k v o gate up down
-TOTAL_CTAS = 400
+TOTAL_CTAS = 386
 
 
 def time_layer(M, bits, rank, steps, pool_layers=3, total_ctas=TOTAL_CTAS):
