@@ -551,7 +551,9 @@ __host__ __device__ inline void unit_range(int r, int R, int rank, int nkc, int 
 // kTWarps warps each take blocks of up to eight rows of A of one 1024-wide k chunk: rows by bulk copies
 // (requested before the wait on the previous kernel), the chunk of x by coalesced loads, then m16n8k16 MMAs
 // whose rows are the tokens; fp32 atomics into t, and the last of these CTAs raises the "t complete" flag.
-constexpr int kTWarps = 4;
+constexpr int kTWarps = 8;
+constexpr int kTcK = 512;                     // k extent of a block of a t CTA
+constexpr int kTcPitch = kTcK + 8;            // elements between rows in its shared memory (16 bytes past a multiple of 128)
 template <typename T>
 __device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
 {
@@ -568,17 +570,17 @@ __device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
         pdl_launch_dependents();
         return;
     }
-    const int area = (8 + p.M) * kAPitch;                                     // elements per warp: 8 rows of A, M rows of x
-    T *s_Aw = reinterpret_cast<T *>(smem + 1024) + (size_t)warp * area, *s_xw = s_Aw + 8 * kAPitch;
+    const int area = (8 + p.M) * kTcPitch;                                     // elements per warp: 8 rows of A, M rows of x
+    T *s_Aw = reinterpret_cast<T *>(smem + 1024) + (size_t)warp * area, *s_xw = s_Aw + 8 * kTcPitch;
     const uint32_t bar = bar0 + 8u * warp;
-    const int bpr = (p.rank + 7) / 8, nkc = (p.K + kTUnitK - 1) / kTUnitK, nblocks = nkc * bpr;
+    const int bpr = (p.rank + 7) / 8, nkc = (p.K + kTcK - 1) / kTcK, nblocks = nkc * bpr;
     const T *A = static_cast<const T *>(p.A), *x = static_cast<const T *>(p.x);
     bool waited = false, dead = false;
     int round = 0;
 #pragma unroll 1
     for (int b = cta * kTWarps + warp; b < nblocks; b += p.n_t * kTWarps, ++round) {
         const int kc = b / bpr, j0 = (b - kc * bpr) * 8, nrows = min(8, p.rank - j0);
-        const int kbeg = kc * kTUnitK, nk = min(kTUnitK, p.K - kbeg);            // a multiple of 128
+        const int kbeg = kc * kTcK, nk = min(kTcK, p.K - kbeg);                // a multiple of 128
         __syncwarp();
         if (lane == 0) {
             if (round > 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the last block's reads are done
@@ -586,7 +588,7 @@ __device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
         }
         __syncwarp();
         if (lane < nrows)
-            bulk_g2s(smem_u32(s_Aw + (size_t)lane * kAPitch), A + (size_t)(j0 + lane) * p.K + kbeg, (uint32_t)nk * 2u, bar);
+            bulk_g2s(smem_u32(s_Aw + (size_t)lane * kTcPitch), A + (size_t)(j0 + lane) * p.K + kbeg, (uint32_t)nk * 2u, bar);
         if (!waited) {                                                         // x may come from the previous kernel
             pdl_wait();
             pdl_launch_dependents();
@@ -594,11 +596,11 @@ __device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
         }
 #pragma unroll 1
         for (int m = 0; m < p.M; m += 2) {
-            uint4 v[2][4];
+            uint4 v[2][kTcK / 256];
 #pragma unroll
             for (int mm = 0; mm < 2; ++mm)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < kTcK / 256; ++i) {
                     const int k = lane * 8 + 256 * i;
                     v[mm][i] = make_uint4(0u, 0u, 0u, 0u);
                     if (k < nk && m + mm < p.M) v[mm][i] = __ldcg(reinterpret_cast<const uint4 *>(x + (size_t)(m + mm) * p.K + kbeg + k));
@@ -606,16 +608,16 @@ __device__ __noinline__ void t_cta_body(const DecodeParams &p, const int cta)
 #pragma unroll
             for (int mm = 0; mm < 2; ++mm)
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (m + mm < p.M) *reinterpret_cast<uint4 *>(s_xw + (size_t)(m + mm) * kAPitch + lane * 8 + 256 * i) = v[mm][i];
+                for (int i = 0; i < kTcK / 256; ++i)
+                    if (m + mm < p.M) *reinterpret_cast<uint4 *>(s_xw + (size_t)(m + mm) * kTcPitch + lane * 8 + 256 * i) = v[mm][i];
         }
         __syncwarp();
         if (!mbar_wait(bar, (uint32_t)round & 1u)) {
             dead = true;
             break;
         }
-        const uint32_t *arow = reinterpret_cast<const uint32_t *>(s_Aw + (size_t)g * kAPitch);
-        const uint32_t *xa = reinterpret_cast<const uint32_t *>(s_xw + (size_t)g * kAPitch);
+        const uint32_t *arow = reinterpret_cast<const uint32_t *>(s_Aw + (size_t)g * kTcPitch);
+        const uint32_t *xa = reinterpret_cast<const uint32_t *>(s_xw + (size_t)g * kTcPitch);
         const bool col_ok = g < nrows, ra_ok = g < p.M;
         float d[4][4];
 #pragma unroll
@@ -1844,7 +1846,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         // t from a few CTAs at the head of the grid (M <= 4; over all of K, whatever the K slices): then the others hold no A
         pl.n_t = 0;
         if (a.rank > 0 && a.M <= kTMmaMaxM && !g_t_late && tune.t_ctas != 0) {
-            const int nblocks = ((a.K + kTUnitK - 1) / kTUnitK) * ((a.rank + 7) / 8);      // over all of K
+            const int nblocks = ((a.K + kTcK - 1) / kTcK) * ((a.rank + 7) / 8);            // over all of K
             pl.n_t = min(12, (nblocks + kTWarps - 1) / kTWarps);
             pl.a_cap = 0;
             tu_max = 0;
@@ -1898,7 +1900,7 @@ Plan make_plan(const LinearArgs &a, const DecodeTuning &tune)
         pl.NS = ns_want;
         while (pl.NS > 2 && off + (size_t)pl.NS * pl.stage_bytes > budget) --pl.NS;
         off += (size_t)pl.NS * pl.stage_bytes;
-        if (pl.n_t > 0) off = max(off, (size_t)1024 + (size_t)kTWarps * (8 + a.M) * kAPitch * 2);   // what a t CTA needs
+        if (pl.n_t > 0) off = max(off, (size_t)1024 + (size_t)kTWarps * (8 + a.M) * kTcPitch * 2);  // what a t CTA needs
         pl.smem = off;
         return nseg_max <= kMaxSeg && pl.smem <= budget;
     };
