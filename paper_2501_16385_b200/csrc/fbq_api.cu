@@ -24,6 +24,8 @@ std::atomic<long long> g_launches{0};
 struct Options {
     int force_kernel = -1;
     DecodeTuning decode;
+    GemvTuning gemv;
+    int use_gemv = 1;
     int decode_t_late = 0;
     int decode_t_wait = 1;
     int batch_ctas = 400;
@@ -122,6 +124,25 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
     int launches = 0;
     cudaError_t e = cudaSuccess;
 
+    if (kernel == FBQ_KERNEL_DECODE && g_opt.use_gemv && gemv_supported(a)) {
+        GemvTuning gt = g_opt.gemv;
+        gt.pdl = g_opt.decode.pdl;
+        if (tune.max_ctas > 0) gt.max_ctas = tune.max_ctas;
+        size_t pf = 0;
+        int nc = 0;
+        gemv_workspace_need(a, gt, &pf, &nc);
+        size_t have_c = (size_t)ws->n_counters;
+        if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        ws->n_counters = (int)have_c;
+        e = launch_gemv(a, *ws, gt, s, &launches);
+        if (e == cudaSuccess) {
+            g_launches += launches;
+            return FBQ_OK;
+        }
+        if (e != cudaErrorInvalidConfiguration) return FBQ_ERR_CUDA;
+        (void)cudaGetLastError();                 // no plan fits: the other decode kernel
+    }
     if (kernel == FBQ_KERNEL_DECODE) {
         size_t pf = 0;
         int nc = 0;
@@ -179,6 +200,10 @@ int *option_slot(const char *name)
 {
     if (!name) return nullptr;
     if (!strcmp(name, "force_kernel")) return &g_opt.force_kernel;
+    if (!strcmp(name, "gemv")) return &g_opt.use_gemv;
+    if (!strcmp(name, "gemv_ctas")) return &g_opt.gemv.max_ctas;
+    if (!strcmp(name, "t_poll_limit")) return &g_opt.gemv.poll_limit;
+    if (!strcmp(name, "test_skip_t_arrive")) return &g_opt.gemv.test_skip_arrive;
     if (!strcmp(name, "decode_sk")) return &g_opt.decode.sk;
     if (!strcmp(name, "decode_chunk")) return &g_opt.decode.chunk;
     if (!strcmp(name, "decode_depth")) return &g_opt.decode.depth;

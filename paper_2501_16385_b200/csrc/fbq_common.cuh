@@ -84,6 +84,17 @@ cudaError_t launch_decode(const LinearArgs &a, Workspace &ws, const DecodeTuning
 void decode_workspace_need(const LinearArgs &a, const DecodeTuning &tune, size_t *partial_floats,
                            int *counters);
 
+// The streaming decode kernel (fbq_gemv.cu).
+struct GemvTuning {
+    int max_ctas = 0;          // 0: one main CTA per SM
+    int pdl = 1;
+    int poll_limit = 0;        // 0: default number of looks at the "t complete" counter
+    int test_skip_arrive = 0;  // test switch: the t CTAs do not report their arrival (the wait for t must run out)
+};
+bool gemv_supported(const LinearArgs &a);
+void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters);
+cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tune, cudaStream_t s, int *launches);
+
 int decode_batch_max();
 bool decode_batch_need(const LinearArgs *a, int count, const int *ctas, const DecodeTuning &tune, size_t *partial_floats,
                        size_t *t_floats, int *counters);

@@ -1,0 +1,924 @@
+// Streaming decode kernel (few tokens) of the FBQuant linear, sm_100a.
+//
+// One launch computes  y = x.dequant(Q,s,z)^T + (x.A^T).B^T  (Algorithm 1 step 6 of the paper;
+// Section 4.3 fuses dequantisation, main product and up-projection and leaves t = x.A^T to a second
+// launch; here t comes from a few CTAs of the same grid).  The kernel is built around what a launch
+// of a few microseconds costs besides streaming its weights:
+//
+//   * Everything that comes from the WEIGHTS (packed codes, scales, zero points, B, A) is requested
+//     before the kernel waits for the preceding kernel of its stream (programmatic dependent
+//     launch); a CTA takes half an SM's shared memory at most, so the CTAs of the next launch are
+//     resident and prefetching while this launch still computes.
+//   * No table is built per CTA: scales and zero points of a 16-row tile arrive as they are stored
+//     (two bulk copies per tile) and are converted where they are used.
+//   * The weight stream is one TMA tensor copy per stage (16 groups x 16 rows of packed codes) into
+//     an mbarrier ring; eight compute warps share every stage.
+//
+// Main CTAs (one per SM by default) own contiguous ranges of 16-row tiles.  Integer form (M <= 2):
+// a code masked out of its word is an unsigned byte operand of the 8-bit integer MMA as it stands
+// (four codes per register, at most one shift per word); x is fixed point per group of 128 (three
+// signed base-256 digits, exact integer sums), and scale and zero point are applied per group to the
+// integer sums in fp32.  At M = 1 an MMA's eight columns hold the digits of TWO groups (columns 0-2
+// and 4-6), so the per-group fp32 work is done once per pair of groups.
+// The epilogue warp of a CTA adds the eight warps' partial tiles (fixed order), adds t.B^T on tensor
+// cores (t as two 16-bit terms, rows of B by TMA with the 128-byte swizzle), rounds once, stores y.
+//
+// t CTAs (the first n_t blocks of the grid): each holds a k-chunk of all rows of A (TMA, swizzled,
+// requested before the wait), multiplies it with its chunk of x on tensor cores and stores its
+// partial t to scratch; an arrival counter tells the main CTAs' epilogue warps when all chunks are
+// there (bounded polling; FBQ_ERR_TIMEOUT instead of a hang), which then add the chunks in order.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <mutex>
+#include <type_traits>
+#include <vector>
+
+#include "fbq_common.cuh"
+#include "fbq_ptx.cuh"
+
+namespace fbq {
+namespace {
+using namespace ptx;
+
+constexpr int kCW = 8;                       // compute warps of a main CTA
+constexpr int kEpiWarp = kCW;                // then the epilogue warp
+constexpr int kProdWarp = kCW + 1;           // and the producer warp
+constexpr int kWarps = kCW + 2;
+constexpr int kThreads = kWarps * 32;
+constexpr int kTile = 16;                    // weight rows of a tile
+constexpr int kCHG = 16;                     // quantisation groups of a stage
+constexpr int kMaxNS = 8, kMaxBuf = 8, kMaxB = 4, kMaxMeta = 8;
+constexpr int kTKB = 64;                     // k extent of one block of A in a t CTA (128 bytes: the swizzle span)
+constexpr uint32_t kZeroBytes = 1024;        // zeros that lanes without a digit column read instead
+
+struct GemvParams {
+    const void *x;
+    const __half *scales;
+    const __half *zeros;
+    void *y;
+    float *tpart;       // [n_t][M][rank] partial sums of t, one slot per t CTA
+    int *ctr;           // [0] t CTAs arrived, [1] main CTAs that have read t; both zero on entry and exit
+    int *status;        // receives FBQ_ERR_TIMEOUT when a bounded wait runs out
+    int M, N, K, G, rank;
+    int NT;             // tiles
+    int n_t, n_main;
+    int t_kb;           // blocks of kTKB input channels per t CTA
+    int NS, nbuf, nmeta, nb;
+    int stage_bytes, meta_pitch, b_slot_bytes, b_box_cols, b_swz;
+    int off_bar, off_tab, off_zero, off_x, off_meta, off_seg, off_t, off_B, off_ring;
+    int off_tA, off_tred;                   // t CTA: blocks of A, reduction buffer
+    uint32_t poll_limit;                    // looks at the arrival counter before giving up
+    int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
+};
+
+// barrier slots (8 bytes each) from off_bar
+constexpr int kBarFull = 0, kBarEmpty = kMaxNS, kBarSegFull = 2 * kMaxNS, kBarSegFree = 2 * kMaxNS + kMaxBuf,
+              kBarB = 2 * kMaxNS + 2 * kMaxBuf, kBarA = kBarB + kMaxB, kNumBars = kBarA + 1;
+
+// ------------------------------------------------- integer form: codes as bytes
+// A 3- or 4-bit code masked out of its word where it sits is the unsigned byte q * 2^j (j = the
+// field's offset inside its byte): an operand of the 8-bit integer MMA as it stands.
+//   INT4 word i:  r[2i]   = w & 0x0F0F0F0F          codes 8i+0, 8i+2, 8i+4, 8i+6
+//                 r[2i+1] = w & 0xF0F0F0F0          codes 8i+1, 8i+3, 8i+5, 8i+7   (x 16)
+//   INT3 word i:  r[3i]   = w & 0x0E070E07          codes 10i+0, 10i+3 (x 2), 10i+5, 10i+8 (x 2)
+//                 r[3i+1] = w & 0x70387038          codes 10i+1 (x 8), 10i+4 (x 16), 10i+6 (x 8), 10i+9 (x 16)
+//                 r[3i+2] = (w >> 6) & 0x02070207   codes 10i+2, bit i of code 30 (x 2), 10i+7, bit i of code 31 (x 2)
+// (The three bits of the bit-sliced codes 30 and 31 are operands of their own: 36 byte slots per 32
+// codes.  With and-masks alone no layout of 32 three-bit codes in three words gets by with 32 slots: a
+// byte lane holds two whole fields and two spare bits, and the spare bits of different bytes cannot
+// meet in one lane.)
+template <int BITS> struct Slots {
+    static constexpr int kRegs = (BITS == 4) ? 8 : 9;
+    static constexpr int kWords = (BITS == 4) ? 4 : 3;
+    // code (0..31) of a lane's run whose value sits in byte j of register R
+    static __host__ __device__ constexpr int code(int R, int j)
+    {
+        if (BITS == 4) return 8 * (R >> 1) + 2 * j + (R & 1);
+        const int i = R / 3, f = R % 3;
+        if (f == 2 && (j & 1)) return 30 + (j >> 1);
+        return 10 * i + 5 * (j >> 1) + f + 3 * (j & 1);
+    }
+    // log2 of the factor x is stored with in that slot
+    static __host__ __device__ constexpr int scale_log2(int R, int j)
+    {
+        if (BITS == 4) return (R & 1) ? -4 : 0;
+        const int i = R / 3, f = R % 3;
+        if (f == 2) return (j & 1) ? i - 1 : 0;
+        if (f == 1) return (j & 1) ? -4 : -3;
+        return (j & 1) ? -1 : 0;
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *r)
+    {
+        if (BITS == 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                r[2 * i] = w[i] & 0x0F0F0F0Fu;
+                r[2 * i + 1] = w[i] & 0xF0F0F0F0u;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                r[3 * i] = w[i] & 0x0E070E07u;
+                r[3 * i + 1] = w[i] & 0x70387038u;
+                r[3 * i + 2] = (w[i] >> 6) & 0x02070207u;
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ float half_bits_to_float(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)v)); }
+
+__device__ __forceinline__ void give_up(const GemvParams &p) { atomicExch(p.status, (int)FBQ_ERR_TIMEOUT); }
+
+// ------------------------------------------------------------------ x, integer form
+// x of all K for M tokens as fixed point per group of 128: 2^e puts the group's largest |x| into
+// [2^20, 2^21); per byte slot X = rint(x 2^e 2^-j) (the slot's factor undone) as three signed
+// base-256 digits, X = d0 2^16 + d1 2^8 + d2 (the bytes of (X + 0x808080) ^ 0x808080).  Digit i of
+// token m is MMA column 4m + i (M = 2) or 4 (group parity) + i (M = 1).  Layout in shared memory:
+// 16-byte units [group][register quad 0..1][column 3m+i][lane t] (registers 4p..4p+3 of the
+// unpacked codes), then one word per [group][column][lane t] for register 8 of INT3.  The table
+// holds, per (group, token), two float4: (2^-e 2^16, 2^-e 2^8, sum of x, 0) for the lanes that hold
+// digits 0 and 1 and (2^-e, 0, 0, 0) for the lanes that hold digit 2.  A group with a non-finite x
+// gets NaN there, so that its outputs are NaN as the definition says.
+template <int BITS, typename T, int M>
+__device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, int warp, int lane)
+{
+    constexpr int NR = Slots<BITS>::kRegs;
+    constexpr int ncol = 3 * M;
+    const T *x = static_cast<const T *>(p.x);
+    float4 *s_tab = reinterpret_cast<float4 *>(smem + p.off_tab);
+    uint4 *s_x8 = reinterpret_cast<uint4 *>(smem + p.off_x);
+    uint32_t *s_xt = reinterpret_cast<uint32_t *>(smem + p.off_x) + (size_t)p.G * 2 * ncol * 16;
+    const int runs_per_tok = p.K / 32, nruns = M * runs_per_tok;           // multiples of 4
+    const int upper = warp & 1;
+    if ((p.G & 1) && warp == 0 && lane < 2 * M) s_tab[(size_t)p.G * M * 2 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < nruns; base += (kCW / 2) * 32) {
+        const int idx = base + (warp >> 1) * 32 + lane;                    // whole quads are valid or not
+        const bool valid = idx < nruns;
+        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+        uint4 xv[4];
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + run * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
+        float xf[32];
+        float amax = 0.f, xsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            T xe;
+            *reinterpret_cast<uint16_t *>(&xe) = e[c];
+            xf[c] = ActTraits<T>::to_float(xe);
+            amax = fmaxf(amax, fabsf(xf[c]));
+            xsum += xf[c];
+        }
+        // the four runs of one (token, group) sit in four consecutive lanes
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+        const bool finite = (amax <= 3.0e38f) && (fabsf(xsum) <= 3.4e38f);                // false for Inf and NaN
+        const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 32u), 230u);           // biased exponent of the maximum
+        const float xs = __uint_as_float((274u - ex) << 23);                            // 2^(20 - floor(log2 max))
+        if (valid && !upper && (run & 3) == 0) {
+            const float inv = finite ? __uint_as_float((ex - 20u) << 23) : __uint_as_float(0x7fc00000u);   // 1 / xs
+            float4 *row = s_tab + ((size_t)(run >> 2) * M + m) * 2;
+            row[0] = make_float4(inv * 65536.f, inv * 256.f, xsum, 0.f);
+            row[1] = make_float4(inv, 0.f, 0.f, 0.f);
+        }
+        auto make = [&](auto rbeg, auto rend) {
+            constexpr int R0 = decltype(rbeg)::value, R1 = decltype(rend)::value;
+            uint32_t dg[R1 - R0][3];
+#pragma unroll
+            for (int R = R0; R < R1; ++R) {
+                uint32_t v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    constexpr float kPow[7] = {1.f / 16.f, 1.f / 8.f, 1.f / 4.f, 1.f / 2.f, 1.f, 2.f, 4.f};
+                    const float f = xs * kPow[Slots<BITS>::scale_log2(R, j) + 4];
+                    const int X = __float2int_rn(xf[Slots<BITS>::code(R, j)] * f);
+                    v[j] = ((uint32_t)X + 0x00808080u) ^ 0x00808080u;
+                }
+                // digit i of the four slots -> one register (byte j = slot j)
+                const uint32_t lo01 = __byte_perm(v[0], v[1], 0x5140), lo23 = __byte_perm(v[2], v[3], 0x5140);
+                dg[R - R0][2] = __byte_perm(lo01, lo23, 0x5410);
+                dg[R - R0][1] = __byte_perm(lo01, lo23, 0x7632);
+                dg[R - R0][0] = __byte_perm(__byte_perm(v[0], v[1], 0x0062), __byte_perm(v[2], v[3], 0x0062), 0x5410);
+            }
+            if (valid) {
+                const int gl = run >> 2, lq = run & 3;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const int col = 3 * m + k;
+                    s_x8[(size_t)((gl * 2 + R0 / 4) * ncol + col) * 4 + lq] = make_uint4(dg[0][k], dg[1][k], dg[2][k], dg[3][k]);
+                    if constexpr (R1 - R0 == 5) s_xt[(size_t)(gl * ncol + col) * 4 + lq] = dg[4][k];
+                }
+            }
+        };
+        if (!upper) make(std::integral_constant<int, 0>{}, std::integral_constant<int, 4>{});
+        else make(std::integral_constant<int, 4>{}, std::integral_constant<int, NR>{});
+    }
+}
+
+// --------------------------------------------------------------- compute warps, integer form
+template <int BITS, typename T, int M>
+__device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, int warp, int lane, int tile_first, int ntile)
+{
+    constexpr int NR = Slots<BITS>::kRegs, NW = Slots<BITS>::kWords;
+    constexpr int GB = (BITS == 4) ? 64 : 48;                  // bytes of one group of one row
+    constexpr int ncol = 3 * M;
+    constexpr uint32_t x_gstride = 2u * ncol * 64u;            // bytes of one group's 16-byte units
+    constexpr uint32_t x_chunk1 = ncol * 64u;                  // second register quad
+    constexpr uint32_t xt_gstride = ncol * 16u;
+    const int g = lane >> 2, tq = lane & 3;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + p.off_bar;
+    const int G = p.G, NS = p.NS, SPT = (G + kCHG - 1) / kCHG;
+
+    // ---- per-lane constants.  As an MMA column, this lane is n = g: column block n >> 2 (group parity at
+    // M = 1, token at M = 2), digit n & 3 (3 = no digit: reads zeros).  As an accumulator lane it holds
+    // columns 2tq, 2tq+1: block tq >> 1, digits (0, 1) or (2, none).
+    const int nb = g >> 2, nc = g & 3;
+    const bool has_digit = nc < 3;
+    const uint32_t zero = sbase + p.off_zero;
+    const uint32_t x8 = sbase + p.off_x, xt8 = x8 + (uint32_t)G * x_gstride;
+    uint32_t xa, xb = 0, xsa, xsb = 0, xt, xts;
+    uint32_t tmask0 = 0xffffffffu, tmask1 = 0u;
+    if (M == 1) {
+        // pair of groups (a, b): group a in block 0, group b in block 1
+        xa = (has_digit && nb == 0) ? x8 + (uint32_t)nc * 64u + tq * 16u : zero + tq * 16u;
+        xsa = (has_digit && nb == 0) ? 2u * x_gstride : 0u;
+        xb = (has_digit && nb == 1) ? x8 + x_gstride + (uint32_t)nc * 64u + tq * 16u : zero + tq * 16u;
+        xsb = (has_digit && nb == 1) ? 2u * x_gstride : 0u;
+        xt = has_digit ? xt8 + (uint32_t)nb * xt_gstride + (uint32_t)nc * 16u + tq * 4u : zero;
+        xts = has_digit ? 2u * xt_gstride : 0u;
+        tmask0 = (nb == 0) ? 0xffffffffu : 0u;
+        tmask1 = ~tmask0;
+    } else {
+        xa = has_digit ? x8 + (uint32_t)(3 * nb + nc) * 64u + tq * 16u : zero + tq * 16u;
+        xsa = has_digit ? x_gstride : 0u;
+        xt = has_digit ? xt8 + (uint32_t)(3 * nb + nc) * 16u + tq * 4u : zero;
+        xts = has_digit ? xt_gstride : 0u;
+    }
+    const int ablk = tq >> 1, apar = tq & 1;
+    const uint32_t tab = sbase + p.off_tab + (uint32_t)((M == 1 ? 0 : ablk * 2) + apar) * 16u;     // + group index * (M * 32)
+    const uint32_t w_lane = sbase + p.off_ring + (uint32_t)(g * GB + tq * (GB / 4));
+    const uint32_t meta0 = sbase + p.off_meta;
+    const uint32_t zoff = (uint32_t)p.meta_pitch, row8 = (uint32_t)(8 * G * 2);
+    float *s_seg = reinterpret_cast<float *>(smem + p.off_seg);
+
+    auto load_words = [&](uint32_t wa, uint32_t (&wr)[NW]) {
+        if constexpr (BITS == 4) {
+            const uint4 v = lds_v4(wa);
+            wr[0] = v.x; wr[1] = v.y; wr[2] = v.z; wr[3] = v.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < NW; ++i) wr[i] = lds_u32(wa + 4 * i);
+        }
+    };
+    // the first eight registers of one group's codes (rows g and g + 8) against its digits: four MMAs
+    auto mma8 = [&](int (&d)[4], const uint32_t (&ra)[NR], const uint32_t (&rb)[NR], uint32_t xaddr) {
+        const uint4 x0 = lds_v4(xaddr), x1 = lds_v4(xaddr + x_chunk1);
+        mma_u8s8(d, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
+        mma_u8s8(d, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
+        mma_u8s8(d, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
+        mma_u8s8(d, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
+    };
+    // scale, zero point and the weights of the digits: integer sums of one block -> fp32
+    auto scale = [&](const int (&d)[4], uint32_t tabaddr, uint32_t maddr, float (&acc)[2]) {
+        const float4 tb = lds_f4(tabaddr);
+        const float sg = half_bits_to_float(lds_u16(maddr)), zg = half_bits_to_float(lds_u16(maddr + zoff));
+        const float sh = half_bits_to_float(lds_u16(maddr + row8)), zh = half_bits_to_float(lds_u16(maddr + row8 + zoff));
+        float fg = fmaf((float)d[1], tb.y, (float)d[0] * tb.x);
+        float fh = fmaf((float)d[3], tb.y, (float)d[2] * tb.x);
+        fg = fmaf(-zg, tb.z, fg);
+        fh = fmaf(-zh, tb.z, fh);
+        acc[0] = fmaf(sg, fg, acc[0]);
+        acc[1] = fmaf(sh, fh, acc[1]);
+    };
+
+    int it = 0;
+    for (int ts = 0; ts < ntile; ++ts) {
+        float acc[2] = {0.f, 0.f};
+        const uint32_t mslot = meta0 + (uint32_t)(ts % p.nmeta) * 2u * zoff + (uint32_t)(g * G * 2);
+        for (int st = 0; st < SPT; ++st, ++it) {
+            const int slot = it % NS;
+            if (!mbar_wait(bars + 8u * (kBarFull + slot), (uint32_t)(it / NS) & 1u)) return false;
+            const uint32_t ws = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes;
+            if constexpr (M == 1) {
+                const int pi = st * (kCHG / 2) + warp;                    // pair of the tile
+                const int ga = 2 * pi;
+                if (ga < G) {
+                    const uint32_t wa = ws + (uint32_t)(2 * warp) * (kTile * GB);
+                    uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
+                    int d[4] = {0, 0, 0, 0};
+                    load_words(wa, w0);
+                    load_words(wa + 8 * GB, w1);
+                    Slots<BITS>::run(w0, ra);
+                    Slots<BITS>::run(w1, rb);
+                    mma8(d, ra, rb, xa + (uint32_t)pi * xsa);
+                    uint32_t ta = 0, tb2 = 0;
+                    if constexpr (BITS == 3) {
+                        ta = ra[8];
+                        tb2 = rb[8];
+                    }
+                    load_words(wa + kTile * GB, w0);
+                    load_words(wa + kTile * GB + 8 * GB, w1);
+                    Slots<BITS>::run(w0, ra);
+                    Slots<BITS>::run(w1, rb);
+                    mma8(d, ra, rb, xb + (uint32_t)pi * xsb);
+                    if constexpr (BITS == 3) {
+                        const uint32_t tv = lds_u32(xt + (uint32_t)pi * xts);
+                        mma_u8s8(d, ta, tb2, ra[8], rb[8], tv & tmask0, tv & tmask1);
+                    }
+                    const int grp = min(ga + ablk, G - 1);
+                    scale(d, tab + (uint32_t)(ga + ablk) * 32u, mslot + (uint32_t)grp * 2u, acc);
+                }
+            } else {
+#pragma unroll 1
+                for (int u = 0; u < 2; ++u) {
+                    const int gi = 2 * warp + u, grp = st * kCHG + gi;
+                    if (grp >= G) break;
+                    const uint32_t wa = ws + (uint32_t)gi * (kTile * GB);
+                    uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
+                    int d[4] = {0, 0, 0, 0};
+                    load_words(wa, w0);
+                    load_words(wa + 8 * GB, w1);
+                    Slots<BITS>::run(w0, ra);
+                    Slots<BITS>::run(w1, rb);
+                    mma8(d, ra, rb, xa + (uint32_t)grp * xsa);
+                    if constexpr (BITS == 3) mma_u8s8(d, ra[8], rb[8], 0u, 0u, lds_u32(xt + (uint32_t)grp * xts), 0u);
+                    scale(d, tab + (uint32_t)grp * 64u, mslot + (uint32_t)grp * 2u, acc);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+        }
+        // ---- this warp's partial tile: add the lanes of a block (and, at M = 1, both blocks) ----
+        acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], 1);
+        acc[1] += __shfl_xor_sync(0xffffffffu, acc[1], 1);
+        if (M == 1) {
+            acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], 2);
+            acc[1] += __shfl_xor_sync(0xffffffffu, acc[1], 2);
+        }
+        const int buf = ts % p.nbuf;
+        if (ts >= p.nbuf && !mbar_wait(bars + 8u * (kBarSegFree + buf), (uint32_t)(ts / p.nbuf - 1) & 1u)) return false;
+        if (apar == 0 && ablk < M) {
+            float *dst = s_seg + ((size_t)(buf * kCW + warp) * M + ablk) * kTile;
+            dst[g] = acc[0];
+            dst[g + 8] = acc[1];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFull + buf));
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------ producer
+__device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, const CUtensorMap *wmap, int tile_first, int ntile)
+{
+    const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
+    const uint32_t ring = sbase + p.off_ring, meta0 = sbase + p.off_meta;
+    const int SPT = (p.G + kCHG - 1) / kCHG, NS = p.NS;
+    int it = 0;
+    for (int ts = 0; ts < ntile; ++ts) {
+        const int tile = tile_first + ts;
+        const int rows = min(kTile, p.N - tile * kTile);
+        const uint32_t mbytes = (uint32_t)rows * (uint32_t)p.G * 2u;
+        for (int st = 0; st < SPT; ++st, ++it) {
+            const int slot = it % NS;
+            if (it >= NS && !mbar_wait_idle(bars + 8u * (kBarEmpty + slot), (uint32_t)(it / NS - 1) & 1u)) return false;
+            const uint32_t full = bars + 8u * (kBarFull + slot);
+            mbar_expect_tx(full, (uint32_t)p.stage_bytes + (st == 0 ? 2u * mbytes : 0u));
+            // one box of 16 groups x 16 rows (rows past N and groups past G arrive as zeros)
+            tma_load_3d(ring + (uint32_t)slot * (uint32_t)p.stage_bytes, wmap, 0, tile * kTile, st * kCHG, full);
+            if (st == 0) {
+                const uint32_t ms = meta0 + (uint32_t)(ts % p.nmeta) * 2u * (uint32_t)p.meta_pitch;
+                const size_t off = (size_t)tile * kTile * p.G;
+                bulk_g2s(ms, p.scales + off, mbytes, full);
+                bulk_g2s(ms + (uint32_t)p.meta_pitch, p.zeros + off, mbytes, full);
+            }
+        }
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------ epilogue warp
+// Swizzled byte offset inside a tile that TMA wrote with the 32-, 64- or 128-byte swizzle
+// (mask 1, 3, 7): the 16-byte unit index is XOR-ed with the 128-byte line index.
+__device__ __forceinline__ uint32_t swz(uint32_t off, uint32_t mask) { return off ^ (((off >> 7) & mask) << 4); }
+
+template <typename T>
+__device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, const CUtensorMap *bmap, int lane, int tile_first, int ntile)
+{
+    const int g = lane >> 2, tq = lane & 3;
+    const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
+    const uint32_t bring = sbase + p.off_B;
+    const int rank = p.rank, M = p.M, nkb = rank / 16;
+    const int nbox = (rank + 63) / 64;
+    const uint32_t box_bytes = (uint32_t)kTile * (uint32_t)p.b_box_cols * 2u;
+    auto request_b = [&](int ts) {
+        const uint32_t bar = bars + 8u * (kBarB + ts % p.nb);
+        mbar_expect_tx(bar, (uint32_t)nbox * box_bytes);
+        for (int b = 0; b < nbox; ++b)
+            tma_load_2d(bring + (uint32_t)(ts % p.nb) * (uint32_t)p.b_slot_bytes + (uint32_t)b * box_bytes, bmap, b * 64,
+                        (tile_first + ts) * kTile, bar);
+    };
+    if (rank > 0 && lane == 0)
+        for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
+
+    pdl_wait();
+
+    // ---- t: wait for the t CTAs, add their chunks in order, keep t as MMA column operands ----
+    uint32_t tfrag[8][2];
+    float isc = 1.f;
+    if (rank > 0) {
+        bool ok = false;
+        for (uint32_t i = 0; i < p.poll_limit; ++i) {
+            int seen = 0;
+            if (lane == 0) seen = ld_acquire(p.ctr);
+            seen = __shfl_sync(0xffffffffu, seen, 0);
+            if (seen >= p.n_t) {
+                ok = true;
+                break;
+            }
+            __nanosleep(100);
+        }
+        if (!ok) return false;
+        float *s_t = reinterpret_cast<float *>(smem + p.off_t);
+        float amax = 0.f;
+        for (int i = lane; i < M * rank; i += 32) {
+            float v = 0.f;
+            for (int c = 0; c < p.n_t; ++c) v += __ldcg(p.tpart + (size_t)c * M * rank + i);
+            s_t[i] = v;
+            amax = fmaxf(amax, fabsf(v));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        __syncwarp();
+        // every main CTA tells when it has read t; the last one leaves the counters at zero
+        if (lane == 0) {
+            __threadfence();
+            if (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) {
+                atomicExch(p.ctr, 0);
+                atomicExch(p.ctr + 1, 0);
+            }
+        }
+        // a power of two that puts the largest |t| near 2^14 keeps both terms inside fp16
+        const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 1u), 254u);
+        const uint32_t sb = min(max(268u - ex, 1u), 254u);
+        const float sc = __uint_as_float(sb << 23);
+        isc = __uint_as_float((254u - sb) << 23);
+        const int tok = g >> 1, part = g & 1;        // as an MMA column: token and (rounded value | remainder)
+#pragma unroll
+        for (int kb = 0; kb < 8; ++kb) {
+            tfrag[kb][0] = tfrag[kb][1] = 0u;
+            if (kb < nkb && tok < M) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t pk = 0;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float v = s_t[tok * rank + kb * 16 + h * 8 + 2 * tq + e] * sc;
+                        const T hi = ActTraits<T>::from_float(v);
+                        const T lo = ActTraits<T>::from_float(v - ActTraits<T>::to_float(hi));
+                        const T pick = part ? lo : hi;
+                        pk |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&pick)) << (16 * e);
+                    }
+                    tfrag[kb][h] = pk;
+                }
+            }
+        }
+    }
+
+    const float *s_seg = reinterpret_cast<const float *>(smem + p.off_seg);
+    T *y = static_cast<T *>(p.y);
+    const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
+    for (int ts = 0; ts < ntile; ++ts) {
+        const int buf = ts % p.nbuf;
+        if (!mbar_wait_idle(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
+        float vg = 0.f, vh = 0.f;
+        if (tq < M) {
+            const float *src = s_seg + ((size_t)buf * kCW * M + tq) * kTile;
+#pragma unroll
+            for (int w = 0; w < kCW; ++w) {
+                vg += src[(size_t)w * M * kTile + g];
+                vh += src[(size_t)w * M * kTile + g + 8];
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
+        if (rank > 0) {
+            const int bs = ts % p.nb;
+            if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
+            const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
+            float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kb = 0; kb < 8; ++kb) {
+                if (kb < nkb) {
+                    const uint32_t bx = bt + (uint32_t)(kb >> 2) * box_bytes;
+                    const uint32_t c0 = (uint32_t)((kb & 3) * 32 + tq * 4);               // bytes into the row
+                    const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                    const uint32_t a0 = lds_u32(bx + swz(o0, smask)), a1 = lds_u32(bx + swz(o1, smask));
+                    const uint32_t a2 = lds_u32(bx + swz(o0 + 16u, smask)), a3 = lds_u32(bx + swz(o1 + 16u, smask));
+                    Mma16<T>::run(d, a0, a1, a2, a3, tfrag[kb][0], tfrag[kb][1]);
+                }
+            }
+            vg = fmaf(d[0] + d[1], isc, vg);
+            vh = fmaf(d[2] + d[3], isc, vh);
+            __syncwarp();
+            if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
+        }
+        const int n = (tile_first + ts) * kTile + g;
+        if (tq < M) {
+            if (n < p.N) y[(size_t)tq * p.N + n] = ActTraits<T>::from_float(vg);
+            if (n + 8 < p.N) y[(size_t)tq * p.N + n + 8] = ActTraits<T>::from_float(vh);
+        }
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------ t CTA
+// Block c of the first n_t: t_kb blocks of 64 input channels of all `rank` rows of A in shared memory
+// (TMA, 128-byte swizzle), against the same channels of x read straight from global memory as MMA
+// column operands (tokens are columns).  Warps take the 64-channel blocks round-robin; the eight
+// warps' sums are added in warp order and stored to slot c of tpart.
+template <typename T>
+__device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const CUtensorMap *amap, int c)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    const uint32_t sbase = smem_u32(smem), bar = sbase + p.off_bar + 8u * kBarA;
+    const uint32_t sA = sbase + p.off_tA;
+    const int rank = p.rank, M = p.M, nrb = rank / 16;
+    const int kb0 = c * p.t_kb, nkb = max(0, min(p.t_kb, (p.K + kTKB - 1) / kTKB - kb0));
+    const uint32_t blk_bytes = (uint32_t)rank * 128u;
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        fence_barrier_init();
+        if (nkb > 0) {
+            mbar_expect_tx(bar, (uint32_t)nkb * blk_bytes);
+            for (int b = 0; b < nkb; ++b) tma_load_2d(sA + (uint32_t)b * blk_bytes, amap, (kb0 + b) * kTKB, 0, bar);
+        }
+    }
+    __syncthreads();
+    pdl_wait();
+    float *s_red = reinterpret_cast<float *>(smem + p.off_tred);      // [warp][rank][8 columns]
+    const T *x = static_cast<const T *>(p.x);
+    bool dead = false;
+    for (int tb = 0; tb < (M + 7) / 8; ++tb) {
+        float acc[8][4];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+        const int tok = tb * 8 + g;
+        if (warp < kCW) {
+            for (int b = warp; b < nkb; b += kCW) {
+                uint32_t xb[4][2];
+                const int k0 = (kb0 + b) * kTKB;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const int k = k0 + ks * 16 + 2 * tq;
+                    const bool v = tok < M && k < p.K;
+                    xb[ks][0] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k)) : 0u;
+                    xb[ks][1] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k + 8)) : 0u;
+                }
+                if (!dead && !mbar_wait(bar, 0)) dead = true;
+                if (dead) break;
+                const uint32_t ab = sA + (uint32_t)b * blk_bytes;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    if (r < nrb) {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
+                            Mma16<T>::run(acc[r], lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)),
+                                          lds_u32(ab + swz(o0 + 16u, 7u)), lds_u32(ab + swz(o1 + 16u, 7u)), xb[ks][0], xb[ks][1]);
+                        }
+                    }
+                }
+            }
+            // rows r*16 + g (and + 8) of A, columns 2tq, 2tq+1 (tokens)
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r < nrb) {
+                    float *dst = s_red + ((size_t)warp * rank + r * 16 + g) * 8 + 2 * tq;
+                    dst[0] = acc[r][0];
+                    dst[1] = acc[r][1];
+                    dst[64] = acc[r][2];
+                    dst[65] = acc[r][3];
+                }
+            }
+        }
+        __syncthreads();
+        const int ntok = min(8, M - tb * 8);
+        for (int i = tid; i < ntok * rank; i += kThreads) {
+            const int m = i / rank, j = i - m * rank;
+            float v = 0.f;
+#pragma unroll
+            for (int w = 0; w < kCW; ++w) v += s_red[((size_t)w * rank + j) * 8 + m];
+            p.tpart[((size_t)c * M + tb * 8 + m) * rank + j] = v;
+        }
+        __syncthreads();
+    }
+    if (dead && lane == 0) give_up(p);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0 && !p.test_skip_arrive) atomicAdd(p.ctr, 1);
+}
+
+// ------------------------------------------------------------------------ kernel
+template <int BITS, typename T, int M>
+__global__ void __launch_bounds__(kThreads, 2)
+gemv_kernel(const __grid_constant__ GemvParams p, const __grid_constant__ CUtensorMap wmap,
+            const __grid_constant__ CUtensorMap bmap, const __grid_constant__ CUtensorMap amap)
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);     // the swizzled tiles want 1024-byte alignment
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // the CTAs of the next launch on this stream may become resident as soon as all of ours are
+    pdl_launch_dependents();
+    if ((int)blockIdx.x < p.n_t) {
+        t_cta<T>(p, smem, &amap, (int)blockIdx.x);
+        return;
+    }
+    const int cta = (int)blockIdx.x - p.n_t;
+    const int tile_first = (int)((long long)cta * p.NT / p.n_main);
+    const int ntile = (int)((long long)(cta + 1) * p.NT / p.n_main) - tile_first;
+    const uint32_t bars = smem_u32(smem) + p.off_bar;
+    if (tid == 0) {
+        prefetch_tensormap(&wmap);
+        if (p.rank > 0) prefetch_tensormap(&bmap);
+        for (int i = 0; i < p.NS; ++i) {
+            mbar_init(bars + 8u * (kBarFull + i), 1);
+            mbar_init(bars + 8u * (kBarEmpty + i), kCW);
+        }
+        for (int i = 0; i < p.nbuf; ++i) {
+            mbar_init(bars + 8u * (kBarSegFull + i), kCW);
+            mbar_init(bars + 8u * (kBarSegFree + i), 1);
+        }
+        for (int i = 0; i < p.nb; ++i) mbar_init(bars + 8u * (kBarB + i), 1);
+        fence_barrier_init();
+    }
+    for (uint32_t i = tid; i < kZeroBytes / 4; i += kThreads) reinterpret_cast<uint32_t *>(smem + p.off_zero)[i] = 0u;
+    __syncthreads();
+
+    bool ok = true;
+    if (warp == kProdWarp) {
+        if (lane == 0) ok = produce(p, smem, &wmap, tile_first, ntile);
+    } else if (warp == kEpiWarp) {
+        ok = epilogue<T>(p, smem, &bmap, lane, tile_first, ntile);
+    } else {
+        pdl_wait();                                  // x may come from the preceding kernel
+        convert_x<BITS, T, M>(p, smem, warp, lane);
+        named_barrier_sync(1, kCW * 32);
+        ok = compute_i8<BITS, T, M>(p, smem, warp, lane, tile_first, ntile);
+    }
+    if (!ok && lane == 0) give_up(p);
+}
+
+// ------------------------------------------------------------------ host side
+template <typename X> struct TypeTag { using type = X; };
+
+struct Plan {
+    GemvParams p;
+    size_t smem;
+    bool ok;
+};
+
+int g_sm_count = 0;
+constexpr size_t kSmemHalf = 113 * 1024;     // two CTAs (this launch and the next one) fit on an SM
+constexpr size_t kSmemMax = 227 * 1024;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
+{
+    Plan pl{};
+    pl.ok = false;
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return pl;
+        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return pl;
+    }
+    GemvParams &p = pl.p;
+    const int GB = (a.bits == 4) ? 64 : 48, G = a.K / kGroupFast;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.G = G; p.rank = a.rank;
+    p.NT = (a.N + kTile - 1) / kTile;
+    int want = tune.max_ctas > 0 ? tune.max_ctas : g_sm_count;
+    p.n_main = std::max(1, std::min(want, p.NT));
+    const int nseg = (p.NT + p.n_main - 1) / p.n_main;
+    const int SPT = (G + kCHG - 1) / kCHG;
+    p.stage_bytes = kTile * kCHG * GB;
+    p.meta_pitch = (int)align_up((size_t)kTile * G * 2, 16);
+    // t CTAs: chunks of A of at most 64 KB
+    p.n_t = 0;
+    p.t_kb = 0;
+    const int nblk = (a.K + kTKB - 1) / kTKB;
+    if (a.rank > 0) {
+        const int per = std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128)));
+        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
+        p.t_kb = (nblk + p.n_t - 1) / p.n_t;
+        p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
+    }
+    p.b_box_cols = a.rank <= 16 ? 16 : (a.rank <= 32 ? 32 : 64);      // columns past the rank arrive as zeros
+    p.b_swz = p.b_box_cols >= 64 ? 7 : (p.b_box_cols >= 32 ? 3 : 1);
+    p.b_slot_bytes = (int)align_up((size_t)((a.rank + 63) / 64) * kTile * p.b_box_cols * 2, 1024);
+    p.nbuf = std::min(kMaxBuf, std::max(2, nseg));
+    p.nb = a.rank > 0 ? std::min(kMaxB, std::max(1, nseg)) : 0;
+    const int ncol = 3 * a.M;
+    auto layout = [&](int ns) {
+        p.NS = ns;
+        p.nmeta = std::min(kMaxMeta, (ns - 1) / SPT + 2);
+        size_t off = 0;
+        p.off_bar = (int)off;
+        off += (size_t)kNumBars * 8;
+        off = align_up(off, 16);
+        p.off_tab = (int)off;
+        off += (size_t)(G + 1) * a.M * 32;
+        off = align_up(off, 128);
+        p.off_zero = (int)off;
+        off += kZeroBytes;
+        p.off_x = (int)off;
+        off += (size_t)G * ncol * (a.bits == 4 ? 128 : 144);
+        off = align_up(off, 128);
+        p.off_meta = (int)off;
+        off += (size_t)p.nmeta * 2 * p.meta_pitch;
+        off = align_up(off, 128);
+        p.off_seg = (int)off;
+        off += (size_t)p.nbuf * kCW * a.M * kTile * 4;
+        off = align_up(off, 128);
+        p.off_t = (int)off;
+        off += (size_t)a.M * a.rank * 4;
+        off = align_up(off, 1024);
+        p.off_B = (int)off;
+        off += (size_t)p.nb * p.b_slot_bytes;
+        off = align_up(off, 1024);
+        p.off_ring = (int)off;
+        off += (size_t)ns * p.stage_bytes;
+        return off;
+    };
+    // as many stages as half an SM's shared memory takes (at least three); else the whole SM
+    int ns = kMaxNS;
+    while (ns > 3 && layout(ns) > kSmemHalf) --ns;
+    size_t need = layout(ns);
+    if (need > kSmemHalf) {
+        ns = kMaxNS;
+        while (ns > 2 && layout(ns) > kSmemMax) --ns;
+        need = layout(ns);
+        if (need > kSmemMax) return pl;
+    }
+    // a t CTA: barriers, its blocks of A (1024-byte aligned), the reduction buffer
+    p.off_tA = 1024;
+    p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
+    const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
+    if (need_t > kSmemMax) return pl;
+    pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
+    p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
+    p.test_skip_arrive = tune.test_skip_arrive;
+    pl.ok = true;
+    if (getenv("FBQ_PLAN"))
+        fprintf(stderr, "gemv plan M %d N %d K %d r %d: n_main %d n_t %d (t_kb %d) NS %d nmeta %d nbuf %d nb %d smem %zu (t CTA %zu)\n",
+                a.M, a.N, a.K, a.rank, p.n_main, p.n_t, p.t_kb, p.NS, p.nmeta, p.nbuf, p.nb, need, need_t);
+    return pl;
+}
+
+// Tensor maps are encoded on the host once per (pointer, shape) and kept: they hold addresses and
+// extents only, never data.
+struct MapKey {
+    const void *ptr;
+    int kind, d0, d1, d2, b0, b1;
+    bool operator==(const MapKey &o) const
+    {
+        return ptr == o.ptr && kind == o.kind && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b0 == o.b0 && b1 == o.b1;
+    }
+};
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::mutex g_map_mu;
+std::vector<std::pair<MapKey, CUtensorMap>> g_maps;
+size_t g_map_next = 0;
+
+cudaError_t cached_map(CUtensorMap *out, const MapKey &key, CUtensorMapDataType dt, int ndim, const cuuint64_t *dims,
+                       const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swz_mode)
+{
+    std::lock_guard<std::mutex> lk(g_map_mu);
+    for (const auto &e : g_maps)
+        if (e.first == key) {
+            *out = e.second;
+            return cudaSuccess;
+        }
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (g_encode(out, dt, ndim, const_cast<void *>(key.ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz_mode,
+                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    constexpr size_t kKeep = 1024;
+    if (g_maps.size() < kKeep)
+        g_maps.emplace_back(key, *out);
+    else
+        g_maps[g_map_next++ % kKeep] = std::make_pair(key, *out);
+    return cudaSuccess;
+}
+
+template <int BITS, typename T, int M>
+cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &amap, bool pdl,
+                           cudaStream_t s)
+{
+    auto kern = gemv_kernel<BITS, T, M>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(pl.p.n_t + pl.p.n_main));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, pl.p, wmap, bmap, amap);
+}
+
+}  // namespace
+
+bool gemv_supported(const LinearArgs &a)
+{
+    if (a.group != kGroupFast || a.K % kGroupFast != 0 || a.K < kGroupFast) return false;
+    if (a.M < 1 || a.M > 2) return false;
+    if (a.N % 8 != 0 || a.N < 8) return false;
+    if (a.rank % 16 != 0 || a.rank > 128) return false;
+    auto mis16 = [](const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
+    if (mis16(a.scales) || mis16(a.zeros)) return false;
+    return true;
+}
+
+void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters)
+{
+    const Plan pl = make_plan(a, tune);
+    *tpart_floats = (size_t)std::max(pl.p.n_t, 1) * a.M * std::max(a.rank, 1);
+    *counters = 8;
+}
+
+cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tune, cudaStream_t s, int *launches)
+{
+    Plan pl = make_plan(a, tune);
+    if (!pl.ok) return cudaErrorInvalidConfiguration;
+    GemvParams &p = pl.p;
+    p.x = a.x; p.scales = a.scales; p.zeros = a.zeros; p.y = a.y;
+    p.tpart = ws.partial;
+    p.ctr = ws.counters;
+    p.status = ws.counters + kCtrStatus;
+    CUtensorMap wmap, bmap, amap;
+    {
+        const cuuint32_t wpg = (a.bits == 4) ? 16 : 12;
+        const cuuint64_t dims[3] = {wpg, (cuuint64_t)a.N, (cuuint64_t)p.G};
+        const cuuint64_t strides[2] = {(cuuint64_t)p.G * wpg * 4, (cuuint64_t)wpg * 4};
+        const cuuint32_t box[3] = {wpg, (cuuint32_t)kTile, (cuuint32_t)kCHG};
+        const MapKey key{a.qw, 0, (int)wpg, a.N, p.G, kTile, kCHG};
+        if (cudaError_t e = cached_map(&wmap, key, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+            e != cudaSuccess)
+            return e;
+    }
+    bmap = wmap;
+    amap = wmap;
+    if (a.rank > 0) {
+        const cuuint64_t bd[2] = {(cuuint64_t)a.rank, (cuuint64_t)a.N}, bs[1] = {(cuuint64_t)a.rank * 2};
+        const cuuint32_t bb[2] = {(cuuint32_t)p.b_box_cols, (cuuint32_t)kTile};
+        const CUtensorMapSwizzle sw = p.b_swz == 7 ? CU_TENSOR_MAP_SWIZZLE_128B : (p.b_swz == 3 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        const CUtensorMapDataType dt = a.bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+        if (cudaError_t e = cached_map(&bmap, MapKey{a.B, 1, a.rank, a.N, a.bf16, p.b_box_cols, kTile}, dt, 2, bd, bs, bb, sw); e != cudaSuccess)
+            return e;
+        const cuuint64_t ad[2] = {(cuuint64_t)a.K, (cuuint64_t)a.rank}, as[1] = {(cuuint64_t)a.K * 2};
+        const cuuint32_t ab[2] = {(cuuint32_t)kTKB, (cuuint32_t)a.rank};
+        if (cudaError_t e = cached_map(&amap, MapKey{a.A, 2, a.K, a.rank, a.bf16, kTKB, a.rank}, dt, 2, ad, as, ab, CU_TENSOR_MAP_SWIZZLE_128B);
+            e != cudaSuccess)
+            return e;
+    }
+    const bool pdl = tune.pdl != 0;
+    cudaError_t e = cudaErrorInvalidConfiguration;
+    auto go = [&](auto bits, auto type) {
+        using T = typename decltype(type)::type;
+        constexpr int B = decltype(bits)::value;
+        return a.M == 1 ? launch_variant<B, T, 1>(pl, wmap, bmap, amap, pdl, s) : launch_variant<B, T, 2>(pl, wmap, bmap, amap, pdl, s);
+    };
+    if (a.bits == 4)
+        e = a.bf16 ? go(std::integral_constant<int, 4>{}, TypeTag<__nv_bfloat16>{}) : go(std::integral_constant<int, 4>{}, TypeTag<__half>{});
+    else
+        e = a.bf16 ? go(std::integral_constant<int, 3>{}, TypeTag<__nv_bfloat16>{}) : go(std::integral_constant<int, 3>{}, TypeTag<__half>{});
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
+
+}  // namespace fbq
