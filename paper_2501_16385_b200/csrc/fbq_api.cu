@@ -34,7 +34,7 @@ struct Options {
     int prefill_split = 1;
     int decode_trace = 0;
 } g_opt;
-constexpr size_t kTraceBytes = 512 * 10 * 16 * 8;   // 512 CTAs x 10 warps x 16 marks
+constexpr size_t kTraceBytes = 512 * 18 * 16 * 8;   // 512 CTAs x up to 18 warps x 16 marks
 
 bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -132,9 +132,13 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         int nc = 0;
         gemv_workspace_need(a, gt, &pf, &nc);
         size_t have_c = (size_t)ws->n_counters;
-        if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->tslots, ws->tslots_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
         ws->n_counters = (int)have_c;
+        if (g_opt.decode_trace && !ws->trace) {
+            if (cudaMalloc(&ws->trace, kTraceBytes) != cudaSuccess) return FBQ_ERR_CUDA;
+            cudaMemset(ws->trace, 0, kTraceBytes);
+        }
         e = launch_gemv(a, *ws, gt, s, &launches);
         if (e == cudaSuccess) {
             g_launches += launches;
@@ -202,6 +206,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "force_kernel")) return &g_opt.force_kernel;
     if (!strcmp(name, "gemv")) return &g_opt.use_gemv;
     if (!strcmp(name, "gemv_ctas")) return &g_opt.gemv.max_ctas;
+    if (!strcmp(name, "gemv_dbg")) return &g_opt.gemv.dbg;
     if (!strcmp(name, "t_poll_limit")) return &g_opt.gemv.poll_limit;
     if (!strcmp(name, "test_skip_t_arrive")) return &g_opt.gemv.test_skip_arrive;
     if (!strcmp(name, "decode_sk")) return &g_opt.decode.sk;
@@ -565,6 +570,7 @@ int fbq_poll_status(void *stream)
         // a kernel gave up half way: its bookkeeping is unfinished, start from a clean slate
         cudaMemset(ws->counters, 0, sizeof(int) * (size_t)ws->n_counters);
         if (ws->t) cudaMemset(ws->t, 0, sizeof(float) * ws->t_floats);
+        if (ws->tslots) cudaMemset(ws->tslots, 0, sizeof(float) * ws->tslots_floats);
     }
     return st;
 }
@@ -587,6 +593,7 @@ int fbq_release_workspaces(void)
         cudaFree(w.partial);
         cudaFree(w.t);
         cudaFree(w.t_gen);
+        cudaFree(w.tslots);
         cudaFree(w.counters);
         cudaFree(w.trace);
         cudaFree(w.stage_x);

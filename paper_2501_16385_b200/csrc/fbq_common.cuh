@@ -33,6 +33,8 @@ struct Workspace {
     size_t partial_floats = 0;
     float *t = nullptr;           // down-projection t = x.A^T, [M][rank] fp32 (kept zero between calls)
     float *t_gen = nullptr;       // t of the generic path (no invariant), grows on demand
+    float *tslots = nullptr;      // streaming decode kernel: tagged partial sums of t (all zero between calls)
+    size_t tslots_floats = 0;
     size_t t_floats = 0, t_gen_floats = 0;
     int *counters = nullptr;      // [0]=t arrivals [1]=retired tiles [2]=status [3]=t ready [4]=parked; [8..] per tile
     int n_counters = 0;
@@ -89,6 +91,7 @@ struct GemvTuning {
     int max_ctas = 0;          // 0: one main CTA per SM
     int pdl = 1;
     int poll_limit = 0;        // 0: default number of looks at the "t complete" counter
+    int dbg = 0;
     int test_skip_arrive = 0;  // test switch: the t CTAs do not report their arrival (the wait for t must run out)
 };
 bool gemv_supported(const LinearArgs &a);

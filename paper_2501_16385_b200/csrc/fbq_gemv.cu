@@ -43,13 +43,17 @@ namespace fbq {
 namespace {
 using namespace ptx;
 
-constexpr int kCW = 8;                       // compute warps of a main CTA
+#ifndef FBQ_GEMV_CW
+#define FBQ_GEMV_CW 8
+#endif
+constexpr int kCW = FBQ_GEMV_CW;             // compute warps of a main CTA
+constexpr int kCtasPerSm = (kCW <= 8) ? 2 : 1;   // CTAs of consecutive launches that share an SM
 constexpr int kEpiWarp = kCW;                // then the epilogue warp
 constexpr int kProdWarp = kCW + 1;           // and the producer warp
 constexpr int kWarps = kCW + 2;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTile = 16;                    // weight rows of a tile
-constexpr int kCHG = 16;                     // quantisation groups of a stage
+constexpr int kCHG = 2 * kCW;                // quantisation groups of a stage (one pair per compute warp at M = 1)
 constexpr int kMaxNS = 8, kMaxBuf = 8, kMaxB = 4, kMaxMeta = 8;
 constexpr int kTKB = 64;                     // k extent of one block of A in a t CTA (128 bytes: the swizzle span)
 constexpr uint32_t kZeroBytes = 1024;        // zeros that lanes without a digit column read instead
@@ -59,8 +63,9 @@ struct GemvParams {
     const __half *scales;
     const __half *zeros;
     void *y;
-    float *tpart;       // [n_t][M][rank] partial sums of t, one slot per t CTA
-    int *ctr;           // [0] t CTAs arrived, [1] main CTAs that have read t; both zero on entry and exit
+    float2 *tpart;      // [n_t][M][rank] partial sums of t, one slot per t CTA, each entry (value, tag): tag 1.0f = written by
+                        // this launch; all tags are zero on entry and on exit
+    int *ctr;           // [1] main CTAs that have read t; zero on entry and exit
     int *status;        // receives FBQ_ERR_TIMEOUT when a bounded wait runs out
     int M, N, K, G, rank;
     int NT;             // tiles
@@ -72,11 +77,14 @@ struct GemvParams {
     int off_tA, off_tred;                   // t CTA: blocks of A, reduction buffer
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
+    int dbg;
+    unsigned long long *trace;              // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
 
 // barrier slots (8 bytes each) from off_bar
 constexpr int kBarFull = 0, kBarEmpty = kMaxNS, kBarSegFull = 2 * kMaxNS, kBarSegFree = 2 * kMaxNS + kMaxBuf,
-              kBarB = 2 * kMaxNS + 2 * kMaxBuf, kBarA = kBarB + kMaxB, kNumBars = kBarA + 1;
+              kBarB = 2 * kMaxNS + 2 * kMaxBuf, kBarA = kBarB + kMaxB, kBarXReq = kBarA + 1, kNumBars = kBarXReq + 1;
+constexpr int kEarlyStages = 1;               // weight stages requested before the loads of x are on their way
 
 // ------------------------------------------------- integer form: codes as bytes
 // A 3- or 4-bit code masked out of its word where it sits is the unsigned byte q * 2^j (j = the
@@ -131,6 +139,21 @@ template <int BITS> struct Slots {
 
 __device__ __forceinline__ float half_bits_to_float(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)v)); }
 
+// Tuning aid: the global timer (ns) of this warp at a phase.
+__device__ __forceinline__ void mark(const GemvParams &p, int slot)
+{
+    if (p.trace && (threadIdx.x & 31) == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = t;
+    }
+}
+
+__device__ __forceinline__ void markc(const GemvParams &p, int slot)
+{
+    if (p.trace && (threadIdx.x & 31) == 0) p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = (unsigned long long)clock64();
+}
+
 __device__ __forceinline__ void give_up(const GemvParams &p) { atomicExch(p.status, (int)FBQ_ERR_TIMEOUT); }
 
 // ------------------------------------------------------------------ x, integer form
@@ -146,6 +169,10 @@ __device__ __forceinline__ void give_up(const GemvParams &p) { atomicExch(p.stat
 template <int BITS, typename T, int M>
 __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, int warp, int lane)
 {
+    // Two lanes share a 32-element run of x (the k range of lane t of one group): the even lane makes
+    // the digits of registers 0..3, the odd lane the rest.  Each takes half of the run for the group's
+    // maximum and sum (the eight lanes of a group sit side by side), and converts only the elements
+    // its own slots need.
     constexpr int NR = Slots<BITS>::kRegs;
     constexpr int ncol = 3 * M;
     const T *x = static_cast<const T *>(p.x);
@@ -153,36 +180,46 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     uint4 *s_x8 = reinterpret_cast<uint4 *>(smem + p.off_x);
     uint32_t *s_xt = reinterpret_cast<uint32_t *>(smem + p.off_x) + (size_t)p.G * 2 * ncol * 16;
     const int runs_per_tok = p.K / 32, nruns = M * runs_per_tok;           // multiples of 4
-    const int upper = warp & 1;
     if ((p.G & 1) && warp == 0 && lane < 2 * M) s_tab[(size_t)p.G * M * 2 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int base = 0; base < nruns; base += (kCW / 2) * 32) {
-        const int idx = base + (warp >> 1) * 32 + lane;                    // whole quads are valid or not
+    const int upper = lane & 1;
+#pragma unroll 1
+    for (int base = 0; base < nruns; base += kCW * 16) {
+        const int idx = base + warp * 16 + (lane >> 1);                     // whole groups of eight lanes are valid or not
         const bool valid = idx < nruns;
         const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
         uint4 xv[4];
         const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + run * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        if (base == 0) {                                                     // our loads of x are on their way
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);
+        }
+        if (p.trace && base == 0 && (xv[0].x ^ xv[1].y ^ xv[2].z ^ xv[3].w) != 0x12345677u) mark(p, 9);
         const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
         float xf[32];
-        float amax = 0.f, xsum = 0.f;
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
             T xe;
             *reinterpret_cast<uint16_t *>(&xe) = e[c];
-            xf[c] = ActTraits<T>::to_float(xe);
-            amax = fmaxf(amax, fabsf(xf[c]));
-            xsum += xf[c];
+            xf[c] = ActTraits<T>::to_float(xe);                              // only those that are used below survive
         }
-        // the four runs of one (token, group) sit in four consecutive lanes
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+        float amax = 0.f, xsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const float v = upper ? xf[16 + c] : xf[c];
+            amax = fmaxf(amax, fabsf(v));
+            xsum += v;
+        }
+#pragma unroll
+        for (int o = 1; o < 8; o <<= 1) {
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+        }
         const bool finite = (amax <= 3.0e38f) && (fabsf(xsum) <= 3.4e38f);                // false for Inf and NaN
         const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 32u), 230u);           // biased exponent of the maximum
         const float xs = __uint_as_float((274u - ex) << 23);                            // 2^(20 - floor(log2 max))
-        if (valid && !upper && (run & 3) == 0) {
+        if (valid && (lane & 7) == 0) {
             const float inv = finite ? __uint_as_float((ex - 20u) << 23) : __uint_as_float(0x7fc00000u);   // 1 / xs
             float4 *row = s_tab + ((size_t)(run >> 2) * M + m) * 2;
             row[0] = make_float4(inv * 65536.f, inv * 256.f, xsum, 0.f);
@@ -198,8 +235,9 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
                 for (int j = 0; j < 4; ++j) {
                     constexpr float kPow[7] = {1.f / 16.f, 1.f / 8.f, 1.f / 4.f, 1.f / 2.f, 1.f, 2.f, 4.f};
                     const float f = xs * kPow[Slots<BITS>::scale_log2(R, j) + 4];
-                    const int X = __float2int_rn(xf[Slots<BITS>::code(R, j)] * f);
-                    v[j] = ((uint32_t)X + 0x00808080u) ^ 0x00808080u;
+                    // rint(x f) for |x f| < 2^22 sits in the low bits of x f + 1.5 2^23 (round to nearest even by the FMA)
+                    const uint32_t X = __float_as_uint(fmaf(xf[Slots<BITS>::code(R, j)], f, 12582912.f));
+                    v[j] = (X + 0x00408080u) ^ 0x00808080u;                  // low 24 bits: (X + 0x808080) ^ 0x808080
                 }
                 // digit i of the four slots -> one register (byte j = slot j)
                 const uint32_t lo01 = __byte_perm(v[0], v[1], 0x5140), lo23 = __byte_perm(v[2], v[3], 0x5140);
@@ -242,26 +280,24 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
     // columns 2tq, 2tq+1: block tq >> 1, digits (0, 1) or (2, none).
     const int nb = g >> 2, nc = g & 3;
     const bool has_digit = nc < 3;
-    const uint32_t zero = sbase + p.off_zero;
     const uint32_t x8 = sbase + p.off_x, xt8 = x8 + (uint32_t)G * x_gstride;
-    uint32_t xa, xb = 0, xsa, xsb = 0, xt, xts;
-    uint32_t tmask0 = 0xffffffffu, tmask1 = 0u;
+    // lanes without a digit column, and (M = 1) lanes of the other group's block, load nothing and hold zeros
+    uint32_t xa, xb = 0, xt;
+    uint32_t pa, pb = 0u;
+    constexpr uint32_t xsa = (M == 1) ? 2u * x_gstride : x_gstride, xts = (M == 1) ? 2u * xt_gstride : xt_gstride;
     if (M == 1) {
         // pair of groups (a, b): group a in block 0, group b in block 1
-        xa = (has_digit && nb == 0) ? x8 + (uint32_t)nc * 64u + tq * 16u : zero + tq * 16u;
-        xsa = (has_digit && nb == 0) ? 2u * x_gstride : 0u;
-        xb = (has_digit && nb == 1) ? x8 + x_gstride + (uint32_t)nc * 64u + tq * 16u : zero + tq * 16u;
-        xsb = (has_digit && nb == 1) ? 2u * x_gstride : 0u;
-        xt = has_digit ? xt8 + (uint32_t)nb * xt_gstride + (uint32_t)nc * 16u + tq * 4u : zero;
-        xts = has_digit ? 2u * xt_gstride : 0u;
-        tmask0 = (nb == 0) ? 0xffffffffu : 0u;
-        tmask1 = ~tmask0;
+        pa = (has_digit && nb == 0) ? 1u : 0u;
+        pb = (has_digit && nb == 1) ? 1u : 0u;
+        xa = x8 + (uint32_t)nc * 64u + tq * 16u;
+        xb = xa + x_gstride;
+        xt = xt8 + (uint32_t)nb * xt_gstride + (uint32_t)nc * 16u + tq * 4u;
     } else {
-        xa = has_digit ? x8 + (uint32_t)(3 * nb + nc) * 64u + tq * 16u : zero + tq * 16u;
-        xsa = has_digit ? x_gstride : 0u;
-        xt = has_digit ? xt8 + (uint32_t)(3 * nb + nc) * 16u + tq * 4u : zero;
-        xts = has_digit ? xt_gstride : 0u;
+        pa = has_digit ? 1u : 0u;
+        xa = x8 + (uint32_t)(3 * nb + nc) * 64u + tq * 16u;
+        xt = xt8 + (uint32_t)(3 * nb + nc) * 16u + tq * 4u;
     }
+    const uint32_t pt = has_digit ? 1u : 0u;
     const int ablk = tq >> 1, apar = tq & 1;
     const uint32_t tab = sbase + p.off_tab + (uint32_t)((M == 1 ? 0 : ablk * 2) + apar) * 16u;     // + group index * (M * 32)
     const uint32_t w_lane = sbase + p.off_ring + (uint32_t)(g * GB + tq * (GB / 4));
@@ -279,92 +315,51 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
         }
     };
     // the first eight registers of one group's codes (rows g and g + 8) against its digits: four MMAs
-    auto mma8 = [&](int (&d)[4], const uint32_t (&ra)[NR], const uint32_t (&rb)[NR], uint32_t xaddr) {
-        const uint4 x0 = lds_v4(xaddr), x1 = lds_v4(xaddr + x_chunk1);
-        mma_u8s8(d, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
-        mma_u8s8(d, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
-        mma_u8s8(d, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
-        mma_u8s8(d, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
+    // in two independent chains
+    auto mma8 = [&](int (&d0)[4], int (&d1)[4], const uint32_t (&ra)[NR], const uint32_t (&rb)[NR], const uint4 &x0, const uint4 &x1) {
+        mma_u8s8(d0, ra[0], rb[0], ra[1], rb[1], x0.x, x0.y);
+        mma_u8s8(d1, ra[2], rb[2], ra[3], rb[3], x0.z, x0.w);
+        mma_u8s8(d0, ra[4], rb[4], ra[5], rb[5], x1.x, x1.y);
+        mma_u8s8(d1, ra[6], rb[6], ra[7], rb[7], x1.z, x1.w);
     };
     // scale, zero point and the weights of the digits: integer sums of one block -> fp32
-    auto scale = [&](const int (&d)[4], uint32_t tabaddr, uint32_t maddr, float (&acc)[2]) {
-        const float4 tb = lds_f4(tabaddr);
-        const float sg = half_bits_to_float(lds_u16(maddr)), zg = half_bits_to_float(lds_u16(maddr + zoff));
-        const float sh = half_bits_to_float(lds_u16(maddr + row8)), zh = half_bits_to_float(lds_u16(maddr + row8 + zoff));
-        float fg = fmaf((float)d[1], tb.y, (float)d[0] * tb.x);
-        float fh = fmaf((float)d[3], tb.y, (float)d[2] * tb.x);
-        fg = fmaf(-zg, tb.z, fg);
-        fh = fmaf(-zh, tb.z, fh);
+    struct Meta {
+        float4 tb;
+        uint32_t sg, zg, sh, zh;
+    };
+    auto load_meta = [&](uint32_t tabaddr, uint32_t maddr) {
+        Meta m;
+        m.tb = lds_f4(tabaddr);
+        m.sg = lds_u16(maddr);
+        m.zg = lds_u16(maddr + zoff);
+        m.sh = lds_u16(maddr + row8);
+        m.zh = lds_u16(maddr + row8 + zoff);
+        return m;
+    };
+    auto scale = [&](const int (&d)[4], const Meta &m, float (&acc)[2]) {
+        const float sg = half_bits_to_float(m.sg), zg = half_bits_to_float(m.zg);
+        const float sh = half_bits_to_float(m.sh), zh = half_bits_to_float(m.zh);
+        float fg = fmaf((float)d[1], m.tb.y, (float)d[0] * m.tb.x);
+        float fh = fmaf((float)d[3], m.tb.y, (float)d[2] * m.tb.x);
+        fg = fmaf(-zg, m.tb.z, fg);
+        fh = fmaf(-zh, m.tb.z, fh);
         acc[0] = fmaf(sg, fg, acc[0]);
         acc[1] = fmaf(sh, fh, acc[1]);
     };
 
-    int it = 0;
-    for (int ts = 0; ts < ntile; ++ts) {
-        float acc[2] = {0.f, 0.f};
-        const uint32_t mslot = meta0 + (uint32_t)(ts % p.nmeta) * 2u * zoff + (uint32_t)(g * G * 2);
-        for (int st = 0; st < SPT; ++st, ++it) {
-            const int slot = it % NS;
-            if (!mbar_wait(bars + 8u * (kBarFull + slot), (uint32_t)(it / NS) & 1u)) return false;
-            const uint32_t ws = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes;
-            if constexpr (M == 1) {
-                const int pi = st * (kCHG / 2) + warp;                    // pair of the tile
-                const int ga = 2 * pi;
-                if (ga < G) {
-                    const uint32_t wa = ws + (uint32_t)(2 * warp) * (kTile * GB);
-                    uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
-                    int d[4] = {0, 0, 0, 0};
-                    load_words(wa, w0);
-                    load_words(wa + 8 * GB, w1);
-                    Slots<BITS>::run(w0, ra);
-                    Slots<BITS>::run(w1, rb);
-                    mma8(d, ra, rb, xa + (uint32_t)pi * xsa);
-                    uint32_t ta = 0, tb2 = 0;
-                    if constexpr (BITS == 3) {
-                        ta = ra[8];
-                        tb2 = rb[8];
-                    }
-                    load_words(wa + kTile * GB, w0);
-                    load_words(wa + kTile * GB + 8 * GB, w1);
-                    Slots<BITS>::run(w0, ra);
-                    Slots<BITS>::run(w1, rb);
-                    mma8(d, ra, rb, xb + (uint32_t)pi * xsb);
-                    if constexpr (BITS == 3) {
-                        const uint32_t tv = lds_u32(xt + (uint32_t)pi * xts);
-                        mma_u8s8(d, ta, tb2, ra[8], rb[8], tv & tmask0, tv & tmask1);
-                    }
-                    const int grp = min(ga + ablk, G - 1);
-                    scale(d, tab + (uint32_t)(ga + ablk) * 32u, mslot + (uint32_t)grp * 2u, acc);
-                }
-            } else {
-#pragma unroll 1
-                for (int u = 0; u < 2; ++u) {
-                    const int gi = 2 * warp + u, grp = st * kCHG + gi;
-                    if (grp >= G) break;
-                    const uint32_t wa = ws + (uint32_t)gi * (kTile * GB);
-                    uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
-                    int d[4] = {0, 0, 0, 0};
-                    load_words(wa, w0);
-                    load_words(wa + 8 * GB, w1);
-                    Slots<BITS>::run(w0, ra);
-                    Slots<BITS>::run(w1, rb);
-                    mma8(d, ra, rb, xa + (uint32_t)grp * xsa);
-                    if constexpr (BITS == 3) mma_u8s8(d, ra[8], rb[8], 0u, 0u, lds_u32(xt + (uint32_t)grp * xts), 0u);
-                    scale(d, tab + (uint32_t)grp * 64u, mslot + (uint32_t)grp * 2u, acc);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
-        }
-        // ---- this warp's partial tile: add the lanes of a block (and, at M = 1, both blocks) ----
+    // this warp's partial tile: add the lanes of a block (and, at M = 1, both blocks), hand it to the epilogue warp
+    int dep_buf = 0;
+    uint32_t dep_phase = 1u;                       // parity of the buffer's previous use; unused while dep_first
+    bool dep_first = true;
+    auto deposit = [&](int ts, float (&acc)[2]) -> bool {
         acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], 1);
         acc[1] += __shfl_xor_sync(0xffffffffu, acc[1], 1);
         if (M == 1) {
             acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], 2);
             acc[1] += __shfl_xor_sync(0xffffffffu, acc[1], 2);
         }
-        const int buf = ts % p.nbuf;
-        if (ts >= p.nbuf && !mbar_wait(bars + 8u * (kBarSegFree + buf), (uint32_t)(ts / p.nbuf - 1) & 1u)) return false;
+        const int buf = dep_buf;
+        if (!dep_first && !mbar_wait(bars + 8u * (kBarSegFree + buf), dep_phase)) return false;
         if (apar == 0 && ablk < M) {
             float *dst = s_seg + ((size_t)(buf * kCW + warp) * M + ablk) * kTile;
             dst[g] = acc[0];
@@ -372,6 +367,170 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFull + buf));
+        mark(p, ts == 0 ? 5 : 6);
+        acc[0] = acc[1] = 0.f;
+        if (++dep_buf == p.nbuf) {
+            dep_buf = 0;
+            dep_phase = dep_first ? 0u : dep_phase ^ 1u;
+            dep_first = false;
+        }
+        return true;
+    };
+
+    if constexpr (M == 1) {
+        // One pass = one pair of groups (a, b) of one tile: group a in column block 0, group b in block 1.
+        // Software pipeline over the passes of all tiles: the packed words of the NEXT pass are loaded
+        // while the MMAs of this one are in flight, and the per-group fp32 work follows those loads.
+        const int total = ntile * SPT;
+        const uint32_t woff = (uint32_t)(2 * warp) * (kTile * GB);
+        uint32_t wa0[NW], wa1[NW], wb0[NW], wb1[NW];
+        auto load_pass = [&](int slot) {
+#ifdef HX_NOW
+            for (int i = 0; i < NW; ++i) { wa0[i] = slot * 7 + i; wa1[i] = slot * 11 + i; wb0[i] = slot * 13 + i; wb1[i] = slot * 17 + i; }
+            return;
+#endif
+            const uint32_t wa = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes + woff;
+            load_words(wa, wa0);
+            load_words(wa + 8 * GB, wa1);
+            load_words(wa + kTile * GB, wb0);
+            load_words(wa + kTile * GB + 8 * GB, wb1);
+        };
+        if (total > 0) {
+            if (!mbar_wait(bars + 8u * kBarFull, 0u)) return false;
+            mark(p, 4);
+            if (2 * warp < G) load_pass(0);
+        }
+        float acc[2] = {0.f, 0.f};
+        int ts = 0, st = 0, slot = 0, nslot = (NS > 1) ? 1 : 0;
+        uint32_t npar = (NS > 1) ? 0u : 1u;                           // parity of the next stage's first completion
+        uint32_t mslot = meta0 + (uint32_t)(g * G * 2);
+        int mi = 0;
+        for (int it = 0; it < total; ++it) {
+            const int pi = st * (kCHG / 2) + warp, ga = 2 * pi;
+            const bool live = ga < G;
+            Meta mt;
+            int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0}, d2[4] = {0, 0, 0, 0}, d3[4] = {0, 0, 0, 0};
+            if (live) {
+                const uint32_t xpa = xa + (uint32_t)pi * xsa, xpb = xb + (uint32_t)pi * xsa;
+#ifdef HX_NOX
+                const uint4 xa0 = make_uint4(xpa, xpa * 3, xpa * 5, xpa * 7), xa1 = xa0, xb0 = make_uint4(xpb, xpb * 3, xpb * 5, xpb * 7), xb1 = xb0;
+                uint32_t tv = xpa;
+#else
+                const uint4 xa0 = lds_v4_if(xpa, pa), xa1 = lds_v4_if(xpa + x_chunk1, pa);
+                const uint4 xb0 = lds_v4_if(xpb, pb), xb1 = lds_v4_if(xpb + x_chunk1, pb);
+                uint32_t tv = 0;
+                if constexpr (BITS == 3) tv = lds_u32_if(xt + (uint32_t)pi * xts, pt);
+#endif
+                const int grp = min(ga + ablk, G - 1);
+#ifdef HX_NOMETA
+                mt.tb = make_float4(1.f, 2.f, 3.f, 4.f); mt.sg = mt.zg = mt.sh = mt.zh = 0x3c00u + grp;
+#else
+                mt = load_meta(tab + (uint32_t)(ga + ablk) * 32u, mslot + (uint32_t)grp * 2u);
+#endif
+                uint32_t ra[NR], rb[NR];
+                Slots<BITS>::run(wa0, ra);
+                Slots<BITS>::run(wa1, rb);
+#ifdef HX_NOMMA
+                d0[0] = ra[0] ^ rb[1] ^ ra[2] ^ rb[3] ^ xa0.x; d1[1] = ra[4] ^ rb[5] ^ ra[6] ^ rb[7] ^ xa1.y;
+#else
+                mma8(d0, d1, ra, rb, xa0, xa1);
+#endif
+                uint32_t ta = 0, tb2 = 0;
+                if constexpr (BITS == 3) {
+                    ta = ra[8];
+                    tb2 = rb[8];
+                }
+                Slots<BITS>::run(wb0, ra);
+                Slots<BITS>::run(wb1, rb);
+#ifdef HX_NOMMA
+                d2[0] = ra[0] ^ rb[1] ^ ra[2] ^ rb[3] ^ xb0.x; d3[1] = ra[4] ^ rb[5] ^ ra[6] ^ rb[7] ^ xb1.y ^ ta ^ tb2 ^ ra[8] ^ rb[8] ^ tv;
+#else
+                mma8(d2, d3, ra, rb, xb0, xb1);
+                if constexpr (BITS == 3) mma_u8s8(d0, ta, tb2, ra[8], rb[8], nb == 0 ? tv : 0u, nb == 0 ? 0u : tv);
+#endif
+            }
+            // the next pass's words, while the MMAs run
+            int nst = st + 1, nts = ts;
+            if (nst == SPT) {
+                nst = 0;
+                ++nts;
+            }
+            if (it + 1 < total) {
+#ifndef HX_NOWAIT
+                if (!mbar_wait(bars + 8u * (kBarFull + nslot), npar)) return false;
+#endif
+                if (2 * (nst * (kCHG / 2) + warp) < G) load_pass(nslot);
+            }
+            if (live) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) d0[i] = (d0[i] + d1[i]) + (d2[i] + d3[i]);
+#ifdef HX_NOSCALE
+                acc[0] += (float)(d0[0] + d0[1]) + mt.tb.x + (float)mt.sg; acc[1] += (float)(d0[2] + d0[3]) + (float)mt.zh;
+#else
+                scale(d0, mt, acc);
+#endif
+            }
+#ifndef HX_NOWAIT
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+#endif
+            if (nts != ts) {
+                if (!deposit(ts, acc)) return false;
+                if (++mi == p.nmeta) mi = 0;
+                mslot = meta0 + (uint32_t)mi * 2u * zoff + (uint32_t)(g * G * 2);
+            }
+            st = nst;
+            ts = nts;
+            slot = nslot;
+            if (++nslot == NS) {
+                nslot = 0;
+                npar ^= 1u;
+            }
+        }
+    } else {
+        int slot = 0, mi = 0;
+        uint32_t par = 0u;
+        bool first = true;
+        for (int ts = 0; ts < ntile; ++ts) {
+            float acc[2] = {0.f, 0.f};
+            const uint32_t mslot = meta0 + (uint32_t)mi * 2u * zoff + (uint32_t)(g * G * 2);
+            if (++mi == p.nmeta) mi = 0;
+            for (int st = 0; st < SPT; ++st) {
+                if (!mbar_wait(bars + 8u * (kBarFull + slot), par)) return false;
+                if (first) mark(p, 4);
+                first = false;
+                const uint32_t ws = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes;
+#pragma unroll 1
+                for (int u = 0; u < 2; ++u) {
+                    const int gi = 2 * warp + u, grp = st * kCHG + gi;
+                    if (grp >= G) break;
+                    const uint32_t wa = ws + (uint32_t)gi * (kTile * GB);
+                    uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
+                    load_words(wa, w0);
+                    load_words(wa + 8 * GB, w1);
+                    const uint32_t xp = xa + (uint32_t)grp * xsa;
+                    const uint4 x0 = lds_v4_if(xp, pa), x1 = lds_v4_if(xp + x_chunk1, pa);
+                    uint32_t tv = 0;
+                    if constexpr (BITS == 3) tv = lds_u32_if(xt + (uint32_t)grp * xts, pt);
+                    const Meta mt = load_meta(tab + (uint32_t)grp * 64u, mslot + (uint32_t)grp * 2u);
+                    int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0};
+                    Slots<BITS>::run(w0, ra);
+                    Slots<BITS>::run(w1, rb);
+                    mma8(d0, d1, ra, rb, x0, x1);
+                    if constexpr (BITS == 3) mma_u8s8(d1, ra[8], rb[8], 0u, 0u, tv, 0u);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) d0[i] += d1[i];
+                    scale(d0, mt, acc);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+                if (++slot == NS) {
+                    slot = 0;
+                    par ^= 1u;
+                }
+            }
+            if (!deposit(ts, acc)) return false;
+        }
     }
     return true;
 }
@@ -389,11 +548,15 @@ __device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, cons
         const uint32_t mbytes = (uint32_t)rows * (uint32_t)p.G * 2u;
         for (int st = 0; st < SPT; ++st, ++it) {
             const int slot = it % NS;
+            // Until the compute warps have put their loads of x (which everything waits for) into the memory
+            // system, keep the prefetch shallow: x must not queue behind weights that cannot be used before it.
+            if (it == kEarlyStages && !mbar_wait_idle(bars + 8u * kBarXReq, 0u)) return false;
             if (it >= NS && !mbar_wait_idle(bars + 8u * (kBarEmpty + slot), (uint32_t)(it / NS - 1) & 1u)) return false;
             const uint32_t full = bars + 8u * (kBarFull + slot);
             mbar_expect_tx(full, (uint32_t)p.stage_bytes + (st == 0 ? 2u * mbytes : 0u));
             // one box of 16 groups x 16 rows (rows past N and groups past G arrive as zeros)
             tma_load_3d(ring + (uint32_t)slot * (uint32_t)p.stage_bytes, wmap, 0, tile * kTile, st * kCHG, full);
+            if (it == 0) mark(p, 3);
             if (st == 0) {
                 const uint32_t ms = meta0 + (uint32_t)(ts % p.nmeta) * 2u * (uint32_t)p.meta_pitch;
                 const size_t off = (size_t)tile * kTile * p.G;
@@ -402,6 +565,7 @@ __device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, cons
             }
         }
     }
+    mark(p, 6);
     return true;
 }
 
@@ -430,42 +594,44 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
 
     pdl_wait();
+    mark(p, 2);
 
     // ---- t: wait for the t CTAs, add their chunks in order, keep t as MMA column operands ----
     uint32_t tfrag[8][2];
     float isc = 1.f;
     if (rank > 0) {
-        bool ok = false;
-        for (uint32_t i = 0; i < p.poll_limit; ++i) {
-            int seen = 0;
-            if (lane == 0) seen = ld_acquire(p.ctr);
-            seen = __shfl_sync(0xffffffffu, seen, 0);
-            if (seen >= p.n_t) {
-                ok = true;
-                break;
-            }
-            __nanosleep(100);
-        }
-        if (!ok) return false;
+        // Look at the t CTAs' slots themselves until every entry carries this launch's tag (bounded), adding
+        // the chunks in slot order.
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
         float amax = 0.f;
-        for (int i = lane; i < M * rank; i += 32) {
-            float v = 0.f;
-            for (int c = 0; c < p.n_t; ++c) v += __ldcg(p.tpart + (size_t)c * M * rank + i);
-            s_t[i] = v;
-            amax = fmaxf(amax, fabsf(v));
+        const size_t slot_elems = (size_t)M * rank;
+        bool ok = false;
+        for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
+            bool all = true;
+            amax = 0.f;
+            for (int i = lane; i < M * rank; i += 32) {
+                float v = 0.f;
+                for (int c0 = 0; c0 < p.n_t; c0 += 8) {           // eight slots in flight
+                    float2 part[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v += part[u].x;
+                        all = all && (part[u].y == 1.f);
+                    }
+                }
+                s_t[i] = v;
+                amax = fmaxf(amax, fabsf(v));
+            }
+            ok = __all_sync(0xffffffffu, all);
+            if (!ok && look > 256) __nanosleep(64);
         }
+        if (!ok) return false;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         __syncwarp();
-        // every main CTA tells when it has read t; the last one leaves the counters at zero
-        if (lane == 0) {
-            __threadfence();
-            if (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) {
-                atomicExch(p.ctr, 0);
-                atomicExch(p.ctr + 1, 0);
-            }
-        }
         // a power of two that puts the largest |t| near 2^14 keeps both terms inside fp16
         const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 1u), 254u);
         const uint32_t sb = min(max(268u - ex, 1u), 254u);
@@ -493,12 +659,14 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         }
     }
 
+    mark(p, 3);
     const float *s_seg = reinterpret_cast<const float *>(smem + p.off_seg);
     T *y = static_cast<T *>(p.y);
     const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
     for (int ts = 0; ts < ntile; ++ts) {
         const int buf = ts % p.nbuf;
-        if (!mbar_wait_idle(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
+        if (!mbar_wait_idle_warp(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
+        if (ts == 0) mark(p, 4);
         float vg = 0.f, vh = 0.f;
         if (tq < M) {
             const float *src = s_seg + ((size_t)buf * kCW * M + tq) * kTile;
@@ -514,20 +682,31 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             const int bs = ts % p.nb;
             if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
             const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
-            float d[4] = {0.f, 0.f, 0.f, 0.f};
+            // four 16-wide blocks of the rank at a time: their rows of B first, then the MMAs (two chains)
+            float d[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int kb = 0; kb < 8; ++kb) {
-                if (kb < nkb) {
-                    const uint32_t bx = bt + (uint32_t)(kb >> 2) * box_bytes;
-                    const uint32_t c0 = (uint32_t)((kb & 3) * 32 + tq * 4);               // bytes into the row
-                    const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
-                    const uint32_t a0 = lds_u32(bx + swz(o0, smask)), a1 = lds_u32(bx + swz(o1, smask));
-                    const uint32_t a2 = lds_u32(bx + swz(o0 + 16u, smask)), a3 = lds_u32(bx + swz(o1 + 16u, smask));
-                    Mma16<T>::run(d, a0, a1, a2, a3, tfrag[kb][0], tfrag[kb][1]);
+            for (int kc = 0; kc < 2; ++kc) {
+                if (4 * kc < nkb) {
+                    uint32_t af[4][4];
+                    const uint32_t bx = bt + (uint32_t)kc * box_bytes;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+                        const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                        const bool on = 4 * kc + q < nkb;
+                        af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
+                        af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
+                        af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
+                        af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
+                    }
+                    Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tfrag[4 * kc][0], tfrag[4 * kc][1]);
+                    Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tfrag[4 * kc + 1][0], tfrag[4 * kc + 1][1]);
+                    Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tfrag[4 * kc + 2][0], tfrag[4 * kc + 2][1]);
+                    Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tfrag[4 * kc + 3][0], tfrag[4 * kc + 3][1]);
                 }
             }
-            vg = fmaf(d[0] + d[1], isc, vg);
-            vh = fmaf(d[2] + d[3], isc, vh);
+            vg = fmaf((d[0] + d[1]) + (e[0] + e[1]), isc, vg);
+            vh = fmaf((d[2] + d[3]) + (e[2] + e[3]), isc, vh);
             __syncwarp();
             if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
         }
@@ -535,6 +714,17 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         if (tq < M) {
             if (n < p.N) y[(size_t)tq * p.N + n] = ActTraits<T>::from_float(vg);
             if (n + 8 < p.N) y[(size_t)tq * p.N + n + 8] = ActTraits<T>::from_float(vh);
+        }
+        mark(p, ts == 0 ? 5 : 6);
+    }
+    // every main CTA tells when it has read t; the last one leaves the counters at zero for the next launch
+    if (rank > 0) {
+        int last = 0;
+        if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            for (int i = lane; i < p.n_t * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
+            if (lane == 0) atomicExch(p.ctr + 1, 0);
         }
     }
     return true;
@@ -563,7 +753,9 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
         }
     }
     __syncthreads();
+    mark(p, 1);
     pdl_wait();
+    mark(p, 2);
     float *s_red = reinterpret_cast<float *>(smem + p.off_tred);      // [warp][rank][8 columns]
     const T *x = static_cast<const T *>(p.x);
     bool dead = false;
@@ -585,6 +777,7 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
                 }
                 if (!dead && !mbar_wait(bar, 0)) dead = true;
                 if (dead) break;
+                if (b == warp) mark(p, 3);
                 const uint32_t ab = sA + (uint32_t)b * blk_bytes;
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
@@ -617,20 +810,19 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kCW; ++w) v += s_red[((size_t)w * rank + j) * 8 + m];
-            p.tpart[((size_t)c * M + tb * 8 + m) * rank + j] = v;
+            // value and tag travel in one 8-byte store: whoever sees the tag sees the value
+            p.tpart[((size_t)c * M + tb * 8 + m) * rank + j] = make_float2(v, (p.test_skip_arrive || dead) ? 0.f : 1.f);
         }
         __syncthreads();
     }
     if (dead && lane == 0) give_up(p);
-    __threadfence();
-    __syncthreads();
-    if (tid == 0 && !p.test_skip_arrive) atomicAdd(p.ctr, 1);
+    mark(p, 6);
 }
 
 // ------------------------------------------------------------------------ kernel
 template <int BITS, typename T, int M>
-__global__ void __launch_bounds__(kThreads, 2)
-gemv_kernel(const __grid_constant__ GemvParams p, const __grid_constant__ CUtensorMap wmap,
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
             const __grid_constant__ CUtensorMap bmap, const __grid_constant__ CUtensorMap amap)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -638,6 +830,7 @@ gemv_kernel(const __grid_constant__ GemvParams p, const __grid_constant__ CUtens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // the CTAs of the next launch on this stream may become resident as soon as all of ours are
     pdl_launch_dependents();
+    mark(p, 0);
     if ((int)blockIdx.x < p.n_t) {
         t_cta<T>(p, smem, &amap, (int)blockIdx.x);
         return;
@@ -658,10 +851,12 @@ gemv_kernel(const __grid_constant__ GemvParams p, const __grid_constant__ CUtens
             mbar_init(bars + 8u * (kBarSegFree + i), 1);
         }
         for (int i = 0; i < p.nb; ++i) mbar_init(bars + 8u * (kBarB + i), 1);
+        mbar_init(bars + 8u * kBarXReq, kCW);
         fence_barrier_init();
     }
     for (uint32_t i = tid; i < kZeroBytes / 4; i += kThreads) reinterpret_cast<uint32_t *>(smem + p.off_zero)[i] = 0u;
     __syncthreads();
+    mark(p, 1);
 
     bool ok = true;
     if (warp == kProdWarp) {
@@ -670,8 +865,10 @@ gemv_kernel(const __grid_constant__ GemvParams p, const __grid_constant__ CUtens
         ok = epilogue<T>(p, smem, &bmap, lane, tile_first, ntile);
     } else {
         pdl_wait();                                  // x may come from the preceding kernel
+        mark(p, 2);
         convert_x<BITS, T, M>(p, smem, warp, lane);
         named_barrier_sync(1, kCW * 32);
+        mark(p, 3);
         ok = compute_i8<BITS, T, M>(p, smem, warp, lane, tile_first, ntile);
     }
     if (!ok && lane == 0) give_up(p);
@@ -687,7 +884,6 @@ struct Plan {
 };
 
 int g_sm_count = 0;
-constexpr size_t kSmemHalf = 113 * 1024;     // two CTAs (this launch and the next one) fit on an SM
 constexpr size_t kSmemMax = 227 * 1024;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -705,9 +901,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     const int GB = (a.bits == 4) ? 64 : 48, G = a.K / kGroupFast;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = G; p.rank = a.rank;
     p.NT = (a.N + kTile - 1) / kTile;
-    int want = tune.max_ctas > 0 ? tune.max_ctas : g_sm_count;
-    p.n_main = std::max(1, std::min(want, p.NT));
-    const int nseg = (p.NT + p.n_main - 1) / p.n_main;
+    const int want = tune.max_ctas > 0 ? tune.max_ctas : g_sm_count;
     const int SPT = (G + kCHG - 1) / kCHG;
     p.stage_bytes = kTile * kCHG * GB;
     p.meta_pitch = (int)align_up((size_t)kTile * G * 2, 16);
@@ -721,6 +915,10 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
     }
+    // All CTAs of a launch, t CTAs included, within one per SM: then every CTA of the NEXT launch finds a free half
+    // SM at once.  (Measured: the t CTAs on top of one main CTA per SM cost more, 81 against 72 us per layer step.)
+    p.n_main = std::max(1, std::min(std::max(want - p.n_t, want / 2), p.NT));
+    const int nseg = (p.NT + p.n_main - 1) / p.n_main;
     p.b_box_cols = a.rank <= 16 ? 16 : (a.rank <= 32 ? 32 : 64);      // columns past the rank arrive as zeros
     p.b_swz = p.b_box_cols >= 64 ? 7 : (p.b_box_cols >= 32 ? 3 : 1);
     p.b_slot_bytes = (int)align_up((size_t)((a.rank + 63) / 64) * kTile * p.b_box_cols * 2, 1024);
@@ -758,15 +956,16 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         off += (size_t)ns * p.stage_bytes;
         return off;
     };
-    // as many stages as half an SM's shared memory takes (at least three); else the whole SM
-    int ns = kMaxNS;
-    while (ns > 3 && layout(ns) > kSmemHalf) --ns;
+    // as many stages as fit the CTA's share of an SM's shared memory (all of a CTA's stages where they are few)
+    const size_t budget = (kCtasPerSm == 2 ? 113 * 1024 : kSmemMax) - 2048;
+    int ns = std::min(kMaxNS, std::max(2, nseg * SPT));
+    while (ns > 2 && layout(ns) > budget) --ns;
     size_t need = layout(ns);
-    if (need > kSmemHalf) {
-        ns = kMaxNS;
-        while (ns > 2 && layout(ns) > kSmemMax) --ns;
+    if (need > budget) {                               // x of a long K: the whole SM
+        ns = std::min(kMaxNS, std::max(2, nseg * SPT));
+        while (ns > 2 && layout(ns) > kSmemMax - 2048) --ns;
         need = layout(ns);
-        if (need > kSmemMax) return pl;
+        if (need > kSmemMax - 2048) return pl;
     }
     // a t CTA: barriers, its blocks of A (1024-byte aligned), the reduction buffer
     p.off_tA = 1024;
@@ -776,6 +975,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
+    p.dbg = tune.dbg;
     pl.ok = true;
     if (getenv("FBQ_PLAN"))
         fprintf(stderr, "gemv plan M %d N %d K %d r %d: n_main %d n_t %d (t_kb %d) NS %d nmeta %d nbuf %d nb %d smem %zu (t CTA %zu)\n",
@@ -836,6 +1036,10 @@ cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtens
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
         if (e != cudaSuccess) return e;
+        // Always the largest shared-memory carve-out: launches with different dynamic sizes then share one SM
+        // configuration, so the CTAs of consecutive launches can be resident side by side.
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
         attr_set = true;
     }
     cudaLaunchConfig_t cfg{};
@@ -867,7 +1071,7 @@ bool gemv_supported(const LinearArgs &a)
 void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters)
 {
     const Plan pl = make_plan(a, tune);
-    *tpart_floats = (size_t)std::max(pl.p.n_t, 1) * a.M * std::max(a.rank, 1);
+    *tpart_floats = (size_t)2 * std::max(pl.p.n_t, 1) * a.M * std::max(a.rank, 1);
     *counters = 8;
 }
 
@@ -877,9 +1081,16 @@ cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tu
     if (!pl.ok) return cudaErrorInvalidConfiguration;
     GemvParams &p = pl.p;
     p.x = a.x; p.scales = a.scales; p.zeros = a.zeros; p.y = a.y;
-    p.tpart = ws.partial;
+    p.tpart = reinterpret_cast<float2 *>(ws.tslots);
     p.ctr = ws.counters;
     p.status = ws.counters + kCtrStatus;
+    // tuning aid: consecutive launches write their phase marks to alternate halves of the buffer
+    p.trace = nullptr;
+    if (ws.trace) {
+        static unsigned seq = 0;
+        p.trace = reinterpret_cast<unsigned long long *>(ws.trace) + (size_t)(seq++ & 1u) * 256 * kWarps * 16;
+        if (p.n_t + p.n_main > 256) p.trace = nullptr;
+    }
     CUtensorMap wmap, bmap, amap;
     {
         const cuuint32_t wpg = (a.bits == 4) ? 16 : 12;

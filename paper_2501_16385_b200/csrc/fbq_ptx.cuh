@@ -9,7 +9,14 @@
 namespace fbq {
 namespace ptx {
 
-constexpr uint32_t kWaitLimit = 1u << 22;      // looks at an mbarrier before a wait gives up
+constexpr unsigned long long kWaitNs = 2000000000ull;      // a bounded wait gives up after two seconds
+
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -37,24 +44,42 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-// Bounded wait: false when the limit is hit (never spins forever).
+// Bounded wait: false when the time limit is hit (never spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
 #pragma unroll 1
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitNs) return false;
+    }
 }
 // The same for warps that wait most of the time: they back off between looks so that their polling
 // does not take issue slots from the warps that compute.
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity)
 {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
 #pragma unroll 1
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(64);
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            __nanosleep(200);
+            if (mbar_try_wait(bar, parity)) return true;
+        }
+        if (global_ns() - t0 > kWaitNs) return false;
     }
-    return false;
+}
+// For a whole warp that waits: one lane looks, the others sleep at the warp barrier.
+__device__ __forceinline__ bool mbar_wait_idle_warp(uint32_t bar, uint32_t parity)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait_idle(bar, parity) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -106,6 +131,29 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t a)
 {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+// Predicated forms: lanes with pred == 0 issue no access (and cost no shared-memory bandwidth) and get zeros.
+__device__ __forceinline__ uint4 lds_v4_if(uint32_t a, uint32_t pred)
+{
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %5, 0;\n\t"
+        "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+        : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w)
+        : "r"(a), "r"(pred));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32_if(uint32_t a, uint32_t pred)
+{
+    uint32_t v = 0u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "@p ld.shared.u32 %0, [%1];\n\t}"
+        : "+r"(v)
+        : "r"(a), "r"(pred));
     return v;
 }
 __device__ __forceinline__ float4 lds_f4(uint32_t a)
