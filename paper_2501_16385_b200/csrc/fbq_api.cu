@@ -14,6 +14,7 @@ void decode_set_test_switch(int t_late);
 void decode_set_t_wait(int on);
 void prefill_set_pair(int on);
 void prefill_set_split(int mode);
+void prefill_set_test(int skip_flag, int flag_polls);
 
 namespace {
 
@@ -32,6 +33,7 @@ struct Options {
     int batch_single = 1;
     int prefill_pair = 0;
     int prefill_split = 1;
+    int test_prefill_skip_flag = 0, prefill_flag_polls = 0;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 18 * 16 * 8;   // 512 CTAs x up to 18 warps x 16 marks
@@ -222,6 +224,8 @@ int *option_slot(const char *name)
     if (!strcmp(name, "batch_single")) return &g_opt.batch_single;
     if (!strcmp(name, "prefill_pair")) return &g_opt.prefill_pair;
     if (!strcmp(name, "prefill_split")) return &g_opt.prefill_split;
+    if (!strcmp(name, "test_prefill_skip_flag")) return &g_opt.test_prefill_skip_flag;
+    if (!strcmp(name, "prefill_flag_polls")) return &g_opt.prefill_flag_polls;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
     return nullptr;
 }
@@ -334,6 +338,7 @@ static void apply_kernel_options()
     decode_set_t_wait(g_opt.decode_t_wait);
     prefill_set_pair(g_opt.prefill_pair);
     prefill_set_split(g_opt.prefill_split);
+    prefill_set_test(g_opt.test_prefill_skip_flag, g_opt.prefill_flag_polls);
 }
 
 static int linear_common(const void *x, const uint32_t *qweight, const void *scales, const void *zeros, const void *A,
@@ -448,7 +453,11 @@ static int linear_batch_common(const fbq_problem *problems, int count, int M, in
     int ctas[FBQ_BATCH_MAX];
     for (int i = 0; i < count; ++i)
         ctas[i] = std::max(8, (int)(g_opt.batch_ctas * ((double)a[i].N * a[i].K / total_cost) + 0.5));
-    if (g_opt.batch_single && !host_io && count <= decode_batch_max()) {
+    // Problems in the streaming kernel's domain run as one launch each on the side streams (the same kernel, hence
+    // the same sums, as fbq_linear); the single launch over a problem list is the other decode kernel's.
+    bool all_gemv = g_opt.use_gemv != 0;
+    for (int i = 0; i < count; ++i) all_gemv = all_gemv && gemv_supported(a[i]);
+    if (g_opt.batch_single && !host_io && count <= decode_batch_max() && !all_gemv) {
         // One launch: the decode kernel over a problem list, on the caller's stream.  (With host
         // buffers the per-problem streams below are faster: their small copies overlap.)
         for (int i = 0; i < count; ++i) {

@@ -86,6 +86,8 @@ struct PrefillParams {
     int splitk, splitt;       // K splits of a main tile / of a t tile (1 unless there are few tokens)
     float *part;              // [tile][split][128 rows][TOK] fp32 partial tiles (splitk > 1)
     int *split_ctr;           // [tile] splits that have stored their partial (self-clearing)
+    uint32_t flag_polls;      // looks (256 ns apart) at a token tile's t flag before the wait gives up
+    int test_skip_flag;       // test switch: the t CTAs do not raise the flag (the wait for t must run out)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -576,7 +578,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         const int *flag = p.tflag + m_tile;
                         const int target = 16 * p.rt * p.splitt;
 #pragma unroll 1
-                        for (uint32_t spin = 0; spin < kPfFlagPolls; ++spin) {
+                        for (uint32_t spin = 0; spin < p.flag_polls; ++spin) {
                             asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
                             if (seen >= target) break;
                             __nanosleep(256);
@@ -740,7 +742,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 // this warp's part of t is stored: make it visible, then count the warp in
                 __threadfence();
                 __syncwarp();
-                if (lane == 0) atomicAdd(p.tflag + m_tile, 1);
+                if (lane == 0 && !p.test_skip_flag) atomicAdd(p.tflag + m_tile, 1);
             } else if (p.rank > 0 && tid == 0 && split == 0) {
                 // this CTA has consumed t (its MMAs are complete).  The last main CTA of the token
                 // tile leaves the flag and the count at zero for the next call.
@@ -1173,7 +1175,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_const
                         const int *flag = p.tflag + m_tile;
                         const int target = 16 * p.rt;
 #pragma unroll 1
-                        for (uint32_t spin = 0; spin < kPfFlagPolls; ++spin) {
+                        for (uint32_t spin = 0; spin < p.flag_polls; ++spin) {
                             asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
                             if (seen >= target) break;
                             __nanosleep(256);
@@ -1265,7 +1267,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_const
                 // this warp's part of t is stored: make it visible, then count the warp in
                 __threadfence();
                 __syncwarp();
-                if (lane == 0) atomicAdd(p.tflag + m_tile, 1);
+                if (lane == 0 && !p.test_skip_flag) atomicAdd(p.tflag + m_tile, 1);
             } else if (p.rank > 0 && tid == 0) {
                 // this CTA has consumed t (its MMAs are complete).  The last main CTA of the token
                 // tile leaves the flag and the count at zero for the next call.
@@ -1519,6 +1521,7 @@ cudaError_t make_map(CUtensorMap *map, const void *base, bool elem32, size_t col
 
 // K splits of a main tile when all tokens fit one tile of 128: as many as keep the CTA count near the
 // number of SMs, at most 8, at least 2 groups of K per split.
+int g_pf_skip_flag = 0, g_pf_flag_polls = 0;      // test switches (prefill_set_test)
 int g_split_mode = 1;     // 0: never split K, 1: only deep K (>= 8192), 2: whenever tiles are few
 int prefill_splits(int N, int K)
 {
@@ -1562,6 +1565,8 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
     p.tdone = p.tflag + mt;
     p.split_ctr = p.tdone + mt;
     p.part = ws.partial;
+    p.flag_polls = g_pf_flag_polls > 0 ? (uint32_t)g_pf_flag_polls : kPfFlagPolls;
+    p.test_skip_flag = g_pf_skip_flag;
     CUtensorMap xmap, qmap, amap, bmap, ymap;
     cudaError_t e;
     if ((e = make_map(&xmap, a.x, false, (size_t)a.K, (size_t)a.M, kBK, PAIR ? 128 : TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess)
@@ -1594,6 +1599,11 @@ inline bool aligned16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 
 // 1: token tiles of 256 run on CTA pairs (cta_group::2); 0: single-CTA kernel
 void prefill_set_pair(int on) { g_pair = on ? 1 : 0; }
 void prefill_set_split(int mode) { g_split_mode = mode; }
+void prefill_set_test(int skip_flag, int flag_polls)
+{
+    g_pf_skip_flag = skip_flag;
+    g_pf_flag_polls = flag_polls;
+}
 
 bool prefill_supported(const LinearArgs &a)
 {

@@ -47,7 +47,9 @@ def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M, single
     before = fbq.launch_count()
     fbq.linear_batch(probs, 128, bits)
     torch.cuda.synchronize()
-    assert fbq.launch_count() - before == (1 if single else len(probs))
+    # one launch over the problem list where the other decode kernel runs; the streaming kernel (M <= 2) takes one
+    # launch per problem on the side streams
+    assert fbq.launch_count() - before == (1 if (single and M > 2) else len(probs))
     fbq.set_option("batch_single", 1)
     assert fbq.poll_status() == 0
     for inp, d, pr in zip(inps, devs, probs):
