@@ -81,6 +81,10 @@ cudaError_t grow(P *&ptr, size_t &have, size_t need, size_t elem, cudaStream_t s
 {
     if (need <= have) return cudaSuccess;
     cudaError_t e;
+    // Allocating (and, for a buffer that exists, synchronising and freeing) is illegal while `s` is being
+    // captured into a graph, and a graph captured earlier would keep the old pointers: refuse instead.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone) return cudaErrorStreamCaptureUnsupported;
     if (ptr) {
         if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return e;
         if ((e = cudaFree(ptr)) != cudaSuccess) return e;
@@ -105,6 +109,8 @@ Workspace *workspace_for(cudaStream_t s)
     std::lock_guard<std::mutex> lk(g_mu);
     return &g_ws[std::make_pair(dev, s)];
 }
+
+int grow_status(cudaError_t e) { return e == cudaErrorStreamCaptureUnsupported ? FBQ_ERR_UNSUPPORTED : FBQ_ERR_CUDA; }
 
 // decode_ctas > 0 overrides the decode kernel's grid-size bound for this call.
 int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
@@ -134,8 +140,8 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         int nc = 0;
         gemv_workspace_need(a, gt, &pf, &nc);
         size_t have_c = (size_t)ws->n_counters;
-        if ((e = grow(ws->tslots, ws->tslots_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
-        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->tslots, ws->tslots_floats, pf, sizeof(float), s)) != cudaSuccess) return grow_status(e);
+        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return grow_status(e);
         ws->n_counters = (int)have_c;
         if (g_opt.decode_trace && !ws->trace) {
             if (cudaMalloc(&ws->trace, kTraceBytes) != cudaSuccess) return FBQ_ERR_CUDA;
@@ -154,9 +160,9 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         int nc = 0;
         decode_workspace_need(a, tune, &pf, &nc);
         size_t have_c = (size_t)ws->n_counters;
-        if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
-        if ((e = grow(ws->t, ws->t_floats, (size_t)kDecodeMaxM * kMaxRank, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
-        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->partial, ws->partial_floats, pf, sizeof(float), s)) != cudaSuccess) return grow_status(e);
+        if ((e = grow(ws->t, ws->t_floats, (size_t)kDecodeMaxM * kMaxRank, sizeof(float), s)) != cudaSuccess) return grow_status(e);
+        if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return grow_status(e);
         ws->n_counters = (int)have_c;
         if (g_opt.decode_trace && !ws->trace) {
             if (cudaMalloc(&ws->trace, kTraceBytes) != cudaSuccess) return FBQ_ERR_CUDA;
@@ -180,10 +186,10 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         size_t have_c = (size_t)ws->n_counters, need_t = 0, need_p = 0;
         int need_c = 0;
         prefill_workspace_need(a, &need_c, &need_t, &need_p);
-        if ((e = grow(ws->counters, have_c, (size_t)need_c, sizeof(int), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if ((e = grow(ws->counters, have_c, (size_t)need_c, sizeof(int), s)) != cudaSuccess) return grow_status(e);
         ws->n_counters = (int)have_c;
-        if (need_t > 0 && (e = grow(ws->t_gen, ws->t_gen_floats, need_t, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
-        if (need_p > 0 && (e = grow(ws->partial, ws->partial_floats, need_p, sizeof(float), s)) != cudaSuccess) return FBQ_ERR_CUDA;
+        if (need_t > 0 && (e = grow(ws->t_gen, ws->t_gen_floats, need_t, sizeof(float), s)) != cudaSuccess) return grow_status(e);
+        if (need_p > 0 && (e = grow(ws->partial, ws->partial_floats, need_p, sizeof(float), s)) != cudaSuccess) return grow_status(e);
         e = launch_prefill(a, *ws, s, &launches);
         if (e == cudaErrorInvalidConfiguration) {
             (void)cudaGetLastError();
@@ -233,6 +239,20 @@ int *option_slot(const char *name)
 }  // namespace
 
 void count_launches(int n) { g_launches += n; }
+
+int noalloc_poll_status(int dev);      // fbq_noalloc.cu
+
+// For the no-allocation entry point: the process-wide switches applied, and the decode tuning with
+// everything that sizes scratch left automatic.
+DecodeTuning decode_tuning_for_noalloc()
+{
+    decode_set_test_switch(g_opt.decode_t_late);
+    decode_set_t_wait(g_opt.decode_t_wait);
+    DecodeTuning t = g_opt.decode;
+    t.max_ctas = 0;
+    t.sk = 0;
+    return t;
+}
 
 }  // namespace fbq
 
@@ -572,6 +592,11 @@ int fbq_poll_status(void *stream)
     if (cudaStreamSynchronize(s) != cudaSuccess) return FBQ_ERR_CUDA;
     Workspace *ws = workspace_for(s);
     if (!ws) return FBQ_ERR_CUDA;
+    // the fixed scratch array of fbq_linear_noalloc has a status word of its own (shared by all streams)
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FBQ_ERR_CUDA;
+    const int fixed = noalloc_poll_status(dev);
+    if (fixed != FBQ_OK) return fixed;
     if (!ws->counters) return FBQ_OK;
     int st = 0;
     if (cudaMemcpy(&st, ws->counters + kCtrStatus, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FBQ_ERR_CUDA;

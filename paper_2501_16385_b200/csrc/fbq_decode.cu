@@ -2134,11 +2134,21 @@ bool decode_batch_need(const LinearArgs *a, int count, const int *ctas, const De
     *partial_floats = 0;
     *t_floats = 0;
     *counters = kCtrFirstTile;                      // the shared head (status word) comes first
+    bool i8 = false, heavy = false;
     for (int i = 0; i < count; ++i) {
         DecodeTuning tn = tune;
         tn.max_ctas = ctas[i];
         const Plan pl = make_plan(a[i], tn);
         if (!pl.ok) return false;
+        // One launch runs ONE kernel variant: every problem's shared-memory layout must have been planned for
+        // the same form (integer or 16-bit) and the same sub-branch variant.  Plans that disagree (the form
+        // falls back where x of a long K does not fit) go to one launch per problem instead.
+        if (i == 0) {
+            i8 = pl.i8;
+            heavy = pl.heavy;
+        } else if (pl.i8 != i8 || pl.heavy != heavy) {
+            return false;
+        }
         *partial_floats += (size_t)pl.NT * pl.maxslots * a[i].M * kTileRows;
         *t_floats += (size_t)kDecodeMaxM * kMaxRank;
         *counters += kCtrFirstTile + 2 * pl.NT;

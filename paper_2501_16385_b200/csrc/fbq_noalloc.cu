@@ -19,6 +19,7 @@
 
 namespace fbq {
 void count_launches(int n);
+DecodeTuning decode_tuning_for_noalloc();
 
 namespace {
 
@@ -60,6 +61,23 @@ cudaError_t scratch_base(unsigned char **out)
 }
 
 }  // namespace
+
+// Status word of the fixed array on device `dev` (FBQ_OK when the array was never used there).  A word
+// that is set is returned once: reading clears it and resets the array's counters and t, which a kernel
+// that gave up has left unfinished.  Called by fbq_poll_status after it has synchronised the stream.
+int noalloc_poll_status(int dev)
+{
+    unsigned char *base = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (dev < 0 || dev >= kMaxDevices || !g_base[dev]) return FBQ_OK;
+        base = g_base[dev];
+    }
+    int st = 0;
+    if (cudaMemcpy(&st, base + kCtrStatus * sizeof(int), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FBQ_ERR_CUDA;
+    if (st != 0 && cudaMemset(base, 0, kCtrBytes + kTBytes) != cudaSuccess) return FBQ_ERR_CUDA;
+    return st;
+}
 }  // namespace fbq
 
 using namespace fbq;
@@ -89,7 +107,7 @@ extern "C" int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const 
     a.M = M; a.N = N; a.K = K; a.group = group; a.bits = bits; a.rank = rank;
     a.bf16 = act_is_bf16 != 0;
 
-    const DecodeTuning tune{};                 // automatic plan
+    const DecodeTuning tune = decode_tuning_for_noalloc();     // the process-wide options; scratch-sizing ones automatic
     size_t partial_floats = 0;
     int counters = 0;
     decode_workspace_need(a, tune, &partial_floats, &counters);
@@ -101,7 +119,11 @@ extern "C" int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // Counters, flags and t must be zero when the kernel starts.  The kernel leaves them
     // zero, but the array is shared with every other call, so do not rely on it.
-    if (cudaMemsetAsync(base, 0, kCtrBytes + kTBytes, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    // The status word (counter slot kCtrStatus) is left alone: a time-out of an earlier call stays readable
+    // through fbq_poll_status until it is read.
+    constexpr size_t kHead = (size_t)kCtrStatus * sizeof(int), kTail = ((size_t)kCtrStatus + 1) * sizeof(int);
+    if (cudaMemsetAsync(base, 0, kHead, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    if (cudaMemsetAsync(base + kTail, 0, kCtrBytes + kTBytes - kTail, s) != cudaSuccess) return FBQ_ERR_CUDA;
 
     Workspace ws{};
     ws.counters = reinterpret_cast<int *>(base);

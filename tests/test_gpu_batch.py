@@ -128,3 +128,30 @@ def test_batch_argument_checks(fbq):
     assert L.fbq_linear_batch(arr, 0, 1, 128, 3, 0, 0, None) == 0
     assert L.fbq_linear_batch(arr, 17, 1, 128, 3, 0, 0, None) != 0
     assert L.fbq_linear_batch(None, 1, 1, 128, 3, 0, 0, None) != 0
+
+
+@pytest.mark.parametrize("M", [1, 2, 4, 6])
+def test_full_size_layer_in_one_batch_call(fbq, M):
+    """The seven Llama-2-7B shapes (K = 4096 next to K = 11008) in one fbq_linear_batch call with the
+    single-launch form switched on: whatever mix of plans the problems get, every output (sampled rows at
+    these sizes) matches the oracle."""
+    import torch
+    from workloads import LLAMA2_7B_SHAPES
+    fbq.set_option("batch_single", 1)
+    bits, rank = 3, 16
+    inps = [make_linear(M, N, K, bits, rank, seed=4700 + 10 * M + i) for i, (K, N) in enumerate(LLAMA2_7B_SHAPES)]
+    devs = [DeviceLinear(inp, fbq) for inp in inps]
+    probs = []
+    for d, inp in zip(devs, inps):
+        y = torch.full((M, inp.N), float("nan"), dtype=d.x.dtype, device="cuda")
+        probs.append((d.x, d.qweight, d.scales, d.zeros, d.A, d.B, y))
+    fbq.linear_batch(probs, 128, bits)
+    torch.cuda.synchronize()
+    assert fbq.poll_status() == 0
+    for inp, pr in zip(inps, probs):
+        rows = np.unique(np.concatenate([np.arange(0, inp.N, 37), np.arange(inp.N - 16, inp.N)]))
+        want = oracle.linear_inputs(inp, n_list=rows, threads=8)
+        got = torch_to_f64(pr[6], "f16")
+        assert np.all(np.isfinite(got))
+        rel, mx, lim = compare(got[:, rows], want, inp.x_f64(), inp.K)
+        assert rel <= REL_F_TOL and mx <= lim, (inp.N, inp.K, rel, mx)

@@ -337,3 +337,58 @@ def test_empty_and_status(fbq, torch):
     y0 = fbq.linear(x0, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, 64, 128, 4)
     assert y0.shape == (0, 64)
     assert fbq.poll_status() == 0
+
+
+# ------------------------------------------------------------ contracts the header states
+def test_non_finite_x_reaches_the_outputs(fbq, torch):
+    """An Inf or a NaN in x makes every output of its token non-finite, as the definition says (every output row
+    sums over every input channel) -- also in the integer form, where x passes through fixed point."""
+    for bits, M, rank in ((4, 1, 0), (3, 1, 32), (4, 2, 0)):
+        inp = make_linear(M, 256, 1024, bits, rank, seed=77)
+        dev = DeviceLinear(inp, fbq)
+        for bad in (float("inf"), float("nan")):
+            x = dev.x.clone()
+            x[M - 1, 300] = bad
+            y = torch_to_f64(dev.run(fbq, x=x), "f16")
+            assert not np.any(np.isfinite(y[M - 1])), (bits, M, rank, bad)
+            if M > 1:
+                assert np.all(np.isfinite(y[0]))           # the other token is untouched
+        assert fbq.poll_status() == 0
+
+
+def test_growing_scratch_inside_a_capture_is_refused(fbq, torch):
+    """A call that would have to allocate scratch while its stream is being captured returns
+    FBQ_ERR_UNSUPPORTED and queues nothing; the capture itself stays valid."""
+    fbq.release_workspaces()
+    inp = make_linear(1, 256, 1024, 4, 32, seed=78)
+    dev = DeviceLinear(inp, fbq)
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            with pytest.raises(fbq.FbqError) as err:
+                fbq.linear(dev.x, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, inp.N, 128, 4, stream=st)
+            assert err.value.code == -2
+        st.synchronize()
+        y = fbq.linear(dev.x, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, inp.N, 128, 4, stream=st)   # outside: allocates
+        g2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g2, stream=st):
+            fbq.linear(dev.x, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, inp.N, 128, 4, y=y, stream=st)
+        g2.replay()
+        st.synchronize()
+    want = oracle.linear_inputs(inp, threads=8)
+    rel, mx, lim = compare(torch_to_f64(y, "f16"), want, inp.x_f64(), inp.K)
+    assert rel <= REL_F_TOL and mx <= lim
+
+
+def test_all_rows_full_size_decode_m16(fbq):
+    """Every output of a 13 824 x 5120 projection at M = 16 (no row sampling), through the decode kernel."""
+    inp = make_linear(16, 13824, 5120, 4, 64, seed=79)
+    check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE, threads=16, floor=2e-5)
+
+
+def test_all_rows_full_size_streaming_kernel(fbq):
+    """Every output of the three 7B shapes at M = 1 and of one of them at M = 2."""
+    for M, (K, N), bits in ((1, (4096, 4096), 3), (1, (4096, 11008), 3), (1, (11008, 4096), 3), (2, (11008, 4096), 4)):
+        inp = make_linear(M, N, K, bits, 64, seed=80 + M)
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE, threads=16, floor=2e-5)

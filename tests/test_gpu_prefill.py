@@ -116,3 +116,9 @@ def test_prefill_few_tokens_split_k(fbq, bits, dtype, M, N, K, rank):
     finally:
         fbq.set_option("force_kernel", -1)
         fbq.set_option("prefill_split", 1)
+
+
+def test_all_rows_full_size_prefill(fbq):
+    """Every output of a 4096 x 4096 projection at M = 1024 (no row sampling), fp16."""
+    inp = make_linear(1024, 4096, 4096, 4, 64, seed=90)
+    check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, threads=16, floor=2e-5)

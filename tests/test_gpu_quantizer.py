@@ -126,3 +126,38 @@ def test_quantizer_rejects_bad_requests(fbq):
     assert L.fbq_quantize_feedback(*args(32, 5, 0)) != 0
     assert L.fbq_quantize_feedback(*args(32, 4, 8)) != 0        # rank > 0 without A, B
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("bits", [3, 4])
+@pytest.mark.parametrize("dtype,M", [("f16", 1), ("f16", 2), ("f16", 4), ("f16", 64), ("bf16", 64)])
+def test_zero_points_outside_the_code_range_run_on_every_kernel(fbq, bits, dtype, M):
+    """Groups that do not straddle zero get zero points the quantiser does not clamp: negative for an
+    all-positive group, beyond 2^bits - 1 for an all-negative one.  Every kernel must take them as they are
+    stored (fp16 integers of either sign): the streaming decode kernel (M <= 2), the other decode kernel
+    (M = 4), the prefill kernel in fp16 and bf16 -- checked against the oracle on the quantiser's output."""
+    import torch
+    N, K, rank = 272, 1024, 16
+    rng = np.random.default_rng(5300 + bits)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    W[0::3] = np.abs(W[0::3]) + 0.05           # all-positive rows: z = rint(-min/s) < 0
+    W[1::3] = -np.abs(W[1::3]) - 0.05          # all-negative rows: z > 2^bits - 1
+    _, A, B = _inputs(N, K, rank, dtype, seed=5310 + bits)
+    codes, s, z, wf, dev = _run(fbq, W, A, B, 128, bits, dtype)
+    zf = z.view(np.float16).astype(np.float64)
+    assert zf.min() < 0 and zf.max() > (1 << bits) - 1 and np.all(zf == np.rint(zf))
+    Wd, Ad, Bd, codes_d, s_d, z_d = dev
+    x32 = np.random.default_rng(2).standard_normal((M, K)).astype(np.float32)
+    x_bits = f32_to_bf16_bits(x32) if dtype == "bf16" else x32.astype(np.float16).view(np.uint16)
+    xd = _dev16(x_bits, dtype)
+    y = fbq.linear(xd, fbq.pack(codes_d, bits), s_d, z_d, Ad, Bd, N, 128, bits)
+    torch.cuda.synchronize()
+    assert fbq.poll_status() == 0
+    got = y.float().cpu().numpy().astype(np.float64)
+    want = oracle.linear(x_bits, oracle.pack(codes, bits), s, z, A, B, M, N, K, 128, bits, rank, dtype=dtype, threads=8)
+    rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+    assert rel <= 5e-3, rel
+    xmax = float(np.max(np.abs(x32)))
+    lim = 1e-2 * xmax * np.sqrt(K) / 64.0
+    if dtype == "bf16":
+        lim += 2.0 ** -8 * float(np.max(np.abs(want)))
+    assert np.max(np.abs(got - want)) <= lim

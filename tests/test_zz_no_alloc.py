@@ -2,11 +2,14 @@
 (all of it already given to their own pool, or no room for the synchronisation an
 allocation may imply).  Its scratch is a fixed array inside the library, so its results
 must equal those of fbq_linear, whose scratch is allocated per stream -- on a first call
-and again on a second one, which finds the array as the first call left it.
+and again on a second one, which finds the array as the first call left it -- and, like
+every other path, the CPU oracle's within the layer's tolerance.
 
 Collected last on purpose: a failure here leaves every other test already run."""
 import numpy as np
 import pytest
+
+import oracle
 
 from workloads import make_linear
 
@@ -24,12 +27,15 @@ def test_noalloc_matches_allocating_entry_point_twice():
     for inp in cases:
         dev = DeviceLinear(inp, fbq)
         fbq.set_option("force_kernel", fbq.KERNEL_DECODE)     # the same kernel, whatever the dispatcher prefers at this M
+        fbq.set_option("gemv", 0)                             # ... and not the streaming kernel, which the fixed array does not serve
         try:
             want = dev.run(fbq)                               # existing entry point
         finally:
             fbq.set_option("force_kernel", -1)
+            fbq.set_option("gemv", 1)
         torch.cuda.synchronize()
         want64 = torch_to_f64(want, inp.dtype)
+        y_or = oracle.linear_inputs(inp, threads=8)           # the definition itself
         for call in range(2):                                 # two calls in a row share the array
             y = torch.full((inp.M, inp.N), float("nan"), dtype=want.dtype, device="cuda")
             fbq.linear_noalloc(dev.x, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, inp.N, inp.group,
@@ -39,6 +45,11 @@ def test_noalloc_matches_allocating_entry_point_twice():
             assert np.all(np.isfinite(got64)), "call %d left outputs unwritten" % call
             rel, mx, lim = compare(got64, want64, inp.x_f64(), inp.K)
             assert rel <= REL_F_TOL and mx <= lim, (call, rel, mx)
+            rel, mx, lim = compare(got64, y_or, inp.x_f64(), inp.K)
+            if inp.dtype == "bf16":                           # half an ulp of a bf16 output alone can exceed the bound
+                lim += 2.0 ** -8 * float(np.max(np.abs(y_or)))
+            assert rel <= REL_F_TOL and mx <= lim, ("oracle", call, rel, mx)
+            assert fbq.poll_status() == 0                     # the fixed array's own status word is clean
             if inp.rank == 0:
                 assert torch.equal(y, want)                   # no atomics on this path: bit for bit
 
