@@ -50,13 +50,14 @@ typedef enum {
     FBQ_ERR_UNSUPPORTED = -2, /* shape outside every kernel's domain                     */
     FBQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned                        */
     FBQ_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, launch error)    */
-    FBQ_ERR_TIMEOUT = -5      /* device side: a bounded wait on a bulk copy expired      */
+    FBQ_ERR_TIMEOUT = -5      /* device side: a bounded wait (on a copy, on another CTA's
+                                 part of t) expired; read with fbq_poll_status           */
 } fbq_status;
 
 typedef enum {
     FBQ_KERNEL_NONE = -1,
     FBQ_KERNEL_GENERIC = 0,   /* any supported shape, CUDA cores, two launches if rank>0 */
-    FBQ_KERNEL_DECODE = 1,    /* M <= 16 (chosen for M <= 6): fused streaming kernel, one launch */
+    FBQ_KERNEL_DECODE = 1,    /* M <= 16 (chosen for M <= 6): fused streaming kernels, one launch */
     FBQ_KERNEL_PREFILL = 2    /* tcgen05 / TMEM tensor-core kernel, one launch (chosen from M = 7) */
 } fbq_kernel;
 
@@ -85,21 +86,32 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  *   rank == 0: A and B are ignored (may be NULL); y is the main path alone.
  *   M == 0: nothing is done.
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128
- * and rank a multiple of 8 not above 256 -> decode kernel for M <= 4 with rank <= 128 and for
+ * and rank a multiple of 8 not above 256 -> decode kernels for M <= 4 with rank <= 128 and for
  * M = 5, 6 with M * rank <= 128, else prefill kernel (N a multiple of 8 and 16-byte aligned operands; otherwise the decode
  * kernel up to M = 16); everything else that is well formed -> generic kernel.
+ * Of the decode kernels the streaming one ("gemv" option, default on) runs M <= 2 with N a multiple of
+ * 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; the other decode kernel takes the rest.
  * Well formed means bits in {3,4}, group a multiple of 8 (4 bits) or 32
- * (3 bits) dividing K, rank >= 0.  The decode and prefill kernels assume
- * integer-valued zero points in [0, 127]; the generic kernel accepts any
- * fp16 value.  Accumulation is fp32; t = x.A^T stays fp32 in the decode and
- * generic kernels (where the decode kernel multiplies it with B on tensor cores it enters as
+ * (3 bits) dividing K, rank >= 0.  Zero points are taken as stored: every kernel accepts
+ * integer-valued fp16 zero points of either sign and beyond 2^bits - 1 (what fbq_quantize_feedback
+ * produces for groups that do not straddle zero); the decode and generic kernels any fp16 value.
+ * Accumulation is fp32; t = x.A^T stays fp32 in the decode and
+ * generic kernels (where a decode kernel multiplies it with B on tensor cores it enters as
  * two 16-bit terms, the rounded value and the remainder) and is rounded once to the activation
  * type in the prefill kernel (which also rounds the dequantised weights s*(q-z) once to that
- * type).  At M <= 2 the decode kernel reads x in fixed point per group of 128, exact to 2^-17
- * of the group's largest element ("decode_i8").
- * Summation order is fixed for a given shape (results are
- * reproducible run to run) except for t in the decode kernel, which is
- * accumulated with floating-point atomics. */
+ * type).  At M <= 2 the decode kernels read x in fixed point per group of 128, exact to 2^-17
+ * of the group's largest element; a group that holds an Inf or a NaN makes its token's outputs NaN.
+ * Summation order is fixed for a given shape and grid size (results are
+ * reproducible run to run), except for t in the decode kernel of M >= 3, which is
+ * accumulated with floating-point atomics.
+ * Scratch and CUDA graphs: the library keeps scratch buffers per (device, stream) and grows them
+ * the first time a stream sees a larger shape.  Growing allocates (and, for a buffer that exists,
+ * synchronises the stream and frees the old one): a call that would have to grow scratch while
+ * `stream` is being captured returns FBQ_ERR_UNSUPPORTED and queues nothing, and a graph captured
+ * EARLIER on that stream keeps pointers to a buffer that a later, larger call replaces.  So: run
+ * the largest shape of every kind once on a stream, outside capture, before capturing on it.
+ * After FBQ_ERR_TIMEOUT the stream's counters are unfinished: call fbq_poll_status (it resets
+ * them) before issuing more work on that stream. */
 int fbq_linear(const void *x, const uint32_t *qweight, const void *scales, const void *zeros,
                const void *A, const void *B, void *y, int M, int N, int K, int group, int bits,
                int rank, void *stream);
@@ -137,7 +149,13 @@ int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *s
  *     zero (a memset queued on `stream`).  Calls that can overlap on the GPU (different
  *     streams, or several host threads) therefore race on it: run them one after another.
  *   - Arguments, layouts, dtypes (act_is_bf16 selects bf16 x, A, B, y) and results are
- *     those of fbq_linear / fbq_linear_bf16. */
+ *     those of fbq_linear / fbq_linear_bf16 with the "gemv" option off (the streaming kernel
+ *     of M <= 2 is not served by the fixed array; the other decode kernel runs every M <= 16).
+ *     The process-wide options apply ("pdl", "decode_i8", "decode_t_ctas", ...), except those
+ *     that size scratch ("decode_ctas", "decode_sk"), which stay automatic.
+ *   - A device-side time-out lands in a status word inside the array; fbq_poll_status(any
+ *     stream) of that device returns it once (FBQ_ERR_TIMEOUT), clears it and resets the array.
+ *     The per-call clearing leaves that word alone, so a time-out stays readable until polled. */
 int fbq_linear_noalloc(const void *x, const uint32_t *qweight, const void *scales,
                        const void *zeros, const void *A, const void *B, void *y, int M, int N,
                        int K, int group, int bits, int rank, int act_is_bf16, void *stream);
@@ -232,6 +250,15 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
 /* Tuning and test switches (host side, process wide).  Known names:
  *   "force_kernel"  -1 = automatic, else an fbq_kernel value (shapes outside the
  *                   forced kernel's domain still fall back to the generic one)
+ *   "gemv"          1 (default) = M <= 2 runs the streaming decode kernel where its domain allows (see fbq_linear),
+ *                   0 = the other decode kernel at every M
+ *   "gemv_ctas"     0 = automatic (one main CTA per SM), else an upper bound on the streaming kernel's grid
+ *   "t_poll_limit"  0 = default, else the number of looks the streaming kernel takes at the t CTAs' slots
+ *                   before it gives up with FBQ_ERR_TIMEOUT
+ *   "test_skip_t_arrive", "test_prefill_skip_flag", "prefill_flag_polls"
+ *                   test switches of the failure-detection tests: the CTAs that compute t = x.A^T do not
+ *                   report it (streaming decode kernel / prefill kernel), and the prefill kernel's number
+ *                   of looks at its flag; with them a bounded wait runs out on purpose
  *   "decode_sk"     0 = automatic, else the number of K slices of the decode kernel
  *   "decode_chunk"  0 = automatic, else quantisation groups per smem stage
  *   "decode_depth"  0 = automatic, else stages in flight per warp
@@ -258,6 +285,8 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *                   every tile through the parked-tile branch of the combine protocol
  *   "decode_trace"  tuning aid: 1 = the decode kernel records, per CTA and warp, the SM cycle
  *                   counter at its phases, read with fbq_debug_read_trace
+ * Options are plain process-wide integers read when a call is issued: set them before issuing work, not while
+ * other host threads are inside the library.
  * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name.
  * (Tuning aid outside this interface: with the environment variable FBQ_PLAN set, every plan of the
  * decode kernel is printed to stderr: K slices, CTAs, stage size and count, shared-memory layout, form.) */
@@ -268,14 +297,16 @@ int fbq_get_option(const char *name, int *value);
 long long fbq_launch_count(void);
 
 /* Synchronises `stream` and returns the device-side status word of its scratch
- * space: FBQ_OK, or FBQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up
- * (the affected outputs are then undefined).  Reading clears the word. */
+ * space (or of the fixed array of fbq_linear_noalloc, if that one is set): FBQ_OK, or
+ * FBQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the affected outputs are then
+ * undefined).  Reading clears the word and resets the counters the kernel left unfinished. */
 int fbq_poll_status(void *stream);
 
 /* Tuning aid: copies the phase marks of the last decode launch on `stream` (recorded while
- * "decode_trace" is 1) to host_buf: uint64 [cta][10 warps][16 marks] of SM cycle counts, zero
- * where a mark was not reached; mark 15 of warp 0 is the global timer (ns) at kernel entry.
- * bytes <= 512*10*16*8.  Synchronises the stream. */
+ * "decode_trace" is 1) to host_buf.  The streaming kernel writes uint64 [2][256 CTAs][10 warps][16 marks]
+ * of global-timer values (ns), consecutive launches alternating between the two halves; the other
+ * decode kernel uint64 [cta][10 warps][16 marks] of SM cycle counts with mark 15 of warp 0 the global
+ * timer at kernel entry.  Zero where a mark was not reached.  bytes <= 512*18*16*8.  Synchronises the stream. */
 int fbq_debug_read_trace(void *stream, void *host_buf, size_t bytes);
 
 /* Frees every per-stream scratch buffer (synchronises the device first). */

@@ -42,9 +42,10 @@
 // (Section 4.3 of the paper adds the up-projection into the shared output):
 // their token operand is t = x.A^T (fp32 scratch, rounded once to the activation
 // type by the producers), their weight operand is B as stored.  t itself comes
-// from the same kernel in down-projection mode (K split over CTAs, fp32 atomics
-// into scratch) one launch earlier; the main launch may start while that one
-// drains and waits for it only before its sub-branch blocks.
+// from the SAME launch: the first blocks of the grid run in down-projection mode
+// (both operands by TMA, all of K or a K split each, plain fp32 stores to scratch)
+// and raise a flag per token tile; the main CTAs look at the flag (bounded) only
+// before their sub-branch blocks, at the very end of their K loop.
 // All waits are bounded: a wait that runs out raises FBQ_ERR_TIMEOUT in the
 // status word and every role falls through to the common exit.
 #include <cuda.h>
