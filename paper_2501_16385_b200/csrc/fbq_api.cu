@@ -136,11 +136,12 @@ int run_linear(const LinearArgs &a, cudaStream_t s, int decode_ctas = 0)
         GemvTuning gt = g_opt.gemv;
         gt.pdl = g_opt.decode.pdl;
         if (tune.max_ctas > 0) gt.max_ctas = tune.max_ctas;
-        size_t pf = 0;
+        size_t pf = 0, partf = 0;
         int nc = 0;
-        gemv_workspace_need(a, gt, &pf, &nc);
+        gemv_workspace_need(a, gt, &pf, &nc, &partf);
         size_t have_c = (size_t)ws->n_counters;
         if ((e = grow(ws->tslots, ws->tslots_floats, pf, sizeof(float), s)) != cudaSuccess) return grow_status(e);
+        if (partf > 0 && (e = grow(ws->partial, ws->partial_floats, partf, sizeof(float), s)) != cudaSuccess) return grow_status(e);
         if ((e = grow(ws->counters, have_c, (size_t)nc, sizeof(int), s)) != cudaSuccess) return grow_status(e);
         ws->n_counters = (int)have_c;
         if (g_opt.decode_trace && !ws->trace) {

@@ -95,7 +95,7 @@ struct GemvTuning {
     int test_skip_arrive = 0;  // test switch: the t CTAs do not report their arrival (the wait for t must run out)
 };
 bool gemv_supported(const LinearArgs &a);
-void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters);
+void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters, size_t *partial_floats);
 cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tune, cudaStream_t s, int *launches);
 
 int decode_batch_max();

@@ -75,6 +75,13 @@ struct GemvParams {
     int stage_bytes, meta_pitch, b_slot_bytes, b_box_cols, b_swz;
     int off_bar, off_tab, off_zero, off_x, off_meta, off_seg, off_t, off_B, off_ring;
     int off_tA, off_tred;                   // t CTA: blocks of A, reduction buffer
+    // 16-bit form (M >= 3): K may be cut into SK slices (CTA = row block x slice) whose partial tiles meet in scratch
+    int SK, R;                              // n_main = R * SK
+    int slice_groups;                       // groups per K slice (a multiple of the stage's groups; the last slice takes the rest)
+    int x_pitch;                            // elements between tokens of the staged x
+    int off_px, off_tf;                     // (P, X0) table; t as MMA column operands
+    float *part;                            // [tile][slice][M][16] fp32 partial tiles (SK > 1)
+    int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
     int dbg;
@@ -536,11 +543,13 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
 }
 
 // ------------------------------------------------------------------------ producer
-__device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, const CUtensorMap *wmap, int tile_first, int ntile)
+__device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, const CUtensorMap *wmap, int tile_first, int ntile,
+                                        int g_begin = 0, int g_count = -1, int chg = kCHG)
 {
     const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
     const uint32_t ring = sbase + p.off_ring, meta0 = sbase + p.off_meta;
-    const int SPT = (p.G + kCHG - 1) / kCHG, NS = p.NS;
+    if (g_count < 0) g_count = p.G;
+    const int SPT = (g_count + chg - 1) / chg, NS = p.NS;
     int it = 0;
     for (int ts = 0; ts < ntile; ++ts) {
         const int tile = tile_first + ts;
@@ -555,7 +564,7 @@ __device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, cons
             const uint32_t full = bars + 8u * (kBarFull + slot);
             mbar_expect_tx(full, (uint32_t)p.stage_bytes + (st == 0 ? 2u * mbytes : 0u));
             // one box of 16 groups x 16 rows (rows past N and groups past G arrive as zeros)
-            tma_load_3d(ring + (uint32_t)slot * (uint32_t)p.stage_bytes, wmap, 0, tile * kTile, st * kCHG, full);
+            tma_load_3d(ring + (uint32_t)slot * (uint32_t)p.stage_bytes, wmap, 0, tile * kTile, g_begin + st * chg, full);
             if (it == 0) mark(p, 3);
             if (st == 0) {
                 const uint32_t ms = meta0 + (uint32_t)(ts % p.nmeta) * 2u * (uint32_t)p.meta_pitch;
@@ -730,6 +739,491 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
     return true;
 }
 
+
+// =============================================================== 16-bit form (3 <= M <= 16)
+// Codes become packed 16-bit floats with one LOP3 per pair ("bias-free" unpack): a field at bit p of a
+// 16-bit half, OR-ed into the mantissa of MAGIC = 1024 (fp16) or 128 (bf16), is MAGIC + 2^p q.  Nothing is
+// spent per element on removing MAGIC, 2^p or the zero point: x is staged divided by 2^p (exact) and
+// permuted into the order the unpacker produces, so the MMA yields sum x q + sum (MAGIC / 2^p) x; the second
+// sum (P) and sum x (X0) depend on token and group only and are tabulated when x is staged, and a group
+// contributes s (mma - P) - (s z) X0.
+//   INT4: h[4i+e]  = codes (8i+e , 8i+e+4)  of word i          (i = 0..3, e = 0..3)
+//   INT3: h[5i+f]  = codes (10i+f, 10i+5+f) of word i          (i = 0..2, f = 0..4);  h[15] = codes (30, 31)
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv)
+{
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));   // (a & mask) | orv
+    return r;
+}
+template <int BITS, typename T> struct Unpack16;
+template <> struct Unpack16<4, __half> {
+    static constexpr float kMagic = 1024.f;
+    static __device__ __forceinline__ int div_log2(int c) { return ((c & 7) & 1) ? 4 : 0; }   // odd nibbles sit 4 bits up
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t a = w[i], b = w[i] >> 8;
+            h[4 * i + 0] = lop3_and_or(a, 0x000F000Fu, 0x64006400u);
+            h[4 * i + 1] = lop3_and_or(a, 0x00F000F0u, 0x64006400u);
+            h[4 * i + 2] = lop3_and_or(b, 0x000F000Fu, 0x64006400u);
+            h[4 * i + 3] = lop3_and_or(b, 0x00F000F0u, 0x64006400u);
+        }
+    }
+};
+template <> struct Unpack16<4, __nv_bfloat16> {
+    static constexpr float kMagic = 128.f;                     // 0x4300 | q is 128 + q in bf16 (7 mantissa bits)
+    static __device__ __forceinline__ int div_log2(int) { return 0; }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) h[4 * i + e] = lop3_and_or(w[i] >> (4 * e), 0x000F000Fu, 0x43004300u);
+    }
+};
+template <> struct Unpack16<3, __half> {
+    static constexpr float kMagic = 1024.f;
+    static __device__ __forceinline__ int div_log2(int c)
+    {
+        if (c >= 30) return 0;
+        const int f = (c % 10) % 5;                             // fields 0,3: bit 0; 1,4: bit 3; 2: bit 6 (3,4 after >> 9)
+        return (f == 2) ? 6 : ((f == 1 || f == 4) ? 3 : 0);
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const uint32_t a = w[i], b = w[i] >> 9;
+            h[5 * i + 0] = lop3_and_or(a, 0x00070007u, 0x64006400u);
+            h[5 * i + 1] = lop3_and_or(a, 0x00380038u, 0x64006400u);
+            h[5 * i + 2] = lop3_and_or(a, 0x01C001C0u, 0x64006400u);
+            h[5 * i + 3] = lop3_and_or(b, 0x00070007u, 0x64006400u);
+            h[5 * i + 4] = lop3_and_or(b, 0x00380038u, 0x64006400u);
+        }
+        uint32_t l = lop3_and_or(w[0] >> 15, 0x00010001u, 0x64006400u);
+        l = lop3_and_or(w[1] >> 14, 0x00020002u, l);
+        h[15] = lop3_and_or(w[2] >> 13, 0x00040004u, l);
+    }
+};
+template <> struct Unpack16<3, __nv_bfloat16> {
+    static constexpr float kMagic = 128.f;
+    static __device__ __forceinline__ int div_log2(int c)
+    {
+        if (c >= 30) return 0;
+        const int f = (c % 10) % 5;                             // shifts 0, 6, 12: fields 0,2,4 at bit 0; 1,3 at bit 3
+        return (f == 1 || f == 3) ? 3 : 0;
+    }
+    static __device__ __forceinline__ void run(const uint32_t *w, uint32_t *h)
+    {
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const uint32_t a = w[i], b = w[i] >> 6, c = w[i] >> 12;
+            h[5 * i + 0] = lop3_and_or(a, 0x00070007u, 0x43004300u);
+            h[5 * i + 1] = lop3_and_or(a, 0x00380038u, 0x43004300u);
+            h[5 * i + 2] = lop3_and_or(b, 0x00070007u, 0x43004300u);
+            h[5 * i + 3] = lop3_and_or(b, 0x00380038u, 0x43004300u);
+            h[5 * i + 4] = lop3_and_or(c, 0x00070007u, 0x43004300u);
+        }
+        uint32_t l = lop3_and_or(w[0] >> 15, 0x00010001u, 0x43004300u);
+        l = lop3_and_or(w[1] >> 14, 0x00020002u, l);
+        h[15] = lop3_and_or(w[2] >> 13, 0x00040004u, l);
+    }
+};
+// Position of code c (0..31) of a lane's 32-code run in that order: 2 * h_index + (0 = low half, 1 = high half).
+template <int BITS> __device__ __forceinline__ int frag_pos(int c)
+{
+    if (BITS == 4) {
+        const int i = c >> 3, e8 = c & 7;
+        return 2 * (4 * i + (e8 & 3)) + (e8 >> 2);
+    }
+    if (c >= 30) return 2 * 15 + (c - 30);
+    const int i = c / 10, f = c - 10 * i;
+    return (f < 5) ? 2 * (5 * i + f) : 2 * (5 * i + f - 5) + 1;
+}
+constexpr int kCHGW = 8;                     // groups of a stage in the 16-bit form: one per compute warp
+static_assert(kCHGW == kCW, "the 16-bit form gives every compute warp one group of a stage");
+
+// x of this CTA's K slice (groups g_begin .. g_begin + g_count) for M tokens: per token and group the sixteen
+// fragment-order pairs of a lane's run as 16-byte units [h_index / 4][lane t][h_index % 4]; (P, X0) per (group, token).
+template <int BITS, typename T, int MT>
+__device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, int g_begin, int g_count)
+{
+    const int tid = threadIdx.x, lane = tid & 31, nthr = kCW * 32;
+    T *s_x = reinterpret_cast<T *>(smem + p.off_x);
+    float2 *s_px = reinterpret_cast<float2 *>(smem + p.off_px);
+    const T *x = static_cast<const T *>(p.x);
+    const int runs_per_tok = g_count * 4, nruns = p.M * runs_per_tok;        // multiples of 4
+    constexpr int mp = 8 * MT;                                               // token slots of the (P, X0) table
+    for (int i = tid; i < g_count * mp; i += nthr)                           // tokens beyond M contribute nothing
+        if (i % mp >= p.M) s_px[i] = make_float2(0.f, 0.f);
+#pragma unroll 1
+    for (int base = 0; base < nruns; base += nthr) {
+        const int idx = base + tid;                                          // whole quads are valid or not
+        const bool valid = idx < nruns;
+        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+        uint4 xv[4];
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + (size_t)g_begin * kGroupFast + run * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        if (base == 0) {                                                     // our loads of x are on their way
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);
+        }
+        const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
+        uint32_t h[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) h[i] = 0u;
+        float psum = 0.f, xsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const int pos = frag_pos<BITS>(c);                               // folds to a constant
+            T xe;
+            *reinterpret_cast<uint16_t *>(&xe) = e[c];
+            const float xf = ActTraits<T>::to_float(xe);
+            // exact division by the field weight (a power of two; up to fp16 underflow).  P is summed from the
+            // stored value, so the MMA's bias term cancels exactly.
+            const T xs = ActTraits<T>::from_float(ldexpf(xf, -Unpack16<BITS, T>::div_log2(c)));
+            h[pos >> 1] |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&xs)) << (16 * (pos & 1));
+            psum = fmaf(Unpack16<BITS, T>::kMagic, ActTraits<T>::to_float(xs), psum);
+            xsum += xf;
+        }
+        if (valid) {
+            uint4 *dst = reinterpret_cast<uint4 *>(s_x + (size_t)m * p.x_pitch + (run >> 2) * kGroupFast);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) dst[q4 * 4 + (run & 3)] = make_uint4(h[4 * q4], h[4 * q4 + 1], h[4 * q4 + 2], h[4 * q4 + 3]);
+        }
+        // the four runs of one (token, group) sit in four consecutive lanes
+        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+        if (valid && (run & 3) == 0) s_px[(run >> 2) * mp + m] = make_float2(psum, xsum);
+    }
+}
+
+// Compute warps of the 16-bit form: stages of eight groups, one group per warp; MT blocks of eight tokens.
+template <int BITS, typename T, int MT>
+__device__ __forceinline__ bool compute_w16(const GemvParams &p, uint8_t *smem, int warp, int lane, int ntile, int g_begin, int g_count)
+{
+    constexpr int NW = (BITS == 4) ? 4 : 3;
+    constexpr int GB = (BITS == 4) ? 64 : 48;
+    const int g = lane >> 2, tq = lane & 3;
+    const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
+    const int G = p.G, NS = p.NS, M = p.M, SPT = (g_count + kCHGW - 1) / kCHGW;
+    const uint32_t w_lane = sbase + p.off_ring + (uint32_t)(warp * (kTile * GB) + g * GB + tq * (GB / 4));
+    const uint32_t meta0 = sbase + p.off_meta, zoff = (uint32_t)p.meta_pitch, row8 = (uint32_t)(8 * G * 2);
+    const uint32_t px_lane = sbase + p.off_px + (uint32_t)(2 * tq) * 8u;
+    const uint32_t x_lane = sbase + p.off_x + (uint32_t)tq * 16u;
+    const uint32_t x_tok = (uint32_t)p.x_pitch * 2u;
+    float *s_seg = reinterpret_cast<float *>(smem + p.off_seg);
+    int slot = 0, mi = 0, buf = 0;
+    uint32_t par = 0u, dphase = 1u;
+    bool first = true, dfirst = true;
+    for (int ts = 0; ts < ntile; ++ts) {
+        float acc[MT][4];
+#pragma unroll
+        for (int b = 0; b < MT; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+        const uint32_t mslot = meta0 + (uint32_t)mi * 2u * zoff + (uint32_t)(g * G * 2);
+        if (++mi == p.nmeta) mi = 0;
+        for (int st = 0; st < SPT; ++st) {
+            if (!mbar_wait(bars + 8u * (kBarFull + slot), par)) return false;
+            if (first) mark(p, 4);
+            first = false;
+            const int gl = st * kCHGW + warp;                          // group of the slice
+            if (gl < g_count) {
+                const uint32_t wa = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes;
+                uint32_t w0[NW], w1[NW];
+                if constexpr (BITS == 4) {
+                    const uint4 va = lds_v4(wa), vb = lds_v4(wa + 8 * GB);
+                    w0[0] = va.x; w0[1] = va.y; w0[2] = va.z; w0[3] = va.w;
+                    w1[0] = vb.x; w1[1] = vb.y; w1[2] = vb.z; w1[3] = vb.w;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < NW; ++i) {
+                        w0[i] = lds_u32(wa + 4 * i);
+                        w1[i] = lds_u32(wa + 8 * GB + 4 * i);
+                    }
+                }
+                const uint32_t ma = mslot + (uint32_t)(g_begin + gl) * 2u;
+                const float sg = half_bits_to_float(lds_u16(ma)), zg = half_bits_to_float(lds_u16(ma + zoff));
+                const float sh = half_bits_to_float(lds_u16(ma + row8)), zh = half_bits_to_float(lds_u16(ma + row8 + zoff));
+                const float szg = sg * zg, szh = sh * zh;
+                uint32_t ha[16], hb[16];
+                Unpack16<BITS, T>::run(w0, ha);
+                Unpack16<BITS, T>::run(w1, hb);
+#pragma unroll
+                for (int b = 0; b < MT; ++b) {
+                    // (P, X0) of tokens 8b + 2tq and 8b + 2tq + 1 for this group; one MMA chain starts at -P
+                    const float4 px = lds_f4(px_lane + (uint32_t)(gl * 8 * MT + 8 * b) * 8u);
+                    float t0[4] = {-px.x, -px.z, -px.x, -px.z}, t1[4] = {0.f, 0.f, 0.f, 0.f};
+                    const int token = 8 * b + g;                        // as an MMA column
+                    const uint32_t xg = x_lane + (uint32_t)token * x_tok + (uint32_t)gl * (kGroupFast * 2);
+                    const uint32_t on = token < M ? 1u : 0u;
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const uint4 xv = lds_v4_if(xg + (uint32_t)q4 * 64u, on);
+                        if (q4 & 1) {
+                            Mma16<T>::run(t1, ha[4 * q4 + 0], hb[4 * q4 + 0], ha[4 * q4 + 1], hb[4 * q4 + 1], xv.x, xv.y);
+                            Mma16<T>::run(t1, ha[4 * q4 + 2], hb[4 * q4 + 2], ha[4 * q4 + 3], hb[4 * q4 + 3], xv.z, xv.w);
+                        } else {
+                            Mma16<T>::run(t0, ha[4 * q4 + 0], hb[4 * q4 + 0], ha[4 * q4 + 1], hb[4 * q4 + 1], xv.x, xv.y);
+                            Mma16<T>::run(t0, ha[4 * q4 + 2], hb[4 * q4 + 2], ha[4 * q4 + 3], hb[4 * q4 + 3], xv.z, xv.w);
+                        }
+                    }
+                    // s (mma - P) - (s z) X0
+                    acc[b][0] = fmaf(-szg, px.y, fmaf(sg, t0[0] + t1[0], acc[b][0]));
+                    acc[b][1] = fmaf(-szg, px.w, fmaf(sg, t0[1] + t1[1], acc[b][1]));
+                    acc[b][2] = fmaf(-szh, px.y, fmaf(sh, t0[2] + t1[2], acc[b][2]));
+                    acc[b][3] = fmaf(-szh, px.w, fmaf(sh, t0[3] + t1[3], acc[b][3]));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+            if (++slot == NS) {
+                slot = 0;
+                par ^= 1u;
+            }
+        }
+        // ---- this warp's partial tile [token][16 rows] for the epilogue warp ----
+        if (!dfirst && !mbar_wait(bars + 8u * (kBarSegFree + buf), dphase)) return false;
+        float *dst = s_seg + (size_t)(buf * kCW + warp) * M * kTile;
+#pragma unroll
+        for (int b = 0; b < MT; ++b) {
+            const int t0 = 8 * b + 2 * tq;
+            if (t0 < M) {
+                dst[t0 * kTile + g] = acc[b][0];
+                dst[t0 * kTile + g + 8] = acc[b][2];
+            }
+            if (t0 + 1 < M) {
+                dst[(t0 + 1) * kTile + g] = acc[b][1];
+                dst[(t0 + 1) * kTile + g + 8] = acc[b][3];
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFull + buf));
+        mark(p, ts == 0 ? 5 : 6);
+        if (++buf == p.nbuf) {
+            buf = 0;
+            dphase = dfirst ? 0u : dphase ^ 1u;
+            dfirst = false;
+        }
+    }
+    return true;
+}
+
+// Epilogue warp of the 16-bit form.  Lane (g, tq) finishes rows g and g + 8 of the tile for the tokens 4cb + tq
+// (cb = column block of the up-projection MMA, whose columns 2tq, 2tq + 1 are that token's two 16-bit terms).
+// With K slices the tile's partial sums meet in scratch and the slice that arrives last finishes the tile.
+template <typename T>
+__device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem, const CUtensorMap *bmap, int lane, int tile_first,
+                                              int ntile, int slice)
+{
+    const int g = lane >> 2, tq = lane & 3;
+    const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
+    const uint32_t bring = sbase + p.off_B;
+    const int rank = p.rank, M = p.M, nkb = rank / 16, ncb = (M + 3) / 4, SK = p.SK;
+    const int nbox = (rank + 63) / 64;
+    const uint32_t box_bytes = (uint32_t)kTile * (uint32_t)p.b_box_cols * 2u;
+    auto request_b = [&](int ts) {
+        const uint32_t bar = bars + 8u * (kBarB + ts % p.nb);
+        mbar_expect_tx(bar, (uint32_t)nbox * box_bytes);
+        for (int b = 0; b < nbox; ++b)
+            tma_load_2d(bring + (uint32_t)(ts % p.nb) * (uint32_t)p.b_slot_bytes + (uint32_t)b * box_bytes, bmap, b * 64,
+                        (tile_first + ts) * kTile, bar);
+    };
+    if (rank > 0 && lane == 0)
+        for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
+
+    pdl_wait();
+    mark(p, 2);
+
+    float isc = 1.f;
+    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // [cb][kb][lane][2]
+    if (rank > 0) {
+        float *s_t = reinterpret_cast<float *>(smem + p.off_t);
+        float amax = 0.f;
+        const size_t slot_elems = (size_t)M * rank;
+        bool ok = false;
+        for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
+            bool all = true;
+            amax = 0.f;
+            for (int i = lane; i < M * rank; i += 32) {
+                float v = 0.f;
+                for (int c0 = 0; c0 < p.n_t; c0 += 8) {           // eight slots in flight, added in slot order
+                    float2 part[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v += part[u].x;
+                        all = all && (part[u].y == 1.f);
+                    }
+                }
+                s_t[i] = v;
+                amax = fmaxf(amax, fabsf(v));
+            }
+            ok = __all_sync(0xffffffffu, all);
+            if (!ok && look > 256) __nanosleep(64);
+        }
+        if (!ok) return false;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        __syncwarp();
+        const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 1u), 254u);
+        const uint32_t sb = min(max(268u - ex, 1u), 254u);
+        const float sc = __uint_as_float(sb << 23);
+        isc = __uint_as_float((254u - sb) << 23);
+        for (int cb = 0; cb < ncb; ++cb) {
+            const int tok = 4 * cb + (g >> 1), part = g & 1;   // as an MMA column: token and (rounded value | remainder)
+            for (int kb = 0; kb < nkb; ++kb) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t pk = 0;
+                    if (tok < M) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float v = s_t[tok * rank + kb * 16 + h * 8 + 2 * tq + e] * sc;
+                            const T hi = ActTraits<T>::from_float(v);
+                            const T lo = ActTraits<T>::from_float(v - ActTraits<T>::to_float(hi));
+                            const T pick = part ? lo : hi;
+                            pk |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&pick)) << (16 * e);
+                        }
+                    }
+                    s_tf[((size_t)(cb * nkb + kb) * 32 + lane) * 2 + h] = pk;
+                }
+            }
+        }
+        __syncwarp();
+    }
+    mark(p, 3);
+
+    const float *s_seg = reinterpret_cast<const float *>(smem + p.off_seg);
+    T *y = static_cast<T *>(p.y);
+    const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
+    const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
+    for (int ts = 0; ts < ntile; ++ts) {
+        const int buf = ts % p.nbuf, tile = tile_first + ts;
+        if (!mbar_wait_idle_warp(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
+        if (ts == 0) mark(p, 4);
+        float vg[4] = {0.f, 0.f, 0.f, 0.f}, vh[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+            const int tok = 4 * cb + tq;
+            if (tok < M) {
+                const float *src = s_seg + ((size_t)buf * kCW * M + tok) * kTile;
+#pragma unroll
+                for (int w = 0; w < kCW; ++w) {
+                    vg[cb] += src[(size_t)w * M * kTile + g];
+                    vh[cb] += src[(size_t)w * M * kTile + g + 8];
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
+        bool finish = true;
+        if (SK > 1) {
+            // this slice's partial tile to scratch; whoever counts in last adds the slices in order and finishes
+            float *pt = p.part + ((size_t)tile * SK) * M * kTile;
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) {
+                const int tok = 4 * cb + tq;
+                if (tok < M) {
+                    __stcg(pt + ((size_t)slice * M + tok) * kTile + g, vg[cb]);
+                    __stcg(pt + ((size_t)slice * M + tok) * kTile + g + 8, vh[cb]);
+                }
+            }
+            __threadfence();
+            __syncwarp();
+            int last = 0;
+            if (lane == 0) last = (atomicAdd(p.tctr + tile, 1) == SK - 1) ? 1 : 0;
+            last = __shfl_sync(0xffffffffu, last, 0);
+            finish = last != 0;
+            if (finish) {
+                __threadfence();
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) {
+                    const int tok = 4 * cb + tq;
+                    vg[cb] = vh[cb] = 0.f;
+                    if (tok < M)
+                        for (int s2 = 0; s2 < SK; ++s2) {
+                            vg[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g);
+                            vh[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g + 8);
+                        }
+                }
+                if (lane == 0) atomicExch(p.tctr + tile, 0);
+            }
+        }
+        if (rank > 0) {
+            const int bs = ts % p.nb;
+            if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
+            if (finish) {
+                const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
+                float d[4][4];
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) d[cb][0] = d[cb][1] = d[cb][2] = d[cb][3] = 0.f;
+#pragma unroll 1
+                for (int kc = 0; 4 * kc < nkb; ++kc) {
+                    uint32_t af[4][4];
+                    const uint32_t bx = bt + (uint32_t)kc * box_bytes;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+                        const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                        const bool on = 4 * kc + q < nkb;
+                        af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
+                        af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
+                        af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
+                        af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
+                    }
+#pragma unroll
+                    for (int cb = 0; cb < 4; ++cb) {
+                        if (cb < ncb) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                if (4 * kc + q < nkb) {
+                                    const uint32_t ta = tf_lane + (uint32_t)((cb * nkb + 4 * kc + q) * 32) * 8u;
+                                    Mma16<T>::run(d[cb], af[q][0], af[q][1], af[q][2], af[q][3], lds_u32(ta), lds_u32(ta + 4u));
+                                }
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) {
+                    vg[cb] = fmaf(d[cb][0] + d[cb][1], isc, vg[cb]);
+                    vh[cb] = fmaf(d[cb][2] + d[cb][3], isc, vh[cb]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
+        }
+        if (finish) {
+            const int n = tile * kTile + g;
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) {
+                const int tok = 4 * cb + tq;
+                if (tok < M) {
+                    if (n < p.N) y[(size_t)tok * p.N + n] = ActTraits<T>::from_float(vg[cb]);
+                    if (n + 8 < p.N) y[(size_t)tok * p.N + n + 8] = ActTraits<T>::from_float(vh[cb]);
+                }
+            }
+        }
+        mark(p, ts == 0 ? 5 : 6);
+    }
+    if (rank > 0) {
+        int last = 0;
+        if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            for (int i = lane; i < p.n_t * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
+            if (lane == 0) atomicExch(p.ctr + 1, 0);
+        }
+    }
+    return true;
+}
+
 // ------------------------------------------------------------------------ t CTA
 // Block c of the first n_t: t_kb blocks of 64 input channels of all `rank` rows of A in shared memory
 // (TMA, 128-byte swizzle), against the same channels of x read straight from global memory as MMA
@@ -874,6 +1368,61 @@ gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
     if (!ok && lane == 0) give_up(p);
 }
 
+
+// The 16-bit form: main CTA `cta` is row block cta / SK, K slice cta % SK.
+template <int BITS, typename T, int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemv_wide_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap bmap,
+                 const __grid_constant__ CUtensorMap amap)
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();
+    mark(p, 0);
+    if ((int)blockIdx.x < p.n_t) {
+        t_cta<T>(p, smem, &amap, (int)blockIdx.x);
+        return;
+    }
+    const int cta = (int)blockIdx.x - p.n_t;
+    const int rb = cta / p.SK, slice = cta - rb * p.SK;
+    const int tile_first = (int)((long long)rb * p.NT / p.R);
+    const int ntile = (int)((long long)(rb + 1) * p.NT / p.R) - tile_first;
+    const int g_begin = slice * p.slice_groups, g_count = min(p.slice_groups, p.G - g_begin);
+    const uint32_t bars = smem_u32(smem) + p.off_bar;
+    if (tid == 0) {
+        prefetch_tensormap(&wmap);
+        if (p.rank > 0) prefetch_tensormap(&bmap);
+        for (int i = 0; i < p.NS; ++i) {
+            mbar_init(bars + 8u * (kBarFull + i), 1);
+            mbar_init(bars + 8u * (kBarEmpty + i), kCW);
+        }
+        for (int i = 0; i < p.nbuf; ++i) {
+            mbar_init(bars + 8u * (kBarSegFull + i), kCW);
+            mbar_init(bars + 8u * (kBarSegFree + i), 1);
+        }
+        for (int i = 0; i < p.nb; ++i) mbar_init(bars + 8u * (kBarB + i), 1);
+        mbar_init(bars + 8u * kBarXReq, kCW);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    mark(p, 1);
+    bool ok = true;
+    if (warp == kProdWarp) {
+        if (lane == 0) ok = produce(p, smem, &wmap, tile_first, ntile, g_begin, g_count, kCHGW);
+    } else if (warp == kEpiWarp) {
+        ok = epilogue_wide<T>(p, smem, &bmap, lane, tile_first, ntile, slice);
+    } else {
+        pdl_wait();                                  // x may come from the preceding kernel
+        mark(p, 2);
+        convert_x16<BITS, T, MT>(p, smem, g_begin, g_count);
+        named_barrier_sync(1, kCW * 32);
+        mark(p, 3);
+        ok = compute_w16<BITS, T, MT>(p, smem, warp, lane, ntile, g_begin, g_count);
+    }
+    if (!ok && lane == 0) give_up(p);
+}
+
 // ------------------------------------------------------------------ host side
 template <typename X> struct TypeTag { using type = X; };
 
@@ -983,6 +1532,104 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     return pl;
 }
 
+// Plan of the 16-bit form (3 <= M <= 16): one CTA per SM; K in SK slices when x of all K does not fit.
+Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
+{
+    Plan pl{};
+    pl.ok = false;
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return pl;
+        if (cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return pl;
+    }
+    GemvParams &p = pl.p;
+    const int GB = (a.bits == 4) ? 64 : 48, G = a.K / kGroupFast, MT = (a.M + 7) / 8;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.G = G; p.rank = a.rank;
+    p.NT = (a.N + kTile - 1) / kTile;
+    const int want = tune.max_ctas > 0 ? tune.max_ctas : g_sm_count;
+    p.stage_bytes = kTile * kCHGW * GB;
+    p.meta_pitch = (int)align_up((size_t)kTile * G * 2, 16);
+    p.n_t = 0;
+    p.t_kb = 0;
+    const int nblk = (a.K + kTKB - 1) / kTKB;
+    if (a.rank > 0) {
+        const int per = std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128)));
+        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
+        p.t_kb = (nblk + p.n_t - 1) / p.n_t;
+        p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
+    }
+    // K slices: the smallest power of two whose slice of x (16-bit, all tokens) stays below 100 KB
+    int sk = 1;
+    auto slice_of = [&](int k) { return ((G + k - 1) / k + kCHGW - 1) / kCHGW * kCHGW; };
+    while (sk < 16 && (size_t)a.M * ((size_t)slice_of(sk) * kGroupFast + 32) * 2 > 100 * 1024) sk *= 2;
+    p.slice_groups = slice_of(sk);
+    p.SK = (G + p.slice_groups - 1) / p.slice_groups;
+    p.x_pitch = p.slice_groups * kGroupFast + 32;
+    p.R = std::max(1, std::min(std::max(want - p.n_t, want / 2) / p.SK, p.NT));
+    p.n_main = p.R * p.SK;
+    const int nseg = (p.NT + p.R - 1) / p.R;
+    // stages per tile of the shortest slice (the last one): the producer runs at most NS stages ahead, that is
+    // NS / SPT tiles, and every tile ahead holds a slot of scales and zero points
+    const int last_groups = G - (p.SK - 1) * p.slice_groups;
+    const int SPT = (std::min(p.slice_groups, last_groups) + kCHGW - 1) / kCHGW;
+    p.b_box_cols = a.rank <= 16 ? 16 : (a.rank <= 32 ? 32 : 64);
+    p.b_swz = p.b_box_cols >= 64 ? 7 : (p.b_box_cols >= 32 ? 3 : 1);
+    p.b_slot_bytes = (int)align_up((size_t)((a.rank + 63) / 64) * kTile * p.b_box_cols * 2, 1024);
+    p.nbuf = std::min(kMaxBuf, std::max(2, std::min(nseg, 3)));
+    p.nb = a.rank > 0 ? std::min(kMaxB, std::max(1, std::min(nseg, 2))) : 0;
+    const int ncb = (a.M + 3) / 4, nkb = a.rank / 16;
+    auto layout = [&](int ns) {
+        p.NS = ns;
+        p.nmeta = std::min(kMaxMeta, (ns - 1) / SPT + 2);
+        size_t off = 0;
+        p.off_bar = (int)off;
+        off += (size_t)kNumBars * 8;
+        off = align_up(off, 16);
+        p.off_px = (int)off;
+        off += (size_t)p.slice_groups * 8 * MT * 8;
+        off = align_up(off, 128);
+        p.off_x = (int)off;
+        off += (size_t)a.M * p.x_pitch * 2;
+        off = align_up(off, 128);
+        p.off_meta = (int)off;
+        off += (size_t)p.nmeta * 2 * p.meta_pitch;
+        off = align_up(off, 128);
+        p.off_seg = (int)off;
+        off += (size_t)p.nbuf * kCW * a.M * kTile * 4;
+        off = align_up(off, 128);
+        p.off_t = (int)off;
+        off += (size_t)a.M * a.rank * 4;
+        off = align_up(off, 16);
+        p.off_tf = (int)off;
+        off += (size_t)ncb * nkb * 32 * 8;
+        off = align_up(off, 1024);
+        p.off_B = (int)off;
+        off += (size_t)p.nb * p.b_slot_bytes;
+        off = align_up(off, 1024);
+        p.off_ring = (int)off;
+        off += (size_t)ns * p.stage_bytes;
+        return off;
+    };
+    int ns = std::min(kMaxNS, (kMaxMeta - 2) * SPT + 1);
+    while (ns > 2 && layout(ns) > kSmemMax - 2048) --ns;
+    const size_t need = layout(ns);
+    if (need > kSmemMax - 2048) return pl;
+    p.off_tab = p.off_zero = 0;
+    p.off_tA = 1024;
+    p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
+    const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
+    if (need_t > kSmemMax - 2048) return pl;
+    pl.smem = std::max(need, need_t) + 1024;
+    p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
+    p.test_skip_arrive = tune.test_skip_arrive;
+    p.dbg = tune.dbg;
+    pl.ok = true;
+    if (getenv("FBQ_PLAN"))
+        fprintf(stderr, "gemv wide plan M %d N %d K %d r %d: R %d SK %d (slice %d groups) n_t %d NS %d nmeta %d nbuf %d nb %d smem %zu (t CTA %zu)\n",
+                a.M, a.N, a.K, a.rank, p.R, p.SK, p.slice_groups, p.n_t, p.NS, p.nmeta, p.nbuf, p.nb, need, need_t);
+    return pl;
+}
+
 // Tensor maps are encoded on the host once per (pointer, shape) and kept: they hold addresses and
 // extents only, never data.
 struct MapKey {
@@ -1027,6 +1674,31 @@ cudaError_t cached_map(CUtensorMap *out, const MapKey &key, CUtensorMapDataType 
     return cudaSuccess;
 }
 
+template <int BITS, typename T, int MT>
+cudaError_t launch_wide(const Plan &pl, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &amap, bool pdl, cudaStream_t s)
+{
+    auto kern = gemv_wide_kernel<BITS, T, MT>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(pl.p.n_t + pl.p.n_main));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, pl.p, wmap, bmap, amap);
+}
+
 template <int BITS, typename T, int M>
 cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &amap, bool pdl,
                            cudaStream_t s)
@@ -1060,7 +1732,7 @@ cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtens
 bool gemv_supported(const LinearArgs &a)
 {
     if (a.group != kGroupFast || a.K % kGroupFast != 0 || a.K < kGroupFast) return false;
-    if (a.M < 1 || a.M > 2) return false;
+    if (a.M < 1 || a.M > kDecodeMaxM) return false;
     if (a.N % 8 != 0 || a.N < 8) return false;
     if (a.rank % 16 != 0 || a.rank > 128) return false;
     auto mis16 = [](const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
@@ -1068,19 +1740,24 @@ bool gemv_supported(const LinearArgs &a)
     return true;
 }
 
-void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters)
+void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters, size_t *partial_floats)
 {
-    const Plan pl = make_plan(a, tune);
+    const bool wide = a.M > 2;
+    const Plan pl = wide ? make_plan_wide(a, tune) : make_plan(a, tune);
     *tpart_floats = (size_t)2 * std::max(pl.p.n_t, 1) * a.M * std::max(a.rank, 1);
-    *counters = 8;
+    *counters = 8 + (wide ? pl.p.NT : 0);
+    *partial_floats = (wide && pl.p.SK > 1) ? (size_t)pl.p.NT * pl.p.SK * a.M * kTile : 0;
 }
 
 cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tune, cudaStream_t s, int *launches)
 {
-    Plan pl = make_plan(a, tune);
+    const bool wide = a.M > 2;
+    Plan pl = wide ? make_plan_wide(a, tune) : make_plan(a, tune);
     if (!pl.ok) return cudaErrorInvalidConfiguration;
     GemvParams &p = pl.p;
     p.x = a.x; p.scales = a.scales; p.zeros = a.zeros; p.y = a.y;
+    p.part = ws.partial;
+    p.tctr = ws.counters + 8;
     p.tpart = reinterpret_cast<float2 *>(ws.tslots);
     p.ctr = ws.counters;
     p.status = ws.counters + kCtrStatus;
@@ -1096,8 +1773,9 @@ cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tu
         const cuuint32_t wpg = (a.bits == 4) ? 16 : 12;
         const cuuint64_t dims[3] = {wpg, (cuuint64_t)a.N, (cuuint64_t)p.G};
         const cuuint64_t strides[2] = {(cuuint64_t)p.G * wpg * 4, (cuuint64_t)wpg * 4};
-        const cuuint32_t box[3] = {wpg, (cuuint32_t)kTile, (cuuint32_t)kCHG};
-        const MapKey key{a.qw, 0, (int)wpg, a.N, p.G, kTile, kCHG};
+        const int chg = wide ? kCHGW : kCHG;
+        const cuuint32_t box[3] = {wpg, (cuuint32_t)kTile, (cuuint32_t)chg};
+        const MapKey key{a.qw, 0, (int)wpg, a.N, p.G, kTile, chg};
         if (cudaError_t e = cached_map(&wmap, key, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
             e != cudaSuccess)
             return e;
@@ -1122,6 +1800,8 @@ cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tu
     auto go = [&](auto bits, auto type) {
         using T = typename decltype(type)::type;
         constexpr int B = decltype(bits)::value;
+        if (a.M > 8) return launch_wide<B, T, 2>(pl, wmap, bmap, amap, pdl, s);
+        if (a.M > 2) return launch_wide<B, T, 1>(pl, wmap, bmap, amap, pdl, s);
         return a.M == 1 ? launch_variant<B, T, 1>(pl, wmap, bmap, amap, pdl, s) : launch_variant<B, T, 2>(pl, wmap, bmap, amap, pdl, s);
     };
     if (a.bits == 4)
