@@ -57,8 +57,8 @@ typedef enum {
 typedef enum {
     FBQ_KERNEL_NONE = -1,
     FBQ_KERNEL_GENERIC = 0,   /* any supported shape, CUDA cores, two launches if rank>0 */
-    FBQ_KERNEL_DECODE = 1,    /* M <= 16 (chosen for M <= 6): fused streaming kernels, one launch */
-    FBQ_KERNEL_PREFILL = 2    /* tcgen05 / TMEM tensor-core kernel, one launch (chosen from M = 7) */
+    FBQ_KERNEL_DECODE = 1,    /* M <= 16 (chosen for M <= 8, and to 16 at rank 0): fused streaming kernels, one launch */
+    FBQ_KERNEL_PREFILL = 2    /* tcgen05 / TMEM tensor-core kernel, one launch (chosen from M = 9, or 7 outside the streaming kernel's domain) */
 } fbq_kernel;
 
 /* Number of uint32 words of a packed N x K code matrix: N*K/8 (4 bits) or
@@ -85,12 +85,13 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
 /* The fused layer, fp16 activations: x, A, B, y are fp16; scales, zeros fp16.
  *   rank == 0: A and B are ignored (may be NULL); y is the main path alone.
  *   M == 0: nothing is done.
- * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128
- * and rank a multiple of 8 not above 256 -> decode kernels for M <= 4 with rank <= 128 and for
- * M = 5, 6 with M * rank <= 128, else prefill kernel (N a multiple of 8 and 16-byte aligned operands; otherwise the decode
- * kernel up to M = 16); everything else that is well formed -> generic kernel.
- * Of the decode kernels the streaming one ("gemv" option, default on) runs M <= 2 with N a multiple of
- * 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; the other decode kernel takes the rest.
+ * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128 and rank a multiple of 8
+ * not above 256 are the fast kernels' domain.  The streaming decode kernel ("gemv" option, default on)
+ * needs N a multiple of 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; there
+ * it takes M <= 8 at every rank and M <= 16 without a sub-branch.  Elsewhere the other decode kernel
+ * takes M <= 4 with rank <= 128 and M = 5, 6 with M * rank <= 128.  The prefill kernel (N a multiple of
+ * 8) takes the rest of the domain; shapes outside its domain stay with a decode kernel up to M = 16;
+ * everything else that is well formed -> generic kernel.
  * Well formed means bits in {3,4}, group a multiple of 8 (4 bits) or 32
  * (3 bits) dividing K, rank >= 0.  Zero points are taken as stored: every kernel accepts
  * integer-valued fp16 zero points of either sign and beyond 2^bits - 1 (what fbq_quantize_feedback

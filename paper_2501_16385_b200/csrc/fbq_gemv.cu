@@ -82,6 +82,7 @@ struct GemvParams {
     int off_px, off_tf;                     // (P, X0) table; t as MMA column operands
     float *part;                            // [tile][slice][M][16] fp32 partial tiles (SK > 1)
     int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
+    int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
     int dbg;
@@ -857,19 +858,27 @@ __device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, 
     constexpr int mp = 8 * MT;                                               // token slots of the (P, X0) table
     for (int i = tid; i < g_count * mp; i += nthr)                           // tokens beyond M contribute nothing
         if (i % mp >= p.M) s_px[i] = make_float2(0.f, 0.f);
+    auto fetch = [&](int base, uint4 (&v)[4]) {
+        const int idx = base + tid;
+        const bool valid = idx < nruns;
+        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + (size_t)g_begin * kGroupFast + run * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    uint4 xn[4];
+    fetch(0, xn);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);   // our loads of x are on their way
 #pragma unroll 1
     for (int base = 0; base < nruns; base += nthr) {
         const int idx = base + tid;                                          // whole quads are valid or not
         const bool valid = idx < nruns;
         const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
         uint4 xv[4];
-        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + (size_t)g_begin * kGroupFast + run * 32);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
-        if (base == 0) {                                                     // our loads of x are on their way
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);
-        }
+        for (int i = 0; i < 4; ++i) xv[i] = xn[i];
+        if (base + nthr < nruns) fetch(base + nthr, xn);                     // the next batch's loads, before this batch's work
         const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
         uint32_t h[16];
 #pragma unroll
@@ -883,7 +892,7 @@ __device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, 
             const float xf = ActTraits<T>::to_float(xe);
             // exact division by the field weight (a power of two; up to fp16 underflow).  P is summed from the
             // stored value, so the MMA's bias term cancels exactly.
-            const T xs = ActTraits<T>::from_float(ldexpf(xf, -Unpack16<BITS, T>::div_log2(c)));
+            const T xs = ActTraits<T>::from_float(xf * (1.f / (float)(1 << Unpack16<BITS, T>::div_log2(c))));
             h[pos >> 1] |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&xs)) << (16 * (pos & 1));
             psum = fmaf(Unpack16<BITS, T>::kMagic, ActTraits<T>::to_float(xs), psum);
             xsum += xf;
@@ -1044,25 +1053,34 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
         float amax = 0.f;
         const size_t slot_elems = (size_t)M * rank;
+        const int s_first = p.t_final ? p.n_t : 0, s_end = p.t_final ? p.n_t + 1 : p.n_t;
         bool ok = false;
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
-            for (int i = lane; i < M * rank; i += 32) {
-                float v = 0.f;
-                for (int c0 = 0; c0 < p.n_t; c0 += 8) {           // eight slots in flight, added in slot order
+            for (int i0 = 0; i0 < M * rank; i0 += 32 * 8) {      // eight entries per lane (and slot) in flight
+                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                for (int c = s_first; c < s_end; ++c) {           // slots added in order
                     float2 part[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        part[u] = (i < M * rank) ? __ldcg(p.tpart + (size_t)c * slot_elems + i) : make_float2(0.f, 1.f);
+                    }
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        v += part[u].x;
+                        v[u] += part[u].x;
                         all = all && (part[u].y == 1.f);
                     }
                 }
-                s_t[i] = v;
-                amax = fmaxf(amax, fabsf(v));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + u * 32 + lane;
+                    if (i < M * rank) {
+                        s_t[i] = v[u];
+                        amax = fmaxf(amax, fabsf(v[u]));
+                    }
+                }
             }
             ok = __all_sync(0xffffffffu, all);
             if (!ok && look > 256) __nanosleep(64);
@@ -1103,6 +1121,98 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
     T *y = static_cast<T *>(p.y);
     const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
     const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
+    // adds t.B^T (rows of B from slot ts % nb) to the sums of a tile and stores its rows of y
+    auto finish_tile = [&](int ts, float (&vg)[4], float (&vh)[4]) -> bool {
+        const int tile = tile_first + ts;
+        if (rank > 0) {
+            const int bs = ts % p.nb;
+            if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
+            const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
+            float d[4][4];
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) d[cb][0] = d[cb][1] = d[cb][2] = d[cb][3] = 0.f;
+#pragma unroll 1
+            for (int kc = 0; 4 * kc < nkb; ++kc) {
+                uint32_t af[4][4];
+                const uint32_t bx = bt + (uint32_t)kc * box_bytes;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+                    const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                    const bool on = 4 * kc + q < nkb;
+                    af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
+                    af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
+                    af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
+                    af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
+                }
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) {
+                    if (cb < ncb) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (4 * kc + q < nkb) {
+                                const uint32_t ta = tf_lane + (uint32_t)((cb * nkb + 4 * kc + q) * 32) * 8u;
+                                Mma16<T>::run(d[cb], af[q][0], af[q][1], af[q][2], af[q][3], lds_u32(ta), lds_u32(ta + 4u));
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) {
+                vg[cb] = fmaf(d[cb][0] + d[cb][1], isc, vg[cb]);
+                vh[cb] = fmaf(d[cb][2] + d[cb][3], isc, vh[cb]);
+            }
+        }
+        const int n = tile * kTile + g;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+            const int tok = 4 * cb + tq;
+            if (tok < M) {
+                if (n < p.N) y[(size_t)tok * p.N + n] = ActTraits<T>::from_float(vg[cb]);
+                if (n + 8 < p.N) y[(size_t)tok * p.N + n + 8] = ActTraits<T>::from_float(vh[cb]);
+            }
+        }
+        return true;
+    };
+    // B slot of tile ts is free (used or not needed): request the rows of a later tile into it
+    auto release_b = [&](int ts) -> bool {
+        if (rank == 0) return true;
+        // a slice that does not finish the tile never reads its rows of B, but their copy must have landed
+        // before the slot is handed out again
+        if (!mbar_wait(bars + 8u * (kBarB + ts % p.nb), (uint32_t)(ts / p.nb) & 1u)) return false;
+        __syncwarp();
+        if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
+        return true;
+    };
+    // With K slices: whether the tile is ours to finish shows in the arrival count, which is looked at one tile
+    // later so that the round trip of its atomic overlaps the next tile's sums.
+    int pend_ts = -1, pend_old = 0;
+    auto settle = [&](void) -> bool {
+        if (pend_ts < 0) return true;
+        const int last = __shfl_sync(0xffffffffu, pend_old, 0) == SK - 1;
+        if (last) {
+            const int tile = tile_first + pend_ts;
+            const float *pt = p.part + ((size_t)tile * SK) * M * kTile;
+            __threadfence();
+            float vg[4], vh[4];
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) {
+                const int tok = 4 * cb + tq;
+                vg[cb] = vh[cb] = 0.f;
+                if (tok < M)
+                    for (int s2 = 0; s2 < SK; ++s2) {                   // slices added in order, whoever finishes
+                        vg[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g);
+                        vh[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g + 8);
+                    }
+            }
+            if (lane == 0) atomicExch(p.tctr + tile, 0);
+            if (!finish_tile(pend_ts, vg, vh)) return false;
+        }
+        if (!release_b(pend_ts)) return false;
+        pend_ts = -1;
+        return true;
+    };
     for (int ts = 0; ts < ntile; ++ts) {
         const int buf = ts % p.nbuf, tile = tile_first + ts;
         if (!mbar_wait_idle_warp(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
@@ -1122,9 +1232,8 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
-        bool finish = true;
         if (SK > 1) {
-            // this slice's partial tile to scratch; whoever counts in last adds the slices in order and finishes
+            // this slice's partial tile to scratch, then count in
             float *pt = p.part + ((size_t)tile * SK) * M * kTile;
 #pragma unroll
             for (int cb = 0; cb < 4; ++cb) {
@@ -1136,89 +1245,28 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             }
             __threadfence();
             __syncwarp();
-            int last = 0;
-            if (lane == 0) last = (atomicAdd(p.tctr + tile, 1) == SK - 1) ? 1 : 0;
-            last = __shfl_sync(0xffffffffu, last, 0);
-            finish = last != 0;
-            if (finish) {
-                __threadfence();
-#pragma unroll
-                for (int cb = 0; cb < 4; ++cb) {
-                    const int tok = 4 * cb + tq;
-                    vg[cb] = vh[cb] = 0.f;
-                    if (tok < M)
-                        for (int s2 = 0; s2 < SK; ++s2) {
-                            vg[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g);
-                            vh[cb] += __ldcg(pt + ((size_t)s2 * M + tok) * kTile + g + 8);
-                        }
-                }
-                if (lane == 0) atomicExch(p.tctr + tile, 0);
-            }
-        }
-        if (rank > 0) {
-            const int bs = ts % p.nb;
-            if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
-            if (finish) {
-                const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
-                float d[4][4];
-#pragma unroll
-                for (int cb = 0; cb < 4; ++cb) d[cb][0] = d[cb][1] = d[cb][2] = d[cb][3] = 0.f;
-#pragma unroll 1
-                for (int kc = 0; 4 * kc < nkb; ++kc) {
-                    uint32_t af[4][4];
-                    const uint32_t bx = bt + (uint32_t)kc * box_bytes;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
-                        const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
-                        const bool on = 4 * kc + q < nkb;
-                        af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
-                        af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
-                        af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
-                        af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
-                    }
-#pragma unroll
-                    for (int cb = 0; cb < 4; ++cb) {
-                        if (cb < ncb) {
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                if (4 * kc + q < nkb) {
-                                    const uint32_t ta = tf_lane + (uint32_t)((cb * nkb + 4 * kc + q) * 32) * 8u;
-                                    Mma16<T>::run(d[cb], af[q][0], af[q][1], af[q][2], af[q][3], lds_u32(ta), lds_u32(ta + 4u));
-                                }
-                            }
-                        }
-                    }
-                }
-#pragma unroll
-                for (int cb = 0; cb < 4; ++cb) {
-                    vg[cb] = fmaf(d[cb][0] + d[cb][1], isc, vg[cb]);
-                    vh[cb] = fmaf(d[cb][2] + d[cb][3], isc, vh[cb]);
-                }
-            }
-            __syncwarp();
-            if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
-        }
-        if (finish) {
-            const int n = tile * kTile + g;
-#pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
-                const int tok = 4 * cb + tq;
-                if (tok < M) {
-                    if (n < p.N) y[(size_t)tok * p.N + n] = ActTraits<T>::from_float(vg[cb]);
-                    if (n + 8 < p.N) y[(size_t)tok * p.N + n + 8] = ActTraits<T>::from_float(vh[cb]);
-                }
-            }
+            int old = 0;
+            if (lane == 0) old = atomicAdd(p.tctr + tile, 1);
+            if (!settle()) return false;                                 // the tile before this one
+            pend_ts = ts;
+            pend_old = old;
+        } else {
+            if (!finish_tile(ts, vg, vh)) return false;
+            if (!release_b(ts)) return false;
         }
         mark(p, ts == 0 ? 5 : 6);
     }
+    if (!settle()) return false;
     if (rank > 0) {
         int last = 0;
         if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
-            for (int i = lane; i < p.n_t * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
-            if (lane == 0) atomicExch(p.ctr + 1, 0);
+            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
+            if (lane == 0) {
+                atomicExch(p.ctr, 0);
+                atomicExch(p.ctr + 1, 0);
+            }
         }
     }
     return true;
@@ -1310,6 +1358,35 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
         __syncthreads();
     }
     if (dead && lane == 0) give_up(p);
+    if (p.t_final) {
+        // Many entries (tokens x rank x slots): the t CTA that counts in last adds the slots in order into one
+        // more slot, and the main CTAs read that one alone.
+        volatile int *s_last = reinterpret_cast<volatile int *>(smem + 512);       // free space between the barriers and A
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) *s_last = (atomicAdd(p.ctr, 1) == p.n_t - 1) ? 1 : 0;
+        __syncthreads();
+        if (*s_last) {
+            __threadfence();
+            const size_t slot_elems = (size_t)M * rank;
+            for (int i = tid; i < M * rank; i += kThreads) {
+                float v = 0.f;
+                bool all = true;
+                for (int c0 = 0; c0 < p.n_t; c0 += 8) {
+                    float2 part[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v += part[u].x;
+                        all = all && (part[u].y == 1.f);
+                    }
+                }
+                p.tpart[(size_t)p.n_t * slot_elems + i] = make_float2(v, all ? 1.f : 0.f);
+            }
+        }
+    }
     mark(p, 6);
 }
 
@@ -1558,10 +1635,10 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
     }
-    // K slices: the smallest power of two whose slice of x (16-bit, all tokens) stays below 100 KB
+    // K slices: the smallest power of two whose slice of x (16-bit, all tokens) stays below 136 KB
     int sk = 1;
     auto slice_of = [&](int k) { return ((G + k - 1) / k + kCHGW - 1) / kCHGW * kCHGW; };
-    while (sk < 16 && (size_t)a.M * ((size_t)slice_of(sk) * kGroupFast + 32) * 2 > 100 * 1024) sk *= 2;
+    while (sk < 16 && (size_t)a.M * ((size_t)slice_of(sk) * kGroupFast + 32) * 2 > 136 * 1024) sk *= 2;
     p.slice_groups = slice_of(sk);
     p.SK = (G + p.slice_groups - 1) / p.slice_groups;
     p.x_pitch = p.slice_groups * kGroupFast + 32;
@@ -1615,6 +1692,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     const size_t need = layout(ns);
     if (need > kSmemMax - 2048) return pl;
     p.off_tab = p.off_zero = 0;
+    p.t_final = (p.n_t * a.M * a.rank > 2048) ? 1 : 0;
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
@@ -1744,7 +1822,7 @@ void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tp
 {
     const bool wide = a.M > 2;
     const Plan pl = wide ? make_plan_wide(a, tune) : make_plan(a, tune);
-    *tpart_floats = (size_t)2 * std::max(pl.p.n_t, 1) * a.M * std::max(a.rank, 1);
+    *tpart_floats = (size_t)2 * (std::max(pl.p.n_t, 1) + 1) * a.M * std::max(a.rank, 1);
     *counters = 8 + (wide ? pl.p.NT : 0);
     *partial_floats = (wide && pl.p.SK > 1) ? (size_t)pl.p.NT * pl.p.SK * a.M * kTile : 0;
 }

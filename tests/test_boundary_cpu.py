@@ -42,10 +42,15 @@ def test_dispatch_rules():
         assert sel(M, 11008, 4096, 128, 3, 64, bf16=True) == D
     assert sel(6, 4096, 4096, 128, 4, 16) == D and sel(6, 4096, 4096, 128, 4, 0) == D
     assert sel(4, 4096, 4096, 128, 4, 64) == D and sel(4, 4096, 4096, 128, 4, 128) == D and sel(4, 4096, 4096, 128, 4, 256) == P
-    assert sel(5, 4096, 4096, 128, 4, 64) == P and sel(5, 4096, 4096, 128, 4, 24) == D    # M * rank above 128 at M = 5, 6
+    # measured crossover where the streaming decode kernel's domain holds (N a multiple of 8, rank a multiple of 16 up
+    # to 128): it takes M <= 8 at every rank and M <= 16 without a sub-branch; the tensor-core kernel the rest
+    assert sel(5, 4096, 4096, 128, 4, 64) == D and sel(8, 4096, 4096, 128, 4, 128) == D
+    for M in (9, 15, 16):
+        assert sel(M, 4096, 4096, 128, 4, 32) == P and sel(M, 4096, 4096, 128, 4, 0) == D
+    # outside it the other decode kernel's crossover: M * rank above 128 at M = 5, 6 goes to the tensor-core kernel
+    assert sel(5, 4096, 4096, 128, 4, 24) == D and sel(6, 4096, 4096, 128, 4, 24) == P and sel(7, 4096, 4096, 128, 4, 8) == P
     assert sel(2, 4096, 4096, 128, 4, 128) == D
-    for M in (7, 8, 15, 16):                        # measured crossover: the tensor-core kernel wins from M = 7
-        assert sel(M, 4096, 4096, 128, 4, 32) == P
+    for M in (7, 8, 15, 16):
         assert sel(M, 4100, 4096, 128, 4, 32) == D  # N not a multiple of 8: outside the prefill kernel's domain
     assert sel(1, 4096, 4096, 128, 4, 0) == D
     assert sel(17, 4096, 4096, 128, 4, 64) in (P, G)

@@ -37,7 +37,7 @@ def _problems(fbq, M, bits, rank, dtype, seed0):
 
 @pytest.mark.parametrize("single", [1, 0])
 @pytest.mark.parametrize("bits,rank,dtype,M", [(3, 64, "f16", 1), (4, 64, "bf16", 1), (3, 0, "f16", 1), (3, 16, "f16", 5),
-                                              (4, 64, "f16", 2), (3, 16, "bf16", 6)])
+                                              (4, 64, "f16", 2), (3, 16, "bf16", 6), (4, 8, "f16", 3), (3, 24, "f16", 4)])
 def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M, single):
     import torch
     fbq.set_option("batch_single", single)       # 1: the decode kernel over a problem list; 0: one launch per problem
@@ -47,9 +47,9 @@ def test_batch_matches_oracle_and_single_calls(fbq, bits, rank, dtype, M, single
     before = fbq.launch_count()
     fbq.linear_batch(probs, 128, bits)
     torch.cuda.synchronize()
-    # one launch over the problem list where the other decode kernel runs; the streaming kernel (M <= 2) takes one
-    # launch per problem on the side streams
-    assert fbq.launch_count() - before == (1 if (single and M > 2) else len(probs))
+    # one launch over the problem list where the other decode kernel runs (here: ranks that are not a multiple of 16);
+    # problems in the streaming kernel's domain take one launch each on the side streams
+    assert fbq.launch_count() - before == (1 if (single and rank % 16 != 0) else len(probs))
     fbq.set_option("batch_single", 1)
     assert fbq.poll_status() == 0
     for inp, d, pr in zip(inps, devs, probs):
