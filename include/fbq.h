@@ -193,9 +193,8 @@ int fbq_quantize_feedback(const float *W, const void *A, const void *B, uint8_t 
  *   W [N][K], H [K][K], A [rank][K], B [N][rank]: device fp32 (A and B are the master copies and
  *   are updated in place); loss: device float or NULL; workspace: device,
  *   fbq_reconstruct_workspace_floats(N, K, rank) floats, contents meaningless afterwards.
- * The three dense products are fp32 cuBLAS GEMMs (pedantic math); cuBLAS is loaded on first use
- * (make that first call outside a stream capture), and FBQ_ERR_UNSUPPORTED is returned when it
- * cannot be loaded.  Initialise as Algorithm 1 says (A ~ N(0, sigma^2), B = 0), iterate, then
+ * The three dense products (and fbq_gram) are this library's own fp32 GEMM kernels (CUDA cores, fixed summation
+ * order); no other library is loaded or called.  Initialise as Algorithm 1 says (A ~ N(0, sigma^2), B = 0), iterate, then
  * round A and B to the inference type and call fbq_quantize_feedback once more for (codes, s, z). */
 size_t fbq_reconstruct_workspace_floats(int N, int K, int rank);
 int fbq_gram(const float *X, float *H, int T, int K, void *stream);
@@ -243,6 +242,15 @@ int fbq_linear_batch(const fbq_problem *problems, int count, int M, int group, i
  * before reading it).  The end-to-end path of the benchmark. */
 int fbq_linear_batch_hostio(const fbq_problem *problems, int count, int M, int group, int bits, int rank,
                             int act_is_bf16, void *stream);
+
+/* Comparator, not a product path: the UNFUSED low-rank sub-branch of the paper's Section 3.2 / Fig. "kernel-fusion"
+ * (the quantised main path plus separate launches for the branch), which Section 4.3's fused kernel replaces.
+ * After fbq_linear with rank 0 has written y = x.dequant(Q)^T, this call adds the branch with three launches of
+ * its own: t = x.A^T (fp32), u = t.B^T (rounded to the activation type, written out), y += u (y read and
+ * written once more).  x [M][K], A [rank][K], B [N][rank], y [M][N]: device, fp16 or bf16 (act_is_bf16); rank >= 1.
+ * The benchmark times it against the fused call; a test checks that it computes the same layer. */
+int fbq_sub_branch_unfused(const void *x, const void *A, const void *B, void *y, int M, int N, int K,
+                           int rank, int act_is_bf16, void *stream);
 
 /* Which kernel fbq_linear / fbq_linear_bf16 would run for this shape, or
  * FBQ_KERNEL_NONE when the shape is rejected.  Pure host logic. */

@@ -34,6 +34,7 @@ from .binding import (  # noqa: F401
     select_kernel,
     set_option,
     status_string,
+    sub_branch_unfused,
     unpack,
 )
 from .accounting import algorithmic_bytes, algorithmic_flops, byte_floor_overhead  # noqa: F401

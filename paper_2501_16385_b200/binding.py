@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_linear_hostio.argtypes = [vp] * 7 + [i32] * 7 + [vp]
         L.fbq_linear_noalloc.argtypes = [vp] * 7 + [i32] * 7 + [vp]
+        L.fbq_sub_branch_unfused.argtypes = [vp] * 4 + [i32] * 5 + [vp]
         L.fbq_quantize_feedback.argtypes = [vp] * 7 + [i32] * 6 + [vp]
         L.fbq_reconstruct_workspace_floats.restype = ctypes.c_size_t
         L.fbq_reconstruct_workspace_floats.argtypes = [i32, i32, i32]
@@ -165,6 +166,18 @@ def linear_noalloc(x, qweight, scales, zeros, A, B, N: int, group: int, bits: in
     _check(lib().fbq_linear_noalloc(_ptr(x), _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(A), _ptr(B),
                                     _ptr(y), M, N, K, group, bits, rank, bf16, _stream(stream)),
            "fbq_linear_noalloc")
+    return y
+
+
+def sub_branch_unfused(x, A, B, y, stream=None):
+    """fbq_sub_branch_unfused: adds (x.A^T).B^T to y with three separate launches (the paper's unfused
+    comparison layer); y must already hold the main path (fbq_linear at rank 0)."""
+    import torch
+    M, K = x.shape
+    rank, N = A.shape[0], y.shape[1]
+    bf16 = 1 if x.dtype == torch.bfloat16 else 0
+    _check(lib().fbq_sub_branch_unfused(_ptr(x), _ptr(A), _ptr(B), _ptr(y), M, N, K, rank, bf16, _stream(stream)),
+           "fbq_sub_branch_unfused")
     return y
 
 

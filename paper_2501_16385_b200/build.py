@@ -19,7 +19,7 @@ SOURCES = ["fbq_api.cu", "fbq_pack.cu", "fbq_generic.cu", "fbq_decode.cu", "fbq_
            "fbq_quant.cu", "fbq_reconstruct.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMPILE_FLAGS = ARCH + ["-lineinfo", "-O3", "-std=c++17", "-Xptxas=-v", "-Xcompiler", "-fPIC", "-rdc=false"]
-LINK_FLAGS = ARCH + ["-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-ldl"]
+LINK_FLAGS = ARCH + ["-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
 
 def _headers():

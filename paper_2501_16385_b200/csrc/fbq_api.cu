@@ -352,7 +352,7 @@ int fbq_reconstruct_step(const float *W, const float *H, float *A, float *B, flo
     if (bits != 3 && bits != 4) return FBQ_ERR_BADARG;
     if (!W || !H || !A || !B || !workspace) return FBQ_ERR_BADARG;
     const int rc = run_reconstruct_step(W, H, A, B, lr, loss, workspace, N, K, group, bits, rank, static_cast<cudaStream_t>(stream));
-    if (rc == FBQ_OK) g_launches += loss ? 5 : 3;       // own kernels: quantiser, (two-stage reduction), two updates
+    if (rc == FBQ_OK) g_launches += loss ? 8 : 6;       // quantiser, three GEMMs, (two-stage reduction), two updates
     return rc;
 }
 
@@ -565,6 +565,24 @@ int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *s
     const int rc = linear_common(sx, qweight, scales, zeros, A, B, sy, M, N, K, group, bits, rank, act_is_bf16 != 0, stream);
     if (rc != FBQ_OK) return rc;
     if (cudaMemcpyAsync(y_host, sy, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    return FBQ_OK;
+}
+
+int fbq_sub_branch_unfused(const void *x, const void *A, const void *B, void *y, int M, int N, int K, int rank, int act_is_bf16,
+                            void *stream)
+{
+    if (M < 0 || N < 1 || K < 1 || rank < 1) return FBQ_ERR_BADARG;
+    if (M == 0) return FBQ_OK;
+    if (!x || !A || !B || !y) return FBQ_ERR_BADARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace *ws = workspace_for(s);
+    if (!ws) return FBQ_ERR_CUDA;
+    cudaError_t e;
+    if ((e = grow(ws->t_gen, ws->t_gen_floats, (size_t)M * rank + ((size_t)M * N + 1) / 2 + 4, sizeof(float), s)) != cudaSuccess)
+        return grow_status(e);
+    int launches = 0;
+    if (launch_sub_branch_unfused(x, A, B, y, M, N, K, rank, act_is_bf16 != 0, *ws, s, &launches) != cudaSuccess) return FBQ_ERR_CUDA;
+    g_launches += launches;
     return FBQ_OK;
 }
 

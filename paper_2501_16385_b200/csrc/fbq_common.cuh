@@ -64,6 +64,8 @@ cudaError_t launch_unpack(const uint32_t *qw, uint8_t *codes, int N, int K, int 
 cudaError_t launch_dequant(const uint32_t *qw, const __half *sc, const __half *ze, float *W, int N,
                            int K, int group, int bits, cudaStream_t s);
 cudaError_t launch_generic(const LinearArgs &a, Workspace &ws, cudaStream_t s, int *launches);
+cudaError_t launch_sub_branch_unfused(const void *x, const void *A, const void *B, void *y, int M, int N, int K, int rank, bool bf16,
+                                      Workspace &ws, cudaStream_t s, int *launches);
 cudaError_t launch_quantize_feedback(const float *W, const void *A, const void *B, uint8_t *codes, __half *scales,
                                      __half *zeros, float *WF, float *Delta, int N, int K, int group, int bits, int rank,
                                      int ab_kind, cudaStream_t s);

@@ -120,6 +120,38 @@ gen_main_kernel(const T *__restrict__ x, const uint32_t *__restrict__ qw, const 
     }
 }
 
+// The unfused sub-branch of the paper's comparison (Section 3.2, Fig. "kernel-fusion": the low-rank branch as
+// separate launches next to the quantised main path).  u = t.B^T, rounded to the activation type and written out ...
+template <typename T>
+__global__ void gen_up_kernel(const float *__restrict__ t, const T *__restrict__ B, T *__restrict__ u, int N, int rank)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x, m = blockIdx.y;
+    if (n >= N) return;
+    float acc = 0.f;
+    for (int j = 0; j < rank; ++j) acc = fmaf(t[(size_t)m * rank + j], ActTraits<T>::to_float(B[(size_t)n * rank + j]), acc);
+    u[(size_t)m * N + n] = ActTraits<T>::from_float(acc);
+}
+// ... and y += u as a launch of its own (the extra read and write of the layer output that fusion removes).
+template <typename T>
+__global__ void gen_add_kernel(T *__restrict__ y, const T *__restrict__ u, size_t count)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) y[i] = ActTraits<T>::from_float(ActTraits<T>::to_float(y[i]) + ActTraits<T>::to_float(u[i]));
+}
+
+template <typename T>
+cudaError_t run_unfused(const void *x, const void *A, const void *B, void *y, float *t, void *u, int M, int N, int K, int rank,
+                        cudaStream_t s, int *launches)
+{
+    gen_down_kernel<T><<<dim3(rank, M), 128, 0, s>>>((const T *)x, (const T *)A, t, K, rank);
+    gen_up_kernel<T><<<dim3((N + 127) / 128, M), 128, 0, s>>>(t, (const T *)B, (T *)u, N, rank);
+    const size_t count = (size_t)M * N;
+    gen_add_kernel<T><<<(unsigned)((count + 255) / 256), 256, 0, s>>>((T *)y, (const T *)u, count);
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) *launches += 3;
+    return e;
+}
+
 template <typename T>
 cudaError_t run_generic(const LinearArgs &a, float *t, cudaStream_t s, int *launches)
 {
@@ -148,6 +180,16 @@ cudaError_t launch_generic(const LinearArgs &a, Workspace &ws, cudaStream_t s, i
     // ws.t_gen holds M x rank floats (allocated by the caller of this function)
     return a.bf16 ? run_generic<__nv_bfloat16>(a, ws.t_gen, s, launches)
                   : run_generic<__half>(a, ws.t_gen, s, launches);
+}
+
+// t (M x rank floats) and u (M x N activation-type values) live in ws.t_gen, sized by the caller.
+cudaError_t launch_sub_branch_unfused(const void *x, const void *A, const void *B, void *y, int M, int N, int K, int rank, bool bf16,
+                                      Workspace &ws, cudaStream_t s, int *launches)
+{
+    float *t = ws.t_gen;
+    void *u = ws.t_gen + (size_t)M * rank;
+    return bf16 ? run_unfused<__nv_bfloat16>(x, A, B, y, t, u, M, N, K, rank, s, launches)
+                : run_unfused<__half>(x, A, B, y, t, u, M, N, K, rank, s, launches);
 }
 
 }  // namespace fbq

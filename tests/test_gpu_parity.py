@@ -392,3 +392,22 @@ def test_all_rows_full_size_streaming_kernel(fbq):
     for M, (K, N), bits in ((1, (4096, 4096), 3), (1, (4096, 11008), 3), (1, (11008, 4096), 3), (2, (11008, 4096), 4)):
         inp = make_linear(M, N, K, bits, 64, seed=80 + M)
         check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE, threads=16, floor=2e-5)
+
+
+@pytest.mark.parametrize("M,bits,rank,dtype", [(1, 3, 64, "f16"), (2, 4, 32, "f16"), (8, 4, 64, "bf16")])
+def test_unfused_comparator_computes_the_same_layer(fbq, torch, M, bits, rank, dtype):
+    """The paper's unfused layer (main path, then the low-rank branch as launches of its own), built from this
+    library's kernels for the benchmark's comparison, against the oracle: same tolerance as the fused call (its
+    extra rounding of u and of y is far inside it)."""
+    inp = make_linear(M, 1024, 2048, bits, rank, dtype=dtype, seed=91)
+    dev = DeviceLinear(inp, fbq)
+    before = fbq.launch_count()
+    y = fbq.linear(dev.x, dev.qweight, dev.scales, dev.zeros, None, None, inp.N, 128, bits)
+    fbq.sub_branch_unfused(dev.x, dev.A, dev.B, y)
+    torch.cuda.synchronize()
+    assert fbq.launch_count() - before == 4                  # four kernels instead of one
+    want = oracle.linear_inputs(inp, threads=8)
+    rel, mx, lim = compare(torch_to_f64(y, dtype), want, inp.x_f64(), inp.K)
+    if dtype == "bf16":
+        lim += 2.0 ** -7 * float(np.max(np.abs(want)))
+    assert rel <= REL_F_TOL and mx <= lim
