@@ -187,16 +187,25 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     float4 *s_tab = reinterpret_cast<float4 *>(smem + p.off_tab);
     uint4 *s_x8 = reinterpret_cast<uint4 *>(smem + p.off_x);
     uint32_t *s_xt = reinterpret_cast<uint32_t *>(smem + p.off_x) + (size_t)p.G * 2 * ncol * 16;
-    const int runs_per_tok = p.K / 32, nruns = M * runs_per_tok;           // multiples of 4
-    if ((p.G & 1) && warp == 0 && lane < 2 * M) s_tab[(size_t)p.G * M * 2 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // Every compute warp stages exactly the groups it will multiply (the pairs st * 8 + warp of every stage, the same
+    // for every tile), so no warp waits for another one's part of x.
+    const int G = p.G, SPT = (G + kCHG - 1) / kCHG;
+    const int per_tok = SPT * 8;                                            // runs of this warp per token (4 per group)
+    const int nruns = M * per_tok;
     const int upper = lane & 1;
 #pragma unroll 1
-    for (int base = 0; base < nruns; base += kCW * 16) {
-        const int idx = base + warp * 16 + (lane >> 1);                     // whole groups of eight lanes are valid or not
-        const bool valid = idx < nruns;
-        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+    for (int base = 0; base < nruns; base += 16) {
+        const int idx = base + (lane >> 1);                                 // whole groups of eight lanes are valid or not
+        const int m = idx / per_tok, rem = idx - m * per_tok;
+        const int li = rem >> 2, grp = kCHG * (li >> 1) + 2 * warp + (li & 1);
+        const bool valid = idx < nruns && grp < G;
+        const int run = valid ? grp * 4 + (rem & 3) : 0;
+        if (idx < nruns && grp == G && (lane & 7) == 0) {                  // the partner of the last group when G is odd
+            s_tab[((size_t)G * M + m) * 2] = make_float4(0.f, 0.f, 0.f, 0.f);
+            s_tab[((size_t)G * M + m) * 2 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         uint4 xv[4];
-        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + run * 32);
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)(valid ? m : 0) * p.K + run * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
         if (base == 0) {                                                     // our loads of x are on their way
@@ -1438,7 +1447,7 @@ gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
         pdl_wait();                                  // x may come from the preceding kernel
         mark(p, 2);
         convert_x<BITS, T, M>(p, smem, warp, lane);
-        named_barrier_sync(1, kCW * 32);
+        __syncwarp();                                // a warp multiplies only what it has staged itself
         mark(p, 3);
         ok = compute_i8<BITS, T, M>(p, smem, warp, lane, tile_first, ntile);
     }
