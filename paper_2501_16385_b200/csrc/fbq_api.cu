@@ -219,7 +219,6 @@ int *option_slot(const char *name)
     if (!strcmp(name, "force_kernel")) return &g_opt.force_kernel;
     if (!strcmp(name, "gemv")) return &g_opt.use_gemv;
     if (!strcmp(name, "gemv_ctas")) return &g_opt.gemv.max_ctas;
-    if (!strcmp(name, "gemv_dbg")) return &g_opt.gemv.dbg;
     if (!strcmp(name, "t_poll_limit")) return &g_opt.gemv.poll_limit;
     if (!strcmp(name, "test_skip_t_arrive")) return &g_opt.gemv.test_skip_arrive;
     if (!strcmp(name, "decode_sk")) return &g_opt.decode.sk;

@@ -93,7 +93,6 @@ struct GemvTuning {
     int max_ctas = 0;          // 0: one main CTA per SM
     int pdl = 1;
     int poll_limit = 0;        // 0: default number of looks at the "t complete" counter
-    int dbg = 0;
     int test_skip_arrive = 0;  // test switch: the t CTAs do not report their arrival (the wait for t must run out)
 };
 bool gemv_supported(const LinearArgs &a);

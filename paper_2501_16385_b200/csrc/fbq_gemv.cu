@@ -85,7 +85,6 @@ struct GemvParams {
     int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
-    int dbg;
     unsigned long long *trace;              // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
 
@@ -147,19 +146,17 @@ template <int BITS> struct Slots {
 
 __device__ __forceinline__ float half_bits_to_float(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)v)); }
 
-// Tuning aid: the global timer (ns) of this warp at a phase.
+// Tuning aid, compiled in with -DFBQ_GEMV_TRACE only (the marks cost code size, which this kernel feels): the
+// global timer (ns) of this warp at a phase.
 __device__ __forceinline__ void mark(const GemvParams &p, int slot)
 {
+#ifdef FBQ_GEMV_TRACE
     if (p.trace && (threadIdx.x & 31) == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
         p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = t;
     }
-}
-
-__device__ __forceinline__ void markc(const GemvParams &p, int slot)
-{
-    if (p.trace && (threadIdx.x & 31) == 0) p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = (unsigned long long)clock64();
+#endif
 }
 
 __device__ __forceinline__ void give_up(const GemvParams &p) { atomicExch(p.status, (int)FBQ_ERR_TIMEOUT); }
@@ -212,7 +209,6 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);
         }
-        if (p.trace && base == 0 && (xv[0].x ^ xv[1].y ^ xv[2].z ^ xv[3].w) != 0x12345677u) mark(p, 9);
         const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
         float xf[32];
 #pragma unroll
@@ -402,10 +398,6 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
         const uint32_t woff = (uint32_t)(2 * warp) * (kTile * GB);
         uint32_t wa0[NW], wa1[NW], wb0[NW], wb1[NW];
         auto load_pass = [&](int slot) {
-#ifdef HX_NOW
-            for (int i = 0; i < NW; ++i) { wa0[i] = slot * 7 + i; wa1[i] = slot * 11 + i; wb0[i] = slot * 13 + i; wb1[i] = slot * 17 + i; }
-            return;
-#endif
             const uint32_t wa = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes + woff;
             load_words(wa, wa0);
             load_words(wa + 8 * GB, wa1);
@@ -429,29 +421,16 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
             int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0}, d2[4] = {0, 0, 0, 0}, d3[4] = {0, 0, 0, 0};
             if (live) {
                 const uint32_t xpa = xa + (uint32_t)pi * xsa, xpb = xb + (uint32_t)pi * xsa;
-#ifdef HX_NOX
-                const uint4 xa0 = make_uint4(xpa, xpa * 3, xpa * 5, xpa * 7), xa1 = xa0, xb0 = make_uint4(xpb, xpb * 3, xpb * 5, xpb * 7), xb1 = xb0;
-                uint32_t tv = xpa;
-#else
                 const uint4 xa0 = lds_v4_if(xpa, pa), xa1 = lds_v4_if(xpa + x_chunk1, pa);
                 const uint4 xb0 = lds_v4_if(xpb, pb), xb1 = lds_v4_if(xpb + x_chunk1, pb);
                 uint32_t tv = 0;
                 if constexpr (BITS == 3) tv = lds_u32_if(xt + (uint32_t)pi * xts, pt);
-#endif
                 const int grp = min(ga + ablk, G - 1);
-#ifdef HX_NOMETA
-                mt.tb = make_float4(1.f, 2.f, 3.f, 4.f); mt.sg = mt.zg = mt.sh = mt.zh = 0x3c00u + grp;
-#else
                 mt = load_meta(tab + (uint32_t)(ga + ablk) * 32u, mslot + (uint32_t)grp * 2u);
-#endif
                 uint32_t ra[NR], rb[NR];
                 Slots<BITS>::run(wa0, ra);
                 Slots<BITS>::run(wa1, rb);
-#ifdef HX_NOMMA
-                d0[0] = ra[0] ^ rb[1] ^ ra[2] ^ rb[3] ^ xa0.x; d1[1] = ra[4] ^ rb[5] ^ ra[6] ^ rb[7] ^ xa1.y;
-#else
                 mma8(d0, d1, ra, rb, xa0, xa1);
-#endif
                 uint32_t ta = 0, tb2 = 0;
                 if constexpr (BITS == 3) {
                     ta = ra[8];
@@ -459,12 +438,8 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                 }
                 Slots<BITS>::run(wb0, ra);
                 Slots<BITS>::run(wb1, rb);
-#ifdef HX_NOMMA
-                d2[0] = ra[0] ^ rb[1] ^ ra[2] ^ rb[3] ^ xb0.x; d3[1] = ra[4] ^ rb[5] ^ ra[6] ^ rb[7] ^ xb1.y ^ ta ^ tb2 ^ ra[8] ^ rb[8] ^ tv;
-#else
                 mma8(d2, d3, ra, rb, xb0, xb1);
                 if constexpr (BITS == 3) mma_u8s8(d0, ta, tb2, ra[8], rb[8], nb == 0 ? tv : 0u, nb == 0 ? 0u : tv);
-#endif
             }
             // the next pass's words, while the MMAs run
             int nst = st + 1, nts = ts;
@@ -473,24 +448,16 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                 ++nts;
             }
             if (it + 1 < total) {
-#ifndef HX_NOWAIT
                 if (!mbar_wait(bars + 8u * (kBarFull + nslot), npar)) return false;
-#endif
                 if (2 * (nst * (kCHG / 2) + warp) < G) load_pass(nslot);
             }
             if (live) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) d0[i] = (d0[i] + d1[i]) + (d2[i] + d3[i]);
-#ifdef HX_NOSCALE
-                acc[0] += (float)(d0[0] + d0[1]) + mt.tb.x + (float)mt.sg; acc[1] += (float)(d0[2] + d0[3]) + (float)mt.zh;
-#else
                 scale(d0, mt, acc);
-#endif
             }
-#ifndef HX_NOWAIT
             __syncwarp();
             if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
-#endif
             if (nts != ts) {
                 if (!deposit(ts, acc)) return false;
                 if (++mi == p.nmeta) mi = 0;
@@ -593,13 +560,13 @@ __device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, cons
 // (mask 1, 3, 7): the 16-byte unit index is XOR-ed with the 128-byte line index.
 __device__ __forceinline__ uint32_t swz(uint32_t off, uint32_t mask) { return off ^ (((off >> 7) & mask) << 4); }
 
-template <typename T>
+template <typename T, bool RANKED>
 __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, const CUtensorMap *bmap, int lane, int tile_first, int ntile)
 {
     const int g = lane >> 2, tq = lane & 3;
     const uint32_t sbase = smem_u32(smem), bars = sbase + p.off_bar;
     const uint32_t bring = sbase + p.off_B;
-    const int rank = p.rank, M = p.M, nkb = rank / 16;
+    const int rank = RANKED ? p.rank : 0, M = p.M, nkb = rank / 16;
     const int nbox = (rank + 63) / 64;
     const uint32_t box_bytes = (uint32_t)kTile * (uint32_t)p.b_box_cols * 2u;
     auto request_b = [&](int ts) {
@@ -609,16 +576,16 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             tma_load_2d(bring + (uint32_t)(ts % p.nb) * (uint32_t)p.b_slot_bytes + (uint32_t)b * box_bytes, bmap, b * 64,
                         (tile_first + ts) * kTile, bar);
     };
-    if (rank > 0 && lane == 0)
+    if (RANKED && lane == 0)
         for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
 
     pdl_wait();
     mark(p, 2);
 
     // ---- t: wait for the t CTAs, add their chunks in order, keep t as MMA column operands ----
-    uint32_t tfrag[8][2];
     float isc = 1.f;
-    if (rank > 0) {
+    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // t as MMA column operands [rank block][lane][2]
+    if constexpr (RANKED) {
         // Look at the t CTAs' slots themselves until every entry carries this launch's tag (bounded), adding
         // the chunks in slot order.
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
@@ -657,13 +624,12 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         const float sc = __uint_as_float(sb << 23);
         isc = __uint_as_float((254u - sb) << 23);
         const int tok = g >> 1, part = g & 1;        // as an MMA column: token and (rounded value | remainder)
+#pragma unroll 1
+        for (int kb = 0; kb < nkb; ++kb) {
 #pragma unroll
-        for (int kb = 0; kb < 8; ++kb) {
-            tfrag[kb][0] = tfrag[kb][1] = 0u;
-            if (kb < nkb && tok < M) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t pk = 0;
+            for (int h = 0; h < 2; ++h) {
+                uint32_t pk = 0;
+                if (tok < M) {
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const float v = s_t[tok * rank + kb * 16 + h * 8 + 2 * tq + e] * sc;
@@ -672,10 +638,11 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
                         const T pick = part ? lo : hi;
                         pk |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&pick)) << (16 * e);
                     }
-                    tfrag[kb][h] = pk;
                 }
+                s_tf[((size_t)kb * 32 + lane) * 2 + h] = pk;
             }
         }
+        __syncwarp();
     }
 
     mark(p, 3);
@@ -697,32 +664,33 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
-        if (rank > 0) {
+        if constexpr (RANKED) {
             const int bs = ts % p.nb;
             if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
             const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
             // four 16-wide blocks of the rank at a time: their rows of B first, then the MMAs (two chains)
             float d[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
+#pragma unroll 1
+            for (int kc = 0; 4 * kc < nkb; ++kc) {
+                uint32_t af[4][4], tf[4][2];
+                const uint32_t bx = bt + (uint32_t)kc * box_bytes;
 #pragma unroll
-            for (int kc = 0; kc < 2; ++kc) {
-                if (4 * kc < nkb) {
-                    uint32_t af[4][4];
-                    const uint32_t bx = bt + (uint32_t)kc * box_bytes;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
-                        const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
-                        const bool on = 4 * kc + q < nkb;
-                        af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
-                        af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
-                        af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
-                        af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
-                    }
-                    Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tfrag[4 * kc][0], tfrag[4 * kc][1]);
-                    Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tfrag[4 * kc + 1][0], tfrag[4 * kc + 1][1]);
-                    Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tfrag[4 * kc + 2][0], tfrag[4 * kc + 2][1]);
-                    Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tfrag[4 * kc + 3][0], tfrag[4 * kc + 3][1]);
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+                    const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                    const bool on = 4 * kc + q < nkb;
+                    af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
+                    af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
+                    af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
+                    af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
+                    tf[q][0] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u) : 0u;
+                    tf[q][1] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u + 4u) : 0u;
                 }
+                Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tf[0][0], tf[0][1]);
+                Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tf[1][0], tf[1][1]);
+                Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tf[2][0], tf[2][1]);
+                Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tf[3][0], tf[3][1]);
             }
             vg = fmaf((d[0] + d[1]) + (e[0] + e[1]), isc, vg);
             vh = fmaf((d[2] + d[3]) + (e[2] + e[3]), isc, vh);
@@ -737,7 +705,7 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         mark(p, ts == 0 ? 5 : 6);
     }
     // every main CTA tells when it has read t; the last one leaves the counters at zero for the next launch
-    if (rank > 0) {
+    if constexpr (RANKED) {
         int last = 0;
         if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
         last = __shfl_sync(0xffffffffu, last, 0);
@@ -1311,47 +1279,40 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
     const T *x = static_cast<const T *>(p.x);
     bool dead = false;
     for (int tb = 0; tb < (M + 7) / 8; ++tb) {
-        float acc[8][4];
-#pragma unroll
-        for (int r = 0; r < 8; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
         const int tok = tb * 8 + g;
         if (warp < kCW) {
-            for (int b = warp; b < nkb; b += kCW) {
-                uint32_t xb[4][2];
-                const int k0 = (kb0 + b) * kTKB;
+            // this warp's block of 64 channels (a t CTA holds at most one per warp): its x as column operands ...
+            const bool mine = warp < nkb;
+            uint32_t xb[4][2];
+            const int k0 = (kb0 + warp) * kTKB;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const int k = k0 + ks * 16 + 2 * tq;
-                    const bool v = tok < M && k < p.K;
-                    xb[ks][0] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k)) : 0u;
-                    xb[ks][1] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k + 8)) : 0u;
-                }
-                if (!dead && !mbar_wait(bar, 0)) dead = true;
-                if (dead) break;
-                if (b == warp) mark(p, 3);
-                const uint32_t ab = sA + (uint32_t)b * blk_bytes;
+            for (int ks = 0; ks < 4; ++ks) {
+                const int k = k0 + ks * 16 + 2 * tq;
+                const bool v = mine && tok < M && k < p.K;
+                xb[ks][0] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k)) : 0u;
+                xb[ks][1] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k + 8)) : 0u;
+            }
+            if (mine && !mbar_wait(bar, 0)) dead = true;
+            if (tb == 0) mark(p, 3);
+            const uint32_t ab = sA + (uint32_t)warp * blk_bytes;
+            // ... against sixteen rows of A at a time
+#pragma unroll 1
+            for (int r = 0; r < nrb; ++r) {
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                if (mine && !dead) {
 #pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    if (r < nrb) {
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
-                            Mma16<T>::run(acc[r], lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)),
-                                          lds_u32(ab + swz(o0 + 16u, 7u)), lds_u32(ab + swz(o1 + 16u, 7u)), xb[ks][0], xb[ks][1]);
-                        }
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
+                        Mma16<T>::run(acc, lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)), lds_u32(ab + swz(o0 + 16u, 7u)),
+                                      lds_u32(ab + swz(o1 + 16u, 7u)), xb[ks][0], xb[ks][1]);
                     }
                 }
-            }
-            // rows r*16 + g (and + 8) of A, columns 2tq, 2tq+1 (tokens)
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                if (r < nrb) {
-                    float *dst = s_red + ((size_t)warp * rank + r * 16 + g) * 8 + 2 * tq;
-                    dst[0] = acc[r][0];
-                    dst[1] = acc[r][1];
-                    dst[64] = acc[r][2];
-                    dst[65] = acc[r][3];
-                }
+                // rows r*16 + g (and + 8) of A, columns 2tq, 2tq+1 (tokens)
+                float *dst = s_red + ((size_t)warp * rank + r * 16 + g) * 8 + 2 * tq;
+                dst[0] = acc[0];
+                dst[1] = acc[1];
+                dst[64] = acc[2];
+                dst[65] = acc[3];
             }
         }
         __syncthreads();
@@ -1400,7 +1361,7 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
 }
 
 // ------------------------------------------------------------------------ kernel
-template <int BITS, typename T, int M>
+template <int BITS, typename T, int M, bool RANKED>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
             const __grid_constant__ CUtensorMap bmap, const __grid_constant__ CUtensorMap amap)
@@ -1411,9 +1372,11 @@ gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
     // the CTAs of the next launch on this stream may become resident as soon as all of ours are
     pdl_launch_dependents();
     mark(p, 0);
-    if ((int)blockIdx.x < p.n_t) {
-        t_cta<T>(p, smem, &amap, (int)blockIdx.x);
-        return;
+    if constexpr (RANKED) {
+        if ((int)blockIdx.x < p.n_t) {
+            t_cta<T>(p, smem, &amap, (int)blockIdx.x);
+            return;
+        }
     }
     const int cta = (int)blockIdx.x - p.n_t;
     const int tile_first = (int)((long long)cta * p.NT / p.n_main);
@@ -1442,7 +1405,7 @@ gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
     if (warp == kProdWarp) {
         if (lane == 0) ok = produce(p, smem, &wmap, tile_first, ntile);
     } else if (warp == kEpiWarp) {
-        ok = epilogue<T>(p, smem, &bmap, lane, tile_first, ntile);
+        ok = epilogue<T, RANKED>(p, smem, &bmap, lane, tile_first, ntile);
     } else {
         pdl_wait();                                  // x may come from the preceding kernel
         mark(p, 2);
@@ -1545,7 +1508,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     p.t_kb = 0;
     const int nblk = (a.K + kTKB - 1) / kTKB;
     if (a.rank > 0) {
-        const int per = std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128)));
+        const int per = std::min(kCW, std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128))));     // at most one block per warp
         p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
@@ -1583,6 +1546,9 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         off = align_up(off, 128);
         p.off_t = (int)off;
         off += (size_t)a.M * a.rank * 4;
+        off = align_up(off, 16);
+        p.off_tf = (int)off;
+        off += (size_t)(a.rank / 16) * 32 * 8;
         off = align_up(off, 1024);
         p.off_B = (int)off;
         off += (size_t)p.nb * p.b_slot_bytes;
@@ -1610,7 +1576,6 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
-    p.dbg = tune.dbg;
     pl.ok = true;
     if (getenv("FBQ_PLAN"))
         fprintf(stderr, "gemv plan M %d N %d K %d r %d: n_main %d n_t %d (t_kb %d) NS %d nmeta %d nbuf %d nb %d smem %zu (t CTA %zu)\n",
@@ -1639,7 +1604,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     p.t_kb = 0;
     const int nblk = (a.K + kTKB - 1) / kTKB;
     if (a.rank > 0) {
-        const int per = std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128)));
+        const int per = std::min(kCW, std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128))));     // at most one block per warp
         p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
@@ -1709,7 +1674,6 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     pl.smem = std::max(need, need_t) + 1024;
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
-    p.dbg = tune.dbg;
     pl.ok = true;
     if (getenv("FBQ_PLAN"))
         fprintf(stderr, "gemv wide plan M %d N %d K %d r %d: R %d SK %d (slice %d groups) n_t %d NS %d nmeta %d nbuf %d nb %d smem %zu (t CTA %zu)\n",
@@ -1786,11 +1750,11 @@ cudaError_t launch_wide(const Plan &pl, const CUtensorMap &wmap, const CUtensorM
     return cudaLaunchKernelEx(&cfg, kern, pl.p, wmap, bmap, amap);
 }
 
-template <int BITS, typename T, int M>
+template <int BITS, typename T, int M, bool RANKED>
 cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtensorMap &bmap, const CUtensorMap &amap, bool pdl,
                            cudaStream_t s)
 {
-    auto kern = gemv_kernel<BITS, T, M>;
+    auto kern = gemv_kernel<BITS, T, M, RANKED>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -1889,7 +1853,9 @@ cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tu
         constexpr int B = decltype(bits)::value;
         if (a.M > 8) return launch_wide<B, T, 2>(pl, wmap, bmap, amap, pdl, s);
         if (a.M > 2) return launch_wide<B, T, 1>(pl, wmap, bmap, amap, pdl, s);
-        return a.M == 1 ? launch_variant<B, T, 1>(pl, wmap, bmap, amap, pdl, s) : launch_variant<B, T, 2>(pl, wmap, bmap, amap, pdl, s);
+        if (a.rank == 0)
+            return a.M == 1 ? launch_variant<B, T, 1, false>(pl, wmap, bmap, amap, pdl, s) : launch_variant<B, T, 2, false>(pl, wmap, bmap, amap, pdl, s);
+        return a.M == 1 ? launch_variant<B, T, 1, true>(pl, wmap, bmap, amap, pdl, s) : launch_variant<B, T, 2, true>(pl, wmap, bmap, amap, pdl, s);
     };
     if (a.bits == 4)
         e = a.bf16 ? go(std::integral_constant<int, 4>{}, TypeTag<__nv_bfloat16>{}) : go(std::integral_constant<int, 4>{}, TypeTag<__half>{});

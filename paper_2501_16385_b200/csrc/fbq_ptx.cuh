@@ -44,34 +44,32 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-// Bounded wait: false when the time limit is hit (never spins forever).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: false when the time limit is hit (never spins forever).  The first look is inline; the
+// polling loop is one out-of-line function, so that the many wait sites cost little code.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t sleep_ns)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
 #pragma unroll 1
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
+        for (int i = 0; i < 32; ++i) {
+            if (sleep_ns) __nanosleep(sleep_ns);
             if (mbar_try_wait(bar, parity)) return true;
+        }
         if (global_ns() - t0 > kWaitNs) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, 0u);
 }
 // The same for warps that wait most of the time: they back off between looks so that their polling
 // does not take issue slots from the warps that compute.
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-#pragma unroll 1
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i) {
-            __nanosleep(200);
-            if (mbar_try_wait(bar, parity)) return true;
-        }
-        if (global_ns() - t0 > kWaitNs) return false;
-    }
+    return mbar_wait_slow(bar, parity, 200u);
 }
 // For a whole warp that waits: one lane looks, the others sleep at the warp barrier.
 __device__ __forceinline__ bool mbar_wait_idle_warp(uint32_t bar, uint32_t parity)
