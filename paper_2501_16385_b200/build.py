@@ -2,7 +2,8 @@
 
 Every source file is compiled to an object of its own (in parallel, and only
 when it or a header changed), then the objects are linked into the shared
-library.
+library.  FBQ_EXTRA_NVCC_FLAGS adds compile flags for a build by hand (with
+`--force`), e.g. -DFBQ_GEMV_TRACE for the streaming decode kernel's phase marks.
 """
 from __future__ import annotations
 
@@ -59,7 +60,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if not _stale_obj(src, force):
             return src, 0, ""
         tmp = _obj(src) + ".tmp%d" % os.getpid()
-        res = subprocess.run([nvcc] + COMPILE_FLAGS + ["-c", "-o", tmp, os.path.join(CSRC, src)], capture_output=True, text=True)
+        res = subprocess.run([nvcc] + COMPILE_FLAGS + os.environ.get("FBQ_EXTRA_NVCC_FLAGS", "").split() + ["-c", "-o", tmp, os.path.join(CSRC, src)], capture_output=True, text=True)
         if res.returncode == 0:
             os.replace(tmp, _obj(src))
         return src, res.returncode, res.stdout + res.stderr

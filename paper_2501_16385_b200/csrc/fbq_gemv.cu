@@ -55,8 +55,8 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kTile = 16;                    // weight rows of a tile
 constexpr int kCHG = 2 * kCW;                // quantisation groups of a stage (one pair per compute warp at M = 1)
 constexpr int kMaxNS = 8, kMaxBuf = 8, kMaxB = 4, kMaxMeta = 8;
+constexpr int kMaxSub = 8;                   // tiles whose t.B^T may be formed ahead of their main sums
 constexpr int kTKB = 64;                     // k extent of one block of A in a t CTA (128 bytes: the swizzle span)
-constexpr uint32_t kZeroBytes = 1024;        // zeros that lanes without a digit column read instead
 
 struct GemvParams {
     const void *x;
@@ -73,13 +73,14 @@ struct GemvParams {
     int t_kb;           // blocks of kTKB input channels per t CTA
     int NS, nbuf, nmeta, nb;
     int stage_bytes, meta_pitch, b_slot_bytes, b_box_cols, b_swz;
-    int off_bar, off_tab, off_zero, off_x, off_meta, off_seg, off_t, off_B, off_ring;
+    int off_bar, off_tab, off_x, off_meta, off_seg, off_t, off_B, off_ring;
     int off_tA, off_tred;                   // t CTA: blocks of A, reduction buffer
     // 16-bit form (M >= 3): K may be cut into SK slices (CTA = row block x slice) whose partial tiles meet in scratch
     int SK, R;                              // n_main = R * SK
     int slice_groups;                       // groups per K slice (a multiple of the stage's groups; the last slice takes the rest)
     int x_pitch;                            // elements between tokens of the staged x
     int off_px, off_tf;                     // (P, X0) table; t as MMA column operands
+    int off_sub;                            // t.B^T of the tiles ahead (integer form)
     float *part;                            // [tile][slice][M][16] fp32 partial tiles (SK > 1)
     int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
     int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
@@ -155,6 +156,11 @@ __device__ __forceinline__ void mark(const GemvParams &p, int slot)
         unsigned long long t;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
         p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + slot] = t;
+        if (slot == 0) {                                      // and where the CTA runs
+            unsigned sm;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+            p.trace[((size_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * 16 + 15] = sm;
+        }
     }
 #endif
 }
@@ -187,28 +193,58 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     // Every compute warp stages exactly the groups it will multiply (the pairs st * 8 + warp of every stage, the same
     // for every tile), so no warp waits for another one's part of x.
     const int G = p.G, SPT = (G + kCHG - 1) / kCHG;
-    const int per_tok = SPT * 8;                                            // runs of this warp per token (4 per group)
-    const int nruns = M * per_tok;
+    const int units = M * SPT * 2;                                          // (group, token) units of this warp, token fastest
     const int upper = lane & 1;
+    // unit u of the warp: eight lanes share it
+    auto locate = [&](int it, int &m, int &run, bool &valid, bool &pad) {
+        const int u = it * 4 + (lane >> 3);
+        const int li = u / M;
+        m = u - li * M;
+        const int grp = kCHG * (li >> 1) + 2 * warp + (li & 1);
+        valid = u < units && grp < G;
+        pad = u < units && grp == G;                                        // the partner of the last group when G is odd
+        run = valid ? grp * 4 + ((lane >> 1) & 3) : 0;
+    };
+    // All of the warp's x is requested at once, as whole 128-byte lines (every CTA of the grid reads the same x at
+    // the same moment: the fewer requests per line, the shorter the queue at its L2 slice), straight into shared
+    // memory: the 256 bytes of (group, token m) land at byte 256 m of that group's digit area.  A batch of four
+    // units holds all tokens of its groups, and a batch writes digits only after all its lanes have read their raw
+    // x, so the digits never overwrite raw x that is still needed.
+    const uint32_t xarea = smem_u32(smem) + p.off_x;
+    constexpr uint32_t garea = 2u * ncol * 64u;                             // bytes of one group's digit area
+    const int nbatch = (units + 3) >> 2;
+    for (int it = 0; it < nbatch; ++it) {
+        int m, run;
+        bool valid, pad;
+        locate(it, m, run, valid, pad);
+        if (valid) {
+            const T *src = x + (size_t)m * p.K + (size_t)(run >> 2) * 128 + (lane & 7) * 8;
+            const uint32_t dst = xarea + (uint32_t)(run >> 2) * garea + (uint32_t)m * 256u + (uint32_t)(lane & 7) * 16u;
+            cp_async16(dst, src);
+            cp_async16(dst + 128u, src + 64);
+        }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);    // our loads of x are on their way
+    cp_async_wait_all();
+    __syncwarp();
 #pragma unroll 1
-    for (int base = 0; base < nruns; base += 16) {
-        const int idx = base + (lane >> 1);                                 // whole groups of eight lanes are valid or not
-        const int m = idx / per_tok, rem = idx - m * per_tok;
-        const int li = rem >> 2, grp = kCHG * (li >> 1) + 2 * warp + (li & 1);
-        const bool valid = idx < nruns && grp < G;
-        const int run = valid ? grp * 4 + (rem & 3) : 0;
-        if (idx < nruns && grp == G && (lane & 7) == 0) {                  // the partner of the last group when G is odd
+    for (int it = 0; it < nbatch; ++it) {
+        int m, run;
+        bool valid, pad;
+        locate(it, m, run, valid, pad);
+        if (pad && (lane & 7) == 0) {
             s_tab[((size_t)G * M + m) * 2] = make_float4(0.f, 0.f, 0.f, 0.f);
             s_tab[((size_t)G * M + m) * 2 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         uint4 xv[4];
-        const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)(valid ? m : 0) * p.K + run * 32);
+        {
+            const uint32_t src = xarea + (uint32_t)(run >> 2) * garea + (uint32_t)m * 256u + (uint32_t)(run & 3) * 64u;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xv[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
-        if (base == 0) {                                                     // our loads of x are on their way
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(smem) + p.off_bar + 8u * kBarXReq);
+            for (int i = 0; i < 4; ++i) xv[i] = valid ? lds_v4(src + 16u * i) : make_uint4(0u, 0u, 0u, 0u);
         }
+        __syncwarp();                                                       // every lane holds its raw x: digits may go there
+        if (it == 0) mark(p, 9);
         const uint16_t *e = reinterpret_cast<const uint16_t *>(xv);
         float xf[32];
 #pragma unroll
@@ -555,6 +591,16 @@ __device__ __forceinline__ bool produce(const GemvParams &p, uint8_t *smem, cons
     return true;
 }
 
+// Before the wait for the preceding kernel: up to 64 lines of x per CTA are asked into L2 (the CTAs of a launch
+// start at different lines, so that together they cover a large x).  The preceding kernel may still be writing x:
+// its stores meet the lines in L2 then.  Saves the compute warps the cold miss on their first read of x.
+__device__ __forceinline__ void prefetch_x(const GemvParams &p, int cta, int lane, int elem_bytes)
+{
+    const int nlines = (int)(((size_t)p.M * p.K * elem_bytes + 127) / 128);
+    const char *x = static_cast<const char *>(p.x);
+    for (int j = lane; j < min(nlines, 64); j += 32) prefetch_l2(x + (size_t)((cta * 64 + j) % nlines) * 128);
+}
+
 // ------------------------------------------------------------------------ epilogue warp
 // Swizzled byte offset inside a tile that TMA wrote with the 32-, 64- or 128-byte swizzle
 // (mask 1, 3, 7): the 16-byte unit index is XOR-ed with the 128-byte line index.
@@ -578,6 +624,7 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
     };
     if (RANKED && lane == 0)
         for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
+    prefetch_x(p, (int)blockIdx.x - p.n_t, lane, (int)sizeof(T));
 
     pdl_wait();
     mark(p, 2);
@@ -591,30 +638,41 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
         float amax = 0.f;
         const size_t slot_elems = (size_t)M * rank;
+        const int s_first = p.t_final ? p.n_t : 0, s_end = p.t_final ? p.n_t + 1 : p.n_t;    // the slots to add (or the one that holds their sum)
         bool ok = false;
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
-            for (int i = lane; i < M * rank; i += 32) {
-                float v = 0.f;
-                for (int c0 = 0; c0 < p.n_t; c0 += 8) {           // eight slots in flight
-                    float2 part[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+            for (int i = lane; i < M * rank; i += 64) {                 // two entries x eight slots in flight, added in slot order
+                const bool two = i + 32 < M * rank;
+                float v0 = 0.f, v1 = 0.f;
+                for (int c0 = s_first; c0 < s_end; c0 += 8) {
+                    float2 pa[8], pb[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        v += part[u].x;
-                        all = all && (part[u].y == 1.f);
+                        const bool in = c0 + u < s_end;
+                        pa[u] = in ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+                        pb[u] = (in && two) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i + 32) : make_float2(0.f, 1.f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v0 += pa[u].x;
+                        v1 += pb[u].x;
+                        all = all && (pa[u].y == 1.f) && (pb[u].y == 1.f);
                     }
                 }
-                s_t[i] = v;
-                amax = fmaxf(amax, fabsf(v));
+                s_t[i] = v0;
+                if (two) s_t[i + 32] = v1;
+                amax = fmaxf(amax, fmaxf(fabsf(v0), fabsf(v1)));
             }
             ok = __all_sync(0xffffffffu, all);
             if (!ok && look > 256) __nanosleep(64);
         }
         if (!ok) return false;
+        // Every main CTA tells when it has read t, right away: the last one leaves slots and counters at zero for the
+        // next launch while the others are still at their tiles, not at the end of the kernel.
+        int ack = 0;
+        if (lane == 0) ack = atomicAdd(p.ctr + 1, 1);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         __syncwarp();
@@ -643,15 +701,67 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             }
         }
         __syncwarp();
+        if (__shfl_sync(0xffffffffu, ack, 0) == p.n_main - 1) {
+            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
+            if (lane == 0) {
+                atomicExch(p.ctr, 0);
+                atomicExch(p.ctr + 1, 0);
+            }
+        }
     }
 
     mark(p, 3);
     const float *s_seg = reinterpret_cast<const float *>(smem + p.off_seg);
     T *y = static_cast<T *>(p.y);
     const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
+    // t.B^T of a tile needs t and the tile's rows of B only, so it is formed ahead of the tile's main sums, while the
+    // compute warps are still at them: what is left to do when a tile's sums arrive is short.
+    float2 *s_sub = reinterpret_cast<float2 *>(smem + p.off_sub) + lane;       // [tile % kMaxSub][lane]: rows g and g + 8
+    int nsub = 0;
+    auto sub_tile = [&](int j) -> bool {
+        const int bs = j % p.nb;
+        if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(j / p.nb) & 1u)) return false;
+        const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
+        // four 16-wide blocks of the rank at a time: their rows of B first, then the MMAs (two chains)
+        float d[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
+#pragma unroll 1
+        for (int kc = 0; 4 * kc < nkb; ++kc) {
+            uint32_t af[4][4], tf[4][2];
+            const uint32_t bx = bt + (uint32_t)kc * box_bytes;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+                const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+                const bool on = 4 * kc + q < nkb;
+                af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
+                af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
+                af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
+                af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
+                tf[q][0] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u) : 0u;
+                tf[q][1] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u + 4u) : 0u;
+            }
+            Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tf[0][0], tf[0][1]);
+            Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tf[1][0], tf[1][1]);
+            Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tf[2][0], tf[2][1]);
+            Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tf[3][0], tf[3][1]);
+        }
+        s_sub[(size_t)(j % kMaxSub) * 32] = make_float2((d[0] + d[1]) + (e[0] + e[1]), (d[2] + d[3]) + (e[2] + e[3]));
+        __syncwarp();
+        if (lane == 0 && j + p.nb < ntile) request_b(j + p.nb);
+        return true;
+    };
     for (int ts = 0; ts < ntile; ++ts) {
         const int buf = ts % p.nbuf;
-        if (!mbar_wait_idle_warp(bars + 8u * (kBarSegFull + buf), (uint32_t)(ts / p.nbuf) & 1u)) return false;
+        const uint32_t seg_bar = bars + 8u * (kBarSegFull + buf), seg_par = (uint32_t)(ts / p.nbuf) & 1u;
+        if constexpr (RANKED) {
+            while (nsub < ntile && nsub - ts < kMaxSub) {
+                if (nsub > ts && __any_sync(0xffffffffu, mbar_try_wait(seg_bar, seg_par))) break;     // this tile's sums are there: finish it first
+                if (!sub_tile(nsub)) return false;
+                ++nsub;
+            }
+        }
+        if (!mbar_wait_idle_warp(seg_bar, seg_par)) return false;
         if (ts == 0) mark(p, 4);
         float vg = 0.f, vh = 0.f;
         if (tq < M) {
@@ -665,37 +775,9 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
         if constexpr (RANKED) {
-            const int bs = ts % p.nb;
-            if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(ts / p.nb) & 1u)) return false;
-            const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
-            // four 16-wide blocks of the rank at a time: their rows of B first, then the MMAs (two chains)
-            float d[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};
-            const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
-#pragma unroll 1
-            for (int kc = 0; 4 * kc < nkb; ++kc) {
-                uint32_t af[4][4], tf[4][2];
-                const uint32_t bx = bt + (uint32_t)kc * box_bytes;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
-                    const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
-                    const bool on = 4 * kc + q < nkb;
-                    af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
-                    af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
-                    af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
-                    af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
-                    tf[q][0] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u) : 0u;
-                    tf[q][1] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u + 4u) : 0u;
-                }
-                Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tf[0][0], tf[0][1]);
-                Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tf[1][0], tf[1][1]);
-                Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tf[2][0], tf[2][1]);
-                Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tf[3][0], tf[3][1]);
-            }
-            vg = fmaf((d[0] + d[1]) + (e[0] + e[1]), isc, vg);
-            vh = fmaf((d[2] + d[3]) + (e[2] + e[3]), isc, vh);
-            __syncwarp();
-            if (lane == 0 && ts + p.nb < ntile) request_b(ts + p.nb);
+            const float2 sb = s_sub[(size_t)(ts % kMaxSub) * 32];
+            vg = fmaf(sb.x, isc, vg);
+            vh = fmaf(sb.y, isc, vh);
         }
         const int n = (tile_first + ts) * kTile + g;
         if (tq < M) {
@@ -703,16 +785,6 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             if (n + 8 < p.N) y[(size_t)tq * p.N + n + 8] = ActTraits<T>::from_float(vh);
         }
         mark(p, ts == 0 ? 5 : 6);
-    }
-    // every main CTA tells when it has read t; the last one leaves the counters at zero for the next launch
-    if constexpr (RANKED) {
-        int last = 0;
-        if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            for (int i = lane; i < p.n_t * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
-            if (lane == 0) atomicExch(p.ctr + 1, 0);
-        }
     }
     return true;
 }
@@ -1021,6 +1093,7 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
     if (rank > 0 && lane == 0)
         for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
 
+    prefetch_x(p, (int)blockIdx.x - p.n_t, lane, (int)sizeof(T));
     pdl_wait();
     mark(p, 2);
 
@@ -1252,8 +1325,8 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
 // ------------------------------------------------------------------------ t CTA
 // Block c of the first n_t: t_kb blocks of 64 input channels of all `rank` rows of A in shared memory
 // (TMA, 128-byte swizzle), against the same channels of x read straight from global memory as MMA
-// column operands (tokens are columns).  Warps take the 64-channel blocks round-robin; the eight
-// warps' sums are added in warp order and stored to slot c of tpart.
+// column operands (tokens are columns).  Warps take the 64-channel blocks round-robin (two each at
+// most); the eight warps' sums are added in warp order and stored to slot c of tpart.
 template <typename T>
 __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const CUtensorMap *amap, int c)
 {
@@ -1271,48 +1344,60 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             for (int b = 0; b < nkb; ++b) tma_load_2d(sA + (uint32_t)b * blk_bytes, amap, (kb0 + b) * kTKB, 0, bar);
         }
     }
+    for (int i = tid; i < nkb * M; i += kThreads)      // this CTA's part of x into L2, like the main CTAs' prefetch
+        prefetch_l2(static_cast<const T *>(p.x) + (size_t)(i / nkb) * p.K + (size_t)(kb0 + i % nkb) * kTKB);
     __syncthreads();
     mark(p, 1);
     pdl_wait();
     mark(p, 2);
-    float *s_red = reinterpret_cast<float *>(smem + p.off_tred);      // [warp][rank][8 columns]
+    float *s_red = reinterpret_cast<float *>(smem + p.off_tred);      // [warp][rank][columns in use]
+    const int ncol = M <= 2 ? 2 : 8;
     const T *x = static_cast<const T *>(p.x);
     bool dead = false;
     for (int tb = 0; tb < (M + 7) / 8; ++tb) {
         const int tok = tb * 8 + g;
         if (warp < kCW) {
-            // this warp's block of 64 channels (a t CTA holds at most one per warp): its x as column operands ...
-            const bool mine = warp < nkb;
-            uint32_t xb[4][2];
-            const int k0 = (kb0 + warp) * kTKB;
+            // this warp's blocks of 64 channels (warp and warp + kCW of the CTA's: two at most): their x as column operands ...
+            uint32_t xb[2][4][2];
+            bool mine[2];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const int k = k0 + ks * 16 + 2 * tq;
-                const bool v = mine && tok < M && k < p.K;
-                xb[ks][0] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k)) : 0u;
-                xb[ks][1] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k + 8)) : 0u;
+            for (int u = 0; u < 2; ++u) {
+                mine[u] = warp + u * kCW < nkb;
+                const int k0 = (kb0 + warp + u * kCW) * kTKB;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const int k = k0 + ks * 16 + 2 * tq;
+                    const bool v = mine[u] && tok < M && k < p.K;
+                    xb[u][ks][0] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k)) : 0u;
+                    xb[u][ks][1] = v ? __ldcg(reinterpret_cast<const uint32_t *>(x + (size_t)tok * p.K + k + 8)) : 0u;
+                }
             }
-            if (mine && !mbar_wait(bar, 0)) dead = true;
+            if (mine[0] && !mbar_wait(bar, 0)) dead = true;
             if (tb == 0) mark(p, 3);
-            const uint32_t ab = sA + (uint32_t)warp * blk_bytes;
             // ... against sixteen rows of A at a time
 #pragma unroll 1
             for (int r = 0; r < nrb; ++r) {
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                if (mine && !dead) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
-                        Mma16<T>::run(acc, lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)), lds_u32(ab + swz(o0 + 16u, 7u)),
-                                      lds_u32(ab + swz(o1 + 16u, 7u)), xb[ks][0], xb[ks][1]);
+                for (int u = 0; u < 2; ++u) {
+                    if (mine[u] && !dead) {
+                        const uint32_t ab = sA + (uint32_t)(warp + u * kCW) * blk_bytes;
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
+                            Mma16<T>::run(acc, lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)), lds_u32(ab + swz(o0 + 16u, 7u)),
+                                          lds_u32(ab + swz(o1 + 16u, 7u)), xb[u][ks][0], xb[u][ks][1]);
+                        }
                     }
                 }
                 // rows r*16 + g (and + 8) of A, columns 2tq, 2tq+1 (tokens)
-                float *dst = s_red + ((size_t)warp * rank + r * 16 + g) * 8 + 2 * tq;
-                dst[0] = acc[0];
-                dst[1] = acc[1];
-                dst[64] = acc[2];
-                dst[65] = acc[3];
+                if (2 * tq < ncol) {
+                    float *dst = s_red + ((size_t)warp * rank + r * 16 + g) * ncol + 2 * tq;
+                    dst[0] = acc[0];
+                    dst[1] = acc[1];
+                    dst[8 * ncol] = acc[2];
+                    dst[8 * ncol + 1] = acc[3];
+                }
             }
         }
         __syncthreads();
@@ -1321,7 +1406,7 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             const int m = i / rank, j = i - m * rank;
             float v = 0.f;
 #pragma unroll
-            for (int w = 0; w < kCW; ++w) v += s_red[((size_t)w * rank + j) * 8 + m];
+            for (int w = 0; w < kCW; ++w) v += s_red[((size_t)w * rank + j) * ncol + m];
             // value and tag travel in one 8-byte store: whoever sees the tag sees the value
             p.tpart[((size_t)c * M + tb * 8 + m) * rank + j] = make_float2(v, (p.test_skip_arrive || dead) ? 0.f : 1.f);
         }
@@ -1397,7 +1482,6 @@ gemv_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap,
         mbar_init(bars + 8u * kBarXReq, kCW);
         fence_barrier_init();
     }
-    for (uint32_t i = tid; i < kZeroBytes / 4; i += kThreads) reinterpret_cast<uint32_t *>(smem + p.off_zero)[i] = 0u;
     __syncthreads();
     mark(p, 1);
 
@@ -1486,6 +1570,19 @@ constexpr size_t kSmemMax = 227 * 1024;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Fewer t CTAs (two blocks per warp, chunks of A up to 192 KB) where that saves every main CTA a tile: the main
+// CTAs are what is left of one CTA per SM, and a launch takes as long as the CTA with the most tiles.
+int balanced_t_ctas(int n_t, int nblk, int rank, int tiles, int want)
+{
+    const int per_max = std::min(2 * kCW, std::max(1, (int)(((getenv("FBQ_T_KB2") ? atoi(getenv("FBQ_T_KB2")) : 192) * 1024) / ((size_t)rank * 128))));
+    const int n_min = (nblk + per_max - 1) / per_max;
+    auto most = [&](int nt) { const int m = std::max(1, std::max(want - nt, want / 2)); return (tiles + m - 1) / m; };
+    if (n_min >= n_t || most(n_min) >= most(n_t)) return n_t;
+    int best = n_min;
+    while (best + 1 < n_t && most(best + 1) == most(n_min)) ++best;
+    return best;
+}
+
 Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
 {
     Plan pl{};
@@ -1503,13 +1600,14 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     const int SPT = (G + kCHG - 1) / kCHG;
     p.stage_bytes = kTile * kCHG * GB;
     p.meta_pitch = (int)align_up((size_t)kTile * G * 2, 16);
-    // t CTAs: chunks of A of at most 64 KB
+    // t CTAs: chunks of A of at most 128 KB (measured at rank 128: 84 us per layer step against 94 with 64 KB chunks)
     p.n_t = 0;
     p.t_kb = 0;
     const int nblk = (a.K + kTKB - 1) / kTKB;
     if (a.rank > 0) {
-        const int per = std::min(kCW, std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128))));     // at most one block per warp
-        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
+        int per = std::min(getenv("FBQ_T_CAP") ? atoi(getenv("FBQ_T_CAP")) : kCW, std::max(1, (int)(((getenv("FBQ_T_KB") ? atoi(getenv("FBQ_T_KB")) : 128) * 1024) / ((size_t)a.rank * 128))));
+        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, getenv("FBQ_T_MIN") ? atoi(getenv("FBQ_T_MIN")) : 8)));
+        p.n_t = balanced_t_ctas(p.n_t, nblk, a.rank, p.NT, want);
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
     }
@@ -1533,8 +1631,6 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         p.off_tab = (int)off;
         off += (size_t)(G + 1) * a.M * 32;
         off = align_up(off, 128);
-        p.off_zero = (int)off;
-        off += kZeroBytes;
         p.off_x = (int)off;
         off += (size_t)G * ncol * (a.bits == 4 ? 128 : 144);
         off = align_up(off, 128);
@@ -1549,6 +1645,8 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         off = align_up(off, 16);
         p.off_tf = (int)off;
         off += (size_t)(a.rank / 16) * 32 * 8;
+        p.off_sub = (int)off;
+        off += a.rank > 0 ? (size_t)kMaxSub * 32 * 8 : 0;
         off = align_up(off, 1024);
         p.off_B = (int)off;
         off += (size_t)p.nb * p.b_slot_bytes;
@@ -1571,8 +1669,9 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     // a t CTA: barriers, its blocks of A (1024-byte aligned), the reduction buffer
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
-    const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
+    const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 2 * 4 : 0;      // M <= 2: two columns
     if (need_t > kSmemMax) return pl;
+    p.t_final = (p.n_t * a.M * a.rank > 1024) ? 1 : 0;    // many entries: one t CTA adds the slots for everybody
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
@@ -1604,8 +1703,9 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     p.t_kb = 0;
     const int nblk = (a.K + kTKB - 1) / kTKB;
     if (a.rank > 0) {
-        const int per = std::min(kCW, std::max(1, (int)((64 * 1024) / ((size_t)a.rank * 128))));     // at most one block per warp
+        const int per = std::min(kCW, std::max(1, (int)((128 * 1024) / ((size_t)a.rank * 128))));     // one block per warp
         p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
+        p.n_t = balanced_t_ctas(p.n_t, nblk, a.rank, p.NT, want);
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
     }
@@ -1665,7 +1765,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     while (ns > 2 && layout(ns) > kSmemMax - 2048) --ns;
     const size_t need = layout(ns);
     if (need > kSmemMax - 2048) return pl;
-    p.off_tab = p.off_zero = 0;
+    p.off_tab = 0;
     p.t_final = (p.n_t * a.M * a.rank > 2048) ? 1 : 0;
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;

@@ -75,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ bool mbar_wait_idle_warp(uint32_t bar, uint32_t parity)
 {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait_idle(bar, parity) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = (mbar_try_wait(bar, parity) || mbar_wait_slow(bar, parity, 200u)) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
@@ -106,6 +106,17 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
+
+// Asynchronous 16-byte copy global -> shared of the issuing thread (through L2 only), and the wait for all of them.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Brings the line that holds `a` into L2.  L2 is the device's point of coherence, so this is harmless on memory
+// that an earlier kernel may still be writing.
+__device__ __forceinline__ void prefetch_l2(const void *a) { asm volatile("prefetch.global.L2 [%0];" ::"l"(a)); }
 
 // Programmatic dependent launch: wait() returns once the preceding kernel of the stream has completed
 // and its writes are visible; launch_dependents() lets the following kernel's CTAs become resident.
