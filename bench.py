@@ -511,7 +511,7 @@ def decode_line(args, fbq, torch, wl, peaks, peak_kind, world, rank_id, local, b
                 naive = T(naive_issue(fbq, torch, wl, pool))["ms"] / args.steps
                 extra["naive_sub_branch"] = {
                     "what": "rank-0 fbq_linear + separate down-projection and up-projection-add launches of this library "
-                            "per linear (3 launches), one stream in layer order, same graph replay",
+                            "per linear (4 kernels instead of 1), one stream in layer order, same graph replay",
                     "ms_per_step": naive, "slowdown_vs_fused": naive / ms_step, "overhead_vs_rank0": naive / seq0 - 1.0,
                     "extra_latency_removed_by_fusion": 1.0 - (ms_step - seq0) / (naive - seq0) if naive > seq0 else None}
             plain_steps = min(args.steps, 500)
@@ -547,7 +547,7 @@ def decode_line(args, fbq, torch, wl, peaks, peak_kind, world, rank_id, local, b
         "gpu_launches": args.steps * n_lin * seq["repeats"],     # one fused launch per linear per step, all timed repeats
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": value / world / peaks["hbm_gbs"], "of": peak_kind,
-                     "kernel": "gemv_kernel (one launch per linear)",
+                     "kernel": "gemv_kernel<bits, T, M, ranked> (streaming decode kernel, one launch per linear)",
                      "algorithmic_bytes_per_step": bytes_step,
                      "traffic": TRAFFIC_BYTES_PER_STEP if (wl.bits, wl.rank, wl.M, n_lin) == (3, 64, 1, 7) else None},
         "clocks": clocks,
@@ -559,9 +559,9 @@ def decode_line(args, fbq, torch, wl, peaks, peak_kind, world, rank_id, local, b
     return line
 
 
-# DRAM bytes (read + write) per step measured with ncu on the seven launches of one step
-# (profiles/: the decode summary of the bench workload).
-TRAFFIC_BYTES_PER_STEP = 92_969_000
+# DRAM bytes (read + write) per step measured with ncu on the three shapes of a step, one linear each
+# (4 x 7.941 + 2 x 20.325 + 20.338 MB; profiles/: the streaming decode kernel's summary).
+TRAFFIC_BYTES_PER_STEP = 92_752_000
 
 
 def gpu_arm(args):
