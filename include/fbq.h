@@ -88,7 +88,7 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128 and rank a multiple of 8
  * not above 256 are the fast kernels' domain.  The streaming decode kernel ("gemv" option, default on)
  * needs N a multiple of 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; there
- * it takes M <= 8 at every rank and M <= 16 without a sub-branch.  Elsewhere the other decode kernel
+ * it takes M <= 8 at every rank and M <= 16 at rank <= 64.  Elsewhere the other decode kernel
  * takes M <= 4 with rank <= 128 and M = 5, 6 with M * rank <= 128.  The prefill kernel (N a multiple of
  * 8) takes the rest of the domain; shapes outside its domain stay with a decode kernel up to M = 16;
  * everything else that is well formed -> generic kernel.
@@ -286,8 +286,9 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "prefill_split" the prefill kernel at M <= 128, where a shape has fewer 128-row tiles than SMs: K is cut
  *                   into up to 8 slices, one CTA each, which store fp32 partial tiles to the stream's scratch;
  *                   the CTA that finishes last adds them in slice order and writes y (results do not depend
- *                   on timing).  0 = never, 1 (default) = only for K >= 8192, 2 = whenever the tiles are
- *                   few (faster for a linear that runs alone, slower when several run side by side)
+ *                   on timing).  0 = never, 1 = only for K >= 8192, 2 (default) = whenever the tiles are
+ *                   few (faster for linears that run one after another; when several run side by side on
+ *                   streams of their own, 1 is faster)
  *   "batch_single"  1 = such a batch of up to 8 problems is one launch (default), 0 = one launch per problem
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives

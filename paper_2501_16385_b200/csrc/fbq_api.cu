@@ -32,7 +32,7 @@ struct Options {
     int batch_ctas = 400;
     int batch_single = 1;
     int prefill_pair = 0;
-    int prefill_split = 1;
+    int prefill_split = 2;
     int test_prefill_skip_flag = 0, prefill_flag_polls = 0;
     int decode_trace = 0;
 } g_opt;
@@ -61,16 +61,17 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     if (g_opt.force_kernel == FBQ_KERNEL_DECODE && decode_ok) return FBQ_KERNEL_DECODE;
     if (g_opt.force_kernel == FBQ_KERNEL_PREFILL && prefill_ok) return FBQ_KERNEL_PREFILL;
     if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
-    // Measured on B200 (7B layer, INT4, one stream in layer order, us per layer step, rank 64 / rank 0):
-    //   streaming decode kernel   M = 4: 130 / 79    M = 8: 149 / 100    M = 16: 233 / 141
-    //   tensor-core kernel        M = 4: 213         M = 8: 211          M = 16: 196 (K split whenever tiles are few)
-    //   the other decode kernel   M = 4: 129         M = 8: 258          M = 16: 3204
-    // so where the streaming kernel's domain allows it takes M <= 8 at every rank and M <= 16 without a sub-branch.
+    // Measured on B200 (7B layer, INT4, one stream in layer order, us per layer step, rank 16 / 64 / 128 / 0):
+    //   streaming decode kernel   M = 4: 98 / 118 / 113 / 76   M = 8: 131 / 125 / 164 / 95   M = 12: 156 / 173 / 233   M = 16: 169 / 199 / 272 / 134
+    //   tensor-core kernel        M = 4: 213                   M = 8: 211                    M = 12: 192 / 212 / 222   M = 16: 176 / 196 / 200
+    //                             (K split whenever tiles are few, the default; 227 - 257 with the split only for K >= 8192)
+    //   the other decode kernel   M = 4: 129                   M = 8: 258                    M = 16: 3204
+    // so where the streaming kernel's domain allows it takes M <= 8 at every rank and M <= 16 up to rank 64.
     // Outside that domain the other decode kernel keeps its own crossover: up to M = 4 it gets t from CTAs at the
     // head of its grid and wins at every rank up to 128; at M = 5 and 6 every CTA contributes to t and the tiles
     // wait for it, work that grows with M * rank, so M * rank above 128 goes to the tensor-core kernel.
     const bool streaming = g_opt.use_gemv != 0 && decode_ok && gemv_supported(a);
-    const bool decode_pays = streaming ? (M <= 8 || rank == 0)
+    const bool decode_pays = streaming ? (M <= 8 || rank <= 64)
                                        : (M <= kDecodePreferM && (M <= 4 ? rank <= 128 : M * rank <= 128));
     if (decode_ok && (decode_pays || !prefill_ok)) return FBQ_KERNEL_DECODE;
     if (prefill_ok) return FBQ_KERNEL_PREFILL;

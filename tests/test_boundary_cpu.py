@@ -43,10 +43,11 @@ def test_dispatch_rules():
     assert sel(6, 4096, 4096, 128, 4, 16) == D and sel(6, 4096, 4096, 128, 4, 0) == D
     assert sel(4, 4096, 4096, 128, 4, 64) == D and sel(4, 4096, 4096, 128, 4, 128) == D and sel(4, 4096, 4096, 128, 4, 256) == P
     # measured crossover where the streaming decode kernel's domain holds (N a multiple of 8, rank a multiple of 16 up
-    # to 128): it takes M <= 8 at every rank and M <= 16 without a sub-branch; the tensor-core kernel the rest
+    # to 128): it takes M <= 8 at every rank and M <= 16 up to rank 64; the tensor-core kernel the rest
     assert sel(5, 4096, 4096, 128, 4, 64) == D and sel(8, 4096, 4096, 128, 4, 128) == D
     for M in (9, 15, 16):
-        assert sel(M, 4096, 4096, 128, 4, 32) == P and sel(M, 4096, 4096, 128, 4, 0) == D
+        assert sel(M, 4096, 4096, 128, 4, 32) == D and sel(M, 4096, 4096, 128, 4, 64) == D and sel(M, 4096, 4096, 128, 4, 0) == D
+        assert sel(M, 4096, 4096, 128, 4, 128) == P and sel(M, 4096, 4096, 128, 4, 80) == P
     # outside it the other decode kernel's crossover: M * rank above 128 at M = 5, 6 goes to the tensor-core kernel
     assert sel(5, 4096, 4096, 128, 4, 24) == D and sel(6, 4096, 4096, 128, 4, 24) == P and sel(7, 4096, 4096, 128, 4, 8) == P
     assert sel(2, 4096, 4096, 128, 4, 128) == D
@@ -81,7 +82,7 @@ def test_documented_options_exist_with_their_defaults():
     # every switch named in include/fbq.h is known to the library and starts at the documented value
     defaults = {"force_kernel": -1, "decode_sk": 0, "decode_chunk": 0, "decode_depth": 0, "decode_ctas": 0,
                 "decode_i8": 1, "decode_t_ctas": 1, "decode_t_wait": 1, "batch_ctas": 400, "batch_single": 1,
-                "prefill_pair": 0, "prefill_split": 1, "pdl": 1, "decode_t_late": 0, "decode_trace": 0}
+                "prefill_pair": 0, "prefill_split": 2, "pdl": 1, "decode_t_late": 0, "decode_trace": 0}
     header = open(os.path.join(os.path.dirname(__file__), "..", "include", "fbq.h")).read()
     for name, value in defaults.items():
         assert '"%s"' % name in header, name

@@ -111,11 +111,12 @@ def test_prefill_few_tokens_split_k(fbq, bits, dtype, M, N, K, rank):
         torch.cuda.synchronize()
         assert fbq.poll_status() == 0
         assert torch.equal(ys[0], ys[1]) and torch.equal(ys[1], ys[2])      # partials are added in split order
-        fbq.set_option("prefill_split", 0)                                  # and the unsplit kernel on the same input
-        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, floor=2e-5 if dtype == "f16" else 5e-4)
+        for mode in (0, 1):                                                 # the unsplit kernel, and the split for deep K only
+            fbq.set_option("prefill_split", mode)
+            check_parity(inp, fbq, expect_kernel=fbq.KERNEL_PREFILL, floor=2e-5 if dtype == "f16" else 5e-4)
     finally:
         fbq.set_option("force_kernel", -1)
-        fbq.set_option("prefill_split", 1)
+        fbq.set_option("prefill_split", 2)
 
 
 def test_all_rows_full_size_prefill(fbq):
