@@ -1108,27 +1108,48 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
-            for (int i0 = 0; i0 < M * rank; i0 += 32 * 8) {      // eight entries per lane (and slot) in flight
-                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                for (int c = s_first; c < s_end; ++c) {           // slots added in order
-                    float2 part[8];
+            if (s_end - s_first > 1) {
+                for (int i = lane; i < M * rank; i += 128) {            // four entries x eight slots in flight, added in slot order
+                    float v[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int c0 = s_first; c0 < s_end; c0 += 8) {
+                        float2 pa[4][8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        part[u] = (i < M * rank) ? __ldcg(p.tpart + (size_t)c * slot_elems + i) : make_float2(0.f, 1.f);
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                pa[e][u] = (c0 + u < s_end && i + 32 * e < M * rank) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i + 32 * e)
+                                                                                    : make_float2(0.f, 1.f);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                v[e] += pa[e][u].x;
+                                all = all && (pa[e][u].y == 1.f);
+                            }
                     }
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        v[u] += part[u].x;
-                        all = all && (part[u].y == 1.f);
-                    }
+                    for (int e = 0; e < 4; ++e)
+                        if (i + 32 * e < M * rank) {
+                            s_t[i + 32 * e] = v[e];
+                            amax = fmaxf(amax, fabsf(v[e]));
+                        }
                 }
+            } else {
+                for (int i0 = 0; i0 < M * rank; i0 += 32 * 16) {     // one slot: sixteen entries per lane in flight
+                    float2 part[16];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int i = i0 + u * 32 + lane;
-                    if (i < M * rank) {
-                        s_t[i] = v[u];
-                        amax = fmaxf(amax, fabsf(v[u]));
+                    for (int u = 0; u < 16; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        part[u] = (i < M * rank) ? __ldcg(p.tpart + (size_t)s_first * slot_elems + i) : make_float2(0.f, 1.f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        all = all && (part[u].y == 1.f);
+                        if (i < M * rank) {
+                            s_t[i] = part[u].x;
+                            amax = fmaxf(amax, fabsf(part[u].x));
+                        }
                     }
                 }
             }
@@ -1136,6 +1157,10 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             if (!ok && look > 256) __nanosleep(64);
         }
         if (!ok) return false;
+        // every main CTA tells when it has read t, right away: the last one leaves slots and counters at zero for the
+        // next launch while the others are still at their tiles
+        int ack = 0;
+        if (lane == 0) ack = atomicAdd(p.ctr + 1, 1);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         __syncwarp();
@@ -1164,6 +1189,13 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             }
         }
         __syncwarp();
+        if (__shfl_sync(0xffffffffu, ack, 0) == p.n_main - 1) {
+            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
+            if (lane == 0) {
+                atomicExch(p.ctr, 0);
+                atomicExch(p.ctr + 1, 0);
+            }
+        }
     }
     mark(p, 3);
 
@@ -1307,18 +1339,6 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         mark(p, ts == 0 ? 5 : 6);
     }
     if (!settle()) return false;
-    if (rank > 0) {
-        int last = 0;
-        if (lane == 0) last = (atomicAdd(p.ctr + 1, 1) == p.n_main - 1) ? 1 : 0;
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
-            if (lane == 0) {
-                atomicExch(p.ctr, 0);
-                atomicExch(p.ctr + 1, 0);
-            }
-        }
-    }
     return true;
 }
 
