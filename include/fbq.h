@@ -88,7 +88,8 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128 and rank a multiple of 8
  * not above 256 are the fast kernels' domain.  The streaming decode kernel ("gemv" option, default on)
  * needs N a multiple of 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; there
- * it takes M <= 8 at every rank and M <= 16 at rank <= 64.  Elsewhere the other decode kernel
+ * it takes M <= 8 at every rank, and M <= 16 at rank <= 64 while M * K * 2 bytes stay within 136 KB (x of
+ * all K in shared memory).  Elsewhere the other decode kernel
  * takes M <= 4 with rank <= 128 and M = 5, 6 with M * rank <= 128.  The prefill kernel (N a multiple of
  * 8) takes the rest of the domain; shapes outside its domain stay with a decode kernel up to M = 16;
  * everything else that is well formed -> generic kernel.
@@ -293,8 +294,11 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol
- *   "decode_trace"  tuning aid: 1 = the decode kernel records, per CTA and warp, the SM cycle
- *                   counter at its phases, read with fbq_debug_read_trace
+ *   "decode_trace"  tuning aid: 1 = the decode kernels record, per CTA and warp, a time stamp at
+ *                   their phases, read with fbq_debug_read_trace.  The streaming kernel's marks
+ *                   are compiled in only when the library is built with -DFBQ_GEMV_TRACE
+ *                   (FBQ_EXTRA_NVCC_FLAGS of the build script); a normal build leaves its part of
+ *                   the buffer zero
  * Options are plain process-wide integers read when a call is issued: set them before issuing work, not while
  * other host threads are inside the library.
  * Returns FBQ_OK or FBQ_ERR_BADARG for an unknown name.
@@ -313,7 +317,7 @@ long long fbq_launch_count(void);
 int fbq_poll_status(void *stream);
 
 /* Tuning aid: copies the phase marks of the last decode launch on `stream` (recorded while
- * "decode_trace" is 1) to host_buf.  The streaming kernel writes uint64 [2][256 CTAs][10 warps][16 marks]
+ * "decode_trace" is 1) to host_buf.  The streaming kernel (in a -DFBQ_GEMV_TRACE build) writes uint64 [2][256 CTAs][10 warps][16 marks]
  * of global-timer values (ns), consecutive launches alternating between the two halves; the other
  * decode kernel uint64 [cta][10 warps][16 marks] of SM cycle counts with mark 15 of warp 0 the global
  * timer at kernel entry.  Zero where a mark was not reached.  bytes <= 512*18*16*8.  Synchronises the stream. */

@@ -66,12 +66,15 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     //   tensor-core kernel        M = 4: 213                   M = 8: 211                    M = 12: 192 / 212 / 222   M = 16: 176 / 196 / 200
     //                             (K split whenever tiles are few, the default; 227 - 257 with the split only for K >= 8192)
     //   the other decode kernel   M = 4: 129                   M = 8: 258                    M = 16: 3204
-    // so where the streaming kernel's domain allows it takes M <= 8 at every rank and M <= 16 up to rank 64.
+    // and on the 13B layer (K = 5120 / 13824; rank 64 / 0): streaming M = 8: 150 / 125, M = 12: 208 / 163, M = 16: 411 / 307;
+    // tensor-core M = 8: 256 / 232, M = 12: 258 / 231, M = 16: 234 / 206.  Above eight tokens the streaming kernel
+    // pays only while x of all K fits its shared memory (one K slice: M * K * 2 bytes up to 136 KB), so where its
+    // domain allows it takes M <= 8 at every rank, and M <= 16 up to rank 64 for shapes it does not have to slice.
     // Outside that domain the other decode kernel keeps its own crossover: up to M = 4 it gets t from CTAs at the
     // head of its grid and wins at every rank up to 128; at M = 5 and 6 every CTA contributes to t and the tiles
     // wait for it, work that grows with M * rank, so M * rank above 128 goes to the tensor-core kernel.
     const bool streaming = g_opt.use_gemv != 0 && decode_ok && gemv_supported(a);
-    const bool decode_pays = streaming ? (M <= 8 || rank <= 64)
+    const bool decode_pays = streaming ? (M <= 8 || (rank <= 64 && gemv_k_slices(M, K) == 1))
                                        : (M <= kDecodePreferM && (M <= 4 ? rank <= 128 : M * rank <= 128));
     if (decode_ok && (decode_pays || !prefill_ok)) return FBQ_KERNEL_DECODE;
     if (prefill_ok) return FBQ_KERNEL_PREFILL;

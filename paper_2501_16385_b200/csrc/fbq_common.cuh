@@ -95,6 +95,7 @@ struct GemvTuning {
     int poll_limit = 0;        // 0: default number of looks at the "t complete" counter
     int test_skip_arrive = 0;  // test switch: the t CTAs do not report their arrival (the wait for t must run out)
 };
+int gemv_k_slices(int M, int K);      // K slices the streaming decode kernel cuts a shape into (1: x of all K fits)
 bool gemv_supported(const LinearArgs &a);
 void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tpart_floats, int *counters, size_t *partial_floats);
 cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tune, cudaStream_t s, int *launches);

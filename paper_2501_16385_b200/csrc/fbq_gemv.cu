@@ -1702,6 +1702,16 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     return pl;
 }
 
+// Groups per K slice of the 16-bit form: the smallest power-of-two count of slices whose part of x (16-bit, all
+// tokens, whole stages) stays below 136 KB of shared memory.
+int wide_slice_groups(int M, int G)
+{
+    int sk = 1;
+    auto slice_of = [&](int k) { return ((G + k - 1) / k + kCHGW - 1) / kCHGW * kCHGW; };
+    while (sk < 16 && (size_t)M * ((size_t)slice_of(sk) * kGroupFast + 32) * 2 > 136 * 1024) sk *= 2;
+    return slice_of(sk);
+}
+
 // Plan of the 16-bit form (3 <= M <= 16): one CTA per SM; K in SK slices when x of all K does not fit.
 Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
 {
@@ -1730,10 +1740,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
     }
     // K slices: the smallest power of two whose slice of x (16-bit, all tokens) stays below 136 KB
-    int sk = 1;
-    auto slice_of = [&](int k) { return ((G + k - 1) / k + kCHGW - 1) / kCHGW * kCHGW; };
-    while (sk < 16 && (size_t)a.M * ((size_t)slice_of(sk) * kGroupFast + 32) * 2 > 136 * 1024) sk *= 2;
-    p.slice_groups = slice_of(sk);
+    p.slice_groups = wide_slice_groups(a.M, G);
     p.SK = (G + p.slice_groups - 1) / p.slice_groups;
     p.x_pitch = p.slice_groups * kGroupFast + 32;
     p.R = std::max(1, std::min(std::max(want - p.n_t, want / 2) / p.SK, p.NT));
@@ -1899,6 +1906,13 @@ cudaError_t launch_variant(const Plan &pl, const CUtensorMap &wmap, const CUtens
 }
 
 }  // namespace
+
+int gemv_k_slices(int M, int K)
+{
+    if (M <= 2 || K < kGroupFast) return 1;
+    const int G = K / kGroupFast, sg = wide_slice_groups(M, G);
+    return (G + sg - 1) / sg;
+}
 
 bool gemv_supported(const LinearArgs &a)
 {
