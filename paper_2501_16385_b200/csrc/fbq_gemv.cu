@@ -606,6 +606,35 @@ __device__ __forceinline__ void prefetch_x(const GemvParams &p, int cta, int lan
 // (mask 1, 3, 7): the 16-byte unit index is XOR-ed with the 128-byte line index.
 __device__ __forceinline__ uint32_t swz(uint32_t off, uint32_t mask) { return off ^ (((off >> 7) & mask) << 4); }
 
+// One look at exactly eight t slots with at most 32 E entries: straight-line code, all 8 E loads of a lane in
+// flight (the common shapes: the looks are what a main CTA's epilogue waits with, and a lean look is a fast look).
+// Adds the slots in slot order into s_t, returns whether every entry carried its tag; amax = largest |sum|.
+template <int E>
+__device__ __forceinline__ bool look8(const float2 *slots, size_t slot_elems, int nent, int lane, float *s_t, float &amax)
+{
+    float2 pv[E][8];
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int i = min(lane + 32 * e, nent - 1);          // lanes past the last entry repeat it (and do not store)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) pv[e][u] = __ldcg(slots + (size_t)u * slot_elems + i);
+    }
+    bool all = true;
+    amax = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        float v = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            v += pv[e][u].x;
+            all = all && (pv[e][u].y == 1.f);
+        }
+        if (lane + 32 * e < nent) s_t[lane + 32 * e] = v;
+        amax = fmaxf(amax, fabsf(v));
+    }
+    return all;
+}
+
 template <typename T, bool RANKED>
 __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, const CUtensorMap *bmap, int lane, int tile_first, int ntile)
 {
@@ -643,6 +672,10 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
+            if (s_end - s_first == 8 && M * rank <= 64) {
+                all = (M * rank <= 32) ? look8<1>(p.tpart + (size_t)s_first * slot_elems, slot_elems, M * rank, lane, s_t, amax)
+                                       : look8<2>(p.tpart + (size_t)s_first * slot_elems, slot_elems, M * rank, lane, s_t, amax);
+            } else
             for (int i = lane; i < M * rank; i += 64) {                 // two entries x eight slots in flight, added in slot order
                 const bool two = i + 32 < M * rank;
                 float v0 = 0.f, v1 = 0.f;
