@@ -644,16 +644,30 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
     const int rank = RANKED ? p.rank : 0, M = p.M, nkb = rank / 16;
     const int nbox = (rank + 63) / 64;
     const uint32_t box_bytes = (uint32_t)kTile * (uint32_t)p.b_box_cols * 2u;
-    auto request_b = [&](int ts) {
-        const uint32_t bar = bars + 8u * (kBarB + ts % p.nb);
+    auto request_b = [&](int ts, int slot) {
+        const uint32_t bar = bars + 8u * (kBarB + slot);
         mbar_expect_tx(bar, (uint32_t)nbox * box_bytes);
         for (int b = 0; b < nbox; ++b)
-            tma_load_2d(bring + (uint32_t)(ts % p.nb) * (uint32_t)p.b_slot_bytes + (uint32_t)b * box_bytes, bmap, b * 64,
+            tma_load_2d(bring + (uint32_t)slot * (uint32_t)p.b_slot_bytes + (uint32_t)b * box_bytes, bmap, b * 64,
                         (tile_first + ts) * kTile, bar);
     };
     if (RANKED && lane == 0)
-        for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
+        for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts, ts);   // rows of B are weights: before the wait
     prefetch_x(p, (int)blockIdx.x - p.n_t, lane, (int)sizeof(T));
+    // Everything this warp does per tile runs alone on its latencies, so what does not depend on the tile is done
+    // once, and before the wait: this lane's (swizzled) byte offsets into a tile of B, as MMA row fragments of the
+    // four 16-wide blocks of a 64-column box.
+    const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
+    uint32_t aoff[4][4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
+        const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
+        aoff[q][0] = swz(o0, smask);
+        aoff[q][1] = swz(o1, smask);
+        aoff[q][2] = swz(o0 + 16u, smask);
+        aoff[q][3] = swz(o1 + 16u, smask);
+    }
 
     pdl_wait();
     mark(p, 2);
@@ -706,11 +720,12 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         // next launch while the others are still at their tiles, not at the end of the kernel.
         int ack = 0;
         if (lane == 0) ack = atomicAdd(p.ctr + 1, 1);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        // the largest |sum| of the warp: non-negative floats order like their bit patterns, so one integer reduction does
+        // (a NaN or Inf among them ends up at the top and is clamped below, as before)
+        const uint32_t amax_bits = __reduce_max_sync(0xffffffffu, __float_as_uint(amax));
         __syncwarp();
         // a power of two that puts the largest |t| near 2^14 keeps both terms inside fp16
-        const uint32_t ex = min(max(__float_as_uint(amax) >> 23, 1u), 254u);
+        const uint32_t ex = min(max(amax_bits >> 23, 1u), 254u);
         const uint32_t sb = min(max(268u - ex, 1u), 254u);
         const float sc = __uint_as_float(sb << 23);
         isc = __uint_as_float((254u - sb) << 23);
@@ -746,47 +761,65 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
     mark(p, 3);
     const float *s_seg = reinterpret_cast<const float *>(smem + p.off_seg);
     T *y = static_cast<T *>(p.y);
-    const uint32_t smask = (uint32_t)p.b_swz, pitch = (uint32_t)p.b_box_cols * 2u;
     // t.B^T of a tile needs t and the tile's rows of B only, so it is formed ahead of the tile's main sums, while the
     // compute warps are still at them: what is left to do when a tile's sums arrive is short.
     float2 *s_sub = reinterpret_cast<float2 *>(smem + p.off_sub) + lane;       // [tile % kMaxSub][lane]: rows g and g + 8
-    int nsub = 0;
+    int nsub = 0, sb_slot = 0;
+    uint32_t sb_par = 0u;
+    // t as column operands of the first four rank blocks stays in registers for all tiles
+    uint32_t tfr[4][2] = {{0u, 0u}, {0u, 0u}, {0u, 0u}, {0u, 0u}};
+    if constexpr (RANKED) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            tfr[q][0] = q < nkb ? s_tf[((size_t)q * 32 + lane) * 2] : 0u;
+            tfr[q][1] = q < nkb ? s_tf[((size_t)q * 32 + lane) * 2 + 1] : 0u;
+        }
+    }
     auto sub_tile = [&](int j) -> bool {
-        const int bs = j % p.nb;
-        if (!mbar_wait(bars + 8u * (kBarB + bs), (uint32_t)(j / p.nb) & 1u)) return false;
-        const uint32_t bt = bring + (uint32_t)bs * (uint32_t)p.b_slot_bytes;
+        if (!mbar_wait(bars + 8u * (kBarB + sb_slot), sb_par)) return false;
+        const uint32_t bt = bring + (uint32_t)sb_slot * (uint32_t)p.b_slot_bytes;
         // four 16-wide blocks of the rank at a time: their rows of B first, then the MMAs (two chains)
         float d[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
-#pragma unroll 1
-        for (int kc = 0; 4 * kc < nkb; ++kc) {
+        {
+            uint32_t af[4][4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) af[q][r] = q < nkb ? lds_u32(bt + aoff[q][r]) : 0u;
+            Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tfr[0][0], tfr[0][1]);
+            Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tfr[1][0], tfr[1][1]);
+            Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tfr[2][0], tfr[2][1]);
+            Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tfr[3][0], tfr[3][1]);
+        }
+        if (nkb > 4) {                                                          // rank above 64: the second box
+            const uint32_t bx = bt + box_bytes, tf_lane = sbase + p.off_tf + (uint32_t)lane * 8u;
             uint32_t af[4][4], tf[4][2];
-            const uint32_t bx = bt + (uint32_t)kc * box_bytes;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const uint32_t c0 = (uint32_t)(q * 32 + tq * 4);                  // bytes into the row
-                const uint32_t o0 = (uint32_t)g * pitch + c0, o1 = o0 + 8u * pitch;
-                const bool on = 4 * kc + q < nkb;
-                af[q][0] = on ? lds_u32(bx + swz(o0, smask)) : 0u;
-                af[q][1] = on ? lds_u32(bx + swz(o1, smask)) : 0u;
-                af[q][2] = on ? lds_u32(bx + swz(o0 + 16u, smask)) : 0u;
-                af[q][3] = on ? lds_u32(bx + swz(o1 + 16u, smask)) : 0u;
-                tf[q][0] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u) : 0u;
-                tf[q][1] = on ? lds_u32(tf_lane + (uint32_t)((4 * kc + q) * 32) * 8u + 4u) : 0u;
+                const bool on = 4 + q < nkb;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) af[q][r] = on ? lds_u32(bx + aoff[q][r]) : 0u;
+                tf[q][0] = on ? lds_u32(tf_lane + (uint32_t)((4 + q) * 32) * 8u) : 0u;
+                tf[q][1] = on ? lds_u32(tf_lane + (uint32_t)((4 + q) * 32) * 8u + 4u) : 0u;
             }
             Mma16<T>::run(d, af[0][0], af[0][1], af[0][2], af[0][3], tf[0][0], tf[0][1]);
             Mma16<T>::run(e, af[1][0], af[1][1], af[1][2], af[1][3], tf[1][0], tf[1][1]);
             Mma16<T>::run(d, af[2][0], af[2][1], af[2][2], af[2][3], tf[2][0], tf[2][1]);
             Mma16<T>::run(e, af[3][0], af[3][1], af[3][2], af[3][3], tf[3][0], tf[3][1]);
         }
-        s_sub[(size_t)(j % kMaxSub) * 32] = make_float2((d[0] + d[1]) + (e[0] + e[1]), (d[2] + d[3]) + (e[2] + e[3]));
+        s_sub[(size_t)(j & (kMaxSub - 1)) * 32] = make_float2((d[0] + d[1]) + (e[0] + e[1]), (d[2] + d[3]) + (e[2] + e[3]));
         __syncwarp();
-        if (lane == 0 && j + p.nb < ntile) request_b(j + p.nb);
+        if (lane == 0 && j + p.nb < ntile) request_b(j + p.nb, sb_slot);        // the slot just read
+        if (++sb_slot == p.nb) {
+            sb_slot = 0;
+            sb_par ^= 1u;
+        }
         return true;
     };
+    int buf = 0;
+    uint32_t seg_par = 0u;
     for (int ts = 0; ts < ntile; ++ts) {
-        const int buf = ts % p.nbuf;
-        const uint32_t seg_bar = bars + 8u * (kBarSegFull + buf), seg_par = (uint32_t)(ts / p.nbuf) & 1u;
+        const uint32_t seg_bar = bars + 8u * (kBarSegFull + buf);
         if constexpr (RANKED) {
             while (nsub < ntile && nsub - ts < kMaxSub) {
                 if (nsub > ts && __any_sync(0xffffffffu, mbar_try_wait(seg_bar, seg_par))) break;     // this tile's sums are there: finish it first
@@ -798,17 +831,28 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         if (ts == 0) mark(p, 4);
         float vg = 0.f, vh = 0.f;
         if (tq < M) {
+            // the eight warps' partial sums, added pairwise in a fixed order (a short chain: this warp runs alone on its latencies)
             const float *src = s_seg + ((size_t)buf * kCW * M + tq) * kTile;
+            float pg[kCW], ph[kCW];
 #pragma unroll
             for (int w = 0; w < kCW; ++w) {
-                vg += src[(size_t)w * M * kTile + g];
-                vh += src[(size_t)w * M * kTile + g + 8];
+                pg[w] = src[(size_t)w * M * kTile + g];
+                ph[w] = src[(size_t)w * M * kTile + g + 8];
             }
+#pragma unroll
+            for (int span = 1; span < kCW; span *= 2)
+#pragma unroll
+                for (int w = 0; w + span < kCW; w += 2 * span) {
+                    pg[w] += pg[w + span];
+                    ph[w] += ph[w + span];
+                }
+            vg = pg[0];
+            vh = ph[0];
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
         if constexpr (RANKED) {
-            const float2 sb = s_sub[(size_t)(ts % kMaxSub) * 32];
+            const float2 sb = s_sub[(size_t)(ts & (kMaxSub - 1)) * 32];
             vg = fmaf(sb.x, isc, vg);
             vh = fmaf(sb.y, isc, vh);
         }
@@ -818,6 +862,10 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             if (n + 8 < p.N) y[(size_t)tq * p.N + n + 8] = ActTraits<T>::from_float(vh);
         }
         mark(p, ts == 0 ? 5 : 6);
+        if (++buf == p.nbuf) {
+            buf = 0;
+            seg_par ^= 1u;
+        }
     }
     return true;
 }
