@@ -1475,20 +1475,27 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             }
             if (mine[0] && !mbar_wait(bar, 0)) dead = true;
             if (tb == 0) mark(p, 3);
-            // ... against sixteen rows of A at a time
+            // ... against sixteen rows of A at a time.  Rows are 128 bytes, so the 128-byte swizzle XORs the 16-byte
+            // unit index with the row's low three bits, which are this lane's g for all its rows: the swizzled column
+            // offsets are constants of the lane.
+            const uint32_t xr = (uint32_t)(g & 7) << 4, rowb = (uint32_t)g * 128u;
+            uint32_t col[4][2];
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                col[ks][0] = ((uint32_t)(ks * 32 + tq * 4) ^ xr) + rowb;
+                col[ks][1] = ((uint32_t)(ks * 32 + tq * 4 + 16) ^ xr) + rowb;
+            }
 #pragma unroll 1
             for (int r = 0; r < nrb; ++r) {
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     if (mine[u] && !dead) {
-                        const uint32_t ab = sA + (uint32_t)(warp + u * kCW) * blk_bytes;
+                        const uint32_t ab = sA + (uint32_t)(warp + u * kCW) * blk_bytes + (uint32_t)r * 2048u;
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint32_t o0 = (uint32_t)(r * 16 + g) * 128u + (uint32_t)(ks * 32 + tq * 4), o1 = o0 + 8u * 128u;
-                            Mma16<T>::run(acc, lds_u32(ab + swz(o0, 7u)), lds_u32(ab + swz(o1, 7u)), lds_u32(ab + swz(o0 + 16u, 7u)),
-                                          lds_u32(ab + swz(o1 + 16u, 7u)), xb[u][ks][0], xb[u][ks][1]);
-                        }
+                        for (int ks = 0; ks < 4; ++ks)
+                            Mma16<T>::run(acc, lds_u32(ab + col[ks][0]), lds_u32(ab + col[ks][0] + 1024u), lds_u32(ab + col[ks][1]),
+                                          lds_u32(ab + col[ks][1] + 1024u), xb[u][ks][0], xb[u][ks][1]);
                     }
                 }
                 // rows r*16 + g (and + 8) of A, columns 2tq, 2tq+1 (tokens)
