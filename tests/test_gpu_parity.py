@@ -411,3 +411,31 @@ def test_unfused_comparator_computes_the_same_layer(fbq, torch, M, bits, rank, d
     if dtype == "bf16":
         lim += 2.0 ** -7 * float(np.max(np.abs(want)))
     assert rel <= REL_F_TOL and mx <= lim
+
+
+# The streaming decode kernel's branches by shape: the straight-line look at eight t slots (up to 32 entries, up to 64,
+# a ragged second half), the general look (more entries, fewer slots), the two-level t reduction, t CTAs with two
+# blocks of A per warp, the up-projection's second box of B (rank above 64), and K slices of the 16-bit form.
+@pytest.mark.parametrize("M,N,K,bits,rank,dtype", [
+    (1, 512, 4096, 3, 16, "f16"), (1, 528, 4096, 4, 32, "bf16"), (2, 512, 4096, 3, 32, "f16"), (1, 520, 4096, 4, 48, "f16"),
+    (2, 512, 4096, 3, 48, "f16"), (1, 256, 384, 3, 64, "f16"), (2, 1024, 11008, 4, 128, "f16"), (1, 512, 4096, 4, 80, "bf16"),
+    (1, 1040, 11008, 3, 64, "f16"), (2, 512, 2048, 4, 128, "f16"), (4, 512, 4096, 3, 64, "f16"), (8, 520, 11008, 4, 64, "f16"),
+    (16, 512, 4096, 3, 128, "bf16"), (6, 256, 13824, 4, 32, "f16")])
+def test_streaming_kernel_branches(fbq, M, N, K, bits, rank, dtype):
+    inp = make_linear(M, N, K, bits, rank, dtype=dtype, seed=5100 + 7 * M + rank)
+    fbq.set_option("force_kernel", fbq.KERNEL_DECODE)
+    try:
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE, floor=2e-5 if dtype == "f16" else 5e-4)
+        assert fbq.poll_status() == 0
+        # and the same call again: slots and counters were left clean
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE, floor=2e-5 if dtype == "f16" else 5e-4)
+    finally:
+        fbq.set_option("force_kernel", -1)
+
+
+@pytest.mark.parametrize("M,K,bits,rank", [(1, 4096, 3, 32), (2, 4096, 4, 64), (1, 11008, 4, 64), (2, 2048, 3, 128)])
+def test_streaming_kernel_exact_class_is_bitwise(fbq, M, K, bits, rank):
+    inp = make_exact_class(M, 528, K, bits, rank, seed=5300 + M + rank, x_nnz=32, x_max=2)
+    dev = DeviceLinear(inp, fbq)
+    y = torch_to_f64(dev.run(fbq), "f16")
+    assert np.array_equal(y, oracle.linear_inputs(inp, threads=8))
