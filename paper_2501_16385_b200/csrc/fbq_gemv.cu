@@ -85,6 +85,7 @@ struct GemvParams {
     int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
     int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
+    int t_cleaner;                          // 1: a t CTA clears slots and counters once every reader has told (integer form)
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
     unsigned long long *trace;              // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
@@ -716,10 +717,8 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             if (!ok && look > 256) __nanosleep(64);
         }
         if (!ok) return false;
-        // Every main CTA tells when it has read t, right away: the last one leaves slots and counters at zero for the
-        // next launch while the others are still at their tiles, not at the end of the kernel.
-        int ack = 0;
-        if (lane == 0) ack = atomicAdd(p.ctr + 1, 1);
+        // Tell that this CTA has read t (nobody waits for the add; a t CTA clears up once all have told).
+        if (lane == 0) atomicAdd(p.ctr + 1, 1);
         // the largest |sum| of the warp: non-negative floats order like their bit patterns, so one integer reduction does
         // (a NaN or Inf among them ends up at the top and is clamped below, as before)
         const uint32_t amax_bits = __reduce_max_sync(0xffffffffu, __float_as_uint(amax));
@@ -749,13 +748,6 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             }
         }
         __syncwarp();
-        if (__shfl_sync(0xffffffffu, ack, 0) == p.n_main - 1) {
-            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
-            if (lane == 0) {
-                atomicExch(p.ctr, 0);
-                atomicExch(p.ctr + 1, 0);
-            }
-        }
     }
 
     mark(p, 3);
@@ -1551,6 +1543,37 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
         }
     }
     mark(p, 6);
+    // Clearing up for the next launch: the readers only tell that they have read t (an add that nobody waits for);
+    // one t CTA, which has nothing else left to do, waits until all of them have (bounded), and leaves slots and
+    // counters at zero.  That is the CTA that added the slots, or CTA 0 when every reader adds them itself.
+    if (p.t_cleaner) {
+        volatile int *s_last = reinterpret_cast<volatile int *>(smem + 512);
+        const bool cleaner = p.t_final ? (*s_last != 0) : (c == 0);
+        if (cleaner) {
+            volatile int *s_ok = s_last + 1;
+            if (tid == 0) {
+                int ok = 0;
+                const unsigned long long t0 = global_ns();
+                for (;;) {
+                    if (ld_acquire(p.ctr + 1) >= p.n_main) {
+                        ok = 1;
+                        break;
+                    }
+                    if (global_ns() - t0 > kWaitNs) break;
+                    __nanosleep(100);
+                }
+                *s_ok = ok;
+            }
+            __syncthreads();
+            if (*s_ok) {
+                for (int i = tid; i < (p.n_t + 1) * M * rank; i += kThreads) p.tpart[i] = make_float2(0.f, 0.f);
+                if (tid == 0) {
+                    p.ctr[0] = 0;
+                    p.ctr[1] = 0;
+                }
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------------ kernel
@@ -1780,6 +1803,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 2 * 4 : 0;      // M <= 2: two columns
     if (need_t > kSmemMax) return pl;
     p.t_final = (p.n_t * a.M * a.rank > 1024) ? 1 : 0;    // many entries: one t CTA adds the slots for everybody
+    p.t_cleaner = 1;
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
@@ -1882,6 +1906,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     if (need > kSmemMax - 2048) return pl;
     p.off_tab = 0;
     p.t_final = (p.n_t * a.M * a.rank > 2048) ? 1 : 0;
+    p.t_cleaner = 0;
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
