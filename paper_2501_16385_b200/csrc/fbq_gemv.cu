@@ -85,7 +85,6 @@ struct GemvParams {
     int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
     int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
-    int t_cleaner;                          // 1: a t CTA clears slots and counters once every reader has told (integer form)
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
     unsigned long long *trace;              // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
@@ -1230,10 +1229,8 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             if (!ok && look > 256) __nanosleep(64);
         }
         if (!ok) return false;
-        // every main CTA tells when it has read t, right away: the last one leaves slots and counters at zero for the
-        // next launch while the others are still at their tiles
-        int ack = 0;
-        if (lane == 0) ack = atomicAdd(p.ctr + 1, 1);
+        // tell that this CTA has read t (nobody waits for the add; a t CTA clears up once all have told)
+        if (lane == 0) atomicAdd(p.ctr + 1, 1);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         __syncwarp();
@@ -1262,13 +1259,6 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             }
         }
         __syncwarp();
-        if (__shfl_sync(0xffffffffu, ack, 0) == p.n_main - 1) {
-            for (int i = lane; i < (p.n_t + 1) * M * rank; i += 32) p.tpart[i] = make_float2(0.f, 0.f);
-            if (lane == 0) {
-                atomicExch(p.ctr, 0);
-                atomicExch(p.ctr + 1, 0);
-            }
-        }
     }
     mark(p, 3);
 
@@ -1546,7 +1536,7 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
     // Clearing up for the next launch: the readers only tell that they have read t (an add that nobody waits for);
     // one t CTA, which has nothing else left to do, waits until all of them have (bounded), and leaves slots and
     // counters at zero.  That is the CTA that added the slots, or CTA 0 when every reader adds them itself.
-    if (p.t_cleaner) {
+    {
         volatile int *s_last = reinterpret_cast<volatile int *>(smem + 512);
         const bool cleaner = p.t_final ? (*s_last != 0) : (c == 0);
         if (cleaner) {
@@ -1803,7 +1793,6 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 2 * 4 : 0;      // M <= 2: two columns
     if (need_t > kSmemMax) return pl;
     p.t_final = (p.n_t * a.M * a.rank > 1024) ? 1 : 0;    // many entries: one t CTA adds the slots for everybody
-    p.t_cleaner = 1;
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
     p.test_skip_arrive = tune.test_skip_arrive;
@@ -1906,7 +1895,6 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     if (need > kSmemMax - 2048) return pl;
     p.off_tab = 0;
     p.t_final = (p.n_t * a.M * a.rank > 2048) ? 1 : 0;
-    p.t_cleaner = 0;
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 8 * 4 : 0;
