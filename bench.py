@@ -577,8 +577,8 @@ def decode_line(args, fbq, torch, wl, peaks, peak_kind, world, rank_id, local, b
 
 
 # DRAM bytes (read + write) per step measured with ncu on the three shapes of a step, one linear each
-# (4 x 7.941 + 2 x 20.325 + 20.338 MB; profiles/: the streaming decode kernel's summary).
-TRAFFIC_BYTES_PER_STEP = 92_752_000
+# (4 x 7.940 + 2 x 20.323 + 20.337 MB; profiles/: the streaming decode kernel's summary).
+TRAFFIC_BYTES_PER_STEP = 92_743_000
 
 
 def gpu_arm(args):
