@@ -291,6 +291,9 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *                   few (faster for linears that run one after another; when several run side by side on
  *                   streams of their own, 1 is faster)
  *   "batch_single"  1 = such a batch of up to 8 problems is one launch (default), 0 = one launch per problem
+ *   "hostio_direct_y" 1 (default) = the host-buffer entry points let the kernel write a y of up to 256 KB straight
+ *                   into the caller's buffer when that is pinned, GPU-addressable host memory (no copy queued
+ *                   behind the kernel); 0 = y always goes through the stream's staging buffer and a copy
  *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol

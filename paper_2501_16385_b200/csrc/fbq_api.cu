@@ -33,12 +33,29 @@ struct Options {
     int batch_single = 1;
     int prefill_pair = 0;
     int prefill_split = 2;
+    int hostio_direct_y = 1;
     int test_prefill_skip_flag = 0, prefill_flag_polls = 0;
     int decode_trace = 0;
 } g_opt;
 constexpr size_t kTraceBytes = 512 * 18 * 16 * 8;   // 512 CTAs x up to 18 warps x 16 marks
 
 bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// The host-buffer entry points write a small y straight into the caller's buffer when that is pinned host memory
+// which the GPU can address (unified addressing): the kernel's stores cross the bus instead of a copy that would
+// have to be queued behind the kernel.  Returns the buffer's device alias, or nullptr (pageable memory, unaligned,
+// large, switched off): then y goes through the stream's staging buffer and a copy.
+void *direct_y_alias(void *y_host, size_t bytes)
+{
+    if (!g_opt.hostio_direct_y || bytes > (256u << 10)) return nullptr;
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, y_host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer || misaligned16(at.devicePointer)) return nullptr;
+    return at.devicePointer;
+}
 
 bool well_formed(int M, int N, int K, int group, int bits, int rank)
 {
@@ -238,6 +255,7 @@ int *option_slot(const char *name)
     if (!strcmp(name, "batch_single")) return &g_opt.batch_single;
     if (!strcmp(name, "prefill_pair")) return &g_opt.prefill_pair;
     if (!strcmp(name, "prefill_split")) return &g_opt.prefill_split;
+    if (!strcmp(name, "hostio_direct_y")) return &g_opt.hostio_direct_y;
     if (!strcmp(name, "test_prefill_skip_flag")) return &g_opt.test_prefill_skip_flag;
     if (!strcmp(name, "prefill_flag_polls")) return &g_opt.prefill_flag_polls;
     if (!strcmp(name, "decode_trace")) return &g_opt.decode_trace;
@@ -454,16 +472,22 @@ static int linear_batch_common(const fbq_problem *problems, int count, int M, in
         const size_t xb = (size_t)M * la.K * 2, yb = (size_t)M * la.N * 2;
         char *sx = static_cast<char *>(ws->stage_x), *sy = static_cast<char *>(ws->stage_y);
         if (grow(sx, ws->stage_x_bytes, xb, 1, st) != cudaSuccess) return FBQ_ERR_CUDA;
-        if (grow(sy, ws->stage_y_bytes, yb, 1, st) != cudaSuccess) return FBQ_ERR_CUDA;
         ws->stage_x = sx;
-        ws->stage_y = sy;
         if (cudaMemcpyAsync(sx, la.x, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FBQ_ERR_CUDA;
         la.x = sx;
+        if (void *alias = direct_y_alias(la.y, yb)) {
+            la.y = alias;                             // the kernel writes the caller's buffer itself
+            return FBQ_OK;
+        }
+        if (grow(sy, ws->stage_y_bytes, yb, 1, st) != cudaSuccess) return FBQ_ERR_CUDA;
+        ws->stage_y = sy;
         la.y = sy;
         return FBQ_OK;
     };
     auto stage_out = [&](const LinearArgs &la, void *y_host, cudaStream_t st) -> int {
         if (!host_io) return FBQ_OK;
+        Workspace *ws = workspace_for(st);
+        if (!ws || la.y != ws->stage_y) return FBQ_OK;      // written in place
         return cudaMemcpyAsync(y_host, la.y, (size_t)M * la.N * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess ? FBQ_OK : FBQ_ERR_CUDA;
     };
     if (!all_decode) {
@@ -561,10 +585,12 @@ int fbq_linear_hostio(const void *x_host, const uint32_t *qweight, const void *s
     const size_t xb = (size_t)M * K * 2, yb = (size_t)M * N * 2;
     char *sx = static_cast<char *>(ws->stage_x), *sy = static_cast<char *>(ws->stage_y);
     if (grow(sx, ws->stage_x_bytes, xb, 1, s) != cudaSuccess) return FBQ_ERR_CUDA;
-    if (grow(sy, ws->stage_y_bytes, yb, 1, s) != cudaSuccess) return FBQ_ERR_CUDA;
     ws->stage_x = sx;
-    ws->stage_y = sy;
     if (cudaMemcpyAsync(sx, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    if (void *alias = direct_y_alias(y_host, yb))       // the kernel writes the caller's buffer itself
+        return linear_common(sx, qweight, scales, zeros, A, B, alias, M, N, K, group, bits, rank, act_is_bf16 != 0, stream);
+    if (grow(sy, ws->stage_y_bytes, yb, 1, s) != cudaSuccess) return FBQ_ERR_CUDA;
+    ws->stage_y = sy;
     const int rc = linear_common(sx, qweight, scales, zeros, A, B, sy, M, N, K, group, bits, rank, act_is_bf16 != 0, stream);
     if (rc != FBQ_OK) return rc;
     if (cudaMemcpyAsync(y_host, sy, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FBQ_ERR_CUDA;

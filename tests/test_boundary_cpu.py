@@ -85,7 +85,7 @@ def test_documented_options_exist_with_their_defaults():
     # every switch named in include/fbq.h is known to the library and starts at the documented value
     defaults = {"force_kernel": -1, "decode_sk": 0, "decode_chunk": 0, "decode_depth": 0, "decode_ctas": 0,
                 "decode_i8": 1, "decode_t_ctas": 1, "decode_t_wait": 1, "batch_ctas": 400, "batch_single": 1,
-                "prefill_pair": 0, "prefill_split": 2, "pdl": 1, "decode_t_late": 0, "decode_trace": 0}
+                "prefill_pair": 0, "prefill_split": 2, "hostio_direct_y": 1, "pdl": 1, "decode_t_late": 0, "decode_trace": 0}
     header = open(os.path.join(os.path.dirname(__file__), "..", "include", "fbq.h")).read()
     for name, value in defaults.items():
         assert '"%s"' % name in header, name

@@ -312,7 +312,29 @@ def test_hostio_entry_point(fbq, torch):
     yh = torch.empty((2, 512), dtype=torch.float16).pin_memory()
     fbq.linear_hostio(xh, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, yh, 512, 128, 4)
     torch.cuda.synchronize()
-    assert torch.equal(yh, dev.run(fbq).cpu())
+    ref = dev.run(fbq).cpu()
+    assert torch.equal(yh, ref)
+    # y in pageable memory, and the direct write switched off: both go through the staging buffer and a copy
+    yp = torch.zeros((2, 512), dtype=torch.float16)
+    fbq.linear_hostio(xh, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, yp, 512, 128, 4)
+    torch.cuda.synchronize()
+    assert torch.equal(yp, ref)
+    fbq.set_option("hostio_direct_y", 0)
+    try:
+        yh.zero_()
+        fbq.linear_hostio(xh, dev.qweight, dev.scales, dev.zeros, dev.A, dev.B, yh, 512, 128, 4)
+        torch.cuda.synchronize()
+        assert torch.equal(yh, ref)
+    finally:
+        fbq.set_option("hostio_direct_y", 1)
+    # a y too large to be written across the bus by the kernel (prefill-sized): staged
+    big = make_linear(300, 512, 1024, 4, 16, seed=302)
+    dbig = DeviceLinear(big, fbq)
+    yb = torch.zeros((300, 512), dtype=torch.float16).pin_memory()
+    fbq.linear_hostio(dbig.x.cpu().pin_memory(), dbig.qweight, dbig.scales, dbig.zeros, dbig.A, dbig.B, yb, 512, 128, 4)
+    torch.cuda.synchronize()
+    assert torch.equal(yb, dbig.run(fbq).cpu())
+    assert fbq.poll_status() == 0
 
 
 def test_launch_counter_counts_kernels(fbq, torch):
