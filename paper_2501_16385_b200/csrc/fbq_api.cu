@@ -79,7 +79,7 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     if (g_opt.force_kernel == FBQ_KERNEL_PREFILL && prefill_ok) return FBQ_KERNEL_PREFILL;
     if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
     // Measured on B200 (7B layer, INT4, one stream in layer order, us per layer step, rank 16 / 64 / 128 / 0):
-    //   streaming decode kernel   M = 4: 83 / 86 / 101 / 74    M = 8: 107 / 112 / 144 / 95   M = 12: 156 / 173 / 233   M = 16: 152 / 179 / 272 / 126
+    //   streaming decode kernel   M = 4: 84 / 87 / 101 / 75    M = 8: 107 / 113 / 144 / 96   M = 12: 142 / 157 / 203 / 119   M = 16: 160 / 179 / 240 / 134
     //   tensor-core kernel        M = 4: 213                   M = 8: 211                    M = 12: 192 / 212 / 222   M = 16: 176 / 196 / 200
     //                             (K split whenever tiles are few, the default; 227 - 257 with the split only for K >= 8192)
     //   the other decode kernel   M = 4: 129                   M = 8: 258                    M = 16: 3204
