@@ -1695,7 +1695,7 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // CTAs are what is left of one CTA per SM, and a launch takes as long as the CTA with the most tiles.
 int balanced_t_ctas(int n_t, int nblk, int rank, int tiles, int want)
 {
-    const int per_max = std::min(2 * kCW, std::max(1, (int)(((getenv("FBQ_T_KB2") ? atoi(getenv("FBQ_T_KB2")) : 192) * 1024) / ((size_t)rank * 128))));
+    const int per_max = std::min(2 * kCW, std::max(1, (int)((192 * 1024) / ((size_t)rank * 128))));
     const int n_min = (nblk + per_max - 1) / per_max;
     auto most = [&](int nt) { const int m = std::max(1, std::max(want - nt, want / 2)); return (tiles + m - 1) / m; };
     if (n_min >= n_t || most(n_min) >= most(n_t)) return n_t;
@@ -1726,8 +1726,8 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     p.t_kb = 0;
     const int nblk = (a.K + kTKB - 1) / kTKB;
     if (a.rank > 0) {
-        int per = std::min(getenv("FBQ_T_CAP") ? atoi(getenv("FBQ_T_CAP")) : kCW, std::max(1, (int)(((getenv("FBQ_T_KB") ? atoi(getenv("FBQ_T_KB")) : 128) * 1024) / ((size_t)a.rank * 128))));
-        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, getenv("FBQ_T_MIN") ? atoi(getenv("FBQ_T_MIN")) : 8)));
+        const int per = std::min(kCW, std::max(1, (int)((128 * 1024) / ((size_t)a.rank * 128))));     // one block per warp
+        p.n_t = std::min(64, std::max((nblk + per - 1) / per, std::min(nblk, 8)));
         p.n_t = balanced_t_ctas(p.n_t, nblk, a.rank, p.NT, want);
         p.t_kb = (nblk + p.n_t - 1) / p.n_t;
         p.n_t = (nblk + p.t_kb - 1) / p.t_kb;
