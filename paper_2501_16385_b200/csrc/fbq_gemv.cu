@@ -520,7 +520,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                 if (first) mark(p, 4);
                 first = false;
                 const uint32_t ws = w_lane + (uint32_t)slot * (uint32_t)p.stage_bytes;
-#pragma unroll 1
+#pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int gi = 2 * warp + u, grp = st * kCHG + gi;
                     if (grp >= G) break;
