@@ -85,6 +85,7 @@ struct GemvParams {
     int *tctr;                              // [tile] slices that have stored their partial (zero on entry and exit)
     int t_final;                            // 1: the t CTA that arrives last adds the slots into slot n_t, and the main CTAs read only that one
     uint32_t poll_limit;                    // looks at the arrival counter before giving up
+    int pair;                               // 16-bit form: CTAs come in clusters of two that stage half of x each
     int test_skip_arrive;                   // test switch: t CTAs do not report their arrival
     unsigned long long *trace;              // optional phase timestamps [cta][warp][16] (tuning aid), else NULL
 };
@@ -975,14 +976,21 @@ __device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, 
     T *s_x = reinterpret_cast<T *>(smem + p.off_x);
     float2 *s_px = reinterpret_cast<float2 *>(smem + p.off_px);
     const T *x = static_cast<const T *>(p.x);
-    const int runs_per_tok = g_count * 4, nruns = p.M * runs_per_tok;        // multiples of 4
+    // In a pair (cluster of two CTAs with the same x) this CTA converts every other group and stores the result into
+    // both CTAs' shared memory: every CTA of the grid reads all of x from L2 otherwise, which is what staging costs.
+    const int crank = p.pair ? (int)cluster_ctarank() : 0, cstep = p.pair ? 2 : 1;
+    const int my_groups = (g_count - crank + cstep - 1) / cstep;             // groups crank, crank + cstep, ...
+    const int runs_per_tok = my_groups * 4, nruns = p.M * runs_per_tok;      // multiples of 4
+    const uint32_t peer_x = p.pair ? mapa_shared(smem_u32(s_x), (uint32_t)(crank ^ 1)) : 0u;
+    const uint32_t peer_px = p.pair ? mapa_shared(smem_u32(s_px), (uint32_t)(crank ^ 1)) : 0u;
     constexpr int mp = 8 * MT;                                               // token slots of the (P, X0) table
     for (int i = tid; i < g_count * mp; i += nthr)                           // tokens beyond M contribute nothing
         if (i % mp >= p.M) s_px[i] = make_float2(0.f, 0.f);
     auto fetch = [&](int base, uint4 (&v)[4]) {
         const int idx = base + tid;
         const bool valid = idx < nruns;
-        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+        const int m = valid ? idx / runs_per_tok : 0, mr = valid ? idx - m * runs_per_tok : 0;
+        const int run = ((mr >> 2) * cstep + crank) * 4 + (mr & 3);         // run of the slice: group, quarter
         const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m * p.K + (size_t)g_begin * kGroupFast + run * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) v[i] = valid ? __ldcg(src + i) : make_uint4(0u, 0u, 0u, 0u);
@@ -995,7 +1003,8 @@ __device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, 
     for (int base = 0; base < nruns; base += nthr) {
         const int idx = base + tid;                                          // whole quads are valid or not
         const bool valid = idx < nruns;
-        const int m = valid ? idx / runs_per_tok : 0, run = valid ? idx - m * runs_per_tok : 0;
+        const int m = valid ? idx / runs_per_tok : 0, mr = valid ? idx - m * runs_per_tok : 0;
+        const int run = ((mr >> 2) * cstep + crank) * 4 + (mr & 3);
         uint4 xv[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) xv[i] = xn[i];
@@ -1019,16 +1028,24 @@ __device__ __forceinline__ void convert_x16(const GemvParams &p, uint8_t *smem, 
             xsum += xf;
         }
         if (valid) {
-            uint4 *dst = reinterpret_cast<uint4 *>(s_x + (size_t)m * p.x_pitch + (run >> 2) * kGroupFast);
+            const size_t eoff = (size_t)m * p.x_pitch + (run >> 2) * kGroupFast;    // elements into the staged x
+            uint4 *dst = reinterpret_cast<uint4 *>(s_x + eoff);
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) dst[q4 * 4 + (run & 3)] = make_uint4(h[4 * q4], h[4 * q4 + 1], h[4 * q4 + 2], h[4 * q4 + 3]);
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const uint4 v = make_uint4(h[4 * q4], h[4 * q4 + 1], h[4 * q4 + 2], h[4 * q4 + 3]);
+                dst[q4 * 4 + (run & 3)] = v;
+                if (p.pair) st_cluster_v4(peer_x + (uint32_t)(eoff * 2) + (uint32_t)(q4 * 4 + (run & 3)) * 16u, v);
+            }
         }
         // the four runs of one (token, group) sit in four consecutive lanes
         psum += __shfl_xor_sync(0xffffffffu, psum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         psum += __shfl_xor_sync(0xffffffffu, psum, 2);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
-        if (valid && (run & 3) == 0) s_px[(run >> 2) * mp + m] = make_float2(psum, xsum);
+        if (valid && (run & 3) == 0) {
+            s_px[(run >> 2) * mp + m] = make_float2(psum, xsum);
+            if (p.pair) st_cluster_f2(peer_px + (uint32_t)((run >> 2) * mp + m) * 8u, make_float2(psum, xsum));
+        }
     }
 }
 
@@ -1635,6 +1652,7 @@ gemv_wide_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap, c
     pdl_launch_dependents();
     mark(p, 0);
     if ((int)blockIdx.x < p.n_t) {
+        if (p.pair) cluster_arrive();                // the cluster's barrier counts every thread; nobody here waits on it
         t_cta<T>(p, smem, &amap, (int)blockIdx.x);
         return;
     }
@@ -1663,14 +1681,21 @@ gemv_wide_kernel(const GemvParams p, const __grid_constant__ CUtensorMap wmap, c
     mark(p, 1);
     bool ok = true;
     if (warp == kProdWarp) {
+        if (p.pair) cluster_arrive();
         if (lane == 0) ok = produce(p, smem, &wmap, tile_first, ntile, g_begin, g_count, kCHGW);
     } else if (warp == kEpiWarp) {
+        if (p.pair) cluster_arrive();
         ok = epilogue_wide<T>(p, smem, &bmap, lane, tile_first, ntile, slice);
     } else {
         pdl_wait();                                  // x may come from the preceding kernel
         mark(p, 2);
         convert_x16<BITS, T, MT>(p, smem, g_begin, g_count);
-        named_barrier_sync(1, kCW * 32);
+        if (p.pair) {                                // both CTAs' halves of x are in both CTAs' shared memory
+            cluster_arrive();
+            cluster_wait();
+        } else {
+            named_barrier_sync(1, kCW * 32);
+        }
         mark(p, 3);
         ok = compute_w16<BITS, T, MT>(p, smem, warp, lane, ntile, g_begin, g_count);
     }
@@ -1844,7 +1869,12 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     p.slice_groups = wide_slice_groups(a.M, G);
     p.SK = (G + p.slice_groups - 1) / p.slice_groups;
     p.x_pitch = p.slice_groups * kGroupFast + 32;
+    // One K slice: the main CTAs all stage the same x, so they come in clusters of two that stage half of it each (an
+    // even number of t CTAs, the odd one out idle, and of main CTAs keeps the clusters among their own kind).
+    p.pair = (p.SK == 1 && p.NT >= 2 && want >= 4) ? 1 : 0;
+    if (p.pair && (p.n_t & 1)) ++p.n_t;
     p.R = std::max(1, std::min(std::max(want - p.n_t, want / 2) / p.SK, p.NT));
+    if (p.pair && (p.R & 1)) --p.R;
     p.n_main = p.R * p.SK;
     const int nseg = (p.NT + p.R - 1) / p.R;
     // stages per tile of the shortest slice (the last one): the producer runs at most NS stages ahead, that is
@@ -1970,11 +2000,22 @@ cudaError_t launch_wide(const Plan &pl, const CUtensorMap &wmap, const CUtensorM
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = s;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute at[2];
+    unsigned na = 0;
+    if (pdl) {
+        at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (pl.p.pair) {
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = 2;
+        at[na].val.clusterDim.y = 1;
+        at[na].val.clusterDim.z = 1;
+        ++na;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kern, pl.p, wmap, bmap, amap);
 }
 
