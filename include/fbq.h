@@ -88,8 +88,8 @@ int fbq_dequant(const uint32_t *qweight, const uint16_t *scales, const uint16_t 
  * Dispatch (fbq_select_kernel tells which kernel a shape gets): group == 128 and rank a multiple of 8
  * not above 256 are the fast kernels' domain.  The streaming decode kernel ("gemv" option, default on)
  * needs N a multiple of 8, rank a multiple of 16 up to 128 and 16-byte aligned scales and zeros; there
- * it takes M <= 8 at every rank, and M <= 16 at rank <= 64 while M * K * 2 bytes stay within 136 KB (x of
- * all K in shared memory).  Elsewhere the other decode kernel
+ * it takes M <= 8 for every shape, and M <= 16 while M * K * 2 bytes stay within 136 KB (x of all K in
+ * shared memory).  Elsewhere the other decode kernel
  * takes M <= 4 with rank <= 128 and M = 5, 6 with M * rank <= 128.  The prefill kernel (N a multiple of
  * 8) takes the rest of the domain; shapes outside its domain stay with a decode kernel up to M = 16;
  * everything else that is well formed -> generic kernel.

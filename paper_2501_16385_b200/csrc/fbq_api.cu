@@ -79,19 +79,21 @@ int select_kernel(int M, int N, int K, int group, int bits, int rank, bool bf16)
     if (g_opt.force_kernel == FBQ_KERNEL_PREFILL && prefill_ok) return FBQ_KERNEL_PREFILL;
     if (g_opt.force_kernel >= 0) return FBQ_KERNEL_GENERIC;
     // Measured on B200 (7B layer, INT4, one stream in layer order, us per layer step, rank 16 / 64 / 128 / 0):
-    //   streaming decode kernel   M = 4: 84 / 87 / 101 / 75    M = 8: 107 / 113 / 144 / 96   M = 12: 142 / 157 / 203 / 119   M = 16: 160 / 179 / 240 / 134
-    //   tensor-core kernel        M = 4: 213                   M = 8: 211                    M = 12: 192 / 212 / 222   M = 16: 176 / 196 / 200
+    //   streaming decode kernel   M = 4: 84 / 87 / 101 / 74    M = 8: 107 / 112 / 144 / 91   M = 12: 142 / 156 / 202 / 114   M = 16: 160 / 176 / 236 / 125
+    //   tensor-core kernel        M = 4: 213                   M = 8: 211                    M = 12: 192 / 207 / 213 / 178   M = 16: 176 / 197 / 201 / 166
     //                             (K split whenever tiles are few, the default; 227 - 257 with the split only for K >= 8192)
     //   the other decode kernel   M = 4: 129                   M = 8: 258                    M = 16: 3204
+    // per shape at rank 128 (us per launch, 4096 -> 4096 / 4096 -> 11008 / 11008 -> 4096): streaming M = 12: 21.7 / 29.6 / 58.6,
+    // M = 16: 24.9 / 34.0 / 68.9; tensor-core M = 12: 23.6 / 40.1 / 35.1, M = 16: 23.7 / 35.4 / 35.3;
     // and on the 13B layer (K = 5120 / 13824; rank 64 / 0): streaming M = 8: 150 / 125, M = 12: 208 / 163, M = 16: 411 / 307;
     // tensor-core M = 8: 256 / 232, M = 12: 258 / 231, M = 16: 234 / 206.  Above eight tokens the streaming kernel
     // pays only while x of all K fits its shared memory (one K slice: M * K * 2 bytes up to 136 KB), so where its
-    // domain allows it takes M <= 8 at every rank, and M <= 16 up to rank 64 for shapes it does not have to slice.
+    // domain allows it takes M <= 8 for every shape, and M <= 16 for the shapes it does not have to slice.
     // Outside that domain the other decode kernel keeps its own crossover: up to M = 4 it gets t from CTAs at the
     // head of its grid and wins at every rank up to 128; at M = 5 and 6 every CTA contributes to t and the tiles
     // wait for it, work that grows with M * rank, so M * rank above 128 goes to the tensor-core kernel.
     const bool streaming = g_opt.use_gemv != 0 && decode_ok && gemv_supported(a);
-    const bool decode_pays = streaming ? (M <= 8 || (rank <= 64 && gemv_k_slices(M, K) == 1))
+    const bool decode_pays = streaming ? (M <= 8 || gemv_k_slices(M, K) == 1)
                                        : (M <= kDecodePreferM && (M <= 4 ? rank <= 128 : M * rank <= 128));
     if (decode_ok && (decode_pays || !prefill_ok)) return FBQ_KERNEL_DECODE;
     if (prefill_ok) return FBQ_KERNEL_PREFILL;

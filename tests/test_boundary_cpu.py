@@ -43,13 +43,13 @@ def test_dispatch_rules():
     assert sel(6, 4096, 4096, 128, 4, 16) == D and sel(6, 4096, 4096, 128, 4, 0) == D
     assert sel(4, 4096, 4096, 128, 4, 64) == D and sel(4, 4096, 4096, 128, 4, 128) == D and sel(4, 4096, 4096, 128, 4, 256) == P
     # measured crossover where the streaming decode kernel's domain holds (N a multiple of 8, rank a multiple of 16 up
-    # to 128): it takes M <= 8 at every rank, and M <= 16 up to rank 64 while x of all K fits its shared memory
+    # to 128): it takes M <= 8 for every shape, and M <= 16 while x of all K fits its shared memory
     # (M * K * 2 bytes up to 136 KB: no K slices); the tensor-core kernel the rest
     assert sel(5, 4096, 4096, 128, 4, 64) == D and sel(8, 4096, 4096, 128, 4, 128) == D and sel(8, 5120, 13824, 128, 3, 64) == D
     for M in (9, 15, 16):
         assert sel(M, 4096, 4096, 128, 4, 32) == D and sel(M, 4096, 4096, 128, 4, 64) == D and sel(M, 4096, 4096, 128, 4, 0) == D
-        assert sel(M, 4096, 4096, 128, 4, 128) == P and sel(M, 4096, 4096, 128, 4, 80) == P
-        assert sel(M, 4096, 11008, 128, 4, 64) == P and sel(M, 4096, 11008, 128, 4, 0) == P      # K too deep for one slice
+        assert sel(M, 4096, 4096, 128, 4, 128) == D and sel(M, 4096, 4096, 128, 4, 80) == D and sel(M, 4096, 4096, 128, 4, 256) == P
+        assert sel(M, 4096, 11008, 128, 4, 64) == P and sel(M, 4096, 11008, 128, 4, 128) == P and sel(M, 4096, 11008, 128, 4, 0) == P      # K too deep for one slice
     assert sel(12, 5120, 5120, 128, 4, 64) == D and sel(16, 5120, 5120, 128, 4, 64) == P and sel(16, 5120, 5120, 128, 4, 0) == P
     # outside it the other decode kernel's crossover: M * rank above 128 at M = 5, 6 goes to the tensor-core kernel
     assert sel(5, 4096, 4096, 128, 4, 24) == D and sel(6, 4096, 4096, 128, 4, 24) == P and sel(7, 4096, 4096, 128, 4, 8) == P
