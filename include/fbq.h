@@ -294,7 +294,11 @@ int fbq_select_kernel(int M, int N, int K, int group, int bits, int rank, int ac
  *   "hostio_direct_y" 1 (default) = the host-buffer entry points let the kernel write a y of up to 256 KB straight
  *                   into the caller's buffer when that is pinned, GPU-addressable host memory (no copy queued
  *                   behind the kernel); 0 = y always goes through the stream's staging buffer and a copy
- *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain
+ *   "pdl"           1 = launch with programmatic dependent launch (default), 0 = plain.  With 1 a decode or
+ *                   prefill kernel may start while the kernel before it on the stream still runs: it sets
+ *                   itself up, and the decode kernels already fetch qweight, scales, zeros, A and B, before
+ *                   they wait for that kernel; x, y and the scratch are touched only after the wait.  So
+ *                   the weight operands must not be written by the launch directly before (x may be)
  *   "decode_t_late" test switch: 1 = contribute to t after the main loop, which drives
  *                   every tile through the parked-tile branch of the combine protocol
  *   "decode_trace"  tuning aid: 1 = the decode kernels record, per CTA and warp, a time stamp at

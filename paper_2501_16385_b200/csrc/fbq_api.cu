@@ -14,6 +14,7 @@ void decode_set_test_switch(int t_late);
 void decode_set_t_wait(int on);
 void prefill_set_pair(int on);
 void prefill_set_split(int mode);
+void prefill_set_pdl(int on);
 void prefill_set_test(int skip_flag, int flag_polls);
 
 namespace {
@@ -386,6 +387,7 @@ static void apply_kernel_options()
     decode_set_t_wait(g_opt.decode_t_wait);
     prefill_set_pair(g_opt.prefill_pair);
     prefill_set_split(g_opt.prefill_split);
+    prefill_set_pdl(g_opt.decode.pdl);
     prefill_set_test(g_opt.test_prefill_skip_flag, g_opt.prefill_flag_polls);
 }
 
