@@ -670,12 +670,17 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         aoff[q][3] = swz(o1 + 16u, smask);
     }
 
+    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // t as MMA column operands [rank block][lane][2]
+    if constexpr (RANKED) {
+        for (int i = lane; i < nkb * 64; i += 32) s_tf[i] = 0u;
+        __syncwarp();
+    }
+
     pdl_wait();
     mark(p, 2);
 
     // ---- t: wait for the t CTAs, add their chunks in order, keep t as MMA column operands ----
     float isc = 1.f;
-    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // t as MMA column operands [rank block][lane][2]
     if constexpr (RANKED) {
         // Look at the t CTAs' slots themselves until every entry carries this launch's tag (bounded), adding
         // the chunks in slot order.
@@ -728,24 +733,22 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         const uint32_t sb = min(max(268u - ex, 1u), 254u);
         const float sc = __uint_as_float(sb << 23);
         isc = __uint_as_float((254u - sb) << 23);
-        const int tok = g >> 1, part = g & 1;        // as an MMA column: token and (rounded value | remainder)
-#pragma unroll 1
-        for (int kb = 0; kb < nkb; ++kb) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t pk = 0;
-                if (tok < M) {
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float v = s_t[tok * rank + kb * 16 + h * 8 + 2 * tq + e] * sc;
-                        const T hi = ActTraits<T>::from_float(v);
-                        const T lo = ActTraits<T>::from_float(v - ActTraits<T>::to_float(hi));
-                        const T pick = part ? lo : hi;
-                        pk |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&pick)) << (16 * e);
-                    }
-                }
-                s_tf[((size_t)kb * 32 + lane) * 2 + h] = pk;
-            }
+        // t as MMA column operands: column 2 tok holds the rounded values of token tok, column 2 tok + 1 what the
+        // rounding left; a lane takes pairs of consecutive rank indices (all lanes busy: this runs on the critical
+        // path of the launch), the columns beyond the tokens were set to zero before the wait.
+        const int half_rank = rank >> 1;
+        for (int idx = lane; idx < M * half_rank; idx += 32) {
+            const int tok = idx / half_rank, k0 = 2 * (idx - tok * half_rank);
+            const float2 tv = *reinterpret_cast<const float2 *>(s_t + tok * rank + k0);
+            const float v0 = tv.x * sc, v1 = tv.y * sc;
+            const T h0 = ActTraits<T>::from_float(v0), h1 = ActTraits<T>::from_float(v1);
+            const T l0 = ActTraits<T>::from_float(v0 - ActTraits<T>::to_float(h0));
+            const T l1 = ActTraits<T>::from_float(v1 - ActTraits<T>::to_float(h1));
+            const uint32_t pk_hi = (uint32_t)(*reinterpret_cast<const uint16_t *>(&h0)) | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&h1)) << 16);
+            const uint32_t pk_lo = (uint32_t)(*reinterpret_cast<const uint16_t *>(&l0)) | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&l1)) << 16);
+            const int kb = k0 >> 4, h = (k0 >> 3) & 1, q = (k0 & 7) >> 1;      // rank block, half of it, lane's quarter
+            s_tf[((size_t)kb * 32 + (2 * tok) * 4 + q) * 2 + h] = pk_hi;
+            s_tf[((size_t)kb * 32 + (2 * tok + 1) * 4 + q) * 2 + h] = pk_lo;
         }
         __syncwarp();
     }
