@@ -33,7 +33,7 @@ struct Workspace {
     size_t partial_floats = 0;
     float *t = nullptr;           // down-projection t = x.A^T, [M][rank] fp32 (kept zero between calls)
     float *t_gen = nullptr;       // t of the generic path (no invariant), grows on demand
-    float *tslots = nullptr;      // streaming decode kernel: tagged partial sums of t (all zero between calls)
+    float *tslots = nullptr;      // streaming decode kernel: partial sums of t, one encoded word per entry (all zero between calls)
     size_t tslots_floats = 0;
     size_t t_floats = 0, t_gen_floats = 0;
     int *counters = nullptr;      // [0]=t arrivals [1]=retired tiles [2]=status [3]=t ready [4]=parked; [8..] per tile

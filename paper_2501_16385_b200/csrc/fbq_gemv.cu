@@ -63,8 +63,11 @@ struct GemvParams {
     const __half *scales;
     const __half *zeros;
     void *y;
-    float2 *tpart;      // [n_t][M][rank] partial sums of t, one slot per t CTA, each entry (value, tag): tag 1.0f = written by
-                        // this launch; all tags are zero on entry and on exit
+    int slot_elems;     // words from one slot of tpart to the next: M * rank rounded up to whole 128-byte lines (slots
+                        // that share a line make the line a hot spot: every main CTA polls it while a t CTA writes it)
+    uint32_t *tpart;    // [n_t (+ 1)][M][rank] partial sums of t, one slot per t CTA (and one for their sum), each entry
+                        // one word: the fp32 value with +0.0 stored as -0.0, so a word is zero exactly while it has not been written
+                        // by this launch; all words are zero on entry and on exit
     int *ctr;           // [1] main CTAs that have read t; zero on entry and exit
     int *status;        // receives FBQ_ERR_TIMEOUT when a bounded wait runs out
     int M, N, K, G, rank;
@@ -607,33 +610,66 @@ __device__ __forceinline__ void prefetch_x(const GemvParams &p, int cta, int lan
 // (mask 1, 3, 7): the 16-byte unit index is XOR-ed with the 128-byte line index.
 __device__ __forceinline__ uint32_t swz(uint32_t off, uint32_t mask) { return off ^ (((off >> 7) & mask) << 4); }
 
-// One look at exactly eight t slots with at most 32 E entries: straight-line code, all 8 E loads of a lane in
-// flight (the common shapes: the looks are what a main CTA's epilogue waits with, and a lean look is a fast look).
-// Adds the slots in slot order into s_t, returns whether every entry carried its tag; amax = largest |sum|.
-template <int E>
-__device__ __forceinline__ bool look8(const float2 *slots, size_t slot_elems, int nent, int lane, float *s_t, float &amax)
+// An entry of a t slot is the fp32 value itself, with +0.0 stored as -0.0: the word is never zero once written, so
+// value and "written" travel in one 4-byte store, a reader may fetch four entries with one 16-byte load, add them as
+// they are (-0.0 adds like +0.0, and a sum that starts at +0.0 stays +0.0) and check each word by itself; memory that
+// is zero means "not yet".
+constexpr uint32_t kTNone = 0x80000000u;                     // -0.0: what a slot that does not exist reads as
+__device__ __forceinline__ uint32_t t_enc(float v) { const uint32_t w = __float_as_uint(v); return w ? w : kTNone; }
+__device__ __forceinline__ uint32_t t_min(uint32_t m, const uint4 &w) { return __vimin3_u32(m, __vimin3_u32(w.x, w.y, w.z), w.w); }
+
+// One look at exactly eight t slots with at most 128 entries: straight-line code, a lane takes four consecutive
+// entries and has its eight 16-byte loads in flight at once (the common shapes: the looks are what a main CTA's
+// epilogue waits with, and a lean look is a fast look).  Adds the slots in slot order into s_t, returns whether
+// every entry was there; amax = largest |sum|.
+__device__ __forceinline__ bool look8(const uint32_t *slots, size_t slot_elems, int nent, int lane, float *s_t, float &amax)
 {
-    float2 pv[E][8];
+    const int nq = nent >> 2, q = min(lane, nq - 1);          // lanes past the last four entries repeat them (and do not store)
+    uint4 pv[8];
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int i = min(lane + 32 * e, nent - 1);          // lanes past the last entry repeat it (and do not store)
+    for (int u = 0; u < 8; ++u) pv[u] = __ldcg(reinterpret_cast<const uint4 *>(slots + (size_t)u * slot_elems) + q);
+    uint32_t mn = 0xFFFFFFFFu;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) pv[e][u] = __ldcg(slots + (size_t)u * slot_elems + i);
+    for (int u = 0; u < 8; ++u) {
+        mn = t_min(mn, pv[u]);
+        v.x += __uint_as_float(pv[u].x);
+        v.y += __uint_as_float(pv[u].y);
+        v.z += __uint_as_float(pv[u].z);
+        v.w += __uint_as_float(pv[u].w);
     }
-    bool all = true;
+    if (lane < nq) *reinterpret_cast<float4 *>(s_t + 4 * lane) = v;
+    amax = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+    return mn != 0u;
+}
+
+// The same for any number of slots and entries: four entries x eight slots in flight per lane, added in slot order.
+__device__ __forceinline__ bool look_slots(const uint32_t *tpart, size_t slot_elems, int s_first, int s_end, int nent, int lane,
+                                           float *s_t, float &amax)
+{
+    uint32_t mn = 0xFFFFFFFFu;
     amax = 0.f;
+    for (int q = lane; 4 * q < nent; q += 32) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = s_first; c0 < s_end; c0 += 8) {
+            uint4 pa[8];
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        float v = 0.f;
+            for (int u = 0; u < 8; ++u)
+                pa[u] = (c0 + u < s_end) ? __ldcg(reinterpret_cast<const uint4 *>(tpart + (size_t)(c0 + u) * slot_elems) + q)
+                                         : make_uint4(kTNone, kTNone, kTNone, kTNone);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            v += pv[e][u].x;
-            all = all && (pv[e][u].y == 1.f);
+            for (int u = 0; u < 8; ++u) {
+                mn = t_min(mn, pa[u]);
+                v.x += __uint_as_float(pa[u].x);
+                v.y += __uint_as_float(pa[u].y);
+                v.z += __uint_as_float(pa[u].z);
+                v.w += __uint_as_float(pa[u].w);
+            }
         }
-        if (lane + 32 * e < nent) s_t[lane + 32 * e] = v;
-        amax = fmaxf(amax, fabsf(v));
+        *reinterpret_cast<float4 *>(s_t + 4 * q) = v;
+        amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
     }
-    return all;
+    return mn != 0u;
 }
 
 template <typename T, bool RANKED>
@@ -686,38 +722,16 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
         // the chunks in slot order.
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
         float amax = 0.f;
-        const size_t slot_elems = (size_t)M * rank;
+        const size_t slot_elems = (size_t)p.slot_elems;
         const int s_first = p.t_final ? p.n_t : 0, s_end = p.t_final ? p.n_t + 1 : p.n_t;    // the slots to add (or the one that holds their sum)
         bool ok = false;
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
-            if (s_end - s_first == 8 && M * rank <= 64) {
-                all = (M * rank <= 32) ? look8<1>(p.tpart + (size_t)s_first * slot_elems, slot_elems, M * rank, lane, s_t, amax)
-                                       : look8<2>(p.tpart + (size_t)s_first * slot_elems, slot_elems, M * rank, lane, s_t, amax);
-            } else
-            for (int i = lane; i < M * rank; i += 64) {                 // two entries x eight slots in flight, added in slot order
-                const bool two = i + 32 < M * rank;
-                float v0 = 0.f, v1 = 0.f;
-                for (int c0 = s_first; c0 < s_end; c0 += 8) {
-                    float2 pa[8], pb[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const bool in = c0 + u < s_end;
-                        pa[u] = in ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
-                        pb[u] = (in && two) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i + 32) : make_float2(0.f, 1.f);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        v0 += pa[u].x;
-                        v1 += pb[u].x;
-                        all = all && (pa[u].y == 1.f) && (pb[u].y == 1.f);
-                    }
-                }
-                s_t[i] = v0;
-                if (two) s_t[i + 32] = v1;
-                amax = fmaxf(amax, fmaxf(fabsf(v0), fabsf(v1)));
-            }
+            if (s_end - s_first == 8 && M * rank <= 128)
+                all = look8(p.tpart + (size_t)s_first * slot_elems, slot_elems, M * rank, lane, s_t, amax);
+            else
+                all = look_slots(p.tpart, slot_elems, s_first, s_end, M * rank, lane, s_t, amax);
             ok = __all_sync(0xffffffffu, all);
             if (!ok && look > 256) __nanosleep(64);
         }
@@ -1186,61 +1200,42 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         for (int ts = 0; ts < min(ntile, p.nb); ++ts) request_b(ts);   // rows of B are weights: before the wait
 
     prefetch_x(p, (int)blockIdx.x - p.n_t, lane, (int)sizeof(T));
+    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // [cb][kb][lane][2]
+    for (int i = lane; i < ncb * nkb * 64; i += 32) s_tf[i] = 0u;
+    __syncwarp();
     pdl_wait();
     mark(p, 2);
 
     float isc = 1.f;
-    uint32_t *s_tf = reinterpret_cast<uint32_t *>(smem + p.off_tf);      // [cb][kb][lane][2]
     if (rank > 0) {
         float *s_t = reinterpret_cast<float *>(smem + p.off_t);
         float amax = 0.f;
-        const size_t slot_elems = (size_t)M * rank;
+        const size_t slot_elems = (size_t)p.slot_elems;
         const int s_first = p.t_final ? p.n_t : 0, s_end = p.t_final ? p.n_t + 1 : p.n_t;
         bool ok = false;
         for (uint32_t look = 0; look < p.poll_limit && !ok; ++look) {
             bool all = true;
             amax = 0.f;
             if (s_end - s_first > 1) {
-                for (int i = lane; i < M * rank; i += 128) {            // four entries x eight slots in flight, added in slot order
-                    float v[4] = {0.f, 0.f, 0.f, 0.f};
-                    for (int c0 = s_first; c0 < s_end; c0 += 8) {
-                        float2 pa[4][8];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-#pragma unroll
-                            for (int u = 0; u < 8; ++u)
-                                pa[e][u] = (c0 + u < s_end && i + 32 * e < M * rank) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i + 32 * e)
-                                                                                    : make_float2(0.f, 1.f);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) {
-                                v[e] += pa[e][u].x;
-                                all = all && (pa[e][u].y == 1.f);
-                            }
-                    }
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (i + 32 * e < M * rank) {
-                            s_t[i + 32 * e] = v[e];
-                            amax = fmaxf(amax, fabsf(v[e]));
-                        }
-                }
+                all = look_slots(p.tpart, slot_elems, s_first, s_end, M * rank, lane, s_t, amax);
             } else {
-                for (int i0 = 0; i0 < M * rank; i0 += 32 * 16) {     // one slot: sixteen entries per lane in flight
-                    float2 part[16];
+                const uint4 *slot = reinterpret_cast<const uint4 *>(p.tpart + (size_t)s_first * slot_elems);
+                for (int q0 = 0; 4 * q0 < M * rank; q0 += 32 * 8) {  // one slot: eight times four entries per lane in flight
+                    uint4 part[8];
 #pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        part[u] = (i < M * rank) ? __ldcg(p.tpart + (size_t)s_first * slot_elems + i) : make_float2(0.f, 1.f);
+                    for (int u = 0; u < 8; ++u) {
+                        const int q = q0 + u * 32 + lane;
+                        part[u] = (4 * q < M * rank) ? __ldcg(slot + q) : make_uint4(kTNone, kTNone, kTNone, kTNone);
                     }
 #pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        all = all && (part[u].y == 1.f);
-                        if (i < M * rank) {
-                            s_t[i] = part[u].x;
-                            amax = fmaxf(amax, fabsf(part[u].x));
+                    for (int u = 0; u < 8; ++u) {
+                        const int q = q0 + u * 32 + lane;
+                        all = all && t_min(0xFFFFFFFFu, part[u]) != 0u;
+                        if (4 * q < M * rank) {
+                            const float4 v = make_float4(__uint_as_float(part[u].x), __uint_as_float(part[u].y), __uint_as_float(part[u].z),
+                                                         __uint_as_float(part[u].w));
+                            *reinterpret_cast<float4 *>(s_t + 4 * q) = v;
+                            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
                         }
                     }
                 }
@@ -1258,25 +1253,23 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
         const uint32_t sb = min(max(268u - ex, 1u), 254u);
         const float sc = __uint_as_float(sb << 23);
         isc = __uint_as_float((254u - sb) << 23);
-        for (int cb = 0; cb < ncb; ++cb) {
-            const int tok = 4 * cb + (g >> 1), part = g & 1;   // as an MMA column: token and (rounded value | remainder)
-            for (int kb = 0; kb < nkb; ++kb) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t pk = 0;
-                    if (tok < M) {
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const float v = s_t[tok * rank + kb * 16 + h * 8 + 2 * tq + e] * sc;
-                            const T hi = ActTraits<T>::from_float(v);
-                            const T lo = ActTraits<T>::from_float(v - ActTraits<T>::to_float(hi));
-                            const T pick = part ? lo : hi;
-                            pk |= (uint32_t)(*reinterpret_cast<const uint16_t *>(&pick)) << (16 * e);
-                        }
-                    }
-                    s_tf[((size_t)(cb * nkb + kb) * 32 + lane) * 2 + h] = pk;
-                }
-            }
+        // t as MMA column operands [column block of four tokens][rank block][lane][2]: column 2 (tok % 4) holds the
+        // rounded values of token tok, the next column what the rounding left; a lane takes pairs of consecutive rank
+        // indices and forms both terms once; the columns of tokens beyond M were set to zero before the wait.
+        const int half_rank = rank >> 1;
+        for (int idx = lane; idx < M * half_rank; idx += 32) {
+            const int tok = idx / half_rank, k0 = 2 * (idx - tok * half_rank);
+            const float2 tv = *reinterpret_cast<const float2 *>(s_t + tok * rank + k0);
+            const float v0 = tv.x * sc, v1 = tv.y * sc;
+            const T h0 = ActTraits<T>::from_float(v0), h1 = ActTraits<T>::from_float(v1);
+            const T l0 = ActTraits<T>::from_float(v0 - ActTraits<T>::to_float(h0));
+            const T l1 = ActTraits<T>::from_float(v1 - ActTraits<T>::to_float(h1));
+            const uint32_t pk_hi = (uint32_t)(*reinterpret_cast<const uint16_t *>(&h0)) | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&h1)) << 16);
+            const uint32_t pk_lo = (uint32_t)(*reinterpret_cast<const uint16_t *>(&l0)) | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&l1)) << 16);
+            const int cb = tok >> 2, kb = k0 >> 4, h = (k0 >> 3) & 1, q = (k0 & 7) >> 1;
+            uint32_t *dst = s_tf + ((size_t)(cb * nkb + kb) * 32 + (2 * (tok & 3)) * 4 + q) * 2 + h;
+            dst[0] = pk_hi;
+            dst[8] = pk_lo;                                     // four lanes on: the remainder's column
         }
         __syncwarp();
     }
@@ -1517,8 +1510,8 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kCW; ++w) v += s_red[((size_t)w * rank + j) * ncol + m];
-            // value and tag travel in one 8-byte store: whoever sees the tag sees the value
-            p.tpart[((size_t)c * M + tb * 8 + m) * rank + j] = make_float2(v, (p.test_skip_arrive || dead) ? 0.f : 1.f);
+            // the value, encoded so that the word is not zero: whoever sees the word sees the value
+            p.tpart[(size_t)c * p.slot_elems + (size_t)(tb * 8 + m) * rank + j] = (p.test_skip_arrive || dead) ? 0u : t_enc(v);
         }
         __syncthreads();
     }
@@ -1533,22 +1526,21 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
         __syncthreads();
         if (*s_last) {
             __threadfence();
-            const size_t slot_elems = (size_t)M * rank;
+            const size_t slot_elems = (size_t)p.slot_elems;
             for (int i = tid; i < M * rank; i += kThreads) {
                 float v = 0.f;
                 bool all = true;
                 for (int c0 = 0; c0 < p.n_t; c0 += 8) {
-                    float2 part[8];
+                    uint32_t part[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : make_float2(0.f, 1.f);
+                    for (int u = 0; u < 8; ++u) part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : kTNone;
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        v += part[u].x;
-                        all = all && (part[u].y == 1.f);
+                        v += __uint_as_float(part[u]);
+                        all = all && (part[u] != 0u);
                     }
                 }
-                p.tpart[(size_t)p.n_t * slot_elems + i] = make_float2(v, all ? 1.f : 0.f);
+                p.tpart[(size_t)p.n_t * slot_elems + i] = all ? t_enc(v) : 0u;
             }
         }
     }
@@ -1576,7 +1568,8 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
             }
             __syncthreads();
             if (*s_ok) {
-                for (int i = tid; i < (p.n_t + 1) * M * rank; i += kThreads) p.tpart[i] = make_float2(0.f, 0.f);
+                uint4 *z = reinterpret_cast<uint4 *>(p.tpart);            // 16 bytes per store: this is the kernel's tail
+                for (int i = tid; i < (p.n_t + 1) * (p.slot_elems >> 2); i += kThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
                 if (tid == 0) {
                     p.ctr[0] = 0;
                     p.ctr[1] = 0;
@@ -1820,6 +1813,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
     const size_t need_t = a.rank > 0 ? (size_t)p.off_tred + (size_t)kCW * a.rank * 2 * 4 : 0;      // M <= 2: two columns
     if (need_t > kSmemMax) return pl;
+    p.slot_elems = (a.M * a.rank + 31) / 32 * 32;
     p.t_final = (p.n_t * a.M * a.rank > 1024) ? 1 : 0;    // many entries: one t CTA adds the slots for everybody
     pl.smem = std::max(need, need_t) + 1024;       // slack for the alignment of the dynamic window
     p.poll_limit = tune.poll_limit > 0 ? (uint32_t)tune.poll_limit : (1u << 20);
@@ -1927,6 +1921,7 @@ Plan make_plan_wide(const LinearArgs &a, const GemvTuning &tune)
     const size_t need = layout(ns);
     if (need > kSmemMax - 2048) return pl;
     p.off_tab = 0;
+    p.slot_elems = (a.M * a.rank + 31) / 32 * 32;
     p.t_final = (p.n_t * a.M * a.rank > 2048) ? 1 : 0;
     p.off_tA = 1024;
     p.off_tred = p.off_tA + p.t_kb * a.rank * 128;
@@ -2074,7 +2069,7 @@ void gemv_workspace_need(const LinearArgs &a, const GemvTuning &tune, size_t *tp
 {
     const bool wide = a.M > 2;
     const Plan pl = wide ? make_plan_wide(a, tune) : make_plan(a, tune);
-    *tpart_floats = (size_t)2 * (std::max(pl.p.n_t, 1) + 1) * a.M * std::max(a.rank, 1);
+    *tpart_floats = (size_t)(std::max(pl.p.n_t, 1) + 1) * std::max(pl.p.slot_elems, 32);
     *counters = 8 + (wide ? pl.p.NT : 0);
     *partial_floats = (wide && pl.p.SK > 1) ? (size_t)pl.p.NT * pl.p.SK * a.M * kTile : 0;
 }
@@ -2088,7 +2083,7 @@ cudaError_t launch_gemv(const LinearArgs &a, Workspace &ws, const GemvTuning &tu
     p.x = a.x; p.scales = a.scales; p.zeros = a.zeros; p.y = a.y;
     p.part = ws.partial;
     p.tctr = ws.counters + 8;
-    p.tpart = reinterpret_cast<float2 *>(ws.tslots);
+    p.tpart = reinterpret_cast<uint32_t *>(ws.tslots);
     p.ctr = ws.counters;
     p.status = ws.counters + kCtrStatus;
     // tuning aid: consecutive launches write their phase marks to alternate halves of the buffer
