@@ -134,6 +134,26 @@ def test_decode_rank0_and_zero_branches_agree(fbq, torch, bits):
     check_parity(inp0, fbq, expect_kernel=fbq.KERNEL_DECODE)
 
 
+@pytest.mark.parametrize("M,N,K,rank", [(1, 512, 4096, 64), (2, 256, 4096, 128), (1, 256, 11008, 64), (8, 512, 4096, 64),
+                                        (16, 256, 4096, 128), (4, 256, 11008, 32)])
+def test_streaming_kernel_zero_t_is_not_taken_for_missing(fbq, torch, M, N, K, rank):
+    # x = 0 makes every partial sum of t an exact zero.  The t slots announce themselves by being non-zero (a zero
+    # is stored as -0.0), so an all-zero t must neither time out nor change y: one slot per t CTA, the slot of the
+    # sum where there are many entries (K = 11008), both forms of the kernel
+    inp = make_linear(M, N, K, 3, rank, seed=31 * M + rank)
+    dev = DeviceLinear(inp, fbq)
+    fbq.set_option("force_kernel", fbq.KERNEL_DECODE)
+    try:
+        for x in (torch.zeros_like(dev.x), -torch.zeros_like(dev.x)):
+            y = dev.run(fbq, x=x)
+            torch.cuda.synchronize()
+            assert fbq.poll_status() == 0
+            assert torch.count_nonzero(y).item() == 0
+        check_parity(inp, fbq, expect_kernel=fbq.KERNEL_DECODE)       # and the slots are clean for the next call
+    finally:
+        fbq.set_option("force_kernel", -1)
+
+
 @pytest.mark.parametrize("bits,dtype", [(4, "f16"), (3, "f16"), (4, "bf16"), (3, "bf16")])
 def test_decode_sub_branch_alone(fbq, bits, dtype):
     # codes == zero points: the main path vanishes and y is the low-rank product alone,
