@@ -89,6 +89,9 @@ struct PrefillParams {
     int *split_ctr;           // [tile] splits that have stored their partial (self-clearing)
     uint32_t flag_polls;      // looks (256 ns apart) at a token tile's t flag before the wait gives up
     int test_skip_flag;       // test switch: the t CTAs do not raise the flag (the wait for t must run out)
+    void *t16;                // [M][rank_pad] t rounded to the activation type, written by the t CTAs and read by the main
+                              // CTAs' TMA copies as one more token operand (NULL: t32 and the producers' conversion)
+    int rank_pad;             // columns of t16: rank rounded up to whole K blocks of 64 (the padding is zero)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -412,11 +415,12 @@ template <int TOK> struct Smem {
 // amap: A [rank][K], boxes of 128 rows x 64 elements, 128-byte swizzle (t CTAs)
 // bmap: B [N][rank], boxes of 128 rows x 64 elements, 128-byte swizzle (main CTAs, rank > 0)
 // ymap: y [M][N], boxes of TOK/4 rows x 128 elements, no swizzle (stores)
+// tmap: t16 [M][rank_pad], boxes like xmap's (main CTAs, rank > 0, one K split of t)
 template <int BITS, typename T, int TOK>
 __global__ void __launch_bounds__(kPfThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
                const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
-               const __grid_constant__ CUtensorMap ymap, const PrefillParams p)
+               const __grid_constant__ CUtensorMap ymap, const __grid_constant__ CUtensorMap tmap, const PrefillParams p)
 {
     using L = Smem<TOK>;
     constexpr uint32_t kXBytes = L::kXBytes, kStageBytes = L::kStageBytes;
@@ -486,6 +490,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&amap)) : "memory");
         } else {
             if (p.rank > 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&bmap)) : "memory");
+            if (p.t16) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ymap)) : "memory");
         }
     }
@@ -581,6 +586,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             for (int i = kb_x + h; i < nkb && !dead; i += 2) {
                 const int s = i % kStages;
                 if (i >= kStages && !pf_mbar_wait(empty0 + 8u * s, (uint32_t)(i / kStages - 1) & 1u)) { dead = true; break; }
+                if (p.t16) {                                 // both operands of this block arrive by TMA: nothing to write
+                    __syncwarp();
+                    if (lane == 0) pf_mbar_arrive(full0 + 8u * s);
+                    continue;
+                }
                 if (!t_ready) {                              // every warp of every t CTA of this token tile has stored its part
                     int seen = 0;
                     if (lane == 0) {
@@ -721,6 +731,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         unsigned short *sp = reinterpret_cast<unsigned short *>(smem + (size_t)c * (kBN * 2)) + 32 * q + lane;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) sp[j * kBN] = to_bits16<T>(__uint_as_float(v[j]));
+                    } else if (p.t16) {
+                        if (nn < p.rank_pad) {               // rounded once, here; rows of A beyond the rank are zero fill
+                            unsigned short *tp = static_cast<unsigned short *>(p.t16) + (size_t)(m0 + c) * p.rank_pad + nn;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (m0 + c + j < p.M) tp[(size_t)j * p.rank_pad] = to_bits16<T>(__uint_as_float(v[j]));
+                        }
                     } else {
                         if (nn < p.rank) {                   // 32 lanes = 32 consecutive rank indices: 128-byte stores
                             float *tp = p.t32 + (size_t)split * p.M * p.rank + (size_t)(m0 + c) * p.rank + nn;
@@ -748,7 +765,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 }
             }
             if (t_role) {
-                // this warp's part of t is stored: make it visible, then count the warp in
+                // this warp's part of t is stored: make it visible (to the main CTAs' TMA copies as well), then count the warp in
+                asm volatile("fence.proxy.async;" ::: "memory");
                 __threadfence();
                 __syncwarp();
                 if (lane == 0 && !p.test_skip_flag) atomicAdd(p.tflag + m_tile, 1);
@@ -816,6 +834,26 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 } else if (kb < kb_x) {
                     pf_mbar_expect_tx(bar, kXBytes);
                     tma_load_2d(xt, &xmap, (kb_begin + kb) * kBK, m0, bar);
+                } else if (p.t16) {
+                    if (kb == kb_x) {                        // every warp of every t CTA of this token tile has stored its part
+                        const int *flag = p.tflag + m_tile;
+                        const int target = 16 * p.rt * p.splitt;
+                        int seen = 0;
+#pragma unroll 1
+                        for (uint32_t spin = 0; spin < p.flag_polls; ++spin) {
+                            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+                            if (seen >= target) break;
+                            __nanosleep(256);
+                        }
+                        if (seen < target) {
+                            dead = true;
+                            break;
+                        }
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                    }
+                    pf_mbar_expect_tx(bar, kXBytes + kWBytes);
+                    tma_load_2d(xt, &tmap, (kb - kb_x) * kBK, m0, bar);   // t as the token operand
+                    tma_load_2d(wt, &bmap, (kb - kb_x) * kBK, n0, bar);   // rows of B
                 } else {
                     pf_mbar_expect_tx(bar, kWBytes);
                     tma_load_2d(wt, &bmap, (kb - kb_x) * kBK, n0, bar);   // rows of B
@@ -876,8 +914,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             for (int t = 0; t < 4; ++t) out[t] = __funnelshift_r(w[t], w[t + 1], (o & 1u) * 16u);
         };
         bool dead = false;
-        fetch(0);
         const uint32_t ring0 = sbase + L::kRingOff, table0 = sbase + L::kTableOff + (uint32_t)(64 * v + lane) * 4u;
+        fetch(0);
 #pragma unroll 1
         for (int c = 0; 8 * c < groups && !dead; ++c) {
             uint32_t sz[2][8];                              // (s | z << 16) of [row][group of this chunk]
@@ -1465,7 +1503,7 @@ int g_pf_pdl = 1;             // launch with programmatic stream serialisation (
 
 template <int BITS, typename T, int TOK>
 cudaError_t launch_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, const CUtensorMap &amap, const CUtensorMap &bmap,
-                          const CUtensorMap &ymap, const PrefillParams &p, unsigned grid, cudaStream_t s)
+                          const CUtensorMap &ymap, const CUtensorMap &tmap, const PrefillParams &p, unsigned grid, cudaStream_t s)
 {
     auto kern = prefill_kernel<BITS, T, TOK>;
     static bool attr_set = false;
@@ -1484,7 +1522,7 @@ cudaError_t launch_kernel(const CUtensorMap &xmap, const CUtensorMap &wmap, cons
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = g_pf_pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, xmap, wmap, amap, bmap, ymap, p);
+    return cudaLaunchKernelEx(&cfg, kern, xmap, wmap, amap, bmap, ymap, tmap, p);
 }
 
 template <int BITS, typename T>
@@ -1597,6 +1635,14 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
         return e;
     if ((e = make_map(&ymap, a.y, false, (size_t)a.N, (size_t)a.M, kBN, TOK / 4, CU_TENSOR_MAP_SWIZZLE_NONE)) != cudaSuccess) return e;
     amap = bmap = xmap;
+    CUtensorMap tmap = xmap;
+    p.t16 = nullptr;
+    p.rank_pad = p.kb_slab * kBK;
+    if (!PAIR && a.rank > 0 && p.splitt == 1) {
+        // t goes from the t CTAs to the main CTAs in the activation type, laid out like x, behind the fp32 slices of t
+        p.t16 = ws.t_gen + (((size_t)a.M * a.rank + 3) & ~(size_t)3);
+        if ((e = make_map(&tmap, p.t16, false, (size_t)p.rank_pad, (size_t)a.M, kBK, TOK, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
+    }
     if (a.rank > 0) {
         if ((e = make_map(&amap, a.A, false, (size_t)a.K, (size_t)a.rank, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
         if ((e = make_map(&bmap, a.B, false, (size_t)a.rank, (size_t)a.N, kBK, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) != cudaSuccess) return e;
@@ -1606,8 +1652,8 @@ cudaError_t run_prefill(const LinearArgs &a, Workspace &ws, cudaStream_t s, int 
         e = (a.bits == 4) ? launch_pair_kernel<4, T>(xmap, qmap, amap, bmap, ymap, p, grid, s)
                           : launch_pair_kernel<3, T>(xmap, qmap, amap, bmap, ymap, p, grid, s);
     else
-        e = (a.bits == 4) ? launch_kernel<4, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s)
-                          : launch_kernel<3, T, TOK>(xmap, qmap, amap, bmap, ymap, p, grid, s);
+        e = (a.bits == 4) ? launch_kernel<4, T, TOK>(xmap, qmap, amap, bmap, ymap, tmap, p, grid, s)
+                          : launch_kernel<3, T, TOK>(xmap, qmap, amap, bmap, ymap, tmap, p, grid, s);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -1640,7 +1686,7 @@ void prefill_workspace_need(const LinearArgs &a, int *counters, size_t *t_floats
     const int mt128 = (a.M + 127) / 128;
     const int splits = (a.M <= 128) ? prefill_splits(a.N, a.K) : 1;
     *counters = kPfCtrBase + 2 * mt128 + nt * mt128 + 2;
-    *t_floats = (size_t)a.M * a.rank * splits;
+    *t_floats = (size_t)a.M * a.rank * splits + 4 + (size_t)a.M * ((a.rank + 63) / 64 * 64) / 2;      // fp32 slices of t, then t in the activation type
     *partial_floats = (splits > 1) ? (size_t)nt * splits * kBN * 128 : 0;
 }
 
