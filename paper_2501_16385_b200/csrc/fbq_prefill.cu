@@ -572,11 +572,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     for (int kc = 0; kc < 4; ++kc)
                         sts128(wdst + (uint32_t)b * kStageBytes + ((((uint32_t)(4 * part + kc)) ^ wsw) << 4), wb[4 * kc], wb[4 * kc + 1], wb[4 * kc + 2],
                                wb[4 * kc + 3]);
-                    pf_fence_proxy_async();                 // generic-proxy stores -> visible to the MMA's reads
-                    __syncwarp();
-                    if (lane == 0) pf_mbar_arrive(fullb + 8u * b);          // one arrival per warp
                 }
                 if (dead) break;
+                pf_fence_proxy_async();                     // generic-proxy stores -> visible to the MMA's reads
+                __syncwarp();
+                if (lane == 0) {                            // one arrival per warp and block
+                    pf_mbar_arrive(fullb);
+                    pf_mbar_arrive(fullb + 8u);
+                }
                 if (g >= 2) ephase ^= 1u;
             }
             // ---- sub-branch blocks: token operand = t (fp32 scratch, rounded once); B arrives by TMA.
