@@ -419,7 +419,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
             dst[g + 8] = acc[1];
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFull + buf));
+        mbar_arrive_if(bars + 8u * (kBarSegFull + buf), lane == 0);
         mark(p, ts == 0 ? 5 : 6);
         acc[0] = acc[1] = 0.f;
         if (++dep_buf == p.nbuf) {
@@ -497,7 +497,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                 scale(d0, mt, acc);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+            mbar_arrive_if(bars + 8u * (kBarEmpty + slot), lane == 0);
             if (nts != ts) {
                 if (!deposit(ts, acc)) return false;
                 if (++mi == p.nmeta) mi = 0;
@@ -547,7 +547,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                     scale(d0, mt, acc);
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+                mbar_arrive_if(bars + 8u * (kBarEmpty + slot), lane == 0);
                 if (++slot == NS) {
                     slot = 0;
                     par ^= 1u;
@@ -859,7 +859,7 @@ __device__ __forceinline__ bool epilogue(const GemvParams &p, uint8_t *smem, con
             vh = ph[0];
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
+        mbar_arrive_if(bars + 8u * (kBarSegFree + buf), lane == 0);
         if constexpr (RANKED) {
             const float2 sb = s_sub[(size_t)(ts & (kMaxSub - 1)) * 32];
             vg = fmaf(sb.x, isc, vg);
@@ -1143,7 +1143,7 @@ __device__ __forceinline__ bool compute_w16(const GemvParams &p, uint8_t *smem, 
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bars + 8u * (kBarEmpty + slot));
+            mbar_arrive_if(bars + 8u * (kBarEmpty + slot), lane == 0);
             if (++slot == NS) {
                 slot = 0;
                 par ^= 1u;
@@ -1165,7 +1165,7 @@ __device__ __forceinline__ bool compute_w16(const GemvParams &p, uint8_t *smem, 
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFull + buf));
+        mbar_arrive_if(bars + 8u * (kBarSegFull + buf), lane == 0);
         mark(p, ts == 0 ? 5 : 6);
         if (++buf == p.nbuf) {
             buf = 0;
@@ -1389,7 +1389,7 @@ __device__ __forceinline__ bool epilogue_wide(const GemvParams &p, uint8_t *smem
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + 8u * (kBarSegFree + buf));
+        mbar_arrive_if(bars + 8u * (kBarSegFree + buf), lane == 0);
         if (SK > 1) {
             // this slice's partial tile to scratch, then count in
             float *pt = p.part + ((size_t)tile * SK) * M * kTile;
