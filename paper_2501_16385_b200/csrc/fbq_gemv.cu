@@ -200,13 +200,13 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     const int units = M * SPT * 2;                                          // (group, token) units of this warp, token fastest
     const int upper = lane & 1;
     // unit u of the warp: eight lanes share it
-    auto locate = [&](int it, int &m, int &run, bool &valid, bool &pad) {
+    auto locate = [&](int it, int &m, int &run, bool &valid, int &pad) {
         const int u = it * 4 + (lane >> 3);
         const int li = u / M;
         m = u - li * M;
         const int grp = kCHG * (li >> 1) + 2 * warp + (li & 1);
         valid = u < units && grp < G;
-        pad = u < units && grp == G;                                        // the partner of the last group when G is odd
+        pad = (u < units && grp >= G) ? grp : -1;                           // a group of the last stage beyond K
         run = valid ? grp * 4 + ((lane >> 1) & 3) : 0;
     };
     // All of the warp's x is requested at once, as whole 128-byte lines (every CTA of the grid reads the same x at
@@ -218,8 +218,8 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     constexpr uint32_t garea = 2u * ncol * 64u;                             // bytes of one group's digit area
     const int nbatch = (units + 3) >> 2;
     for (int it = 0; it < nbatch; ++it) {
-        int m, run;
-        bool valid, pad;
+        int m, run, pad;
+        bool valid;
         locate(it, m, run, valid, pad);
         if (valid) {
             const T *src = x + (size_t)m * p.K + (size_t)(run >> 2) * 128 + (lane & 7) * 8;
@@ -234,12 +234,14 @@ __device__ __forceinline__ void convert_x(const GemvParams &p, uint8_t *smem, in
     __syncwarp();
 #pragma unroll 1
     for (int it = 0; it < nbatch; ++it) {
-        int m, run;
-        bool valid, pad;
+        int m, run, pad;
+        bool valid;
         locate(it, m, run, valid, pad);
-        if (pad && (lane & 7) == 0) {
-            s_tab[((size_t)G * M + m) * 2] = make_float4(0.f, 0.f, 0.f, 0.f);
-            s_tab[((size_t)G * M + m) * 2 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        // The last stage is multiplied whole: its groups beyond K arrive as zero codes (the tensor copy's fill), and
+        // their table entries are zero, so they add nothing whatever stands where their x would be.
+        if (pad >= 0 && (lane & 7) == 0) {
+            s_tab[((size_t)pad * M + m) * 2] = make_float4(0.f, 0.f, 0.f, 0.f);
+            s_tab[((size_t)pad * M + m) * 2 + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         uint4 xv[4];
         {
@@ -447,7 +449,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
         if (total > 0) {
             if (!mbar_wait(bars + 8u * kBarFull, 0u)) return false;
             mark(p, 4);
-            if (2 * warp < G) load_pass(0);
+            load_pass(0);
         }
         float acc[2] = {0.f, 0.f};
         int ts = 0, st = 0, slot = 0, nslot = (NS > 1) ? 1 : 0;
@@ -456,7 +458,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
         int mi = 0;
         for (int it = 0; it < total; ++it) {
             const int pi = st * (kCHG / 2) + warp, ga = 2 * pi;
-            const bool live = ga < G;
+            constexpr bool live = true;                                    // groups beyond K are zero codes with a zero table entry
             Meta mt;
             int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0}, d2[4] = {0, 0, 0, 0}, d3[4] = {0, 0, 0, 0};
             if (live) {
@@ -489,7 +491,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
             }
             if (it + 1 < total) {
                 if (!mbar_wait(bars + 8u * (kBarFull + nslot), npar)) return false;
-                if (2 * (nst * (kCHG / 2) + warp) < G) load_pass(nslot);
+                load_pass(nslot);
             }
             if (live) {
 #pragma unroll
@@ -527,7 +529,6 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int gi = 2 * warp + u, grp = st * kCHG + gi;
-                    if (grp >= G) break;
                     const uint32_t wa = ws + (uint32_t)gi * (kTile * GB);
                     uint32_t w0[NW], w1[NW], ra[NR], rb[NR];
                     load_words(wa, w0);
@@ -536,7 +537,7 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                     const uint4 x0 = lds_v4_if(xp, pa), x1 = lds_v4_if(xp + x_chunk1, pa);
                     uint32_t tv = 0;
                     if constexpr (BITS == 3) tv = lds_u32_if(xt + (uint32_t)grp * xts, pt);
-                    const Meta mt = load_meta(tab + (uint32_t)grp * 64u, mslot + (uint32_t)grp * 2u);
+                    const Meta mt = load_meta(tab + (uint32_t)grp * 64u, mslot + (uint32_t)min(grp, G - 1) * 2u);
                     int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0};
                     Slots<BITS>::run(w0, ra);
                     Slots<BITS>::run(w1, rb);
@@ -1771,7 +1772,7 @@ Plan make_plan(const LinearArgs &a, const GemvTuning &tune)
         off += (size_t)kNumBars * 8;
         off = align_up(off, 16);
         p.off_tab = (int)off;
-        off += (size_t)(G + 1) * a.M * 32;
+        off += (size_t)SPT * kCHG * a.M * 32;                       // the last stage's groups beyond K have (zero) entries too
         off = align_up(off, 128);
         p.off_x = (int)off;
         off += (size_t)G * ncol * (a.bits == 4 ? 128 : 144);
