@@ -489,10 +489,8 @@ __device__ __forceinline__ bool compute_i8(const GemvParams &p, uint8_t *smem, i
                 nst = 0;
                 ++nts;
             }
-            if (it + 1 < total) {
-                if (!mbar_wait(bars + 8u * (kBarFull + nslot), npar)) return false;
-                load_pass(nslot);
-            }
+            if (it + 1 < total && !mbar_wait(bars + 8u * (kBarFull + nslot), npar)) return false;
+            load_pass(nslot);                                               // after the last pass: words that nobody uses
             if (live) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) d0[i] = (d0[i] + d1[i]) + (d2[i] + d3[i]);
