@@ -1526,20 +1526,46 @@ __device__ __forceinline__ void t_cta(const GemvParams &p, uint8_t *smem, const 
         if (*s_last) {
             __threadfence();
             const size_t slot_elems = (size_t)p.slot_elems;
-            for (int i = tid; i < M * rank; i += kThreads) {
-                float v = 0.f;
-                bool all = true;
-                for (int c0 = 0; c0 < p.n_t; c0 += 8) {
-                    uint32_t part[8];
+            if (M * rank <= kThreads) {
+                // few entries: one per thread, so that as many threads as possible share the loads
+                for (int i = tid; i < M * rank; i += kThreads) {
+                    float v = 0.f;
+                    bool all = true;
+                    for (int c0 = 0; c0 < p.n_t; c0 += 8) {
+                        uint32_t part[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : kTNone;
+                        for (int u = 0; u < 8; ++u) part[u] = (c0 + u < p.n_t) ? __ldcg(p.tpart + (size_t)(c0 + u) * slot_elems + i) : kTNone;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        v += __uint_as_float(part[u]);
-                        all = all && (part[u] != 0u);
+                        for (int u = 0; u < 8; ++u) {
+                            v += __uint_as_float(part[u]);
+                            all = all && (part[u] != 0u);
+                        }
                     }
+                    p.tpart[(size_t)p.n_t * slot_elems + i] = all ? t_enc(v) : 0u;
                 }
-                p.tpart[(size_t)p.n_t * slot_elems + i] = all ? t_enc(v) : 0u;
+            } else {
+                // many entries (several tokens): four per thread and load, or the rounds of loads are this CTA's time
+                for (int q = tid; 4 * q < M * rank; q += kThreads) {
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    uint32_t mn = 0xFFFFFFFFu;
+                    for (int c0 = 0; c0 < p.n_t; c0 += 8) {
+                        uint4 part[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            part[u] = (c0 + u < p.n_t) ? __ldcg(reinterpret_cast<const uint4 *>(p.tpart + (size_t)(c0 + u) * slot_elems) + q)
+                                                       : make_uint4(kTNone, kTNone, kTNone, kTNone);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            mn = t_min(mn, part[u]);
+                            v.x += __uint_as_float(part[u].x);
+                            v.y += __uint_as_float(part[u].y);
+                            v.z += __uint_as_float(part[u].z);
+                            v.w += __uint_as_float(part[u].w);
+                        }
+                    }
+                    reinterpret_cast<uint4 *>(p.tpart + (size_t)p.n_t * slot_elems)[q] =
+                        mn != 0u ? make_uint4(t_enc(v.x), t_enc(v.y), t_enc(v.z), t_enc(v.w)) : make_uint4(0u, 0u, 0u, 0u);
+                }
             }
         }
     }
