@@ -304,6 +304,9 @@ def time_plain_steps(torch, issue, steps):
     return e0.elapsed_time(e1)
 
 
+E2E_WARM_S = 0.3          # untimed end-to-end steps before the clock starts (seconds of wall time, at least `warmup` steps)
+
+
 def time_e2e(fbq, torch, wl, pool, steps: int, warmup: int, batched: bool = False):
     """Same steps end to end through the C ABI with HOST buffers (x from pinned host memory, y read back to
     pinned host memory), then a stream synchronise so that the step's results are on the host.  Wall clock.
@@ -328,12 +331,16 @@ def time_e2e(fbq, torch, wl, pool, steps: int, warmup: int, batched: bool = Fals
                 fbq.linear_hostio(xs[li][j], d.qweight, d.scales, d.zeros, d.A, d.B, ys[li][j], d.N, GROUP, wl.bits, stream=main)
         main.synchronize()                            # the step's results are read on the host
 
-    for i in range(max(3, warmup)):
-        one(i)
+    # Untimed steps until the path has settled: on this host the first tenths of a second of such steps (small copies and
+    # kernel writes across the bus, a synchronise per step) run about 30 % slower than all later ones.
+    tw, nw = time.perf_counter(), 0
+    while nw < max(3, warmup) or time.perf_counter() - tw < E2E_WARM_S:
+        one(nw)
+        nw += 1
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for i in range(steps):
-        one(i)
+        one(nw + i)
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
     h2d = sum(K * 2 * wl.M for K, _ in wl.shapes)
@@ -528,13 +535,13 @@ def decode_line(args, fbq, torch, wl, peaks, peak_kind, world, rank_id, local, b
         if world == 1:
             e2e_steps = min(max(args.steps, 50), 500)
             dt, h2d, d2h = time_e2e(fbq, torch, wl, pool, e2e_steps, 3)
-            what = "fbq_linear_hostio per linear in layer order, host buffers, synchronise per step"
+            what = "fbq_linear_hostio per linear in layer order after 0.3 s of untimed steps, host buffers, synchronise per step"
             per_linear_ms = dt * 1e3 / e2e_steps
             if n_lin > 1 and hasattr(fbq, "make_batch"):
                 dtb, _, _ = time_e2e(fbq, torch, wl, pool, e2e_steps, 3, batched=True)
                 if dtb < dt:
                     dt = dtb
-                    what = ("one fbq_linear_batch_hostio call per step (the library's side streams overlap the problems' "
+                    what = ("one fbq_linear_batch_hostio call per step after 0.3 s of untimed steps (the library's side streams overlap the problems' "
                             "small copies), host buffers, synchronise per step")
             extra["e2e"] = {"value": bytes_step * e2e_steps / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                             "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3 / e2e_steps, "steps": e2e_steps,
